@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the fixed-point 8-bit inference path: one step = one forward pass of the
+ResNet-50-shaped fixed-point network on a batch of 256 synthetic 224x224x3 int8 images.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  `value` is images/s with inputs resident in HBM; `e2e` is the same
+metric with the image batch copied from pinned host memory and the logits copied back every step.
+With --impl reference the CPU oracle is timed instead (a deliberately plain program: context only).
+Under torchrun every rank runs the same batch on its own GPU (replicas, no collective on the data
+path); the elapsed time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2202_05239_b200 import synth  # noqa: E402
+
+METRIC = "fixed-point inference images/sec"
+UNIT = "images/s"
+WORKLOAD = "resnet50_fixed_point_b256"
+NET, BATCH, SEED = "resnet50", 256, 0
+INT8_NOMINAL_TOPS = 4500.0
+
+
+# ----------------------------------------------------------------------------- distributed plumbing
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def dist_init(backend: str):
+    import torch.distributed as dist
+    rank, _, world = dist_env()
+    if world > 1 and not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29511")
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(value: float, world: int, device="cpu") -> float:
+    """Maximum of a per-rank scalar (the job is as slow as its slowest rank)."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank_per_step: int, steps: int, world: int, elapsed_ms_max: float) -> float:
+    return units_per_rank_per_step * steps * world / (elapsed_ms_max * 1e-3)
+
+
+# ----------------------------------------------------------------------------- clocks
+
+CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+class ClockSampler:
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.path = os.path.join("/tmp", f"f8_clocks_{os.getpid()}.csv")
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={CLOCK_QUERY}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu_index), "-lms", "100"], stdout=self.f,
+                                         stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.f.close()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    smax.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, flag in zip(names, parts[5:9]):
+                    if flag.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------- reference arm / CPU baseline
+
+def time_oracle(layers, images: int, seed: int):
+    """Times the CPU oracle, as it stands, on `images` images of the workload; returns (images/s, seconds, threads)."""
+    from oracle import f8ref
+    f8ref.lib()
+    x = synth.draw_image(images, seed + 1)
+    t0 = time.perf_counter()
+    f8ref.net_forward(layers, x, keep_all=False)
+    dt = time.perf_counter() - t0
+    return images / dt, dt, f8ref.threads()
+
+
+def cpu_baseline(layers, target_seconds: float = 12.0):
+    ips1, dt1, threads = time_oracle(layers, 1, SEED)
+    n = int(max(2, min(64, round(target_seconds / max(dt1, 1e-3)))))
+    ips, dt, threads = time_oracle(layers, n, SEED)
+    return {"value": ips, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{n} of the {BATCH} images of {WORKLOAD} ({dt:.1f} s); images are independent, so the rate is per image"}
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    layers = synth.make_net(NET, SEED)
+    sample = 4
+    for _ in range(max(0, min(args.warmup, 1))):
+        time_oracle(layers, 1, SEED)
+    t0 = time.perf_counter()
+    threads = 0
+    for _ in range(args.steps):
+        _, _, threads = time_oracle(layers, sample, SEED)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "net": NET, "global_batch": BATCH,
+                       "note": f"each step is a {sample}-image sample of the batch run through the CPU oracle"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": f"{sample} images per step x {args.steps} steps"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- our arm
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured"
+    except (OSError, KeyError, ValueError):
+        return 6650.0, "fallback"
+
+
+def run_ours(args):
+    import torch
+    from paper_2202_05239_b200 import api
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fixed-point path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist_init("nccl")
+
+    layers = synth.make_net(NET, SEED)
+    net = api.Net(layers, BATCH)
+    x_host = torch.from_numpy(synth.draw_image(BATCH, SEED + 1 + rank)).pin_memory()
+    x_dev = x_host.to(dev)
+    out = torch.empty((BATCH, 1000), dtype=torch.int32, device=dev)
+    out_host = torch.empty((BATCH, 1000), dtype=torch.int32).pin_memory()
+    ws = torch.empty(net.workspace_bytes(BATCH), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        net.forward(x_dev, out=out, workspace=ws)
+
+    def step_e2e():
+        x_dev.copy_(x_host, non_blocking=True)
+        net.forward(x_dev, out=out, workspace=ws)
+        out_host.copy_(out, non_blocking=True)
+
+    # ---- device-resident throughput
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    api.f8_device_status()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier(world)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    elapsed_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = net.last_launch_count * args.steps
+    value = whole_job_rate(BATCH, args.steps, world, elapsed_ms)
+
+    # ---- end to end (host buffers, copies inside the timed region)
+    for _ in range(2):
+        step_e2e()
+    torch.cuda.synchronize()
+    barrier(world)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step_e2e()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    e2e_value = whole_job_rate(BATCH, args.steps, world, e2e_ms)
+
+    # ---- per-layer device times of the timed configuration (events between the launches)
+    net.set_profiling(True)
+    reps = max(3, min(10, args.steps))
+    acc_ms = np.zeros(len(layers))
+    tc_flags = None
+    for _ in range(reps):
+        step()
+        ms, tc_flags = net.layer_ms()
+        acc_ms += np.array(ms)
+    net.set_profiling(False)
+    layer_ms = acc_ms / reps
+
+    # ---- attainable INT8 rate of this device (MMA-only probe), same run
+    iters = 4096
+    api.f8_mma_i8_probe(iters)      # warm-up
+    torch.cuda.synchronize()
+    e0.record(stream)
+    ops = api.f8_mma_i8_probe(iters)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    probe_tops = ops / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    api.f8_device_status()
+
+    if rank != 0:
+        return
+    peak_gbs, peak_kind = measured_peaks()
+    tc_bytes = tc_ops = tc_ms = 0.0
+    other_bytes = other_ms = 0.0
+    per_layer = []
+    for l, ms, tc in zip(layers, layer_ms, tc_flags):
+        b = BATCH * l.bytes_per_image() + l.param_bytes()
+        o = 2.0 * BATCH * l.macs_per_image
+        if tc:
+            tc_bytes += b
+            tc_ops += o
+            tc_ms += ms
+        else:
+            other_bytes += b
+            other_ms += ms
+        per_layer.append({"name": l.name, "ms": round(float(ms), 5), "tc": bool(tc),
+                          "gbs": round(b / (ms * 1e-3) / 1e9, 1) if ms > 0 else None,
+                          "tops": round(o / (ms * 1e-3) / 1e12, 1) if ms > 0 else None})
+    achieved = tc_bytes / (tc_ms * 1e-3) / 1e9 if tc_ms > 0 else 0.0
+    total_ops = 2.0 * BATCH * synth.net_macs_per_image(layers)
+    ms_per_step = elapsed_ms / args.steps
+    roofline = {
+        "kernel": "f8_conv_gemm_tc_kernel",
+        "bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
+        "peak_source": f"{peak_kind} HBM copy bandwidth",
+        "traffic": None,
+        "launches_per_step": int(sum(tc_flags)), "kernel_ms_per_step": tc_ms,
+        "algorithmic_bytes_per_step": tc_bytes,
+        "tensor": {"achieved_tops": tc_ops / (tc_ms * 1e-3) / 1e12 if tc_ms > 0 else 0.0,
+                   "probe_peak_tops": probe_tops, "nominal_peak_tops": INT8_NOMINAL_TOPS,
+                   "frac_of_probe": (tc_ops / (tc_ms * 1e-3) / 1e12) / probe_tops if tc_ms > 0 and probe_tops > 0 else None},
+        "other_kernels": {"ms_per_step": other_ms, "gbs": other_bytes / (other_ms * 1e-3) / 1e9 if other_ms > 0 else None},
+        "whole_step": {"tops": total_ops / (ms_per_step * 1e-3) / 1e12,
+                       "gbs": synth.net_bytes(layers, BATCH) / (ms_per_step * 1e-3) / 1e9},
+    }
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int8", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "net": NET, "global_batch": BATCH * world, "batch_per_gpu": BATCH,
+                       "image": "224x224x3 int8 FL=6", "parallelism": f"replicas x{world}",
+                       "l2": "no flush: one step moves %.1f GB of activations, far beyond the 126 MB L2" %
+                             (synth.net_bytes(layers, BATCH) / 1e9)},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel()),
+                    "d2h_bytes_per_step": int(out_host.numel() * 4), "ms_per_step": e2e_ms / args.steps},
+            "gpu_launches": int(launches),
+            "roofline": roofline}
+    if world == 1:
+        line["cpu_baseline"] = cpu_baseline(layers)
+    if args.layers:
+        line["layers"] = per_layer
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", action="store_true", help="add per-layer times to the JSON line")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+    try:
+        import torch.distributed as dist
+        if dist.is_available() and dist.is_initialized():
+            dist.destroy_process_group()
+    except Exception:
+        pass
+
+
+if __name__ == "__main__":
+    main()

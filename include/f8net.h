@@ -1,0 +1,198 @@
+/*
+ * f8net.h -- C ABI of the fixed-point 8-bit inference library for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates the inference arithmetic of F8Net ("Fixed-Point 8-bit Only
+ * Multiplication for Network Quantization"): every tensor element is an 8-bit
+ * integer code q with a per-tensor fractional length FL and stands for q * 2^-FL
+ * (word length 8 everywhere, Sec. 4.3).  A layer multiplies 8-bit activations by
+ * 8-bit effective weights, accumulates in int32, adds the effective bias (Eq. 6),
+ * optionally adds a shortcut tensor after aligning its format by a bit shift
+ * (Sec. 4.3 "Clipping-Level Sharing", Fig. 4), and applies the fixed-point
+ * quantizer of the consumer, Eq. 2 (unsigned, clip [0, 255]; this is also the
+ * ReLU / PACT clip, Eq. 4) or its signed form from the appendix (clip
+ * [-127, 127]).  Because all formats are powers of two, the quantizer is a
+ * rounding arithmetic shift by  s = FL_x + FL_w - FL_y  followed by the clip;
+ * no int32 or floating-point multiplication is used for rescaling.
+ *
+ * For one output element, with FA = FL_x + FL_w:
+ *
+ *     acc = sum_taps x * w + bias                         exact, int32
+ *     if residual:  F = max(FA, FL_r)
+ *                   acc = (acc << (F - FA)) + (r << (F - FL_r)),  FA = F
+ *     s   = FA - FL_y
+ *     t   = s > 0 ? floor((acc + 2^(s-1)) / 2^s) : acc * 2^(-s)    (round half up)
+ *     y   = min(hi, max(lo, t))
+ *
+ * Conventions for every entry point
+ *   - Pointers named x, w, bias, residual, y, workspace are DEVICE pointers unless
+ *     the name starts with host_.  Tensors are dense, NHWC (channel fastest),
+ *     16-byte aligned.  The caller owns every buffer; the library allocates no
+ *     output and keeps no pointer after the call returns (f8_net objects own a
+ *     device copy of their parameters, see f8_net_create).
+ *   - cuda_stream is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls validate their arguments on the host, enqueue work on the stream and
+ *     return without synchronising.
+ *   - Errors are reported by the return code; nothing is launched when validation
+ *     fails.  f8_last_error() gives a message for the calling thread's last
+ *     failure.  Kernels never trap: a wait that does not complete within its
+ *     bound makes the kernel return early and sets a device status word that
+ *     f8_device_status() reads.
+ *   - Preconditions the library cannot check on device data: every accumulator
+ *     (including the aligned residual sum) fits in int32.  f8_net_create checks
+ *     this bound from the host copies of the parameters.
+ */
+#ifndef F8NET_H
+#define F8NET_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    F8_OK = 0,
+    F8_ERR_NULL = 1,          /* a required pointer is NULL */
+    F8_ERR_SHAPE = 2,         /* non-positive or inconsistent extents */
+    F8_ERR_DTYPE = 3,         /* dtype code not valid in this position */
+    F8_ERR_FL_RANGE = 4,      /* fractional length outside the accepted range */
+    F8_ERR_SHIFT_RANGE = 5,   /* a shift amount outside [-8, 31] (requantisation) or [0, 22] (alignment) */
+    F8_ERR_ALIGN = 6,         /* a pointer is not 16-byte aligned */
+    F8_ERR_ACC_BOUND = 7,     /* the int32 accumulator bound cannot be guaranteed */
+    F8_ERR_WORKSPACE = 8,     /* workspace missing or too small */
+    F8_ERR_UNSUPPORTED = 9,   /* valid request the library does not implement */
+    F8_ERR_CUDA = 10,         /* a CUDA runtime / driver call failed */
+    F8_ERR_TIMEOUT = 11       /* a kernel gave up on a bounded wait (see f8_device_status) */
+} f8_status;
+
+typedef enum { F8_U8 = 0, F8_S8 = 1, F8_S32 = 2 } f8_dtype;
+
+/*
+ * One convolution-shaped layer (Eq. 6).  Input x is [n, h, w, c]; the output is
+ * [n, ho, wo, c_out] with ho = (h + 2 pad - kh) / stride + 1 (same for wo);
+ * dilation 1; cross-correlation; taps outside the image contribute 0.
+ *   x_dtype  F8_U8 or F8_S8, format fl_x (0..8 unsigned, 0..7 signed; Eq. 2 and its signed form)
+ *   weights  int8 in [-128, 127], format fl_w (-8..24: the arithmetic only sees the shift)
+ *   y_dtype  F8_U8: quantizer of Eq. 2, clip [0, 255] (this is ReLU + PACT clip);
+ *            F8_S8: signed quantizer, clip [-127, 127];
+ *            F8_S32: raw accumulator in format fl_x + fl_w (fl_y ignored)
+ *   r_dtype / fl_r describe the residual tensor and are read only when the
+ *            residual pointer of the call is not NULL.
+ */
+typedef struct {
+    int n, h, w, c;
+    int c_out, kh, kw, stride, pad;
+    int x_dtype, y_dtype, r_dtype;
+    int fl_x, fl_w, fl_y, fl_r;
+} f8_conv_desc;
+
+/* Dense convolution (Eq. 6; residual add of Sec. 4.3; quantizer Eq. 2 / signed form).
+ *   w_ohwi [c_out, kh, kw, c] int8; bias [c_out] int32 in format fl_x + fl_w or NULL (zero);
+ *   residual NULL or [n, ho, wo, c_out] 8-bit (r_dtype, fl_r); y [n, ho, wo, c_out].
+ * Layers with c % 16 == 0 whose input is at least 128 KiB run on the tensor cores
+ * (tcgen05.mma kind::i8); every other shape takes a CUDA-core kernel with the same
+ * result.  workspace: f8_conv_workspace_bytes(desc) bytes (may be 0 -> NULL allowed). */
+f8_status f8_conv2d_fixed(const f8_conv_desc *desc, const void *x, const int8_t *w_ohwi, const int32_t *bias,
+                          const void *residual, void *y, void *workspace, size_t workspace_bytes,
+                          void *cuda_stream);
+
+/* Depthwise convolution (one kh x kw filter per channel; MobileNet layers of Sec. 5),
+ * c_out must equal c.  w_chw [c, kh, kw] int8.  Everything else as f8_conv2d_fixed. */
+f8_status f8_dwconv_fixed(const f8_conv_desc *desc, const void *x, const int8_t *w_chw, const int32_t *bias,
+                          const void *residual, void *y, void *workspace, size_t workspace_bytes,
+                          void *cuda_stream);
+
+/* Fully connected layer: Eq. 6 with the sum over k inputs.  x [n, k] 8-bit, w_out_k [out, k] int8,
+ * bias [out] int32 (format fl_x + fl_w) or NULL, y [n, out] of y_dtype (F8_S32 = logits in
+ * format fl_x + fl_w, the values "stored in 32-bit" of Sec. 4.3). */
+f8_status f8_linear_fixed(int n, int k, int out, int x_dtype, int y_dtype, int fl_x, int fl_w, int fl_y,
+                          const void *x, const int8_t *w_out_k, const int32_t *bias, void *y,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Max pooling k x k / stride with padding (not in the paper: integer max over the taps inside
+ * the image; codes and format unchanged).  x, y 8-bit NHWC of dtype x_dtype. */
+f8_status f8_maxpool_fixed(int n, int h, int w, int c, int k, int stride, int pad, int x_dtype,
+                           const void *x, void *y, void *cuda_stream);
+
+/* Global average pooling (not in the paper): sum over h*w followed by the quantizer of Eq. 2
+ * (or its signed form) with shift ceil(log2(h*w)) + fl_x - fl_y; y [n, c] of dtype x_dtype. */
+f8_status f8_global_avgpool_fixed(int n, int h, int w, int c, int x_dtype, int fl_x, int fl_y,
+                                  const void *x, void *y, void *cuda_stream);
+
+size_t f8_conv_workspace_bytes(const f8_conv_desc *desc);
+
+/* ---------------------------------------------------------------- whole networks */
+
+typedef enum { F8_LAYER_CONV = 0, F8_LAYER_DWCONV = 1, F8_LAYER_MAXPOOL = 2, F8_LAYER_GAP = 3,
+               F8_LAYER_LINEAR = 4 } f8_layer_kind;
+
+/* Tensor 0 is the network input; layer i writes tensor i + 1.  src / res name tensors
+ * (res = -1: no residual).  conv.n is ignored (the batch is given per call); for
+ * F8_LAYER_LINEAR conv.c = inputs and conv.c_out = outputs; for pooling layers only the
+ * geometry, x_dtype and fl_x / fl_y are read. */
+typedef struct {
+    int kind;
+    int src;
+    int res;
+    f8_conv_desc conv;
+} f8_layer_desc;
+
+typedef struct f8_net f8_net;
+
+/* Builds a network object from HOST copies of the parameters (host_weights[i] / host_bias[i]
+ * may be NULL for layers without parameters).  Validates every layer, checks the int32
+ * accumulator bound of each output channel from the actual weights (F8_ERR_ACC_BOUND),
+ * copies (and where needed re-packs) the parameters to the current device.  The last
+ * layer's output is the network output.  Must be called with the target device current. */
+f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t *const *host_weights,
+                        const int32_t *const *host_bias, int max_batch, f8_net **out);
+
+/* Bytes of device workspace f8_net_forward needs for this batch (all intermediate tensors). */
+size_t f8_net_workspace_bytes(const f8_net *net, int batch);
+
+/* One forward pass (the fixed-point inference path end to end).  x: [batch, h, w, c] network
+ * input; y: the last layer's output ([batch, out] int32 logits for a net ending in a linear
+ * layer).  layer_dump: NULL, or an array of n_layers device pointers; a non-NULL entry i
+ * receives a copy of layer i's output (for parity checks). */
+f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *workspace,
+                         size_t workspace_bytes, void *const *layer_dump, void *cuda_stream);
+
+/* Number of kernels the last f8_net_forward on this object enqueued. */
+int f8_net_last_launch_count(const f8_net *net);
+
+/* Per-layer timing.  With profiling on, f8_net_forward records a CUDA event after every kernel it
+ * enqueues; f8_net_get_layer_ms waits for the last profiled pass and writes the device time of
+ * each layer (ms[n_layers]; a stem's packing pre-pass is added to its layer) and, if
+ * on_tensor_cores is not NULL, 1 for layers that ran on the tcgen05 path. */
+f8_status f8_net_set_profiling(f8_net *net, int on);
+f8_status f8_net_get_layer_ms(f8_net *net, float *ms, int *on_tensor_cores);
+
+void f8_net_destroy(f8_net *net);
+
+/* ---------------------------------------------------------------- diagnostics */
+
+const char *f8_status_str(f8_status s);
+const char *f8_last_error(void);
+
+/* Synchronises the device and returns F8_ERR_TIMEOUT if any kernel since the last call
+ * abandoned a bounded wait (the word is cleared), F8_ERR_CUDA on a CUDA error, else F8_OK. */
+f8_status f8_device_status(void);
+
+/* Number of tensor-core (tcgen05) convolution kernels this process has launched so far; lets a
+ * caller confirm which path a layer took. */
+long long f8_tc_launch_count(void);
+
+/* Test hook: non-zero routes every dense layer to the CUDA-core kernel (same results). */
+void f8_debug_force_direct(int on);
+
+/* Tensor-core probe: every SM issues `iters` back-to-back tcgen05.mma kind::i8
+ * 128 x 256 x 32 instructions on resident shared-memory tiles (no global traffic).
+ * Returns the number of int8 operations (2 per multiply-accumulate) issued in *ops so that
+ * the caller can time the launch and obtain the attainable INT8 rate of the device. */
+f8_status f8_mma_i8_probe(int iters, double *ops, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* F8NET_H */

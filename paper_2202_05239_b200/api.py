@@ -1,0 +1,278 @@
+"""Thin Python binding over the C-ABI CUDA library (``libf8net.so``).
+
+Only argument marshalling happens here: every function forwards device pointers
+of torch tensors (torch supplies memory and streams) to the entry point of the
+same name in ``include/f8net.h``.  There is no CPU fallback: importing this
+module fails if the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import synth
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libf8net.so")
+
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build the CUDA library first "
+        "(python -m paper_2202_05239_b200.build, or __graft_entry__.build())")
+
+_lib = ctypes.CDLL(_LIB_PATH)
+
+F8_OK = 0
+F8_U8, F8_S8, F8_S32 = 0, 1, 2
+STATUS_NAMES = ["F8_OK", "F8_ERR_NULL", "F8_ERR_SHAPE", "F8_ERR_DTYPE", "F8_ERR_FL_RANGE", "F8_ERR_SHIFT_RANGE",
+                "F8_ERR_ALIGN", "F8_ERR_ACC_BOUND", "F8_ERR_WORKSPACE", "F8_ERR_UNSUPPORTED", "F8_ERR_CUDA",
+                "F8_ERR_TIMEOUT"]
+
+
+class ConvDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("n", "h", "w", "c", "c_out", "kh", "kw", "stride", "pad", "x_dtype", "y_dtype", "r_dtype",
+                 "fl_x", "fl_w", "fl_y", "fl_r")]
+
+
+class LayerDesc(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int), ("src", ctypes.c_int), ("res", ctypes.c_int), ("conv", ConvDesc)]
+
+
+class F8Error(RuntimeError):
+    def __init__(self, status: int, message: str):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{name}: {message}")
+
+
+_vp, _ci, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+_lib.f8_conv2d_fixed.argtypes = [ctypes.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.f8_dwconv_fixed.argtypes = _lib.f8_conv2d_fixed.argtypes
+_lib.f8_linear_fixed.argtypes = [_ci] * 8 + [_vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.f8_maxpool_fixed.argtypes = [_ci] * 8 + [_vp, _vp, _vp]
+_lib.f8_global_avgpool_fixed.argtypes = [_ci] * 7 + [_vp, _vp, _vp]
+_lib.f8_conv_workspace_bytes.argtypes = [ctypes.POINTER(ConvDesc)]
+_lib.f8_conv_workspace_bytes.restype = _sz
+_lib.f8_net_create.argtypes = [ctypes.POINTER(LayerDesc), _ci, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _ci,
+                               ctypes.POINTER(_vp)]
+_lib.f8_net_workspace_bytes.argtypes = [_vp, _ci]
+_lib.f8_net_workspace_bytes.restype = _sz
+_lib.f8_net_forward.argtypes = [_vp, _ci, _vp, _vp, _vp, _sz, ctypes.POINTER(_vp), _vp]
+_lib.f8_net_last_launch_count.argtypes = [_vp]
+_lib.f8_net_set_profiling.argtypes = [_vp, _ci]
+_lib.f8_net_get_layer_ms.argtypes = [_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int)]
+_lib.f8_net_destroy.argtypes = [_vp]
+_lib.f8_net_destroy.restype = None
+_lib.f8_status_str.argtypes = [_ci]
+_lib.f8_status_str.restype = ctypes.c_char_p
+_lib.f8_last_error.restype = ctypes.c_char_p
+_lib.f8_mma_i8_probe.argtypes = [_ci, ctypes.POINTER(ctypes.c_double), _vp]
+_lib.f8_debug_force_direct.argtypes = [_ci]
+_lib.f8_debug_force_direct.restype = None
+
+
+def _check(status: int):
+    if status != F8_OK:
+        raise F8Error(status, _lib.f8_last_error().decode())
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("tensors must be contiguous CUDA tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def conv_desc(layer: "synth.Layer", n: int) -> ConvDesc:
+    return ConvDesc(n, layer.h, layer.w, layer.c, layer.c_out, layer.kh, layer.kw, layer.stride, layer.pad,
+                    layer.x_dtype, layer.y_dtype, layer.r_dtype, layer.fl_x, layer.fl_w, layer.fl_y, layer.fl_r)
+
+
+_TORCH_DTYPE = {F8_U8: torch.uint8, F8_S8: torch.int8, F8_S32: torch.int32}
+
+
+def torch_dtype(code: int) -> torch.dtype:
+    return _TORCH_DTYPE[code]
+
+
+def to_device(a: Optional[np.ndarray], device="cuda") -> Optional[torch.Tensor]:
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+# ------------------------------------------------------------------ entry points (same names as the C ABI)
+
+def f8_conv2d_fixed(desc: ConvDesc, x, w, bias, residual, y, workspace=None, stream=None):
+    _check(_lib.f8_conv2d_fixed(ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y),
+                                _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def f8_dwconv_fixed(desc: ConvDesc, x, w, bias, residual, y, workspace=None, stream=None):
+    _check(_lib.f8_dwconv_fixed(ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y),
+                                _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def f8_linear_fixed(n, k, out, x_dtype, y_dtype, fl_x, fl_w, fl_y, x, w, bias, y, workspace=None, stream=None):
+    _check(_lib.f8_linear_fixed(n, k, out, x_dtype, y_dtype, fl_x, fl_w, fl_y, _ptr(x), _ptr(w), _ptr(bias), _ptr(y),
+                                _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def f8_maxpool_fixed(n, h, w, c, k, stride, pad, x_dtype, x, y, stream=None):
+    _check(_lib.f8_maxpool_fixed(n, h, w, c, k, stride, pad, x_dtype, _ptr(x), _ptr(y), _stream(stream)))
+
+
+def f8_global_avgpool_fixed(n, h, w, c, x_dtype, fl_x, fl_y, x, y, stream=None):
+    _check(_lib.f8_global_avgpool_fixed(n, h, w, c, x_dtype, fl_x, fl_y, _ptr(x), _ptr(y), _stream(stream)))
+
+
+def f8_conv_workspace_bytes(desc: ConvDesc) -> int:
+    return int(_lib.f8_conv_workspace_bytes(ctypes.byref(desc)))
+
+
+def f8_device_status():
+    _check(_lib.f8_device_status())
+
+
+def f8_mma_i8_probe(iters: int, stream=None) -> float:
+    ops = ctypes.c_double(0.0)
+    _check(_lib.f8_mma_i8_probe(iters, ctypes.byref(ops), _stream(stream)))
+    return ops.value
+
+
+_lib.f8_tc_launch_count.restype = ctypes.c_longlong
+
+
+def f8_tc_launch_count() -> int:
+    return int(_lib.f8_tc_launch_count())
+
+
+def f8_debug_force_direct(on: bool):
+    _lib.f8_debug_force_direct(1 if on else 0)
+
+
+def exported_symbols() -> List[str]:
+    return ["f8_conv2d_fixed", "f8_dwconv_fixed", "f8_linear_fixed", "f8_maxpool_fixed", "f8_global_avgpool_fixed",
+            "f8_conv_workspace_bytes", "f8_net_create", "f8_net_workspace_bytes", "f8_net_forward",
+            "f8_net_last_launch_count", "f8_net_set_profiling", "f8_net_get_layer_ms", "f8_net_destroy", "f8_status_str", "f8_last_error", "f8_device_status",
+            "f8_mma_i8_probe"]
+
+
+def run_layer(layer: "synth.Layer", x: torch.Tensor, residual: Optional[torch.Tensor] = None, params=None,
+              stream=None) -> torch.Tensor:
+    """One generated layer through the single-layer entry points; returns a new output tensor."""
+    n = x.shape[0]
+    w, b = params if params is not None else (to_device(layer.weight), to_device(layer.bias))
+    if layer.kind in (synth.CONV, synth.DWCONV):
+        y = torch.empty((n, layer.ho, layer.wo, layer.c_out), dtype=torch_dtype(layer.y_dtype), device=x.device)
+        fn = f8_conv2d_fixed if layer.kind == synth.CONV else f8_dwconv_fixed
+        fn(conv_desc(layer, n), x, w, b, residual, y, stream=stream)
+    elif layer.kind == synth.LINEAR:
+        y = torch.empty((n, layer.c_out), dtype=torch_dtype(layer.y_dtype), device=x.device)
+        f8_linear_fixed(n, layer.c, layer.c_out, layer.x_dtype, layer.y_dtype, layer.fl_x, layer.fl_w, layer.fl_y,
+                        x, w, b, y, stream=stream)
+    elif layer.kind == synth.MAXPOOL:
+        y = torch.empty((n, layer.ho, layer.wo, layer.c), dtype=x.dtype, device=x.device)
+        f8_maxpool_fixed(n, layer.h, layer.w, layer.c, layer.kh, layer.stride, layer.pad, layer.x_dtype, x, y,
+                         stream=stream)
+    elif layer.kind == synth.GAP:
+        y = torch.empty((n, layer.c), dtype=x.dtype, device=x.device)
+        f8_global_avgpool_fixed(n, layer.h, layer.w, layer.c, layer.x_dtype, layer.fl_x, layer.fl_y, x, y,
+                                stream=stream)
+    else:
+        raise ValueError(layer.kind)
+    return y
+
+
+class Net:
+    """Owner of an ``f8_net`` object built from generated layer descriptions."""
+
+    def __init__(self, layers: Sequence["synth.Layer"], max_batch: int):
+        self.layers = list(layers)
+        self.max_batch = max_batch
+        n = len(self.layers)
+        descs = (LayerDesc * n)()
+        wptrs = (_vp * n)()
+        bptrs = (_vp * n)()
+        self._keep = []
+        for i, l in enumerate(self.layers):
+            descs[i] = LayerDesc(l.kind, l.src, l.res, conv_desc(l, 1))
+            if l.weight is not None:
+                w = np.ascontiguousarray(l.weight, dtype=np.int8)
+                self._keep.append(w)
+                wptrs[i] = w.ctypes.data
+            if l.bias is not None:
+                b = np.ascontiguousarray(l.bias, dtype=np.int32)
+                self._keep.append(b)
+                bptrs[i] = b.ctypes.data
+        handle = _vp()
+        _check(_lib.f8_net_create(descs, n, wptrs, bptrs, max_batch, ctypes.byref(handle)))
+        self._h = handle
+        self._ws = None
+        last = self.layers[-1]
+        self.out_shape = (last.c_out,) if last.kind in (synth.LINEAR, synth.GAP) else (last.ho, last.wo, last.c_out)
+        self.out_dtype = torch_dtype(last.y_dtype)
+
+    def workspace_bytes(self, batch: int) -> int:
+        return int(_lib.f8_net_workspace_bytes(self._h, batch))
+
+    def layer_output(self, i: int, batch: int, device="cuda") -> torch.Tensor:
+        l = self.layers[i]
+        shape = (batch, l.c_out) if l.kind in (synth.LINEAR, synth.GAP) else (batch, l.ho, l.wo, l.c_out)
+        return torch.empty(shape, dtype=torch_dtype(l.y_dtype), device=device)
+
+    def forward(self, x: torch.Tensor, out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                dump: Optional[Sequence[Optional[torch.Tensor]]] = None, stream=None) -> torch.Tensor:
+        """f8_net_forward: ``x`` [batch,h,w,c] device tensor -> ``out`` (allocated if not given)."""
+        batch = x.shape[0]
+        if out is None:
+            out = torch.empty((batch,) + self.out_shape, dtype=self.out_dtype, device=x.device)
+        need = self.workspace_bytes(batch)
+        if workspace is None:
+            if self._ws is None or self._ws.numel() < need or self._ws.device != x.device:
+                self._ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+            workspace = self._ws
+        dptr = None
+        if dump is not None:
+            dptr = (_vp * len(self.layers))()
+            for i, t in enumerate(dump):
+                if t is not None:
+                    dptr[i] = t.data_ptr()
+        _check(_lib.f8_net_forward(self._h, batch, _ptr(x), _ptr(out), _ptr(workspace), workspace.numel(), dptr,
+                                   _stream(stream)))
+        return out
+
+    def set_profiling(self, on: bool):
+        _check(_lib.f8_net_set_profiling(self._h, 1 if on else 0))
+
+    def layer_ms(self):
+        """(ms per layer, ran-on-tensor-cores flag per layer) of the last profiled forward pass."""
+        n = len(self.layers)
+        ms = (ctypes.c_float * n)()
+        tc = (ctypes.c_int * n)()
+        _check(_lib.f8_net_get_layer_ms(self._h, ms, tc))
+        return list(ms), [bool(v) for v in tc]
+
+    @property
+    def last_launch_count(self) -> int:
+        return int(_lib.f8_net_last_launch_count(self._h))
+
+    def close(self):
+        if self._h:
+            _lib.f8_net_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,701 @@
+// C ABI: argument validation, dispatch to the kernels, and the whole-network executor.
+#include <cuda_runtime.h>
+
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <memory>
+#include <new>
+#include <vector>
+
+#include "f8_internal.h"
+
+namespace {
+
+thread_local char g_err[512] = "";
+bool g_force_direct = false;
+long long g_tc_launches = 0;
+
+f8_status fail(f8_status s, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+f8_status cuda_fail(cudaError_t e, const char *what) {
+    return fail(F8_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
+
+int ceil_log2(long long v) {
+    int d = 0;
+    while ((1ll << d) < v) ++d;
+    return d;
+}
+
+// Validates one conv-shaped descriptor and derives geometry + requantisation parameters.
+f8_status check_conv(const f8_conv_desc *d, bool depthwise, bool has_res, F8ConvGeom *g, F8Requant *q) {
+    if (!d) return fail(F8_ERR_NULL, "descriptor is NULL");
+    if (d->n < 0 || d->h <= 0 || d->w <= 0 || d->c <= 0 || d->c_out <= 0 || d->kh <= 0 || d->kw <= 0 ||
+        d->stride <= 0 || d->pad < 0)
+        return fail(F8_ERR_SHAPE, "non-positive extent in descriptor");
+    if (depthwise && d->c_out != d->c) return fail(F8_ERR_SHAPE, "depthwise layers need c_out == c");
+    const int ho = (d->h + 2 * d->pad - d->kh) / d->stride + 1;
+    const int wo = (d->w + 2 * d->pad - d->kw) / d->stride + 1;
+    if (d->h + 2 * d->pad < d->kh || d->w + 2 * d->pad < d->kw || ho <= 0 || wo <= 0)
+        return fail(F8_ERR_SHAPE, "filter larger than the padded image");
+    if ((long long)d->n * ho * wo * d->c_out >= (1ll << 40) || (long long)d->n * d->h * d->w * d->c >= (1ll << 40))
+        return fail(F8_ERR_SHAPE, "tensor too large");
+    if (d->x_dtype != F8_U8 && d->x_dtype != F8_S8) return fail(F8_ERR_DTYPE, "x_dtype must be F8_U8 or F8_S8");
+    if (d->y_dtype != F8_U8 && d->y_dtype != F8_S8 && d->y_dtype != F8_S32)
+        return fail(F8_ERR_DTYPE, "y_dtype must be F8_U8, F8_S8 or F8_S32");
+    if (d->fl_x < 0 || d->fl_x > (d->x_dtype == F8_U8 ? 8 : 7))
+        return fail(F8_ERR_FL_RANGE, "fl_x = %d outside the 8-bit format range", d->fl_x);
+    if (d->fl_w < -8 || d->fl_w > 24) return fail(F8_ERR_FL_RANGE, "fl_w = %d outside [-8, 24]", d->fl_w);
+    int fa = d->fl_x + d->fl_w;
+    q->sh_acc = q->sh_res = 0;
+    q->has_res = has_res ? 1 : 0;
+    q->r_signed = 0;
+    if (has_res) {
+        if (d->r_dtype != F8_U8 && d->r_dtype != F8_S8) return fail(F8_ERR_DTYPE, "r_dtype must be F8_U8 or F8_S8");
+        if (d->fl_r < 0 || d->fl_r > (d->r_dtype == F8_U8 ? 8 : 7))
+            return fail(F8_ERR_FL_RANGE, "fl_r = %d outside the 8-bit format range", d->fl_r);
+        const int f = std::max(fa, d->fl_r);
+        q->sh_acc = f - fa;
+        q->sh_res = f - d->fl_r;
+        q->r_signed = d->r_dtype == F8_S8;
+        if (q->sh_acc > 22 || q->sh_res > 22)
+            return fail(F8_ERR_SHIFT_RANGE, "residual alignment shift %d / %d exceeds 22", q->sh_acc, q->sh_res);
+        fa = f;
+    }
+    q->y_kind = d->y_dtype;
+    if (d->y_dtype == F8_S32) {
+        q->s = 0;
+        q->lo = q->hi = 0;
+    } else {
+        if (d->fl_y < 0 || d->fl_y > (d->y_dtype == F8_U8 ? 8 : 7))
+            return fail(F8_ERR_FL_RANGE, "fl_y = %d outside the 8-bit format range", d->fl_y);
+        q->s = fa - d->fl_y;
+        if (q->s < -8 || q->s > 31) return fail(F8_ERR_SHIFT_RANGE, "requantisation shift %d outside [-8, 31]", q->s);
+        q->lo = d->y_dtype == F8_U8 ? 0 : -127;
+        q->hi = d->y_dtype == F8_U8 ? 255 : 127;
+    }
+    // shape-level accumulator bound: |sum| <= K * 255 * 128 (or 128 * 128) must leave room for bias / residual
+    const long long k = (long long)d->kh * d->kw * (depthwise ? 1 : d->c);
+    const long long worst = k * (d->x_dtype == F8_U8 ? 255ll : 128ll) * 128ll;
+    if ((worst << q->sh_acc) >= (1ll << 30))
+        return fail(F8_ERR_ACC_BOUND, "K = %lld taps cannot be guaranteed to fit the int32 accumulator", k);
+    g->n = d->n; g->h = d->h; g->w = d->w; g->c = d->c;
+    g->ho = ho; g->wo = wo; g->c_out = d->c_out;
+    g->kh = d->kh; g->kw = d->kw;
+    g->stride_h = g->stride_w = d->stride;
+    g->pad_h = g->pad_w = d->pad;
+    g->x_signed = d->x_dtype == F8_S8;
+    return F8_OK;
+}
+
+F8TcTensorView dense_view(const void *x, const F8ConvGeom &g) {
+    F8TcTensorView v;
+    v.base = x;
+    v.dim_c = g.c; v.dim_w = g.w; v.dim_h = g.h; v.dim_n = g.n;
+    v.stride_w = (uint64_t)g.c;
+    v.stride_h = (uint64_t)g.c * g.w;
+    v.stride_n = (uint64_t)g.c * g.w * g.h;
+    return v;
+}
+
+struct PlanDeleter { void operator()(F8TcPlan *p) const { free(p); } };
+using PlanPtr = std::unique_ptr<F8TcPlan, PlanDeleter>;
+
+// tensor maps inside the plan are 64-byte aligned objects
+PlanPtr alloc_plan() {
+    const size_t size = (f8_tc_plan_size() + 63) / 64 * 64;
+    void *p = aligned_alloc(64, size);
+    if (p) memset(p, 0, size);
+    return PlanPtr((F8TcPlan *)p);
+}
+
+f8_status run_dense(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w, const int32_t *bias,
+                    const void *res, void *y, cudaStream_t st) {
+    if (g.n == 0) return F8_OK;
+    const size_t x_bytes = (size_t)g.n * g.h * g.w * g.c;
+    if (!g_force_direct && f8_tc_supported(g, x_bytes)) {
+        PlanPtr plan = alloc_plan();
+        if (!plan) return fail(F8_ERR_CUDA, "out of host memory");
+        const char *why = "";
+        cudaError_t e = f8_tc_plan_init(plan.get(), g, q, dense_view(x, g), w, bias, res, y, f8_status_word(), &why);
+        if (e == cudaSuccess) {
+            e = f8_tc_launch(plan.get(), st);
+            if (e != cudaSuccess) return cuda_fail(e, "tensor-core conv launch");
+            ++g_tc_launches;
+            return F8_OK;
+        }
+        if (e != cudaErrorInvalidValue && e != cudaErrorNotSupported) return cuda_fail(e, why);
+        // the tensor map could not be encoded for this shape: take the CUDA-core kernel
+    }
+    cudaError_t e = f8_launch_conv_direct(g, q, x, w, bias, res, y, st);
+    if (e != cudaSuccess) return cuda_fail(e, "direct conv launch");
+    return F8_OK;
+}
+
+}   // namespace
+
+int *f8_status_word() {
+    static int *words[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!words[dev]) {
+        int *p = nullptr;
+        if (cudaMalloc(&p, 256) != cudaSuccess) return nullptr;
+        cudaMemset(p, 0, 256);
+        words[dev] = p;
+    }
+    return words[dev];
+}
+
+extern "C" {
+
+const char *f8_status_str(f8_status s) {
+    switch (s) {
+        case F8_OK: return "F8_OK";
+        case F8_ERR_NULL: return "F8_ERR_NULL";
+        case F8_ERR_SHAPE: return "F8_ERR_SHAPE";
+        case F8_ERR_DTYPE: return "F8_ERR_DTYPE";
+        case F8_ERR_FL_RANGE: return "F8_ERR_FL_RANGE";
+        case F8_ERR_SHIFT_RANGE: return "F8_ERR_SHIFT_RANGE";
+        case F8_ERR_ALIGN: return "F8_ERR_ALIGN";
+        case F8_ERR_ACC_BOUND: return "F8_ERR_ACC_BOUND";
+        case F8_ERR_WORKSPACE: return "F8_ERR_WORKSPACE";
+        case F8_ERR_UNSUPPORTED: return "F8_ERR_UNSUPPORTED";
+        case F8_ERR_CUDA: return "F8_ERR_CUDA";
+        case F8_ERR_TIMEOUT: return "F8_ERR_TIMEOUT";
+    }
+    return "F8_ERR_?";
+}
+
+const char *f8_last_error(void) { return g_err; }
+
+long long f8_tc_launch_count(void) { return g_tc_launches; }
+
+// Test hook: non-zero routes every dense layer to the CUDA-core kernel.
+void f8_debug_force_direct(int on) { g_force_direct = on != 0; }
+
+f8_status f8_device_status(void) {
+    int *w = f8_status_word();
+    if (!w) return fail(F8_ERR_CUDA, "no status word");
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+    int v = 0;
+    e = cudaMemcpy(&v, w, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "status read");
+    if (v != 0) {
+        cudaMemset(w, 0, sizeof(int));
+        return fail(F8_ERR_TIMEOUT, "a kernel abandoned a bounded wait (site %d)", v);
+    }
+    return F8_OK;
+}
+
+size_t f8_conv_workspace_bytes(const f8_conv_desc *) { return 0; }
+
+f8_status f8_conv2d_fixed(const f8_conv_desc *desc, const void *x, const int8_t *w, const int32_t *bias,
+                          const void *residual, void *y, void *, size_t, void *cuda_stream) {
+    F8ConvGeom g;
+    F8Requant q;
+    f8_status s = check_conv(desc, false, residual != nullptr, &g, &q);
+    if (s != F8_OK) return s;
+    if (g.n == 0) return F8_OK;
+    if (!x || !w || !y) return fail(F8_ERR_NULL, "x, w and y must not be NULL");
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(residual) || !aligned16(bias))
+        return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    return run_dense(g, q, x, w, bias, residual, y, (cudaStream_t)cuda_stream);
+}
+
+f8_status f8_dwconv_fixed(const f8_conv_desc *desc, const void *x, const int8_t *w, const int32_t *bias,
+                          const void *residual, void *y, void *, size_t, void *cuda_stream) {
+    F8ConvGeom g;
+    F8Requant q;
+    f8_status s = check_conv(desc, true, residual != nullptr, &g, &q);
+    if (s != F8_OK) return s;
+    if (g.n == 0) return F8_OK;
+    if (!x || !w || !y) return fail(F8_ERR_NULL, "x, w and y must not be NULL");
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(residual) || !aligned16(bias))
+        return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    cudaError_t e = f8_launch_dwconv(g, q, x, w, bias, residual, y, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "depthwise launch");
+    return F8_OK;
+}
+
+f8_status f8_linear_fixed(int n, int k, int out, int x_dtype, int y_dtype, int fl_x, int fl_w, int fl_y, const void *x,
+                          const int8_t *w, const int32_t *bias, void *y, void *, size_t, void *cuda_stream) {
+    f8_conv_desc d;
+    memset(&d, 0, sizeof(d));
+    d.n = n; d.h = 1; d.w = 1; d.c = k; d.c_out = out; d.kh = d.kw = 1; d.stride = 1; d.pad = 0;
+    d.x_dtype = x_dtype; d.y_dtype = y_dtype; d.fl_x = fl_x; d.fl_w = fl_w; d.fl_y = fl_y;
+    return f8_conv2d_fixed(&d, x, w, bias, nullptr, y, nullptr, 0, cuda_stream);
+}
+
+f8_status f8_maxpool_fixed(int n, int h, int w, int c, int k, int stride, int pad, int x_dtype, const void *x, void *y,
+                           void *cuda_stream) {
+    if (n < 0 || h <= 0 || w <= 0 || c <= 0 || k <= 0 || stride <= 0 || pad < 0 || pad >= k || h + 2 * pad < k ||
+        w + 2 * pad < k)
+        return fail(F8_ERR_SHAPE, "bad pooling geometry");
+    if (x_dtype != F8_U8 && x_dtype != F8_S8) return fail(F8_ERR_DTYPE, "x_dtype must be F8_U8 or F8_S8");
+    if (n == 0) return F8_OK;
+    if (!x || !y) return fail(F8_ERR_NULL, "x and y must not be NULL");
+    if (!aligned16(x) || !aligned16(y)) return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    cudaError_t e = f8_launch_maxpool(n, h, w, c, k, stride, pad, x_dtype == F8_S8, x, y, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "max-pool launch");
+    return F8_OK;
+}
+
+f8_status f8_global_avgpool_fixed(int n, int h, int w, int c, int x_dtype, int fl_x, int fl_y, const void *x, void *y,
+                                  void *cuda_stream) {
+    if (n < 0 || h <= 0 || w <= 0 || c <= 0 || (long long)h * w > (1 << 22)) return fail(F8_ERR_SHAPE, "bad pooling geometry");
+    if (x_dtype != F8_U8 && x_dtype != F8_S8) return fail(F8_ERR_DTYPE, "x_dtype must be F8_U8 or F8_S8");
+    const int fmax = x_dtype == F8_U8 ? 8 : 7;
+    if (fl_x < 0 || fl_x > fmax || fl_y < 0 || fl_y > fmax) return fail(F8_ERR_FL_RANGE, "fl outside the 8-bit format range");
+    const int s = ceil_log2((long long)h * w) + fl_x - fl_y;
+    if (s < -8 || s > 31) return fail(F8_ERR_SHIFT_RANGE, "shift %d outside [-8, 31]", s);
+    if (n == 0) return F8_OK;
+    if (!x || !y) return fail(F8_ERR_NULL, "x and y must not be NULL");
+    if (!aligned16(x) || !aligned16(y)) return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    cudaError_t e = f8_launch_gap(n, h, w, c, x_dtype == F8_S8, s, x, y, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "global-average-pool launch");
+    return F8_OK;
+}
+
+f8_status f8_mma_i8_probe(int iters, double *ops, void *cuda_stream) {
+    if (!ops) return fail(F8_ERR_NULL, "ops is NULL");
+    if (iters <= 0 || iters > (1 << 24)) return fail(F8_ERR_SHAPE, "iters out of range");
+    cudaError_t e = f8_tc_probe(iters, ops, f8_status_word(), (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "probe launch");
+    return F8_OK;
+}
+
+}   // extern "C"
+
+// ===========================================================================================
+// Whole-network executor
+// ===========================================================================================
+
+namespace {
+
+struct NetLayer {
+    f8_layer_desc d;
+    F8ConvGeom g;            // per-image geometry (n filled per call)
+    F8Requant q;
+    int8_t *w = nullptr;     // device parameters (owned)
+    int32_t *b = nullptr;
+    // stem packing (3-channel inputs on the tensor-core path)
+    bool packed = false;
+    int pack_wp = 0, pack_left = 0, pack_kw8 = 0;
+    int8_t *w_packed = nullptr;
+    size_t out_bytes_per_image = 0;
+};
+
+struct Step {
+    int kind = 0;             // layer kind, or -1 for the stem packing pre-pass
+    int layer = -1;
+    const void *x = nullptr;
+    const void *res = nullptr;
+    void *y = nullptr;
+    bool use_tc = false;
+    PlanPtr plan;
+    F8ConvGeom g;
+};
+
+}   // namespace
+
+struct f8_net {
+    std::vector<NetLayer> layers;
+    std::vector<int> t_h, t_w, t_c, t_elem;     // per tensor: per-image shape and element size
+    int max_batch = 0;
+    // cached execution plan
+    int plan_batch = -1;
+    const void *plan_x = nullptr;
+    void *plan_y = nullptr, *plan_ws = nullptr;
+    bool plan_force_direct = false;
+    std::vector<Step> steps;
+    std::vector<size_t> t_off;                   // workspace offset per tensor
+    size_t pack_off = 0;
+    int last_launches = 0;
+    // optional per-layer timing
+    bool profiling = false;
+    std::vector<cudaEvent_t> events;             // steps + 1 events of the last profiled forward
+    std::vector<int> event_layer;                // layer each step belongs to
+};
+
+namespace {
+
+size_t round256(size_t v) { return (v + 255) / 256 * 256; }
+
+size_t tensor_bytes(const f8_net *net, int t, int batch) {
+    return (size_t)batch * net->t_h[t] * net->t_w[t] * net->t_c[t] * net->t_elem[t];
+}
+
+// Assigns workspace offsets: tensors whose lifetimes do not overlap may share memory (first fit).
+size_t assign_offsets(const f8_net *net, int batch, std::vector<size_t> *off, size_t *pack_off) {
+    const int nt = (int)net->layers.size() + 1;
+    std::vector<int> last(nt, -1);
+    for (int i = 0; i < (int)net->layers.size(); ++i) {
+        last[net->layers[i].d.src] = i;
+        if (net->layers[i].d.res >= 0) last[net->layers[i].d.res] = i;
+    }
+    struct Live { size_t off, size; int until; };
+    std::vector<Live> live;
+    off->assign(nt, 0);
+    size_t top = 0;
+    for (int t = 1; t < nt - 1; ++t) {          // tensor 0 = caller's x, tensor nt-1 = caller's y
+        const int born = t - 1;                 // written by layer t-1
+        const size_t size = round256(tensor_bytes(net, t, batch));
+        live.erase(std::remove_if(live.begin(), live.end(), [&](const Live &l) { return l.until < born; }), live.end());
+        std::sort(live.begin(), live.end(), [](const Live &a, const Live &b) { return a.off < b.off; });
+        size_t pos = 0;
+        for (const Live &l : live) {
+            if (pos + size <= l.off) break;
+            pos = std::max(pos, l.off + l.size);
+        }
+        (*off)[t] = pos;
+        live.push_back({pos, size, std::max(last[t], born)});
+        top = std::max(top, pos + size);
+    }
+    *pack_off = top;
+    size_t pack = 0;
+    for (const NetLayer &l : net->layers)
+        if (l.packed) pack = std::max(pack, round256((size_t)batch * l.g.h * l.pack_wp * 8));
+    return top + pack;
+}
+
+void free_layers(f8_net *net) {
+    for (NetLayer &l : net->layers) {
+        if (l.w) cudaFree(l.w);
+        if (l.b) cudaFree(l.b);
+        if (l.w_packed) cudaFree(l.w_packed);
+    }
+}
+
+}   // namespace
+
+extern "C" {
+
+f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t *const *host_weights,
+                        const int32_t *const *host_bias, int max_batch, f8_net **out) {
+    if (!layers || !out) return fail(F8_ERR_NULL, "layers / out is NULL");
+    if (n_layers <= 0 || max_batch <= 0) return fail(F8_ERR_SHAPE, "n_layers and max_batch must be positive");
+    std::unique_ptr<f8_net> net(new (std::nothrow) f8_net);
+    if (!net) return fail(F8_ERR_CUDA, "out of host memory");
+    net->max_batch = max_batch;
+    net->layers.resize(n_layers);
+    // tensor 0 shape comes from the first layer that reads it
+    net->t_h.assign(n_layers + 1, 0);
+    net->t_w.assign(n_layers + 1, 0);
+    net->t_c.assign(n_layers + 1, 0);
+    net->t_elem.assign(n_layers + 1, 1);
+    std::vector<int> t_dtype(n_layers + 1, -1), t_fl(n_layers + 1, 0);
+    auto cleanup = [&](f8_status s) { free_layers(net.get()); return s; };
+    for (int i = 0; i < n_layers; ++i) {
+        NetLayer &L = net->layers[i];
+        L.d = layers[i];
+        f8_conv_desc &d = L.d.conv;
+        d.n = 1;
+        if (L.d.src < 0 || L.d.src > i) return cleanup(fail(F8_ERR_SHAPE, "layer %d: src %d is not an earlier tensor", i, L.d.src));
+        if (L.d.res > i) return cleanup(fail(F8_ERR_SHAPE, "layer %d: res %d is not an earlier tensor", i, L.d.res));
+        const int kind = L.d.kind;
+        if (kind == F8_LAYER_LINEAR) { d.h = d.w = 1; d.kh = d.kw = 1; d.stride = 1; d.pad = 0; }
+        if (kind == F8_LAYER_GAP) { d.kh = d.kw = 1; d.stride = 1; d.pad = 0; d.c_out = d.c; d.y_dtype = d.x_dtype; d.fl_w = 0; }
+        if (kind == F8_LAYER_MAXPOOL) { d.c_out = d.c; d.y_dtype = d.x_dtype; d.fl_w = 0; d.fl_y = d.fl_x; }
+        const bool has_res = L.d.res >= 0 && (kind == F8_LAYER_CONV || kind == F8_LAYER_DWCONV);
+        f8_status s;
+        switch (kind) {
+            case F8_LAYER_CONV:
+            case F8_LAYER_LINEAR:
+                s = check_conv(&d, false, has_res, &L.g, &L.q);
+                break;
+            case F8_LAYER_DWCONV:
+                s = check_conv(&d, true, has_res, &L.g, &L.q);
+                break;
+            case F8_LAYER_MAXPOOL:
+                if (d.kh != d.kw || d.pad >= d.kh) return cleanup(fail(F8_ERR_SHAPE, "layer %d: bad pooling window", i));
+                s = check_conv(&d, true, false, &L.g, &L.q);
+                break;
+            case F8_LAYER_GAP: {
+                f8_conv_desc t = d;
+                t.kh = t.h; t.kw = t.w;
+                t.fl_w = ceil_log2((long long)d.h * d.w);    // the power-of-two "average" enters as a format shift
+                s = check_conv(&t, true, false, &L.g, &L.q);
+                L.g.kh = L.g.kw = 1;
+                break;
+            }
+            default:
+                return cleanup(fail(F8_ERR_UNSUPPORTED, "layer %d: unknown kind %d", i, kind));
+        }
+        if (s != F8_OK) {
+            char msg[400];
+            snprintf(msg, sizeof(msg), "layer %d: %s", i, g_err);
+            return cleanup(fail(s, "%s", msg));
+        }
+        // shapes / dtypes must chain
+        const int src = L.d.src;
+        if (src == 0 && net->t_h[0] == 0) {
+            net->t_h[0] = d.h; net->t_w[0] = d.w; net->t_c[0] = d.c;
+            t_dtype[0] = d.x_dtype; t_fl[0] = d.fl_x;
+        }
+        if (net->t_h[src] != d.h || net->t_w[src] != d.w || net->t_c[src] != d.c)
+            return cleanup(fail(F8_ERR_SHAPE, "layer %d: input shape does not match tensor %d", i, src));
+        if (t_dtype[src] != d.x_dtype || t_fl[src] != d.fl_x)
+            return cleanup(fail(F8_ERR_DTYPE, "layer %d: x_dtype / fl_x do not match the producer of tensor %d", i, src));
+        const int ho = kind == F8_LAYER_GAP ? 1 : L.g.ho, wo = kind == F8_LAYER_GAP ? 1 : L.g.wo;
+        if (has_res) {
+            const int r = L.d.res;
+            if (net->t_h[r] != ho || net->t_w[r] != wo || net->t_c[r] != d.c_out)
+                return cleanup(fail(F8_ERR_SHAPE, "layer %d: residual tensor %d has the wrong shape", i, r));
+            if (t_dtype[r] != d.r_dtype || t_fl[r] != d.fl_r)
+                return cleanup(fail(F8_ERR_DTYPE, "layer %d: r_dtype / fl_r do not match the producer of tensor %d", i, r));
+        }
+        net->t_h[i + 1] = ho; net->t_w[i + 1] = wo; net->t_c[i + 1] = d.c_out;
+        net->t_elem[i + 1] = d.y_dtype == F8_S32 ? 4 : 1;
+        t_dtype[i + 1] = d.y_dtype;
+        t_fl[i + 1] = d.y_dtype == F8_S32 ? d.fl_x + d.fl_w : d.fl_y;
+        L.out_bytes_per_image = (size_t)ho * wo * d.c_out * net->t_elem[i + 1];
+
+        // parameters
+        const bool has_params = kind == F8_LAYER_CONV || kind == F8_LAYER_DWCONV || kind == F8_LAYER_LINEAR;
+        if (!has_params) continue;
+        const int8_t *hw = host_weights ? host_weights[i] : nullptr;
+        const int32_t *hb = host_bias ? host_bias[i] : nullptr;
+        if (!hw) return cleanup(fail(F8_ERR_NULL, "layer %d: weights missing", i));
+        const size_t per_out = (size_t)d.kh * d.kw * (kind == F8_LAYER_DWCONV ? 1 : d.c);
+        // exact accumulator bound per output channel from the actual parameters
+        const long long xmax = d.x_dtype == F8_U8 ? 255 : 128;
+        const long long rmax = has_res ? (d.r_dtype == F8_U8 ? 255 : 128) : 0;
+        for (int co = 0; co < d.c_out; ++co) {
+            long long sum = 0;
+            for (size_t j = 0; j < per_out; ++j) sum += llabs((long long)hw[co * per_out + j]);
+            long long bound = sum * xmax + (hb ? llabs((long long)hb[co]) : 0);
+            bound = (bound << L.q.sh_acc) + (rmax << L.q.sh_res);
+            if (bound >= (1ll << 31) - 1)
+                return cleanup(fail(F8_ERR_ACC_BOUND, "layer %d channel %d: accumulator bound %lld exceeds int32", i, co, bound));
+        }
+    }
+    // second pass (everything validated): upload the parameters
+    for (int i = 0; i < n_layers; ++i) {
+        NetLayer &L = net->layers[i];
+        const f8_conv_desc &d = L.d.conv;
+        const int kind = L.d.kind;
+        if (kind != F8_LAYER_CONV && kind != F8_LAYER_DWCONV && kind != F8_LAYER_LINEAR) continue;
+        const int8_t *hw = host_weights[i];
+        const int32_t *hb = host_bias ? host_bias[i] : nullptr;
+        const size_t wn = (size_t)d.kh * d.kw * (kind == F8_LAYER_DWCONV ? 1 : d.c) * d.c_out;
+        cudaError_t e = cudaMalloc(&L.w, round256(wn));
+        if (e == cudaSuccess) e = cudaMemcpy(L.w, hw, wn, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess && hb) {
+            e = cudaMalloc(&L.b, round256(4 * (size_t)d.c_out));
+            if (e == cudaSuccess) e = cudaMemcpy(L.b, hb, 4 * (size_t)d.c_out, cudaMemcpyHostToDevice);
+        }
+        if (e != cudaSuccess) return cleanup(cuda_fail(e, "parameter upload"));
+
+        // 3-channel (<= 8) stems with an even stride: widen pixels to 8 bytes so that the kw-tap window of an
+        // output column is one contiguous, 16-byte aligned run of kw8 bytes; the layer then is a kh x 1
+        // convolution over kw8 "channels" of an overlapping strided view, which the tensor-core path takes.
+        if (kind == F8_LAYER_CONV && d.c <= 8 && d.c % 16 != 0 && d.stride % 2 == 0 && d.kw * 8 <= 256) {
+            L.packed = true;
+            L.pack_left = d.pad;
+            L.pack_kw8 = (d.kw * 8 + 31) / 32 * 32;
+            L.pack_wp = std::max(d.w + d.pad, (L.g.wo - 1) * d.stride + L.pack_kw8 / 8);
+            L.pack_wp = (L.pack_wp + 1) / 2 * 2;              // rows stay 16-byte multiples
+            std::vector<int8_t> wp((size_t)d.c_out * d.kh * L.pack_kw8, 0);
+            for (int co = 0; co < d.c_out; ++co)
+                for (int r = 0; r < d.kh; ++r)
+                    for (int s2 = 0; s2 < d.kw; ++s2)
+                        for (int ch = 0; ch < d.c; ++ch)
+                            wp[((size_t)co * d.kh + r) * L.pack_kw8 + s2 * 8 + ch] =
+                                hw[(((size_t)co * d.kh + r) * d.kw + s2) * d.c + ch];
+            e = cudaMalloc(&L.w_packed, round256(wp.size()));
+            if (e == cudaSuccess) e = cudaMemcpy(L.w_packed, wp.data(), wp.size(), cudaMemcpyHostToDevice);
+            if (e != cudaSuccess) return cleanup(cuda_fail(e, "packed stem weights upload"));
+        }
+    }
+    *out = net.release();
+    return F8_OK;
+}
+
+size_t f8_net_workspace_bytes(const f8_net *net, int batch) {
+    if (!net || batch <= 0) return 0;
+    std::vector<size_t> off;
+    size_t pack_off;
+    return assign_offsets(net, batch, &off, &pack_off) + 256;
+}
+
+int f8_net_last_launch_count(const f8_net *net) { return net ? net->last_launches : 0; }
+
+f8_status f8_net_set_profiling(f8_net *net, int on) {
+    if (!net) return fail(F8_ERR_NULL, "net is NULL");
+    net->profiling = on != 0;
+    net->event_layer.clear();
+    return F8_OK;
+}
+
+f8_status f8_net_get_layer_ms(f8_net *net, float *ms, int *on_tensor_cores) {
+    if (!net || !ms) return fail(F8_ERR_NULL, "net / ms is NULL");
+    const int nl = (int)net->layers.size();
+    for (int i = 0; i < nl; ++i) ms[i] = 0.f;
+    if (on_tensor_cores) for (int i = 0; i < nl; ++i) on_tensor_cores[i] = 0;
+    if (net->event_layer.empty()) return fail(F8_ERR_UNSUPPORTED, "no profiled forward pass recorded");
+    cudaError_t e = cudaEventSynchronize(net->events[net->event_layer.size()]);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaEventSynchronize");
+    for (size_t k = 0; k < net->event_layer.size(); ++k) {
+        float t = 0.f;
+        e = cudaEventElapsedTime(&t, net->events[k], net->events[k + 1]);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventElapsedTime");
+        ms[net->event_layer[k]] += t;
+    }
+    if (on_tensor_cores)
+        for (const Step &stp : net->steps)
+            if (stp.kind >= 0 && stp.use_tc) on_tensor_cores[stp.layer] = 1;
+    return F8_OK;
+}
+
+void f8_net_destroy(f8_net *net) {
+    if (!net) return;
+    for (cudaEvent_t ev : net->events) cudaEventDestroy(ev);
+    free_layers(net);
+    delete net;
+}
+
+f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *workspace, size_t workspace_bytes,
+                         void *const *layer_dump, void *cuda_stream) {
+    if (!net) return fail(F8_ERR_NULL, "net is NULL");
+    if (batch < 0 || batch > net->max_batch) return fail(F8_ERR_SHAPE, "batch %d outside [0, %d]", batch, net->max_batch);
+    if (batch == 0) { net->last_launches = 0; return F8_OK; }
+    if (!x || !y) return fail(F8_ERR_NULL, "x and y must not be NULL");
+    if (!aligned16(x) || !aligned16(y) || !aligned16(workspace)) return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    const size_t need = f8_net_workspace_bytes(net, batch);
+    if (need > 256 && (!workspace || workspace_bytes < need))
+        return fail(F8_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, workspace_bytes);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int nl = (int)net->layers.size();
+
+    const bool replan = net->plan_batch != batch || net->plan_x != x || net->plan_y != y || net->plan_ws != workspace ||
+                        net->plan_force_direct != g_force_direct;
+    if (replan) {
+        net->steps.clear();
+        net->plan_batch = -1;
+        assign_offsets(net, batch, &net->t_off, &net->pack_off);
+        auto tensor_ptr = [&](int t) -> void * {
+            if (t == 0) return const_cast<void *>(x);
+            if (t == nl) return y;
+            return (uint8_t *)workspace + net->t_off[t];
+        };
+        for (int i = 0; i < nl; ++i) {
+            NetLayer &L = net->layers[i];
+            Step stp;
+            stp.kind = L.d.kind;
+            stp.layer = i;
+            stp.x = tensor_ptr(L.d.src);
+            stp.res = (L.q.has_res) ? tensor_ptr(L.d.res) : nullptr;
+            stp.y = tensor_ptr(i + 1);
+            stp.g = L.g;
+            stp.g.n = batch;
+            if ((L.d.kind == F8_LAYER_CONV || L.d.kind == F8_LAYER_LINEAR) && !g_force_direct) {
+                const char *why = "";
+                if (L.packed) {
+                    F8ConvGeom pg = stp.g;
+                    pg.c = L.pack_kw8; pg.kw = 1; pg.stride_w = 1; pg.pad_w = 0;
+                    void *pbuf = (uint8_t *)workspace + net->pack_off;
+                    const size_t pbytes = (size_t)batch * L.g.h * L.pack_wp * 8;
+                    if (f8_tc_supported(pg, pbytes)) {
+                        F8TcTensorView v;
+                        v.base = pbuf;
+                        v.dim_c = L.pack_kw8; v.dim_w = L.g.wo; v.dim_h = L.g.h; v.dim_n = batch;
+                        v.stride_w = (uint64_t)L.g.stride_w * 8;
+                        v.stride_h = (uint64_t)L.pack_wp * 8;
+                        v.stride_n = (uint64_t)L.pack_wp * 8 * L.g.h;
+                        PlanPtr plan = alloc_plan();
+                        if (plan && f8_tc_plan_init(plan.get(), pg, L.q, v, L.w_packed, L.b, stp.res, stp.y,
+                                                    f8_status_word(), &why) == cudaSuccess) {
+                            Step pre;
+                            pre.kind = -1;
+                            pre.layer = i;
+                            pre.x = stp.x;
+                            pre.y = pbuf;
+                            pre.g = stp.g;
+                            net->steps.push_back(std::move(pre));
+                            stp.use_tc = true;
+                            stp.plan = std::move(plan);
+                        }
+                    }
+                } else if (f8_tc_supported(stp.g, (size_t)batch * L.g.h * L.g.w * L.g.c)) {
+                    PlanPtr plan = alloc_plan();
+                    if (plan && f8_tc_plan_init(plan.get(), stp.g, L.q, dense_view(stp.x, stp.g), L.w, L.b, stp.res,
+                                                stp.y, f8_status_word(), &why) == cudaSuccess) {
+                        stp.use_tc = true;
+                        stp.plan = std::move(plan);
+                    }
+                }
+            }
+            net->steps.push_back(std::move(stp));
+        }
+        net->plan_batch = batch;
+        net->plan_x = x;
+        net->plan_y = y;
+        net->plan_ws = workspace;
+        net->plan_force_direct = g_force_direct;
+    }
+
+    int launches = 0;
+    const bool prof = net->profiling;
+    if (prof) {
+        while (net->events.size() < net->steps.size() + 1) {
+            cudaEvent_t ev;
+            if (cudaEventCreate(&ev) != cudaSuccess) return fail(F8_ERR_CUDA, "cudaEventCreate failed");
+            net->events.push_back(ev);
+        }
+        net->event_layer.clear();
+        cudaEventRecord(net->events[0], st);
+    }
+    for (Step &stp : net->steps) {
+        NetLayer &L = net->layers[stp.layer];
+        cudaError_t e = cudaSuccess;
+        switch (stp.kind) {
+            case -1:
+                e = f8_launch_pack_stem(batch, L.g.h, L.g.w, L.g.c, L.pack_wp, L.pack_left, stp.x, stp.y, st);
+                break;
+            case F8_LAYER_CONV:
+            case F8_LAYER_LINEAR:
+                if (stp.use_tc) { e = f8_tc_launch(stp.plan.get(), st); ++g_tc_launches; }
+                else e = f8_launch_conv_direct(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st);
+                break;
+            case F8_LAYER_DWCONV:
+                e = f8_launch_dwconv(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st);
+                break;
+            case F8_LAYER_MAXPOOL:
+                e = f8_launch_maxpool(batch, L.g.h, L.g.w, L.g.c, L.d.conv.kh, L.d.conv.stride, L.d.conv.pad, L.g.x_signed,
+                                      stp.x, stp.y, st);
+                break;
+            case F8_LAYER_GAP:
+                e = f8_launch_gap(batch, L.g.h, L.g.w, L.g.c, L.g.x_signed, L.q.s, stp.x, stp.y, st);
+                break;
+        }
+        if (e != cudaSuccess) return cuda_fail(e, "layer launch");
+        ++launches;
+        if (prof) {
+            cudaEventRecord(net->events[launches], st);
+            net->event_layer.push_back(stp.layer);
+        }
+        if (layer_dump && stp.kind >= 0 && layer_dump[stp.layer]) {
+            e = cudaMemcpyAsync(layer_dump[stp.layer], stp.y, (size_t)batch * L.out_bytes_per_image,
+                                cudaMemcpyDeviceToDevice, st);
+            if (e != cudaSuccess) return cuda_fail(e, "layer dump copy");
+        }
+    }
+    net->last_launches = launches;
+    return F8_OK;
+}
+
+}   // extern "C"

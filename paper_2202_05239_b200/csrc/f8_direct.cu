@@ -1,0 +1,345 @@
+// CUDA-core kernels: generic direct convolution (any shape), depthwise convolution, pooling and the
+// stem packing pre-pass.  Depthwise and pooling layers are not dense contractions: they are bound by
+// HBM traffic, so these kernels are organised around wide, coalesced NHWC accesses.
+#include "f8_epilogue.cuh"
+
+namespace {
+
+__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {   // u8 x s8
+    int d;
+    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ int dp4a_ss(uint32_t a, uint32_t b, int c) {   // s8 x s8
+    int d;
+    asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+__device__ __forceinline__ void store_out(void *y, size_t i, int v, int y_kind) {
+    if (y_kind == F8_S32) ((int32_t *)y)[i] = v;
+    else ((uint8_t *)y)[i] = (uint8_t)(v & 0xff);
+}
+
+// ---------------------------------------------------------------------------------------
+// Generic direct convolution: one thread per output element, channel fastest so that a warp
+// shares its input window.  Used for shapes the tensor-core path does not take.
+// ---------------------------------------------------------------------------------------
+template <bool VEC4>
+__global__ void __launch_bounds__(256) conv_direct_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
+                                                          const int8_t *__restrict__ w,
+                                                          const int32_t *__restrict__ bias,
+                                                          const void *__restrict__ res, void *__restrict__ y) {
+    const size_t total = (size_t)g.n * g.ho * g.wo * g.c_out;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int co = (int)(idx % g.c_out);
+        size_t pix = idx / g.c_out;
+        const int ow = (int)(pix % g.wo);
+        pix /= g.wo;
+        const int oh = (int)(pix % g.ho);
+        const int in = (int)(pix / g.ho);
+        int acc = bias ? bias[co] : 0;
+        for (int r = 0; r < g.kh; ++r) {
+            const int ih = oh * g.stride_h + r - g.pad_h;
+            if (ih < 0 || ih >= g.h) continue;
+            for (int s = 0; s < g.kw; ++s) {
+                const int iw = ow * g.stride_w + s - g.pad_w;
+                if (iw < 0 || iw >= g.w) continue;
+                const uint8_t *xp = x + (((size_t)in * g.h + ih) * g.w + iw) * g.c;
+                const int8_t *wp = w + (((size_t)co * g.kh + r) * g.kw + s) * g.c;
+                if (VEC4) {
+                    const uint32_t *x4 = (const uint32_t *)xp;
+                    const uint32_t *w4 = (const uint32_t *)wp;
+                    const int nc = g.c >> 2;
+                    if (g.x_signed) {
+                        for (int c = 0; c < nc; ++c) acc = dp4a_ss(x4[c], w4[c], acc);
+                    } else {
+                        for (int c = 0; c < nc; ++c) acc = dp4a_us(x4[c], w4[c], acc);
+                    }
+                } else {
+                    for (int c = 0; c < g.c; ++c) {
+                        const int xv = g.x_signed ? (int)(int8_t)xp[c] : (int)xp[c];
+                        acc += xv * (int)wp[c];
+                    }
+                }
+            }
+        }
+        const int rv = q.has_res ? f8_load8(res, idx, q.r_signed) : 0;
+        store_out(y, idx, f8_requant(acc, rv, q), q.y_kind);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Depthwise kh x kw convolution.  One thread owns 4 consecutive channels of one output pixel:
+// every tap is one 32-bit load that a warp coalesces into a 128-byte row segment.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) dwconv_vec4_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
+                                                          const int8_t *__restrict__ w,
+                                                          const int32_t *__restrict__ bias,
+                                                          const void *__restrict__ res, void *__restrict__ y) {
+    const int c4 = g.c >> 2;
+    const size_t total = (size_t)g.n * g.ho * g.wo * c4;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int cg = (int)(idx % c4);
+        size_t pix = idx / c4;
+        const int ow = (int)(pix % g.wo);
+        pix /= g.wo;
+        const int oh = (int)(pix % g.ho);
+        const int in = (int)(pix / g.ho);
+        const int c0 = cg * 4;
+        int acc[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[j] = bias ? bias[c0 + j] : 0;
+        const int taps = g.kh * g.kw;
+        for (int r = 0; r < g.kh; ++r) {
+            const int ih = oh * g.stride_h + r - g.pad_h;
+            if (ih < 0 || ih >= g.h) continue;
+            for (int s = 0; s < g.kw; ++s) {
+                const int iw = ow * g.stride_w + s - g.pad_w;
+                if (iw < 0 || iw >= g.w) continue;
+                const uint32_t xw = *(const uint32_t *)(x + (((size_t)in * g.h + ih) * g.w + iw) * g.c + c0);
+                const int t = r * g.kw + s;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    acc[j] += f8_byte(xw, j, g.x_signed) * (int)w[(size_t)(c0 + j) * taps + t];
+            }
+        }
+        const size_t o = (((size_t)in * g.ho + oh) * g.wo + ow) * g.c + c0;
+        uint32_t rw = 0;
+        if (q.has_res) rw = *(const uint32_t *)((const uint8_t *)res + o);
+        int out[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) out[j] = f8_requant(acc[j], f8_byte(rw, j, q.r_signed), q);
+        if (q.y_kind == F8_S32) {
+            *(int4 *)((int32_t *)y + o) = make_int4(out[0], out[1], out[2], out[3]);
+        } else {
+            *(uint32_t *)((uint8_t *)y + o) = f8_pack4(out[0], out[1], out[2], out[3]);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) dwconv_scalar_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
+                                                            const int8_t *__restrict__ w,
+                                                            const int32_t *__restrict__ bias,
+                                                            const void *__restrict__ res, void *__restrict__ y) {
+    const size_t total = (size_t)g.n * g.ho * g.wo * g.c;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(idx % g.c);
+        size_t pix = idx / g.c;
+        const int ow = (int)(pix % g.wo);
+        pix /= g.wo;
+        const int oh = (int)(pix % g.ho);
+        const int in = (int)(pix / g.ho);
+        int acc = bias ? bias[ch] : 0;
+        for (int r = 0; r < g.kh; ++r) {
+            const int ih = oh * g.stride_h + r - g.pad_h;
+            if (ih < 0 || ih >= g.h) continue;
+            for (int s = 0; s < g.kw; ++s) {
+                const int iw = ow * g.stride_w + s - g.pad_w;
+                if (iw < 0 || iw >= g.w) continue;
+                acc += f8_load8(x, (((size_t)in * g.h + ih) * g.w + iw) * g.c + ch, g.x_signed) *
+                       (int)w[((size_t)ch * g.kh + r) * g.kw + s];
+            }
+        }
+        const int rv = q.has_res ? f8_load8(res, idx, q.r_signed) : 0;
+        store_out(y, idx, f8_requant(acc, rv, q), q.y_kind);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Max pooling: one thread per (output pixel, VEC channels); taps outside the image are skipped.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t max4(uint32_t a, uint32_t b, int is_signed) {
+    return is_signed ? __vmaxs4(a, b) : __vmaxu4(a, b);
+}
+
+template <int WORDS>   // WORDS 32-bit words (4 channels each) per thread: 4 -> 16-byte accesses
+__global__ void __launch_bounds__(256) maxpool_kernel(int n, int h, int w, int c, int ho, int wo, int k, int stride,
+                                                      int pad, int x_signed, const uint8_t *__restrict__ x,
+                                                      uint8_t *__restrict__ y) {
+    const int cg = c / (4 * WORDS);
+    const size_t total = (size_t)n * ho * wo * cg;
+    const uint32_t identity = x_signed ? 0x80808080u : 0u;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int g = (int)(idx % cg);
+        size_t pix = idx / cg;
+        const int ow = (int)(pix % wo);
+        pix /= wo;
+        const int oh = (int)(pix % ho);
+        const int in = (int)(pix / ho);
+        uint32_t m[WORDS];
+#pragma unroll
+        for (int j = 0; j < WORDS; ++j) m[j] = identity;
+        for (int r = 0; r < k; ++r) {
+            const int ih = oh * stride + r - pad;
+            if (ih < 0 || ih >= h) continue;
+            for (int s = 0; s < k; ++s) {
+                const int iw = ow * stride + s - pad;
+                if (iw < 0 || iw >= w) continue;
+                const uint32_t *p = (const uint32_t *)(x + (((size_t)in * h + ih) * w + iw) * c) + g * WORDS;
+                if (WORDS == 4) {
+                    const uint4 v = *(const uint4 *)p;
+                    m[0] = max4(m[0], v.x, x_signed);
+                    m[1 % WORDS] = max4(m[1 % WORDS], v.y, x_signed);
+                    m[2 % WORDS] = max4(m[2 % WORDS], v.z, x_signed);
+                    m[3 % WORDS] = max4(m[3 % WORDS], v.w, x_signed);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < WORDS; ++j) m[j] = max4(m[j], p[j], x_signed);
+                }
+            }
+        }
+        uint32_t *o = (uint32_t *)(y + (((size_t)in * ho + oh) * wo + ow) * c) + g * WORDS;
+        if (WORDS == 4) *(uint4 *)o = make_uint4(m[0], m[1 % WORDS], m[2 % WORDS], m[3 % WORDS]);
+        else {
+#pragma unroll
+            for (int j = 0; j < WORDS; ++j) o[j] = m[j];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) maxpool_scalar_kernel(int n, int h, int w, int c, int ho, int wo, int k,
+                                                             int stride, int pad, int x_signed,
+                                                             const uint8_t *__restrict__ x, uint8_t *__restrict__ y) {
+    const size_t total = (size_t)n * ho * wo * c;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(idx % c);
+        size_t pix = idx / c;
+        const int ow = (int)(pix % wo);
+        pix /= wo;
+        const int oh = (int)(pix % ho);
+        const int in = (int)(pix / ho);
+        int m = -1000;
+        for (int r = 0; r < k; ++r) {
+            const int ih = oh * stride + r - pad;
+            if (ih < 0 || ih >= h) continue;
+            for (int s = 0; s < k; ++s) {
+                const int iw = ow * stride + s - pad;
+                if (iw < 0 || iw >= w) continue;
+                m = max(m, f8_load8(x, (((size_t)in * h + ih) * w + iw) * c + ch, x_signed));
+            }
+        }
+        y[idx] = (uint8_t)(m & 0xff);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Global average pooling: sum over h*w, rounding shift, clip.  A block handles one image and a
+// slab of channels; threads run over channels so that every row read is coalesced.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) gap_kernel(int hw, int c, int x_signed, int s, const uint8_t *__restrict__ x,
+                                                  uint8_t *__restrict__ y) {
+    const int in = blockIdx.y;
+    const int ch = blockIdx.x * blockDim.x + threadIdx.x;
+    if (ch >= c) return;
+    const uint8_t *p = x + (size_t)in * hw * c + ch;
+    int sum = 0;
+    for (int i = 0; i < hw; ++i) {
+        const uint8_t b = p[(size_t)i * c];
+        sum += x_signed ? (int)(int8_t)b : (int)b;
+    }
+    F8Requant q;
+    q.sh_acc = q.sh_res = 0;
+    q.s = s;
+    q.lo = x_signed ? -127 : 0;
+    q.hi = x_signed ? 127 : 255;
+    q.y_kind = x_signed ? F8_S8 : F8_U8;
+    q.has_res = 0;
+    q.r_signed = 0;
+    y[(size_t)in * c + ch] = (uint8_t)(f8_requant(sum, 0, q) & 0xff);
+}
+
+// ---------------------------------------------------------------------------------------
+// Stem packing: [n,h,w,c<=8] -> [n,h,wp,8], pixel iw lands at column iw + left; all other bytes 0.
+// One thread writes one 8-byte output pixel.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) pack_stem_kernel(int n, int h, int w, int c, int wp, int left,
+                                                        const uint8_t *__restrict__ x, uint2 *__restrict__ y) {
+    const size_t total = (size_t)n * h * wp;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int col = (int)(idx % wp);
+        const size_t row = idx / wp;           // n*h + ih
+        const int iw = col - left;
+        uint32_t lo = 0, hi = 0;
+        if (iw >= 0 && iw < w) {
+            const uint8_t *p = x + (row * w + iw) * c;
+            for (int j = 0; j < c; ++j) {
+                const uint32_t b = p[j];
+                if (j < 4) lo |= b << (8 * j);
+                else hi |= b << (8 * (j - 4));
+            }
+        }
+        y[idx] = make_uint2(lo, hi);
+    }
+}
+
+inline int grid_for(size_t total, int block) {
+    size_t blocks = (total + block - 1) / block;
+    const size_t cap = 148 * 16;   // a few waves of a grid-stride loop on 148 SMs
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+}   // namespace
+
+cudaError_t f8_launch_conv_direct(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
+                                  const int32_t *bias, const void *res, void *y, cudaStream_t st) {
+    const size_t total = (size_t)g.n * g.ho * g.wo * g.c_out;
+    if (total == 0) return cudaSuccess;
+    const bool vec = (g.c % 4 == 0) && (((uintptr_t)x | (uintptr_t)w) % 4 == 0);
+    if (vec)
+        conv_direct_kernel<true><<<grid_for(total, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
+    else
+        conv_direct_kernel<false><<<grid_for(total, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
+    return cudaGetLastError();
+}
+
+cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
+                             const int32_t *bias, const void *res, void *y, cudaStream_t st) {
+    const size_t total = (size_t)g.n * g.ho * g.wo * g.c;
+    if (total == 0) return cudaSuccess;
+    if (g.c % 4 == 0)
+        dwconv_vec4_kernel<<<grid_for(total / 4, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
+    else
+        dwconv_scalar_kernel<<<grid_for(total, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
+    return cudaGetLastError();
+}
+
+cudaError_t f8_launch_maxpool(int n, int h, int w, int c, int k, int stride, int pad, int x_signed, const void *x,
+                              void *y, cudaStream_t st) {
+    const int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
+    const size_t total = (size_t)n * ho * wo * c;
+    if (total == 0) return cudaSuccess;
+    if (c % 16 == 0)
+        maxpool_kernel<4><<<grid_for(total / 16, 256), 256, 0, st>>>(n, h, w, c, ho, wo, k, stride, pad, x_signed,
+                                                                     (const uint8_t *)x, (uint8_t *)y);
+    else if (c % 4 == 0)
+        maxpool_kernel<1><<<grid_for(total / 4, 256), 256, 0, st>>>(n, h, w, c, ho, wo, k, stride, pad, x_signed,
+                                                                    (const uint8_t *)x, (uint8_t *)y);
+    else
+        maxpool_scalar_kernel<<<grid_for(total, 256), 256, 0, st>>>(n, h, w, c, ho, wo, k, stride, pad, x_signed,
+                                                                    (const uint8_t *)x, (uint8_t *)y);
+    return cudaGetLastError();
+}
+
+cudaError_t f8_launch_gap(int n, int h, int w, int c, int x_signed, int s, const void *x, void *y, cudaStream_t st) {
+    if (n == 0) return cudaSuccess;
+    dim3 grid((c + 255) / 256, n);
+    gap_kernel<<<grid, 256, 0, st>>>(h * w, c, x_signed, s, (const uint8_t *)x, (uint8_t *)y);
+    return cudaGetLastError();
+}
+
+cudaError_t f8_launch_pack_stem(int n, int h, int w, int c, int wp, int left, const void *x, void *y,
+                                cudaStream_t st) {
+    const size_t total = (size_t)n * h * wp;
+    if (total == 0) return cudaSuccess;
+    pack_stem_kernel<<<grid_for(total, 256), 256, 0, st>>>(n, h, w, c, wp, left, (const uint8_t *)x, (uint2 *)y);
+    return cudaGetLastError();
+}

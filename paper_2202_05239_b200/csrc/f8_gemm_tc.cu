@@ -1,0 +1,594 @@
+// Dense convolution / pointwise / fully connected layers as an implicit GEMM on the Blackwell tensor
+// cores:  D[M = output pixels, N = output channels] = A[M, K = taps x channels] * B[N, K]^T.
+//
+//   * A tiles (128 output pixels x KB channels of one filter tap) are gathered straight from the NHWC
+//     activation tensor by TMA in im2col mode (zero fill outside the image and past the last pixel);
+//     B tiles (BN output channels x KB) come from the OHWI weight tensor by tiled TMA.  Both land in
+//     shared memory in the swizzled K-major layout tcgen05.mma reads.
+//   * One thread issues tcgen05.mma.kind::i8 (u8|s8 x s8 -> s32); the 128 x BN int32 accumulator lives
+//     in tensor memory, double buffered so the epilogue of tile i overlaps the main loop of tile i+1.
+//   * Four epilogue warps read the accumulator with tcgen05.ld (one output pixel per thread, 16
+//     consecutive channels per load), add the bias, align and add the residual, apply the rounding
+//     shift and clip (Eq. 2 / signed form applied to Eq. 6) and store 16 output bytes per instruction.
+//   * Persistent CTAs (one per SM) walk the tile list; tiles that share an A tile are adjacent so that
+//     the activation tensor is read from HBM once and from L2 afterwards.
+//
+// Every mbarrier wait is bounded: when a wait does not complete the kernel raises a shared abort flag,
+// writes the device status word, drains what it started and returns; it never spins forever or traps.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <string.h>
+
+#include "f8_epilogue.cuh"
+
+namespace {
+
+constexpr int TILE_M = 128;
+constexpr int NUM_THREADS = 192;           // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr int MAX_STAGES = 8;
+constexpr int TMEM_COLS = 512;
+constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
+constexpr unsigned long long DRAIN_LIMIT_CYCLES = 200000000ull;
+constexpr size_t SMEM_BUDGET = 200 * 1024;
+
+struct TcParams {
+    int M;                    // total output pixels
+    int ho, wo;
+    int c_out;
+    int kh, kw;
+    int stride_h, stride_w, pad_h, pad_w;
+    int c_chunks;             // K chunks per tap
+    int kb;                   // bytes (= int8 elements) of K per stage: 32, 64 or 128
+    int bn;                   // N tile, multiple of 16, <= 256
+    int m_tiles, n_tiles;
+    int stages;
+    uint32_t stage_bytes;     // A + B bytes of one stage (rounded to 1024)
+    uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
+    uint32_t tx_bytes;        // bytes both TMA loads of a stage deliver
+    uint32_t idesc;           // tcgen05 instruction descriptor
+    uint64_t desc_hi;         // constant upper part of the shared-memory matrix descriptors
+    const int32_t *bias;
+    const uint8_t *res;
+    uint8_t *y;
+    int vec_bytes;            // widest aligned store the output rows allow: 16, 8, 4 or 1
+    F8Requant q;
+    int *status;
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false when the kernel is aborting (this wait or another one ran out).
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                       int code, unsigned long long limit = WAIT_LIMIT_CYCLES) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = clock64();
+    unsigned spins = 0;
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0) {
+            if (*abort_flag) return false;
+            if ((unsigned long long)(clock64() - t0) > limit) {
+                *abort_flag = 1;
+                atomicCAS(status, 0, code);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w,
+                                                int h, int n, uint16_t off_w, uint16_t off_h) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
+                                            int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, int8 operands, int32 accumulate.
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// mbarrier arrives once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+
+// 16 consecutive accumulator columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
+        "%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are `kb` bytes long and swizzled with
+// the matching TMA mode: 8-row groups are 8*kb bytes apart (stride byte offset), the leading offset
+// is unused (1), descriptor version 1, layout code 2 / 4 / 6 for 128 / 64 / 32-byte swizzle.
+__host__ __device__ inline uint64_t smem_desc_hi(int kb) {
+    const uint64_t layout = kb == 128 ? 2 : (kb == 64 ? 4 : 6);
+    const uint64_t sbo = (uint64_t)(8 * kb) >> 4;
+    return ((uint64_t)1 << 16) | (sbo << 32) | ((uint64_t)1 << 46) | (layout << 61);
+}
+
+// ----------------------------------------------------------------------------- epilogue helpers
+
+__device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int (&acc)[16], size_t row, int co0,
+                                               bool row_valid) {
+    // how many of the 16 channels exist
+    const int nvalid = min(16, p.c_out - co0);
+    int v[16];
+    uint32_t rw[4] = {0u, 0u, 0u, 0u};
+    const size_t o = row * (size_t)p.c_out + co0;
+    if (p.q.has_res && row_valid) {
+        if (p.vec_bytes == 16 && nvalid == 16) {
+            const uint4 t = *(const uint4 *)(p.res + o);
+            rw[0] = t.x; rw[1] = t.y; rw[2] = t.z; rw[3] = t.w;
+        } else {
+            for (int j = 0; j < nvalid; ++j) rw[j >> 2] |= (uint32_t)p.res[o + j] << (8 * (j & 3));
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int b = (j < nvalid && p.bias) ? __ldg(p.bias + co0 + j) : 0;
+        v[j] = f8_requant(acc[j] + b, f8_byte(rw[j >> 2], j & 3, p.q.r_signed), p.q);
+    }
+    if (!row_valid) return;
+    if (p.q.y_kind == F8_S32) {
+        int32_t *y32 = (int32_t *)p.y + o;
+        if (nvalid == 16 && (p.c_out & 3) == 0) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) *(int4 *)(y32 + 4 * j) = make_int4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        } else {
+            for (int j = 0; j < nvalid; ++j) y32[j] = v[j];
+        }
+        return;
+    }
+    uint32_t ow[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) ow[j] = f8_pack4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    uint8_t *yo = p.y + o;
+    if (nvalid == 16 && p.vec_bytes == 16) {
+        *(uint4 *)yo = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+    } else if (p.vec_bytes >= 8 && (nvalid & 7) == 0) {
+        for (int j = 0; j < nvalid / 8; ++j) *(uint2 *)(yo + 8 * j) = make_uint2(ow[2 * j], ow[2 * j + 1]);
+    } else if (p.vec_bytes >= 4 && (nvalid & 3) == 0) {
+        for (int j = 0; j < nvalid / 4; ++j) *(uint32_t *)(yo + 4 * j) = ow[j];
+    } else {
+        for (int j = 0; j < nvalid; ++j) yo[j] = (uint8_t)(ow[j >> 2] >> (8 * (j & 3)));
+    }
+}
+
+// ----------------------------------------------------------------------------- the kernel
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                       const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // stage buffers need 1024-byte alignment for the 128-byte swizzle
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t full_bar = smem_u32(&bars[0]);
+    const uint32_t empty_bar = smem_u32(&bars[MAX_STAGES]);
+    const uint32_t tfull_bar = smem_u32(&bars[2 * MAX_STAGES]);
+    const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + 2]);
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar + 8 * a, 1);
+            mbar_init(tempty_bar + 8 * a, 128);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int k_iters = p.kh * p.kw * p.c_chunks;
+    volatile int *abortp = &abort_flag;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t issued = 0;            // loads issued so far (for the drain on abort)
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+                const int m0 = m_t * TILE_M;
+                const int ow = m0 % p.wo;
+                const int t1 = m0 / p.wo;
+                const int oh = t1 % p.ho;
+                const int img = t1 / p.ho;
+                const int base_w = ow * p.stride_w - p.pad_w;
+                const int base_h = oh * p.stride_h - p.pad_h;
+                for (int r = 0; ok && r < p.kh; ++r)
+                    for (int s = 0; ok && s < p.kw; ++s)
+                        for (int cc = 0; cc < p.c_chunks; ++cc) {
+                            if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101)) {
+                                ok = false;
+                                break;
+                            }
+                            const uint32_t fb = full_bar + 8 * stage;
+                            const uint32_t a_dst = smem_base + stage * p.stage_bytes;
+                            mbar_expect_tx(fb, p.tx_bytes);
+                            tma_load_im2col(a_dst, &map_a, fb, cc * p.kb, base_w, base_h, img, (uint16_t)s,
+                                            (uint16_t)r);
+                            tma_load_3d(a_dst + p.a_bytes, &map_b, fb, cc * p.kb, r * p.kw + s, n_t * p.bn);
+                            ++issued;
+                            if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                        }
+            }
+            if (!ok) {
+                // Drain: give every load that was issued time to land before the CTA's shared memory goes away.
+                const uint32_t pending = issued < (uint32_t)p.stages ? issued : (uint32_t)p.stages;
+                for (uint32_t i = 0; i < pending; ++i) {
+                    const uint32_t idx = issued - 1 - i;
+                    const int st = (int)(idx % p.stages);
+                    const uint32_t ph = (idx / p.stages) & 1;
+                    const unsigned long long t0 = clock64();
+                    while (!mbar_try_wait(full_bar + 8 * st, ph) &&
+                           (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int local = 0;
+            bool ok = true;
+            bool committed_any = false;
+            int last_acc = 0;
+            uint32_t last_acc_phase = 0;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+                const int acc = local & 1;
+                const uint32_t acc_phase = (local >> 1) & 1;
+                if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, abortp, p.status, 102)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * 256;   // two 256-column accumulators
+                for (int kc = 0; kc < k_iters; ++kc) {
+                    if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, 103)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_base + stage * p.stage_bytes;
+                    const uint32_t b_addr = a_addr + p.a_bytes;
+                    const uint64_t a_desc = p.desc_hi | (uint64_t)((a_addr & 0x3ffffu) >> 4);
+                    const uint64_t b_desc = p.desc_hi | (uint64_t)((b_addr & 0x3ffffu) >> 4);
+                    for (int j = 0; j < p.kb / 32; ++j)   // 32 bytes of K per instruction: +2 in 16-byte units
+                        mma_i8(d_tmem, a_desc + 2 * j, b_desc + 2 * j, p.idesc, (kc | j) != 0 ? 1u : 0u);
+                    mma_commit(empty_bar + 8 * stage);    // frees the stage when these MMAs have read it
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                mma_commit(tfull_bar + 8 * acc);          // accumulator complete
+                committed_any = true;
+                last_acc = acc;
+                last_acc_phase = acc_phase;
+            }
+            if (!ok && committed_any) {
+                // let the tensor pipe finish what was issued before TMEM is released
+                const unsigned long long t0 = clock64();
+                while (!mbar_try_wait(tfull_bar + 8 * last_acc, last_acc_phase) &&
+                       (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 belong to this warp
+        int local = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+            const int acc = local & 1;
+            const uint32_t acc_phase = (local >> 1) & 1;
+            const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+            if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104)) { ok = false; break; }
+            tc_fence_after();
+            const size_t row = (size_t)m_t * TILE_M + quarter * 32 + lane;
+            const bool row_valid = row < (size_t)p.M;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256;
+            const int n0 = n_t * p.bn;
+            for (int ch = 0; ch < p.bn / 16; ++ch) {
+                const int co0 = n0 + ch * 16;
+                if (co0 >= p.c_out) break;          // uniform across the CTA
+                int v[16];
+                tmem_ld16(t_addr + ch * 16, v);
+                tmem_ld_wait();
+                epilogue_chunk(p, v, row, co0, row_valid);
+            }
+            tc_fence_before();
+            mbar_arrive(tempty_bar + 8 * acc);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ----------------------------------------------------------------------------- MMA-only probe
+
+__global__ void __launch_bounds__(NUM_THREADS, 1) f8_mma_probe_kernel(int iters, int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // 128 x 128 A and 256 x 128 B int8 tiles; the values do not matter for a rate measurement
+    for (int i = threadIdx.x; i < (128 + 256) * 128 / 4; i += blockDim.x) ((uint32_t *)smem)[i] = 0x01010101u * (i & 3);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    if (warp == 1 && lane == 0) {
+        const uint32_t a_addr = smem_u32(smem), b_addr = a_addr + 128 * 128;
+        const uint64_t hi = smem_desc_hi(128);
+        const uint64_t a_desc = hi | (uint64_t)((a_addr & 0x3ffffu) >> 4);
+        const uint64_t b_desc = hi | (uint64_t)((b_addr & 0x3ffffu) >> 4);
+        // u8 x s8 -> s32, M 128, N 256
+        const uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+        for (int i = 0; i < iters; ++i)
+            mma_i8(tmem_base + (i & 1) * 256, a_desc + 2 * (i & 3), b_desc + 2 * (i & 3), idesc, i > 1 ? 1u : 0u);
+        mma_commit(smem_u32(&bar));
+        mbar_wait(smem_u32(&bar), 0, &abort_flag, status, 105);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ----------------------------------------------------------------------------- host side
+
+PFN_cuTensorMapEncodeTiled_v12000 g_encode_tiled = nullptr;
+PFN_cuTensorMapEncodeIm2col_v12000 g_encode_im2col = nullptr;
+
+bool load_driver_entry_points() {
+    if (g_encode_tiled && g_encode_im2col) return true;
+    void *f = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qr) != cudaSuccess || !f ||
+        qr != cudaDriverEntryPointSuccess)
+        return false;
+    g_encode_tiled = (PFN_cuTensorMapEncodeTiled_v12000)f;
+    f = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &qr) != cudaSuccess || !f ||
+        qr != cudaDriverEntryPointSuccess)
+        return false;
+    g_encode_im2col = (PFN_cuTensorMapEncodeIm2col_v12000)f;
+    return true;
+}
+
+int choose_kb(int c) { return c >= 96 ? 128 : (c >= 48 ? 64 : 32); }
+
+int choose_bn(int c_out) {
+    if (c_out >= 256) return 256;
+    return (c_out + 15) / 16 * 16;
+}
+
+CUtensorMapSwizzle swizzle_for(int kb) {
+    return kb == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (kb == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+
+}   // namespace
+
+struct F8TcPlan {
+    CUtensorMap map_a;
+    CUtensorMap map_b;
+    TcParams p;
+    int grid;
+    size_t smem;
+};
+
+size_t f8_tc_plan_size() { return sizeof(F8TcPlan); }
+
+bool f8_tc_supported(const F8ConvGeom &g, size_t x_bytes) {
+    if (g.c % 16 != 0) return false;                 // TMA strides are multiples of 16 bytes
+    if (x_bytes < 128 * 1024) return false;          // tiny tensors: latency bound, CUDA-core kernel
+    if (g.kh > 255 || g.kw > 255) return false;
+    if ((long long)g.n * g.ho * g.wo > 0x7fffff00ll) return false;
+    return true;
+}
+
+cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant &q, const F8TcTensorView &xv,
+                            const int8_t *w, const int32_t *bias, const void *res, void *y, int *status_word,
+                            const char **why) {
+    *why = "";
+    if (!load_driver_entry_points()) {
+        *why = "cuTensorMapEncode entry points not available";
+        return cudaErrorNotSupported;
+    }
+    memset(plan, 0, sizeof(*plan));
+    TcParams &p = plan->p;
+    p.M = g.n * g.ho * g.wo;
+    p.ho = g.ho;
+    p.wo = g.wo;
+    p.c_out = g.c_out;
+    p.kh = g.kh;
+    p.kw = g.kw;
+    p.stride_h = g.stride_h;
+    p.stride_w = g.stride_w;
+    p.pad_h = g.pad_h;
+    p.pad_w = g.pad_w;
+    p.kb = choose_kb(g.c);
+    p.c_chunks = (g.c + p.kb - 1) / p.kb;
+    p.bn = choose_bn(g.c_out);
+    p.m_tiles = (p.M + TILE_M - 1) / TILE_M;
+    p.n_tiles = (g.c_out + p.bn - 1) / p.bn;
+    p.a_bytes = (uint32_t)(TILE_M * p.kb + 1023) / 1024 * 1024;
+    const uint32_t b_bytes = (uint32_t)(p.bn * p.kb + 1023) / 1024 * 1024;
+    p.stage_bytes = p.a_bytes + b_bytes;
+    p.tx_bytes = (uint32_t)((TILE_M + p.bn) * p.kb);
+    int stages = (int)(SMEM_BUDGET / p.stage_bytes);
+    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    if (stages < 2) {
+        *why = "stage does not fit";
+        return cudaErrorInvalidValue;
+    }
+    p.stages = stages;
+    // instruction descriptor: D = s32 (2 at bit 4), A format at bit 7 (0 = u8, 1 = s8), B = s8 at bit 10,
+    // both operands K-major, N/8 at bit 17, M/16 at bit 24
+    p.idesc = (2u << 4) | ((g.x_signed ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) |
+              ((uint32_t)(TILE_M >> 4) << 24);
+    p.desc_hi = smem_desc_hi(p.kb);
+    p.bias = bias;
+    p.res = (const uint8_t *)res;
+    p.y = (uint8_t *)y;
+    p.q = q;
+    p.status = status_word;
+    const int ysz = q.y_kind == F8_S32 ? 4 : 1;
+    const size_t row_bytes = (size_t)g.c_out * ysz;
+    p.vec_bytes = (row_bytes % 16 == 0) ? 16 : (row_bytes % 8 == 0 ? 8 : (row_bytes % 4 == 0 ? 4 : 1));
+
+    // A: activation tensor (C, W, H, N) in im2col mode.  Corners follow the usual forward-convolution
+    // rule: lower = -pad, upper = pad - (k - 1); the traversal stride is the convolution stride.
+    {
+        cuuint64_t dims[4] = {xv.dim_c, xv.dim_w, xv.dim_h, xv.dim_n};
+        cuuint64_t strides[3] = {xv.stride_w, xv.stride_h, xv.stride_n};
+        int lower[2] = {-g.pad_w, -g.pad_h};
+        int upper[2] = {g.pad_w - (g.kw - 1), g.pad_h - (g.kh - 1)};
+        cuuint32_t estr[4] = {1, (cuuint32_t)g.stride_w, (cuuint32_t)g.stride_h, 1};
+        CUresult r = g_encode_im2col(&plan->map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(xv.base), dims,
+                                     strides, lower, upper, (cuuint32_t)p.kb, (cuuint32_t)TILE_M, estr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(p.kb), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            *why = "cuTensorMapEncodeIm2col rejected the activation tensor";
+            return cudaErrorInvalidValue;
+        }
+    }
+    // B: weights (C, taps, C_out), box (kb, 1, bn)
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)g.c, (cuuint64_t)(g.kh * g.kw), (cuuint64_t)g.c_out};
+        cuuint64_t strides[2] = {(cuuint64_t)g.c, (cuuint64_t)g.c * g.kh * g.kw};
+        cuuint32_t box[3] = {(cuuint32_t)p.kb, 1, (cuuint32_t)p.bn};
+        cuuint32_t estr[3] = {1, 1, 1};
+        CUresult r = g_encode_tiled(&plan->map_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t *>(w), dims,
+                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(p.kb),
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            *why = "cuTensorMapEncodeTiled rejected the weight tensor";
+            return cudaErrorInvalidValue;
+        }
+    }
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    plan->grid = total_tiles < sms ? total_tiles : sms;
+    // at least half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
+    plan->smem = (size_t)p.stages * p.stage_bytes + 1024;
+    if (plan->smem < 120 * 1024) plan->smem = 120 * 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(SMEM_BUDGET + 2048));
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    return cudaSuccess;
+}
+
+cudaError_t f8_tc_launch(const F8TcPlan *plan, cudaStream_t st) {
+    if (plan->p.M == 0) return cudaSuccess;
+    f8_conv_gemm_tc_kernel<<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p);
+    return cudaGetLastError();
+}
+
+cudaError_t f8_tc_probe(int iters, double *ops, int *status_word, cudaStream_t st) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const size_t smem = 120 * 1024;
+    cudaError_t e = cudaFuncSetAttribute(f8_mma_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    f8_mma_probe_kernel<<<sms, NUM_THREADS, smem, st>>>(iters, status_word);
+    *ops = 2.0 * 128 * 256 * 32 * (double)iters * sms;
+    return cudaGetLastError();
+}

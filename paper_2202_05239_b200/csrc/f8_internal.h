@@ -1,0 +1,68 @@
+// Internal declarations shared by the CUDA sources of the library (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/f8net.h"
+
+// How an int32 accumulator becomes an output element: bias has already been added.
+//   v = has_res ? (acc << sh_acc) + (r << sh_res) : acc
+//   y_kind 2: store v as int32
+//   else    : t = s > 0 ? rounding right shift of v by s : v << -s ; y = clamp(t, lo, hi)
+struct F8Requant {
+    int sh_acc;     // F - (fl_x + fl_w), F = max(fl_x + fl_w, fl_r)   (0 without residual)
+    int sh_res;     // F - fl_r
+    int s;          // F - fl_y   in [-8, 31]
+    int lo, hi;     // clip bounds of the output quantizer
+    int y_kind;     // F8_U8 / F8_S8 / F8_S32
+    int has_res;
+    int r_signed;
+};
+
+// Geometry of one convolution-shaped launch (dense or depthwise).
+struct F8ConvGeom {
+    int n, h, w, c;         // input
+    int ho, wo, c_out;      // output
+    int kh, kw;
+    int stride_h, stride_w;
+    int pad_h, pad_w;
+    int x_signed;
+};
+
+// ---- CUDA-core kernels (f8_direct.cu) -------------------------------------------------
+cudaError_t f8_launch_conv_direct(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
+                                  const int32_t *bias, const void *res, void *y, cudaStream_t st);
+cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
+                             const int32_t *bias, const void *res, void *y, cudaStream_t st);
+cudaError_t f8_launch_maxpool(int n, int h, int w, int c, int k, int stride, int pad, int x_signed,
+                              const void *x, void *y, cudaStream_t st);
+cudaError_t f8_launch_gap(int n, int h, int w, int c, int x_signed, int s, const void *x, void *y,
+                          cudaStream_t st);
+// channel-padding pre-pass for 3-channel stems: [n,h,w,c] -> [n,h,wp,8] with `left` zero pixels in front
+cudaError_t f8_launch_pack_stem(int n, int h, int w, int c, int wp, int left, const void *x, void *y,
+                                cudaStream_t st);
+
+// ---- tensor-core implicit GEMM (f8_gemm_tc.cu) ----------------------------------------
+struct F8TcPlan;   // opaque: tensor maps + launch parameters of one conv launch
+
+// Activation tensor as the TMA sees it: extents and byte strides of (C, W, H, N).
+struct F8TcTensorView {
+    const void *base;
+    uint64_t dim_c, dim_w, dim_h, dim_n;
+    uint64_t stride_w, stride_h, stride_n;   // bytes (stride of C is 1)
+};
+
+// True when this geometry can run on the tensor-core path.
+bool f8_tc_supported(const F8ConvGeom &g, size_t x_bytes);
+size_t f8_tc_plan_size();
+// Encodes tensor maps and tile schedule; returns cudaSuccess or an error (no launch).
+cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant &q, const F8TcTensorView &xv,
+                            const int8_t *w /* [c_out][kh][kw][g.c] */, const int32_t *bias, const void *res,
+                            void *y, int *status_word, const char **why);
+cudaError_t f8_tc_launch(const F8TcPlan *plan, cudaStream_t st);
+cudaError_t f8_tc_probe(int iters, double *ops, int *status_word, cudaStream_t st);
+
+// Device status word (0 = fine); allocated once per process on first use.
+int *f8_status_word();

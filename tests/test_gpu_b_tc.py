@@ -1,0 +1,79 @@
+"""GPU parity (bit-exact) of the tensor-core implicit-GEMM path (tcgen05.mma kind::i8 + TMA im2col)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2202_05239_b200 import synth
+from gpu_util import api, check_layer, random_conv_layer, random_input, random_residual
+
+pytestmark = pytest.mark.gpu
+
+
+def test_tensor_core_probe_runs():
+    a = api()
+    ops = a.f8_mma_i8_probe(64)
+    torch.cuda.synchronize()
+    a.f8_device_status()
+    assert ops == 2.0 * 128 * 256 * 32 * 64 * torch.cuda.get_device_properties(0).multi_processor_count
+
+
+# (h, w, c, c_out, k, stride, pad, n, x_signed, y_dtype, res)
+TC_CASES = [
+    (56, 56, 64, 64, 1, 1, 0, 1, False, synth.U8, False),      # plain GEMM, one K chunk (64-byte swizzle)
+    (28, 28, 128, 128, 1, 1, 0, 2, False, synth.U8, True),     # 128-byte swizzle + residual
+    (28, 28, 256, 64, 1, 1, 0, 1, True, synth.S8, False),      # two K chunks, signed in / out
+    (14, 14, 1024, 256, 1, 1, 0, 3, False, synth.U8, False),   # 8 K chunks, ragged M (588 pixels)
+    (56, 56, 64, 64, 3, 1, 1, 1, False, synth.U8, False),      # 3x3 halo through im2col
+    (28, 28, 128, 128, 3, 2, 1, 2, False, synth.U8, True),     # 3x3 stride 2
+    (56, 56, 256, 512, 1, 2, 0, 1, False, synth.S8, False),    # 1x1 stride 2 (downsample), two N tiles
+    (15, 17, 32, 48, 3, 1, 1, 17, True, synth.U8, False),       # odd sizes, 32-byte swizzle, N tile 48
+    (9, 9, 144, 24, 1, 1, 0, 13, False, synth.S8, True),       # c = 144 (ragged K chunk), c_out = 24
+    (12, 12, 96, 576, 1, 1, 0, 10, True, synth.U8, False),     # three N tiles with a ragged last one
+    (7, 7, 512, 512, 3, 1, 1, 6, False, synth.U8, False),      # 36 K iterations, tiles span several images
+    (8, 8, 2048, 1000, 1, 1, 0, 2, False, synth.S32, False),   # int32 output, ragged N
+    (33, 20, 16, 96, 1, 1, 0, 13, True, synth.U8, False),      # c = 16: half-empty 32-byte K chunk
+    (20, 20, 64, 32, 5, 1, 2, 6, False, synth.U8, False),      # 5x5
+    (31, 31, 64, 64, 3, 2, 0, 3, False, synth.U8, False),      # stride 2 without padding
+]
+
+
+@pytest.mark.parametrize("case", range(len(TC_CASES)))
+def test_tensor_core_conv(ref, case):
+    h, w, c, c_out, k, stride, pad, n, xs, y_dtype, with_res = TC_CASES[case]
+    rng = np.random.default_rng(300 + case)
+    layer = random_conv_layer(rng, h=h, w=w, c=c, c_out=c_out, k=k, stride=stride, pad=pad, x_signed=xs, y_dtype=y_dtype,
+                              with_res=with_res)
+    x = random_input(rng, n, layer)
+    assert x.size >= 128 * 1024, "case must be large enough for the tensor-core path"
+    res = random_residual(rng, n, layer) if with_res else None
+    check_layer(ref, layer, x, res, expect_tc=True)
+
+
+def test_extreme_operands_on_tensor_cores(ref):
+    """-128 weights against 255 / -128 activations: the signedness selection of the MMA must be right."""
+    rng = np.random.default_rng(5)
+    for xs in (False, True):
+        layer = random_conv_layer(rng, h=32, w=32, c=128, c_out=64, k=1, stride=1, pad=0, x_signed=xs, y_dtype=synth.S32,
+                                  with_res=False, wide=True)
+        layer.weight[:] = -128
+        layer.weight[1::2] = 127
+        x = random_input(rng, 1, layer)
+        x[:] = -128 if xs else 255
+        check_layer(ref, layer, x, expect_tc=True)
+
+
+@pytest.mark.parametrize("index", range(6))
+def test_layer_sweep_shapes(ref, index):
+    """The CNN layer-shape sweep at a batch the oracle finishes in seconds."""
+    layer, x = synth.sweep_case(index, batch=6, seed=0)
+    check_layer(ref, layer, x, expect_tc=True)
+
+
+def test_linear_on_tensor_cores(ref):
+    rng = np.random.default_rng(11)
+    n, k, out = 256, 2048, 1000
+    wgt = np.clip(np.round(rng.normal(0, 20, size=(out, k))), -128, 127).astype(np.int8)
+    bias = rng.integers(-5000, 5000, size=out).astype(np.int32)
+    layer = synth.Layer(synth.LINEAR, "fc", 0, -1, 1, 1, k, out, 1, 1, 1, 0, synth.U8, synth.S32, synth.U8, 6, 9, 3, 0, wgt, bias)
+    x = rng.integers(0, 256, size=(n, k)).astype(np.uint8)
+    check_layer(ref, layer, x, expect_tc=True)

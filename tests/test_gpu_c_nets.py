@@ -1,0 +1,84 @@
+"""Whole-network parity through f8_net_forward: every layer's output equals the oracle's, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2202_05239_b200 import synth
+from gpu_util import api
+
+pytestmark = pytest.mark.gpu
+
+
+def _compare_net(ref, name, batch, image, force_direct=False, seed=0):
+    a = api()
+    layers = synth.make_net(name, seed, image=image)
+    x = synth.draw_image(batch, seed + 1, image, image)
+    want = ref.net_forward(layers, x)
+    a.f8_debug_force_direct(force_direct)
+    before = a.f8_tc_launch_count()
+    try:
+        net = a.Net(layers, batch)
+        dump = [net.layer_output(i, batch) for i in range(len(layers))]
+        out = net.forward(a.to_device(x), dump=dump)
+        torch.cuda.synchronize()
+        a.f8_device_status()
+    finally:
+        a.f8_debug_force_direct(False)
+    for i, l in enumerate(layers):
+        got = dump[i].cpu().numpy().reshape(want[i + 1].shape)
+        bad = int((got != want[i + 1]).sum())
+        assert bad == 0, f"{name} layer {i} ({l.name}): {bad} of {got.size} elements differ"
+    assert np.array_equal(out.cpu().numpy(), want[-1])
+    assert net.last_launch_count >= len(layers)
+    tc = a.f8_tc_launch_count() - before
+    if force_direct:
+        assert tc == 0
+    elif image == 224:
+        # every dense layer whose input is at least 128 KiB and has c % 16 == 0 (or is a packed stem)
+        assert tc >= sum(1 for l in layers if l.kind == synth.CONV and l.c % 16 == 0 and batch * l.h * l.w * l.c >= 131072)
+    net.close()
+
+
+@pytest.mark.parametrize("name", ["resnet18", "resnet50", "mobilenetv2"])
+def test_net_parity_cuda_core_path(ref, name):
+    _compare_net(ref, name, 2, 64, force_direct=True)
+
+
+@pytest.mark.parametrize("name,batch,image", [("resnet18", 3, 224), ("resnet50", 2, 224), ("mobilenetv2", 3, 224),
+                                              ("resnet50", 1, 224), ("resnet18", 5, 96)])
+def test_net_parity(ref, name, batch, image):
+    _compare_net(ref, name, batch, image)
+
+
+def test_resnet50_full_batch_sampled_images(ref):
+    """The benchmark configuration (batch 256): images are independent, so the oracle checks a sample of
+    them one by one against the logits of the full-batch launch."""
+    a = api()
+    batch = 256
+    layers = synth.make_net("resnet50", 0)
+    x = synth.draw_image(batch, 1)
+    net = a.Net(layers, batch)
+    out = net.forward(a.to_device(x))
+    torch.cuda.synchronize()
+    a.f8_device_status()
+    got = out.cpu().numpy()
+    for i in (0, 77, 128, 255):
+        want = ref.net_forward(layers, x[i:i + 1], keep_all=False)[-1]
+        assert np.array_equal(got[i:i + 1], want), f"image {i}"
+    # a second pass over the same buffers gives the same bits (no state leaks between calls)
+    out2 = net.forward(a.to_device(x))
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    net.close()
+
+
+def test_workspace_too_small_is_rejected():
+    a = api()
+    layers = synth.make_net("resnet18", 0, image=64)
+    net = a.Net(layers, 2)
+    x = a.to_device(synth.draw_image(2, 0, 64, 64))
+    ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(a.F8Error) as e:
+        net.forward(x, workspace=ws)
+    assert e.value.status == 8
+    net.close()
