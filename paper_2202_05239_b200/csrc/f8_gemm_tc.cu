@@ -7,7 +7,7 @@
 //     shared memory in the swizzled K-major layout tcgen05.mma reads.
 //   * One thread issues tcgen05.mma.kind::i8 (u8|s8 x s8 -> s32); the 128 x BN int32 accumulator lives
 //     in tensor memory, double buffered so the epilogue of tile i overlaps the main loop of tile i+1.
-//   * Four epilogue warps read the accumulator with tcgen05.ld (one output pixel per thread, 16
+//   * Eight epilogue warps read the accumulator with tcgen05.ld (one output pixel per thread, 16
 //     consecutive channels per load), add the bias, align and add the residual, apply the rounding
 //     shift and clip (Eq. 2 / signed form applied to Eq. 6) and store 16 output bytes per instruction.
 //   * Persistent CTAs (one per SM) walk the tile list; tiles that share an A tile are adjacent so that
@@ -25,7 +25,8 @@
 namespace {
 
 constexpr int TILE_M = 128;
-constexpr int NUM_THREADS = 192;           // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr int NUM_EPI_WARPS = 8;           // two warps per TMEM lane quarter, each takes half of the columns
+constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;   // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
 constexpr int MAX_STAGES = 8;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
@@ -52,6 +53,7 @@ struct TcParams {
     const uint8_t *res;
     uint8_t *y;
     int vec_bytes;            // widest aligned store the output rows allow: 16, 8, 4 or 1
+    int fast;                 // 1: 8-bit output, shift >= 1, c_out % 16 == 0 -> branch-free epilogue
     F8Requant q;
     int *status;
 };
@@ -214,6 +216,42 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int (&ac
     }
 }
 
+// Branch-free epilogue for the common case (8-bit output, shift s >= 1, c_out % 16 == 0).
+//   v = acc * 2^sh_acc + bias'          bias' = bias << sh_acc, staged in shared memory
+//   v += r << sh_res                    (RES only)
+//   t = ((v >> (s-1)) + 1) >> 1         = floor((v + 2^(s-1)) / 2^s); cannot overflow because |v| < 2^31 - 1
+//   y = clamp(t, lo, hi)
+template <bool RES>
+__device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], const int4 *bias4, uint4 rw, int mul_acc,
+                                                 int mul_res, int r_signed, int sm1, int lo, int hi) {
+    int t[16];
+    const uint32_t rwords[4] = {rw.x, rw.y, rw.z, rw.w};
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const int4 b = bias4[g];
+        const int bb[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int j = 4 * g + k;
+            int v = acc[j] * mul_acc + bb[k];
+            if (RES) {
+                int r;
+                if (r_signed) asm("bfe.s32 %0, %1, %2, 8;" : "=r"(r) : "r"(rwords[g]), "r"(8 * k));
+                else asm("bfe.u32 %0, %1, %2, 8;" : "=r"(r) : "r"(rwords[g]), "r"(8 * k));
+                v += r * mul_res;
+            }
+            const int u = ((v >> sm1) + 1) >> 1;
+            t[j] = min(max(u, lo), hi);
+        }
+    }
+    uint4 o;
+    o.x = __byte_perm(__byte_perm(t[0], t[1], 0x0040), __byte_perm(t[2], t[3], 0x0040), 0x5410);
+    o.y = __byte_perm(__byte_perm(t[4], t[5], 0x0040), __byte_perm(t[6], t[7], 0x0040), 0x5410);
+    o.z = __byte_perm(__byte_perm(t[8], t[9], 0x0040), __byte_perm(t[10], t[11], 0x0040), 0x5410);
+    o.w = __byte_perm(__byte_perm(t[12], t[13], 0x0040), __byte_perm(t[14], t[15], 0x0040), 0x5410);
+    return o;
+}
+
 // ----------------------------------------------------------------------------- the kernel
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -225,6 +263,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ __align__(16) int bias_stage[NUM_EPI_WARPS][128];   // per warp: bias of its columns, pre-shifted
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -242,7 +281,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
-            mbar_init(tempty_bar + 8 * a, 128);
+            mbar_init(tempty_bar + 8 * a, 32 * NUM_EPI_WARPS);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -347,27 +386,63 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------------ epilogue (warps 2..9)
         const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 belong to this warp
+        const int ew = warp - 2;
+        const int half = ew >> 2;                   // which half of the tile's columns this warp converts
+        const int chunks = p.bn / 16;
+        const int ch_begin = half == 0 ? 0 : (chunks + 1) / 2;
+        const int ch_end = half == 0 ? (chunks + 1) / 2 : chunks;
+        int *bias_w = bias_stage[ew];
+        const int mul_acc = 1 << p.q.sh_acc, mul_res = 1 << p.q.sh_res;
         int local = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
             const int acc = local & 1;
             const uint32_t acc_phase = (local >> 1) & 1;
             const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+            const int n0 = n_t * p.bn;
+            if (p.fast) {
+                // bias of this warp's columns -> shared memory (4 values per lane), before the accumulator is ready
+                __syncwarp();
+                const int c0 = n0 + ch_begin * 16 + lane * 4;
+                int4 b = make_int4(0, 0, 0, 0);
+                if (p.bias && lane * 4 < (ch_end - ch_begin) * 16 && c0 < p.c_out) b = __ldg((const int4 *)(p.bias + c0));
+                b.x <<= p.q.sh_acc; b.y <<= p.q.sh_acc; b.z <<= p.q.sh_acc; b.w <<= p.q.sh_acc;
+                *(int4 *)(bias_w + lane * 4) = b;
+                __syncwarp();
+            }
             if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104)) { ok = false; break; }
             tc_fence_after();
             const size_t row = (size_t)m_t * TILE_M + quarter * 32 + lane;
             const bool row_valid = row < (size_t)p.M;
             const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256;
-            const int n0 = n_t * p.bn;
-            for (int ch = 0; ch < p.bn / 16; ++ch) {
-                const int co0 = n0 + ch * 16;
-                if (co0 >= p.c_out) break;          // uniform across the CTA
-                int v[16];
-                tmem_ld16(t_addr + ch * 16, v);
-                tmem_ld_wait();
-                epilogue_chunk(p, v, row, co0, row_valid);
+            if (p.fast) {
+                const size_t o = row * (size_t)p.c_out + n0;
+                for (int ch = ch_begin; ch < ch_end; ++ch) {
+                    if (n0 + ch * 16 >= p.c_out) break;          // uniform across the CTA
+                    uint4 rw = make_uint4(0, 0, 0, 0);
+                    if (p.q.has_res && row_valid) rw = *(const uint4 *)(p.res + o + ch * 16);
+                    int v[16];
+                    tmem_ld16(t_addr + ch * 16, v);
+                    tmem_ld_wait();
+                    const int4 *b4 = (const int4 *)(bias_w + (ch - ch_begin) * 16);
+                    uint4 out;
+                    if (p.q.has_res)
+                        out = epilogue_fast16<true>(v, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s - 1, p.q.lo, p.q.hi);
+                    else
+                        out = epilogue_fast16<false>(v, b4, rw, 1, 0, 0, p.q.s - 1, p.q.lo, p.q.hi);
+                    if (row_valid) *(uint4 *)(p.y + o + ch * 16) = out;
+                }
+            } else {
+                for (int ch = ch_begin; ch < ch_end; ++ch) {
+                    const int co0 = n0 + ch * 16;
+                    if (co0 >= p.c_out) break;                   // uniform across the CTA
+                    int v[16];
+                    tmem_ld16(t_addr + ch * 16, v);
+                    tmem_ld_wait();
+                    epilogue_chunk(p, v, row, co0, row_valid);
+                }
             }
             tc_fence_before();
             mbar_arrive(tempty_bar + 8 * acc);
@@ -524,6 +599,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.status = status_word;
     const int ysz = q.y_kind == F8_S32 ? 4 : 1;
     const size_t row_bytes = (size_t)g.c_out * ysz;
+    p.fast = (q.y_kind != F8_S32 && q.s >= 1 && g.c_out % 16 == 0) ? 1 : 0;
     p.vec_bytes = (row_bytes % 16 == 0) ? 16 : (row_bytes % 8 == 0 ? 8 : (row_bytes % 4 == 0 ? 4 : 1));
 
     // A: activation tensor (C, W, H, N) in im2col mode.  Corners follow the usual forward-convolution

@@ -1,0 +1,103 @@
+"""Single-layer micro-benchmark: times one fixed-point conv layer through the C ABI.
+
+    python -m paper_2202_05239_b200.layer_bench --sweep            # the six CNN layer shapes at batch 32
+    python -m paper_2202_05239_b200.layer_bench --h 56 --w 56 --c 64 --c-out 256 --k 1 --batch 32 --res
+
+Each layer is run over several copies of its tensors, rotated so that consecutive launches do not find
+their operands in L2 (the copies together exceed twice the L2 size).  Prints one JSON line per layer:
+device time per launch (CUDA events), int8 TOPS and algorithmic GB/s.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+
+import numpy as np
+import torch
+
+from . import api, synth
+
+
+def bench_layer(layer: synth.Layer, batch: int, with_res: bool, iters: int, warmup: int, cold: bool = True):
+    rng = np.random.default_rng(0)
+    x_bytes = batch * layer.h * layer.w * layer.c
+    y_elems = batch * layer.ho * layer.wo * layer.c_out
+    per_set = x_bytes + y_elems * (2 if with_res else 1)
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    sets = max(2, math.ceil(2.2 * l2 / per_set)) if cold else 1
+    sets = min(sets, 64)
+    w = api.to_device(layer.weight)
+    b = api.to_device(layer.bias)
+    xs, rs, ys = [], [], []
+    for _ in range(sets):
+        if layer.x_dtype == synth.S8:
+            x = rng.integers(-128, 128, size=(batch, layer.h, layer.w, layer.c), dtype=np.int64).astype(np.int8)
+        else:
+            x = rng.integers(0, 256, size=(batch, layer.h, layer.w, layer.c), dtype=np.int64).astype(np.uint8)
+        xs.append(api.to_device(x))
+        rs.append(torch.randint(0, 255, (batch, layer.ho, layer.wo, layer.c_out), dtype=torch.uint8, device="cuda")
+                  if with_res else None)
+        ys.append(torch.empty((batch, layer.ho, layer.wo, layer.c_out), dtype=api.torch_dtype(layer.y_dtype),
+                              device="cuda"))
+    desc = api.conv_desc(layer, batch)
+    fn = api.f8_dwconv_fixed if layer.kind == synth.DWCONV else api.f8_conv2d_fixed
+    for i in range(warmup):
+        fn(desc, xs[i % sets], w, b, rs[i % sets], ys[i % sets])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        fn(desc, xs[i % sets], w, b, rs[i % sets], ys[i % sets])
+    e1.record()
+    torch.cuda.synchronize()
+    api.f8_device_status()
+    ms = e0.elapsed_time(e1) / iters
+    macs = batch * layer.macs_per_image
+    ysz = 4 if layer.y_dtype == synth.S32 else 1
+    byts = x_bytes + y_elems * ysz + (y_elems if with_res else 0) + layer.param_bytes()
+    return {"layer": layer.name, "batch": batch, "ms": ms, "tops": 2 * macs / (ms * 1e-3) / 1e12,
+            "gbs": byts / (ms * 1e-3) / 1e9, "macs": macs, "bytes": byts, "buffer_sets": sets}
+
+
+def custom_layer(args) -> synth.Layer:
+    rng = np.random.default_rng(1)
+    depthwise = args.depthwise
+    fan_in = args.k * args.k * (1 if depthwise else args.c)
+    shape = (args.c, args.k, args.k) if depthwise else (args.c_out, args.k, args.k, args.c)
+    wgt, flw = synth.draw_weight(rng, shape, math.sqrt(2.0 / fan_in))
+    bias = synth.draw_bias(rng, args.c_out, 5 + flw)
+    return synth.Layer(synth.DWCONV if depthwise else synth.CONV, f"c{args.k}x{args.k}_{args.h}_{args.c}_{args.c_out}", 0,
+                       1 if args.res else -1, args.h, args.w or args.h, args.c, args.c_out, args.k, args.k, args.stride,
+                       args.k // 2, synth.U8, synth.U8, synth.U8, 5, flw, 5, 5, wgt, bias)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--h", type=int, default=56)
+    ap.add_argument("--w", type=int, default=0)
+    ap.add_argument("--c", type=int, default=64)
+    ap.add_argument("--c-out", type=int, default=64)
+    ap.add_argument("--k", type=int, default=3)
+    ap.add_argument("--stride", type=int, default=1)
+    ap.add_argument("--batch", type=int, default=32)
+    ap.add_argument("--res", action="store_true")
+    ap.add_argument("--depthwise", action="store_true")
+    ap.add_argument("--iters", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--warm-l2", action="store_true", help="reuse one buffer set (operands stay in L2)")
+    args = ap.parse_args()
+    if args.sweep:
+        for i in range(len(synth.SWEEP_SHAPES)):
+            layer, _ = synth.sweep_case(i, batch=1)
+            print(json.dumps(bench_layer(layer, args.batch, False, args.iters, args.warmup, not args.warm_l2)), flush=True)
+    else:
+        if args.depthwise:
+            args.c_out = args.c
+        print(json.dumps(bench_layer(custom_layer(args), args.batch, args.res, args.iters, args.warmup, not args.warm_l2)),
+              flush=True)
+
+
+if __name__ == "__main__":
+    main()
