@@ -7,7 +7,7 @@
 //     shared memory in the swizzled K-major layout tcgen05.mma reads.
 //   * One thread issues tcgen05.mma.kind::i8 (u8|s8 x s8 -> s32); the 128 x BN int32 accumulator lives
 //     in tensor memory, double buffered so the epilogue of tile i overlaps the main loop of tile i+1.
-//   * Eight epilogue warps read the accumulator with tcgen05.ld (one output pixel per thread, 16
+//   * Sixteen epilogue warps read the accumulator with tcgen05.ld (one output pixel per thread, 16
 //     consecutive channels per load), add the bias, align and add the residual, apply the rounding
 //     shift and clip (Eq. 2 / signed form applied to Eq. 6) and store 16 output bytes per instruction.
 //   * Persistent CTAs (one per SM) walk the tile list; tiles that share an A tile are adjacent so that
@@ -25,8 +25,8 @@
 namespace {
 
 constexpr int TILE_M = 128;
-constexpr int NUM_EPI_WARPS = 8;           // two warps per TMEM lane quarter, each takes half of the columns
-constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;   // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
+constexpr int NUM_EPI_WARPS = 16;          // four warps per TMEM lane quarter, each takes a quarter of the columns
+constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;   // warp 0: TMA, warp 1: MMA, warps 2-17: epilogue
 constexpr int MAX_STAGES = 8;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
@@ -263,7 +263,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
-    __shared__ __align__(16) int bias_stage[NUM_EPI_WARPS][128];   // per warp: bias of its columns, pre-shifted
+    __shared__ __align__(16) int bias_stage[NUM_EPI_WARPS][64];   // per warp: bias of its columns, pre-shifted
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -386,13 +386,14 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..9)
+        // ------------------------------------------------------------------ epilogue (warps 2..17)
         const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 belong to this warp
         const int ew = warp - 2;
-        const int half = ew >> 2;                   // which half of the tile's columns this warp converts
+        const int group = ew >> 2;                  // which quarter of the tile's columns this warp converts
         const int chunks = p.bn / 16;
-        const int ch_begin = half == 0 ? 0 : (chunks + 1) / 2;
-        const int ch_end = half == 0 ? (chunks + 1) / 2 : chunks;
+        const int per_group = (chunks + 3) / 4;     // <= 4 chunks of 16 columns per warp
+        const int ch_begin = min(group * per_group, chunks);
+        const int nch = min(ch_begin + per_group, chunks) - ch_begin;
         int *bias_w = bias_stage[ew];
         const int mul_acc = 1 << p.q.sh_acc, mul_res = 1 << p.q.sh_res;
         int local = 0;
@@ -402,44 +403,67 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const uint32_t acc_phase = (local >> 1) & 1;
             const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
             const int n0 = n_t * p.bn;
-            if (p.fast) {
-                // bias of this warp's columns -> shared memory (4 values per lane), before the accumulator is ready
-                __syncwarp();
-                const int c0 = n0 + ch_begin * 16 + lane * 4;
-                int4 b = make_int4(0, 0, 0, 0);
-                if (p.bias && lane * 4 < (ch_end - ch_begin) * 16 && c0 < p.c_out) b = __ldg((const int4 *)(p.bias + c0));
-                b.x <<= p.q.sh_acc; b.y <<= p.q.sh_acc; b.z <<= p.q.sh_acc; b.w <<= p.q.sh_acc;
-                *(int4 *)(bias_w + lane * 4) = b;
-                __syncwarp();
-            }
-            if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104)) { ok = false; break; }
-            tc_fence_after();
             const size_t row = (size_t)m_t * TILE_M + quarter * 32 + lane;
             const bool row_valid = row < (size_t)p.M;
-            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
             if (p.fast) {
-                const size_t o = row * (size_t)p.c_out + n0;
-                for (int ch = ch_begin; ch < ch_end; ++ch) {
-                    if (n0 + ch * 16 >= p.c_out) break;          // uniform across the CTA
-                    uint4 rw = make_uint4(0, 0, 0, 0);
-                    if (p.q.has_res && row_valid) rw = *(const uint4 *)(p.res + o + ch * 16);
-                    int v[16];
-                    tmem_ld16(t_addr + ch * 16, v);
-                    tmem_ld_wait();
-                    const int4 *b4 = (const int4 *)(bias_w + (ch - ch_begin) * 16);
-                    uint4 out;
-                    if (p.q.has_res)
-                        out = epilogue_fast16<true>(v, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s - 1, p.q.lo, p.q.hi);
-                    else
-                        out = epilogue_fast16<false>(v, b4, rw, 1, 0, 0, p.q.s - 1, p.q.lo, p.q.hi);
-                    if (row_valid) *(uint4 *)(p.y + o + ch * 16) = out;
+                // everything that does not depend on the accumulator is fetched before waiting for it:
+                // the bias of this warp's columns (to shared memory) and this thread's residual bytes
+                const int c_first = n0 + ch_begin * 16;
+                const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
+                __syncwarp();
+                if (lane < 16) {
+                    const int c0 = c_first + lane * 4;
+                    int4 b = make_int4(0, 0, 0, 0);
+                    if (p.bias && lane * 4 < my_nch * 16) b = __ldg((const int4 *)(p.bias + c0));
+                    b.x <<= p.q.sh_acc; b.y <<= p.q.sh_acc; b.z <<= p.q.sh_acc; b.w <<= p.q.sh_acc;
+                    *(int4 *)(bias_w + lane * 4) = b;
+                }
+                const size_t o = row * (size_t)p.c_out + c_first;
+                uint4 rw[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    rw[i] = make_uint4(0, 0, 0, 0);
+                    if (p.q.has_res && row_valid && i < my_nch) rw[i] = __ldg((const uint4 *)(p.res + o + i * 16));
+                }
+                __syncwarp();
+                if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104)) { ok = false; break; }
+                tc_fence_after();
+                int va[16], vb[16];
+                if (my_nch > 0) tmem_ld16(t_addr, va);
+#pragma unroll
+                for (int i = 0; i < 4; i += 2) {
+                    if (i < my_nch) {
+                        tmem_ld_wait();
+                        if (i + 1 < my_nch) tmem_ld16(t_addr + (i + 1) * 16, vb);
+                        const int4 *b4 = (const int4 *)(bias_w + i * 16);
+                        uint4 out;
+                        if (p.q.has_res)
+                            out = epilogue_fast16<true>(va, b4, rw[i], mul_acc, mul_res, p.q.r_signed, p.q.s - 1, p.q.lo, p.q.hi);
+                        else
+                            out = epilogue_fast16<false>(va, b4, rw[i], 1, 0, 0, p.q.s - 1, p.q.lo, p.q.hi);
+                        if (row_valid) *(uint4 *)(p.y + o + i * 16) = out;
+                    }
+                    if (i + 1 < my_nch) {
+                        tmem_ld_wait();
+                        if (i + 2 < my_nch) tmem_ld16(t_addr + (i + 2) * 16, va);
+                        const int4 *b4 = (const int4 *)(bias_w + (i + 1) * 16);
+                        uint4 out;
+                        if (p.q.has_res)
+                            out = epilogue_fast16<true>(vb, b4, rw[i + 1], mul_acc, mul_res, p.q.r_signed, p.q.s - 1, p.q.lo, p.q.hi);
+                        else
+                            out = epilogue_fast16<false>(vb, b4, rw[i + 1], 1, 0, 0, p.q.s - 1, p.q.lo, p.q.hi);
+                        if (row_valid) *(uint4 *)(p.y + o + (i + 1) * 16) = out;
+                    }
                 }
             } else {
-                for (int ch = ch_begin; ch < ch_end; ++ch) {
-                    const int co0 = n0 + ch * 16;
-                    if (co0 >= p.c_out) break;                   // uniform across the CTA
+                if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104)) { ok = false; break; }
+                tc_fence_after();
+                for (int i = 0; i < nch; ++i) {
+                    const int co0 = n0 + (ch_begin + i) * 16;
+                    if (co0 >= p.c_out) break;                   // uniform across the warp
                     int v[16];
-                    tmem_ld16(t_addr + ch * 16, v);
+                    tmem_ld16(t_addr + i * 16, v);
                     tmem_ld_wait();
                     epilogue_chunk(p, v, row, co0, row_valid);
                 }
