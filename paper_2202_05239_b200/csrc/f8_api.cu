@@ -479,6 +479,7 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
             for (size_t j = 0; j < per_out; ++j) sum += llabs((long long)hw[co * per_out + j]);
             long long bound = sum * xmax + (hb ? llabs((long long)hb[co]) : 0);
             bound = (bound << L.q.sh_acc) + (rmax << L.q.sh_res);
+            if (L.q.y_kind != F8_S32 && L.q.s >= 1) bound += 1ll << (L.q.s - 1);      // room for the rounding constant
             if (bound >= (1ll << 31) - 1)
                 return cleanup(fail(F8_ERR_ACC_BOUND, "layer %d channel %d: accumulator bound %lld exceeds int32", i, co, bound));
         }

@@ -18,7 +18,10 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <stdlib.h>
 #include <string.h>
+
+#include <algorithm>
 
 #include "f8_epilogue.cuh"
 
@@ -53,7 +56,7 @@ struct TcParams {
     const uint8_t *res;
     uint8_t *y;
     int vec_bytes;            // widest aligned store the output rows allow: 16, 8, 4 or 1
-    int fast;                 // 1: 8-bit output, shift >= 1, c_out % 16 == 0 -> branch-free epilogue
+    int epi;                  // EPI_* epilogue variant
     F8Requant q;
     int *status;
 };
@@ -216,14 +219,16 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int (&ac
     }
 }
 
-// Branch-free epilogue for the common case (8-bit output, shift s >= 1, c_out % 16 == 0).
-//   v = acc * 2^sh_acc + bias'          bias' = bias << sh_acc, staged in shared memory
+// Branch-free epilogue for the common case (8-bit output, 1 <= s <= 24, c_out % 16 == 0).
+//   v = acc * 2^sh_acc + bias'          bias' = (bias << sh_acc) + 2^(s-1), staged in shared memory
 //   v += r << sh_res                    (RES only)
-//   t = ((v >> (s-1)) + 1) >> 1         = floor((v + 2^(s-1)) / 2^s); cannot overflow because |v| < 2^31 - 1
-//   y = clamp(t, lo, hi)
-template <bool RES>
+//   t = v >> s                          = floor((acc' + 2^(s-1)) / 2^s), round half up
+//   y = clamp(t, lo, hi)                saturating pack; the signed quantizer additionally excludes -128
+// cvt.pack.sat packs two saturated values into the low half of d and moves the low half of c above
+// them: d = (c << 16) | (sat(a) << 8) | sat(b).
+template <bool RES, bool SIGNED_OUT>
 __device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], const int4 *bias4, uint4 rw, int mul_acc,
-                                                 int mul_res, int r_signed, int sm1, int lo, int hi) {
+                                                 int mul_res, int r_signed, int s) {
     int t[16];
     const uint32_t rwords[4] = {rw.x, rw.y, rw.z, rw.w};
 #pragma unroll
@@ -233,27 +238,37 @@ __device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], const int
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const int j = 4 * g + k;
-            int v = acc[j] * mul_acc + bb[k];
+            int v = RES ? acc[j] * mul_acc + bb[k] : acc[j] + bb[k];
             if (RES) {
                 int r;
                 if (r_signed) asm("bfe.s32 %0, %1, %2, 8;" : "=r"(r) : "r"(rwords[g]), "r"(8 * k));
                 else asm("bfe.u32 %0, %1, %2, 8;" : "=r"(r) : "r"(rwords[g]), "r"(8 * k));
                 v += r * mul_res;
             }
-            const int u = ((v >> sm1) + 1) >> 1;
-            t[j] = min(max(u, lo), hi);
+            v >>= s;
+            t[j] = SIGNED_OUT ? max(v, -127) : v;
         }
     }
-    uint4 o;
-    o.x = __byte_perm(__byte_perm(t[0], t[1], 0x0040), __byte_perm(t[2], t[3], 0x0040), 0x5410);
-    o.y = __byte_perm(__byte_perm(t[4], t[5], 0x0040), __byte_perm(t[6], t[7], 0x0040), 0x5410);
-    o.z = __byte_perm(__byte_perm(t[8], t[9], 0x0040), __byte_perm(t[10], t[11], 0x0040), 0x5410);
-    o.w = __byte_perm(__byte_perm(t[12], t[13], 0x0040), __byte_perm(t[14], t[15], 0x0040), 0x5410);
-    return o;
+    uint32_t o[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        uint32_t hi2;
+        if (SIGNED_OUT) {
+            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(t[4 * g + 3]), "r"(t[4 * g + 2]));
+            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(o[g]) : "r"(t[4 * g + 1]), "r"(t[4 * g]), "r"(hi2));
+        } else {
+            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(t[4 * g + 3]), "r"(t[4 * g + 2]));
+            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(o[g]) : "r"(t[4 * g + 1]), "r"(t[4 * g]), "r"(hi2));
+        }
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 // ----------------------------------------------------------------------------- the kernel
 
+enum { EPI_GENERIC = 0, EPI_U8 = 1, EPI_U8_RES = 2, EPI_S8 = 3, EPI_S8_RES = 4 };
+
+template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const TcParams p) {
@@ -406,7 +421,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const size_t row = (size_t)m_t * TILE_M + quarter * 32 + lane;
             const bool row_valid = row < (size_t)p.M;
             const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
-            if (p.fast) {
+            if (EPI != EPI_GENERIC) {
+                constexpr bool RES = EPI == EPI_U8_RES || EPI == EPI_S8_RES;
+                constexpr bool SGN = EPI == EPI_S8 || EPI == EPI_S8_RES;
                 // everything that does not depend on the accumulator is fetched before waiting for it:
                 // the bias of this warp's columns (to shared memory) and this thread's residual bytes
                 const int c_first = n0 + ch_begin * 16;
@@ -416,7 +433,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     const int c0 = c_first + lane * 4;
                     int4 b = make_int4(0, 0, 0, 0);
                     if (p.bias && lane * 4 < my_nch * 16) b = __ldg((const int4 *)(p.bias + c0));
-                    b.x <<= p.q.sh_acc; b.y <<= p.q.sh_acc; b.z <<= p.q.sh_acc; b.w <<= p.q.sh_acc;
+                    const int rnd = 1 << (p.q.s - 1);        // rounding constant folded into the bias
+                    b.x = (b.x << p.q.sh_acc) + rnd; b.y = (b.y << p.q.sh_acc) + rnd;
+                    b.z = (b.z << p.q.sh_acc) + rnd; b.w = (b.w << p.q.sh_acc) + rnd;
                     *(int4 *)(bias_w + lane * 4) = b;
                 }
                 const size_t o = row * (size_t)p.c_out + c_first;
@@ -424,7 +443,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     rw[i] = make_uint4(0, 0, 0, 0);
-                    if (p.q.has_res && row_valid && i < my_nch) rw[i] = __ldg((const uint4 *)(p.res + o + i * 16));
+                    if (RES && row_valid && i < my_nch) rw[i] = __ldg((const uint4 *)(p.res + o + i * 16));
                 }
                 __syncwarp();
                 if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104)) { ok = false; break; }
@@ -437,22 +456,14 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         tmem_ld_wait();
                         if (i + 1 < my_nch) tmem_ld16(t_addr + (i + 1) * 16, vb);
                         const int4 *b4 = (const int4 *)(bias_w + i * 16);
-                        uint4 out;
-                        if (p.q.has_res)
-                            out = epilogue_fast16<true>(va, b4, rw[i], mul_acc, mul_res, p.q.r_signed, p.q.s - 1, p.q.lo, p.q.hi);
-                        else
-                            out = epilogue_fast16<false>(va, b4, rw[i], 1, 0, 0, p.q.s - 1, p.q.lo, p.q.hi);
+                        const uint4 out = epilogue_fast16<RES, SGN>(va, b4, rw[i], mul_acc, mul_res, p.q.r_signed, p.q.s);
                         if (row_valid) *(uint4 *)(p.y + o + i * 16) = out;
                     }
                     if (i + 1 < my_nch) {
                         tmem_ld_wait();
                         if (i + 2 < my_nch) tmem_ld16(t_addr + (i + 2) * 16, va);
                         const int4 *b4 = (const int4 *)(bias_w + (i + 1) * 16);
-                        uint4 out;
-                        if (p.q.has_res)
-                            out = epilogue_fast16<true>(vb, b4, rw[i + 1], mul_acc, mul_res, p.q.r_signed, p.q.s - 1, p.q.lo, p.q.hi);
-                        else
-                            out = epilogue_fast16<false>(vb, b4, rw[i + 1], 1, 0, 0, p.q.s - 1, p.q.lo, p.q.hi);
+                        const uint4 out = epilogue_fast16<RES, SGN>(vb, b4, rw[i + 1], mul_acc, mul_res, p.q.r_signed, p.q.s);
                         if (row_valid) *(uint4 *)(p.y + o + (i + 1) * 16) = out;
                     }
                 }
@@ -596,8 +607,10 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.pad_h = g.pad_h;
     p.pad_w = g.pad_w;
     p.kb = choose_kb(g.c);
+    if (const char *e = getenv("F8_TC_KB")) p.kb = atoi(e);
     p.c_chunks = (g.c + p.kb - 1) / p.kb;
     p.bn = choose_bn(g.c_out);
+    if (const char *e = getenv("F8_TC_BN")) p.bn = atoi(e);
     p.m_tiles = (p.M + TILE_M - 1) / TILE_M;
     p.n_tiles = (g.c_out + p.bn - 1) / p.bn;
     p.a_bytes = (uint32_t)(TILE_M * p.kb + 1023) / 1024 * 1024;
@@ -606,6 +619,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.tx_bytes = (uint32_t)((TILE_M + p.bn) * p.kb);
     int stages = (int)(SMEM_BUDGET / p.stage_bytes);
     if (stages > MAX_STAGES) stages = MAX_STAGES;
+    if (const char *e = getenv("F8_TC_STAGES")) stages = std::min(stages, atoi(e));
     if (stages < 2) {
         *why = "stage does not fit";
         return cudaErrorInvalidValue;
@@ -623,7 +637,9 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.status = status_word;
     const int ysz = q.y_kind == F8_S32 ? 4 : 1;
     const size_t row_bytes = (size_t)g.c_out * ysz;
-    p.fast = (q.y_kind != F8_S32 && q.s >= 1 && g.c_out % 16 == 0) ? 1 : 0;
+    p.epi = EPI_GENERIC;
+    if (q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24 && g.c_out % 16 == 0)
+        p.epi = q.y_kind == F8_U8 ? (q.has_res ? EPI_U8_RES : EPI_U8) : (q.has_res ? EPI_S8_RES : EPI_S8);
     p.vec_bytes = (row_bytes % 16 == 0) ? 16 : (row_bytes % 8 == 0 ? 8 : (row_bytes % 4 == 0 ? 4 : 1));
 
     // A: activation tensor (C, W, H, N) in im2col mode.  Corners follow the usual forward-convolution
@@ -667,8 +683,12 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     if (plan->smem < 120 * 1024) plan->smem = 120 * 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(SMEM_BUDGET + 2048));
+        const int bytes = (int)(SMEM_BUDGET + 2048);
+        cudaError_t e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_GENERIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -677,7 +697,13 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
 
 cudaError_t f8_tc_launch(const F8TcPlan *plan, cudaStream_t st) {
     if (plan->p.M == 0) return cudaSuccess;
-    f8_conv_gemm_tc_kernel<<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p);
+    switch (plan->p.epi) {
+        case EPI_U8: f8_conv_gemm_tc_kernel<EPI_U8><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
+        case EPI_U8_RES: f8_conv_gemm_tc_kernel<EPI_U8_RES><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
+        case EPI_S8: f8_conv_gemm_tc_kernel<EPI_S8><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
+        case EPI_S8_RES: f8_conv_gemm_tc_kernel<EPI_S8_RES><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
+        default: f8_conv_gemm_tc_kernel<EPI_GENERIC><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
+    }
     return cudaGetLastError();
 }
 
