@@ -138,6 +138,8 @@ f8_status run_dense(const F8ConvGeom &g, const F8Requant &q, const void *x, cons
         }
         if (e != cudaErrorInvalidValue && e != cudaErrorNotSupported) return cuda_fail(e, why);
         // the tensor map could not be encoded for this shape: take the CUDA-core kernel
+        if (getenv("F8NET_VERBOSE")) fprintf(stderr, "f8net: tensor-core plan rejected (%s: %s), using the CUDA-core kernel\n", why, cudaGetErrorString(e));
+        (void)cudaGetLastError();
     }
     cudaError_t e = f8_launch_conv_direct(g, q, x, w, bias, res, y, st);
     if (e != cudaSuccess) return cuda_fail(e, "direct conv launch");

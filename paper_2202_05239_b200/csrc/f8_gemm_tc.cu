@@ -9,7 +9,10 @@
 //     in tensor memory, double buffered so the epilogue of tile i overlaps the main loop of tile i+1.
 //   * Sixteen epilogue warps read the accumulator with tcgen05.ld (one output pixel per thread, 16
 //     consecutive channels per load), add the bias, align and add the residual, apply the rounding
-//     shift and clip (Eq. 2 / signed form applied to Eq. 6) and store 16 output bytes per instruction.
+//     shift and clip (Eq. 2 / signed form applied to Eq. 6).  The 8-bit result is written to a swizzled
+//     staging tile in shared memory and leaves with one TMA store per 128-byte column slab; the
+//     residual tile arrives the same way (TMA load, two tiles ahead), so global memory only sees
+//     full-line accesses.  Shapes that do not fit this scheme use direct 16-byte stores.
 //   * Persistent CTAs (one per SM) walk the tile list; tiles that share an A tile are adjacent so that
 //     the activation tensor is read from HBM once and from L2 afterwards.
 //
@@ -19,6 +22,7 @@
 #include <cudaTypedefs.h>
 
 #include <stdlib.h>
+#include <stdio.h>
 #include <string.h>
 
 #include <algorithm>
@@ -29,12 +33,19 @@ namespace {
 
 constexpr int TILE_M = 128;
 constexpr int NUM_EPI_WARPS = 16;          // four warps per TMEM lane quarter, each takes a quarter of the columns
-constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;   // warp 0: TMA, warp 1: MMA, warps 2-17: epilogue
+// A thread that issues a TMA load does not get to issue its next one until the first has been served
+// (about one L2 round trip, whatever the box size), so one producer thread caps a CTA at a few tens of
+// bytes per clock.  Loads from different warps overlap: the k-iterations are dealt round-robin to
+// several producer warps.
+constexpr int NUM_PROD_WARPS = 4;
+constexpr int MMA_WARP = NUM_PROD_WARPS;
+constexpr int FIRST_EPI_WARP = NUM_PROD_WARPS + 1;
+constexpr int NUM_THREADS = 32 * (NUM_PROD_WARPS + 1 + NUM_EPI_WARPS);   // producers, MMA issuer, epilogue
 constexpr int MAX_STAGES = 8;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
 constexpr unsigned long long DRAIN_LIMIT_CYCLES = 200000000ull;
-constexpr size_t SMEM_BUDGET = 200 * 1024;
+constexpr size_t SMEM_LIMIT = 220 * 1024;     // dynamic shared memory budget (227 KiB per CTA minus static data)
 
 struct TcParams {
     int M;                    // total output pixels
@@ -46,7 +57,9 @@ struct TcParams {
     int kb;                   // bytes (= int8 elements) of K per stage: 32, 64 or 128
     int bn;                   // N tile, multiple of 16, <= 256
     int m_tiles, n_tiles;
-    int stages;
+    int stages;               // multiple of prod_warps: every stage then has exactly one producer warp, which
+                              // keeps that warp at most one barrier phase ahead of the consumer
+    int prod_warps;           // producer warps in use (<= NUM_PROD_WARPS)
     uint32_t stage_bytes;     // A + B bytes of one stage (rounded to 1024)
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
     uint32_t tx_bytes;        // bytes both TMA loads of a stage deliver
@@ -57,6 +70,14 @@ struct TcParams {
     uint8_t *y;
     int vec_bytes;            // widest aligned store the output rows allow: 16, 8, 4 or 1
     int epi;                  // EPI_* epilogue variant
+    // staged epilogue: the output tile (and the residual tile) pass through shared memory in column
+    // slabs of slab_w bytes per row, written / read by TMA with the matching swizzle
+    int slab_w;               // 16, 32, 64 or 128 bytes
+    int slab_chunks;          // slab_w / 16
+    int n_slabs;              // bn / slab_w
+    uint32_t swz_mask;        // 7, 3, 1 or 0: address bits 7.. XORed into the 16-byte chunk index
+    uint32_t out_bytes;       // TILE_M * bn
+    uint32_t res_off, out_off;   // byte offsets of the two residual / two output buffers behind the stages
     F8Requant q;
     int *status;
 };
@@ -120,6 +141,20 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         " [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
         "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+// shared -> global tile store; rows / columns outside the tensor are clipped by the hardware
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src),
+                 "r"(c0), "r"(c1)
+                 : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -268,16 +303,29 @@ __device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], const int
 
 enum { EPI_GENERIC = 0, EPI_U8 = 1, EPI_U8_RES = 2, EPI_S8 = 3, EPI_S8_RES = 4 };
 
+// Byte offset of 16-byte chunk `chunk` of row `row` inside a staging slab whose rows are slab_w bytes
+// long, in the layout the TMA uses for the matching swizzle mode (chunk index XOR address bits 7..9).
+__device__ __forceinline__ uint32_t slab_offset(int row, int chunk, int slab_w, uint32_t swz_mask) {
+    uint32_t off = (uint32_t)row * slab_w + chunk * 16;
+    return off ^ (((off >> 7) & swz_mask) << 4);
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                       const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_r,
                        const TcParams p) {
+    constexpr bool STAGED = EPI != EPI_GENERIC;                     // output (and residual) through shared memory + TMA
+    constexpr bool RES = EPI == EPI_U8_RES || EPI == EPI_S8_RES;
+    constexpr bool SGN = EPI == EPI_S8 || EPI == EPI_S8_RES;
+
     extern __shared__ uint8_t smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 8];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int epi_abort;
     __shared__ __align__(16) int bias_stage[NUM_EPI_WARPS][64];   // per warp: bias of its columns, pre-shifted
 
     const int warp = threadIdx.x >> 5;
@@ -286,10 +334,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const uint32_t empty_bar = smem_u32(&bars[MAX_STAGES]);
     const uint32_t tfull_bar = smem_u32(&bars[2 * MAX_STAGES]);
     const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + 2]);
+    const uint32_t rfull_bar = smem_u32(&bars[2 * MAX_STAGES + 4]);
+    const uint32_t rempty_bar = smem_u32(&bars[2 * MAX_STAGES + 6]);
     const uint32_t smem_base = smem_u32(smem);
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
+        epi_abort = 0;
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(full_bar + 8 * s, 1);
             mbar_init(empty_bar + 8 * s, 1);
@@ -297,11 +348,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
             mbar_init(tempty_bar + 8 * a, 32 * NUM_EPI_WARPS);
+            mbar_init(rfull_bar + 8 * a, 1);
+            mbar_init(rempty_bar + 8 * a, 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+    if (warp == MMA_WARP) tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -311,16 +364,31 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const int k_iters = p.kh * p.kw * p.c_chunks;
     volatile int *abortp = &abort_flag;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            uint32_t issued = 0;            // loads issued so far (for the drain on abort)
+    if (warp < NUM_PROD_WARPS) {
+        // ------------------------------------------------------------------ TMA producers
+        // k-iteration `it` (counted over all tiles of this CTA) belongs to producer warp it % prod_warps; the
+        // residual tiles all go through warp 0 so that they, too, are requested in order
+        if (lane == 0 && warp < p.prod_warps) {
+            uint32_t it = 0;
+            bool have_last = false;
+            uint32_t last_it = 0;           // this thread's most recent stage load (for the drain on abort)
+            int last_res = -1;              // ... and its most recent residual tile
+            int local = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
                 const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
                 const int m0 = m_t * TILE_M;
+                if (RES && warp == 0) {
+                    // residual tile of this output tile -> staging buffer (local & 1), two tiles ahead of its use
+                    const int b = local & 1;
+                    if (!mbar_wait(rempty_bar + 8 * b, ((local >> 1) & 1) ^ 1, abortp, p.status, 106)) { ok = false; break; }
+                    const uint32_t rb = rfull_bar + 8 * b;
+                    mbar_expect_tx(rb, p.out_bytes);
+                    for (int sl = 0; sl < p.n_slabs; ++sl)
+                        tma_load_2d(smem_base + p.res_off + b * p.out_bytes + sl * (TILE_M * p.slab_w), &map_r, rb,
+                                    n_t * p.bn + sl * p.slab_w, m0);
+                    last_res = local;
+                }
                 const int ow = m0 % p.wo;
                 const int t1 = m0 / p.wo;
                 const int oh = t1 % p.ho;
@@ -329,7 +397,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int base_h = oh * p.stride_h - p.pad_h;
                 for (int r = 0; ok && r < p.kh; ++r)
                     for (int s = 0; ok && s < p.kw; ++s)
-                        for (int cc = 0; cc < p.c_chunks; ++cc) {
+                        for (int cc = 0; cc < p.c_chunks; ++cc, ++it) {
+                            if ((int)(it % (uint32_t)p.prod_warps) != warp) continue;
+                            const int stage = (int)(it % (uint32_t)p.stages);
+                            const uint32_t phase = (it / (uint32_t)p.stages) & 1;
                             if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101)) {
                                 ok = false;
                                 break;
@@ -340,25 +411,28 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                             tma_load_im2col(a_dst, &map_a, fb, cc * p.kb, base_w, base_h, img, (uint16_t)s,
                                             (uint16_t)r);
                             tma_load_3d(a_dst + p.a_bytes, &map_b, fb, cc * p.kb, r * p.kw + s, n_t * p.bn);
-                            ++issued;
-                            if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                            have_last = true;
+                            last_it = it;
                         }
             }
             if (!ok) {
-                // Drain: give every load that was issued time to land before the CTA's shared memory goes away.
-                const uint32_t pending = issued < (uint32_t)p.stages ? issued : (uint32_t)p.stages;
-                for (uint32_t i = 0; i < pending; ++i) {
-                    const uint32_t idx = issued - 1 - i;
-                    const int st = (int)(idx % p.stages);
-                    const uint32_t ph = (idx / p.stages) & 1;
+                // Drain: loads of one thread are served in order, so waiting (bounded) for the most recent one
+                // covers everything this thread has in flight before the CTA's shared memory goes away.
+                if (have_last) {
                     const unsigned long long t0 = clock64();
-                    while (!mbar_try_wait(full_bar + 8 * st, ph) &&
+                    while (!mbar_try_wait(full_bar + 8 * (last_it % (uint32_t)p.stages), (last_it / (uint32_t)p.stages) & 1) &&
+                           (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
+                    }
+                }
+                if (last_res >= 0) {
+                    const unsigned long long t0 = clock64();
+                    while (!mbar_try_wait(rfull_bar + 8 * (last_res & 1), (last_res >> 1) & 1) &&
                            (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
                     }
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == MMA_WARP) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             int stage = 0;
@@ -401,14 +475,16 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..17)
+        // ------------------------------------------------------------------ epilogue warps
         const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 belong to this warp
-        const int ew = warp - 2;
+        const int ew = warp - FIRST_EPI_WARP;
         const int group = ew >> 2;                  // which quarter of the tile's columns this warp converts
         const int chunks = p.bn / 16;
         const int per_group = (chunks + 3) / 4;     // <= 4 chunks of 16 columns per warp
         const int ch_begin = min(group * per_group, chunks);
         const int nch = min(ch_begin + per_group, chunks) - ch_begin;
+        const int tile_row = quarter * 32 + lane;   // this thread's row of the tile
+        const bool issuer = ew == 0 && lane == 0;   // the thread that owns the bulk-store groups
         int *bias_w = bias_stage[ew];
         const int mul_acc = 1 << p.q.sh_acc, mul_res = 1 << p.q.sh_res;
         int local = 0;
@@ -418,54 +494,79 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const uint32_t acc_phase = (local >> 1) & 1;
             const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
             const int n0 = n_t * p.bn;
-            const size_t row = (size_t)m_t * TILE_M + quarter * 32 + lane;
+            const size_t row = (size_t)m_t * TILE_M + tile_row;
             const bool row_valid = row < (size_t)p.M;
             const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
-            if (EPI != EPI_GENERIC) {
-                constexpr bool RES = EPI == EPI_U8_RES || EPI == EPI_S8_RES;
-                constexpr bool SGN = EPI == EPI_S8 || EPI == EPI_S8_RES;
-                // everything that does not depend on the accumulator is fetched before waiting for it:
-                // the bias of this warp's columns (to shared memory) and this thread's residual bytes
+            if (STAGED) {
+                const int b = local & 1;
+                // bias of this warp's columns (+ rounding constant) -> shared memory, before the accumulator is ready
                 const int c_first = n0 + ch_begin * 16;
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
                 __syncwarp();
                 if (lane < 16) {
                     const int c0 = c_first + lane * 4;
-                    int4 b = make_int4(0, 0, 0, 0);
-                    if (p.bias && lane * 4 < my_nch * 16) b = __ldg((const int4 *)(p.bias + c0));
+                    int4 bv = make_int4(0, 0, 0, 0);
+                    if (p.bias && lane * 4 < my_nch * 16) bv = __ldg((const int4 *)(p.bias + c0));
                     const int rnd = 1 << (p.q.s - 1);        // rounding constant folded into the bias
-                    b.x = (b.x << p.q.sh_acc) + rnd; b.y = (b.y << p.q.sh_acc) + rnd;
-                    b.z = (b.z << p.q.sh_acc) + rnd; b.w = (b.w << p.q.sh_acc) + rnd;
-                    *(int4 *)(bias_w + lane * 4) = b;
-                }
-                const size_t o = row * (size_t)p.c_out + c_first;
-                uint4 rw[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    rw[i] = make_uint4(0, 0, 0, 0);
-                    if (RES && row_valid && i < my_nch) rw[i] = __ldg((const uint4 *)(p.res + o + i * 16));
+                    bv.x = (bv.x << p.q.sh_acc) + rnd; bv.y = (bv.y << p.q.sh_acc) + rnd;
+                    bv.z = (bv.z << p.q.sh_acc) + rnd; bv.w = (bv.w << p.q.sh_acc) + rnd;
+                    *(int4 *)(bias_w + lane * 4) = bv;
                 }
                 __syncwarp();
-                if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104)) { ok = false; break; }
+                // A thread whose wait runs out keeps going through this tile (the kernel is aborting and the
+                // whole group leaves together at the next check) so that nobody is left alone at a barrier.
+                mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104);
+                if (RES) mbar_wait(rfull_bar + 8 * b, acc_phase, abortp, p.status, 107);
                 tc_fence_after();
+                if (issuer) {
+                    // the store issued from this output buffer two tiles ago must have finished reading it
+                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    epi_abort = *abortp;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(32 * NUM_EPI_WARPS) : "memory");
+                if (epi_abort) { ok = false; break; }
+                uint8_t *out_buf = smem + p.out_off + b * p.out_bytes;
+                const uint8_t *res_buf = smem + p.res_off + b * p.out_bytes;
                 int va[16], vb[16];
                 if (my_nch > 0) tmem_ld16(t_addr, va);
 #pragma unroll
                 for (int i = 0; i < 4; i += 2) {
                     if (i < my_nch) {
+                        const int ch = ch_begin + i;
+                        const uint32_t so = (uint32_t)(ch / p.slab_chunks) * (TILE_M * p.slab_w) +
+                                            slab_offset(tile_row, ch % p.slab_chunks, p.slab_w, p.swz_mask);
+                        uint4 rw = make_uint4(0, 0, 0, 0);
+                        if (RES) rw = *(const uint4 *)(res_buf + so);
                         tmem_ld_wait();
                         if (i + 1 < my_nch) tmem_ld16(t_addr + (i + 1) * 16, vb);
                         const int4 *b4 = (const int4 *)(bias_w + i * 16);
-                        const uint4 out = epilogue_fast16<RES, SGN>(va, b4, rw[i], mul_acc, mul_res, p.q.r_signed, p.q.s);
-                        if (row_valid) *(uint4 *)(p.y + o + i * 16) = out;
+                        *(uint4 *)(out_buf + so) = epilogue_fast16<RES, SGN>(va, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s);
                     }
                     if (i + 1 < my_nch) {
+                        const int ch = ch_begin + i + 1;
+                        const uint32_t so = (uint32_t)(ch / p.slab_chunks) * (TILE_M * p.slab_w) +
+                                            slab_offset(tile_row, ch % p.slab_chunks, p.slab_w, p.swz_mask);
+                        uint4 rw = make_uint4(0, 0, 0, 0);
+                        if (RES) rw = *(const uint4 *)(res_buf + so);
                         tmem_ld_wait();
                         if (i + 2 < my_nch) tmem_ld16(t_addr + (i + 2) * 16, va);
                         const int4 *b4 = (const int4 *)(bias_w + (i + 1) * 16);
-                        const uint4 out = epilogue_fast16<RES, SGN>(vb, b4, rw[i + 1], mul_acc, mul_res, p.q.r_signed, p.q.s);
-                        if (row_valid) *(uint4 *)(p.y + o + (i + 1) * 16) = out;
+                        *(uint4 *)(out_buf + so) = epilogue_fast16<RES, SGN>(vb, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s);
                     }
+                }
+                // the accumulator has been read: hand it back to the MMA warp
+                tc_fence_before();
+                mbar_arrive(tempty_bar + 8 * acc);
+                // make the generic-proxy writes visible to the TMA, then one thread stores the tile
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                asm volatile("bar.sync 2, %0;" ::"n"(32 * NUM_EPI_WARPS) : "memory");
+                if (issuer) {
+                    for (int sl = 0; sl < p.n_slabs; ++sl)
+                        if (n0 + sl * p.slab_w < p.c_out)
+                            tma_store_2d(&map_y, smem_u32(out_buf) + sl * (TILE_M * p.slab_w), n0 + sl * p.slab_w,
+                                         m_t * TILE_M);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    if (RES) mbar_arrive(rempty_bar + 8 * b);     // everyone is past the barrier: residual buffer is free
                 }
             } else {
                 if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104)) { ok = false; break; }
@@ -478,15 +579,16 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     tmem_ld_wait();
                     epilogue_chunk(p, v, row, co0, row_valid);
                 }
+                tc_fence_before();
+                mbar_arrive(tempty_bar + 8 * acc);
             }
-            tc_fence_before();
-            mbar_arrive(tempty_bar + 8 * acc);
         }
+        if (STAGED && issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == MMA_WARP) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
@@ -509,12 +611,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) f8_mma_probe_kernel(int iters,
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+    if (warp == MMA_WARP) tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
-    if (warp == 1 && lane == 0) {
+    if (warp == MMA_WARP && lane == 0) {
         const uint32_t a_addr = smem_u32(smem), b_addr = a_addr + 128 * 128;
         const uint64_t hi = smem_desc_hi(128);
         const uint64_t a_desc = hi | (uint64_t)((a_addr & 0x3ffffu) >> 4);
@@ -528,7 +630,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) f8_mma_probe_kernel(int iters,
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == MMA_WARP) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
@@ -562,6 +664,15 @@ int choose_bn(int c_out) {
     return (c_out + 15) / 16 * 16;
 }
 
+// N tile of the staged epilogue: a power of two up to 128, or 256 (two 128-byte slabs) when no residual
+// buffers are needed; the TMA store clips columns beyond c_out.
+int choose_bn_staged(int c_out, bool has_res) {
+    if (c_out > 128 && !has_res) return 256;
+    int bn = 16;
+    while (bn < c_out && bn < 128) bn *= 2;
+    return bn;
+}
+
 CUtensorMapSwizzle swizzle_for(int kb) {
     return kb == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (kb == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
 }
@@ -571,6 +682,8 @@ CUtensorMapSwizzle swizzle_for(int kb) {
 struct F8TcPlan {
     CUtensorMap map_a;
     CUtensorMap map_b;
+    CUtensorMap map_y;
+    CUtensorMap map_r;
     TcParams p;
     int grid;
     size_t smem;
@@ -607,24 +720,38 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.pad_h = g.pad_h;
     p.pad_w = g.pad_w;
     p.kb = choose_kb(g.c);
-    if (const char *e = getenv("F8_TC_KB")) p.kb = atoi(e);
     p.c_chunks = (g.c + p.kb - 1) / p.kb;
-    p.bn = choose_bn(g.c_out);
-    if (const char *e = getenv("F8_TC_BN")) p.bn = atoi(e);
+    p.epi = EPI_GENERIC;
+    if (q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24 && g.c_out % 16 == 0)
+        p.epi = q.y_kind == F8_U8 ? (q.has_res ? EPI_U8_RES : EPI_U8) : (q.has_res ? EPI_S8_RES : EPI_S8);
+    const bool staged = p.epi != EPI_GENERIC;
+    p.bn = staged ? choose_bn_staged(g.c_out, q.has_res != 0) : choose_bn(g.c_out);
     p.m_tiles = (p.M + TILE_M - 1) / TILE_M;
     p.n_tiles = (g.c_out + p.bn - 1) / p.bn;
     p.a_bytes = (uint32_t)(TILE_M * p.kb + 1023) / 1024 * 1024;
     const uint32_t b_bytes = (uint32_t)(p.bn * p.kb + 1023) / 1024 * 1024;
     p.stage_bytes = p.a_bytes + b_bytes;
     p.tx_bytes = (uint32_t)((TILE_M + p.bn) * p.kb);
-    int stages = (int)(SMEM_BUDGET / p.stage_bytes);
+    size_t staging = 0;
+    if (staged) {
+        p.slab_w = p.bn < 128 ? p.bn : 128;
+        p.slab_chunks = p.slab_w / 16;
+        p.n_slabs = p.bn / p.slab_w;
+        p.swz_mask = p.slab_w == 128 ? 7u : (p.slab_w == 64 ? 3u : (p.slab_w == 32 ? 1u : 0u));
+        p.out_bytes = (uint32_t)(TILE_M * p.bn);
+        staging = (size_t)p.out_bytes * (q.has_res ? 4 : 2);
+    }
+    int stages = (int)((SMEM_LIMIT - 1024 - staging) / p.stage_bytes);
     if (stages > MAX_STAGES) stages = MAX_STAGES;
-    if (const char *e = getenv("F8_TC_STAGES")) stages = std::min(stages, atoi(e));
     if (stages < 2) {
         *why = "stage does not fit";
         return cudaErrorInvalidValue;
     }
+    p.prod_warps = stages >= NUM_PROD_WARPS ? NUM_PROD_WARPS : stages;
+    stages -= stages % p.prod_warps;
     p.stages = stages;
+    p.res_off = (uint32_t)(p.stages * p.stage_bytes);
+    p.out_off = p.res_off + (q.has_res ? 2 * p.out_bytes : 0);
     // instruction descriptor: D = s32 (2 at bit 4), A format at bit 7 (0 = u8, 1 = s8), B = s8 at bit 10,
     // both operands K-major, N/8 at bit 17, M/16 at bit 24
     p.idesc = (2u << 4) | ((g.x_signed ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) |
@@ -637,9 +764,6 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.status = status_word;
     const int ysz = q.y_kind == F8_S32 ? 4 : 1;
     const size_t row_bytes = (size_t)g.c_out * ysz;
-    p.epi = EPI_GENERIC;
-    if (q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24 && g.c_out % 16 == 0)
-        p.epi = q.y_kind == F8_U8 ? (q.has_res ? EPI_U8_RES : EPI_U8) : (q.has_res ? EPI_S8_RES : EPI_S8);
     p.vec_bytes = (row_bytes % 16 == 0) ? 16 : (row_bytes % 8 == 0 ? 8 : (row_bytes % 4 == 0 ? 4 : 1));
 
     // A: activation tensor (C, W, H, N) in im2col mode.  Corners follow the usual forward-convolution
@@ -673,23 +797,58 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
             return cudaErrorInvalidValue;
         }
     }
+    // output / residual [M, c_out] bytes, one box = one column slab of a tile
+    plan->map_y = plan->map_b;
+    plan->map_r = plan->map_b;
+    if (staged) {
+        cuuint64_t dims[2] = {(cuuint64_t)g.c_out, (cuuint64_t)p.M};
+        cuuint64_t strides[1] = {(cuuint64_t)g.c_out};
+        cuuint32_t box[2] = {(cuuint32_t)p.slab_w, (cuuint32_t)TILE_M};
+        cuuint32_t estr[2] = {1, 1};
+        const CUtensorMapSwizzle sw = p.slab_w == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                      : (p.slab_w == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                         : (p.slab_w == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE));
+        CUresult r = g_encode_tiled(&plan->map_y, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, y, dims, strides, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r == CUDA_SUCCESS && q.has_res)
+            r = g_encode_tiled(&plan->map_r, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(res), dims, strides, box,
+                               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            *why = "cuTensorMapEncodeTiled rejected the output tensor";
+            return cudaErrorInvalidValue;
+        }
+    }
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int total_tiles = p.m_tiles * p.n_tiles;
     plan->grid = total_tiles < sms ? total_tiles : sms;
     // at least half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
-    plan->smem = (size_t)p.stages * p.stage_bytes + 1024;
+    plan->smem = (size_t)p.stages * p.stage_bytes + staging + 1024;
     if (plan->smem < 120 * 1024) plan->smem = 120 * 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        const int bytes = (int)(SMEM_BUDGET + 2048);
+        const int bytes = (int)SMEM_LIMIT;
         cudaError_t e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_GENERIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e != cudaSuccess) return e;
+        if (e != cudaSuccess) {
+            if (getenv("F8NET_VERBOSE")) {
+                cudaFuncAttributes fa;
+                int optin = 0, dev2 = 0;
+                cudaGetDevice(&dev2);
+                cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev2);
+                if (cudaFuncGetAttributes(&fa, f8_conv_gemm_tc_kernel<EPI_U8>) == cudaSuccess)
+                    fprintf(stderr, "f8net: static smem %zu, regs %d, max threads %d, local %zu, optin %d, asked %d\n",
+                            fa.sharedSizeBytes, fa.numRegs, fa.maxThreadsPerBlock, fa.localSizeBytes, optin, bytes);
+            }
+            *why = "cudaFuncSetAttribute(MaxDynamicSharedMemorySize) failed";
+            return e;
+        }
         attr_set = true;
     }
     return cudaSuccess;
@@ -698,11 +857,11 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
 cudaError_t f8_tc_launch(const F8TcPlan *plan, cudaStream_t st) {
     if (plan->p.M == 0) return cudaSuccess;
     switch (plan->p.epi) {
-        case EPI_U8: f8_conv_gemm_tc_kernel<EPI_U8><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
-        case EPI_U8_RES: f8_conv_gemm_tc_kernel<EPI_U8_RES><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
-        case EPI_S8: f8_conv_gemm_tc_kernel<EPI_S8><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
-        case EPI_S8_RES: f8_conv_gemm_tc_kernel<EPI_S8_RES><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
-        default: f8_conv_gemm_tc_kernel<EPI_GENERIC><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->p); break;
+        case EPI_U8: f8_conv_gemm_tc_kernel<EPI_U8><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
+        case EPI_U8_RES: f8_conv_gemm_tc_kernel<EPI_U8_RES><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
+        case EPI_S8: f8_conv_gemm_tc_kernel<EPI_S8><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
+        case EPI_S8_RES: f8_conv_gemm_tc_kernel<EPI_S8_RES><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
+        default: f8_conv_gemm_tc_kernel<EPI_GENERIC><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
     }
     return cudaGetLastError();
 }
