@@ -9,10 +9,11 @@
 //     in tensor memory, double buffered so the epilogue of tile i overlaps the main loop of tile i+1.
 //   * Sixteen epilogue warps read the accumulator with tcgen05.ld (one output pixel per thread, 16
 //     consecutive channels per load), add the bias, align and add the residual, apply the rounding
-//     shift and clip (Eq. 2 / signed form applied to Eq. 6).  The 8-bit result is written to a swizzled
-//     staging tile in shared memory and leaves with one TMA store per 128-byte column slab; the
-//     residual tile arrives the same way (TMA load, two tiles ahead), so global memory only sees
-//     full-line accesses.  Shapes that do not fit this scheme use direct 16-byte stores.
+//     shift and clip (Eq. 2 / signed form applied to Eq. 6).  Each warp writes its 32-row piece of the
+//     8-bit result to a private swizzled staging region and stores it with one TMA instruction; its
+//     piece of the residual tensor arrives the same way, two tiles ahead.  Global memory only sees
+//     full-sector accesses and the warps never synchronise with each other.  Shapes that do not fit
+//     this scheme (int32 output, c_out not a multiple of 16) use direct stores.
 //   * Persistent CTAs (one per SM) walk the tile list; tiles that share an A tile are adjacent so that
 //     the activation tensor is read from HBM once and from L2 afterwards.
 //
@@ -33,15 +34,15 @@ namespace {
 
 constexpr int TILE_M = 128;
 constexpr int NUM_EPI_WARPS = 16;          // four warps per TMEM lane quarter, each takes a quarter of the columns
-// A thread that issues a TMA load does not get to issue its next one until the first has been served
-// (about one L2 round trip, whatever the box size), so one producer thread caps a CTA at a few tens of
-// bytes per clock.  Loads from different warps overlap: the k-iterations are dealt round-robin to
-// several producer warps.
-constexpr int NUM_PROD_WARPS = 4;
+// The TMA serves the loads of one thread strictly one after the other, and one load occupies it for
+// several hundred cycles whatever the box size, so a single issuing thread caps a CTA at roughly ten
+// bytes per clock.  Loads issued by different threads (lanes of one warp included) overlap: every
+// (stage, operand) pair therefore has its own lane of the producer warp.
+constexpr int NUM_PROD_WARPS = 1;
 constexpr int MMA_WARP = NUM_PROD_WARPS;
 constexpr int FIRST_EPI_WARP = NUM_PROD_WARPS + 1;
 constexpr int NUM_THREADS = 32 * (NUM_PROD_WARPS + 1 + NUM_EPI_WARPS);   // producers, MMA issuer, epilogue
-constexpr int MAX_STAGES = 8;
+constexpr int MAX_STAGES = 16;          // two producer lanes per stage
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
 constexpr unsigned long long DRAIN_LIMIT_CYCLES = 200000000ull;
@@ -57,12 +58,10 @@ struct TcParams {
     int kb;                   // bytes (= int8 elements) of K per stage: 32, 64 or 128
     int bn;                   // N tile, multiple of 16, <= 256
     int m_tiles, n_tiles;
-    int stages;               // multiple of prod_warps: every stage then has exactly one producer warp, which
-                              // keeps that warp at most one barrier phase ahead of the consumer
-    int prod_warps;           // producer warps in use (<= NUM_PROD_WARPS)
+    int stages;
     uint32_t stage_bytes;     // A + B bytes of one stage (rounded to 1024)
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
-    uint32_t tx_bytes;        // bytes both TMA loads of a stage deliver
+    uint32_t tx_a, tx_b;      // bytes the A / B load of a stage delivers
     uint32_t idesc;           // tcgen05 instruction descriptor
     uint64_t desc_hi;         // constant upper part of the shared-memory matrix descriptors
     const int32_t *bias;
@@ -70,14 +69,14 @@ struct TcParams {
     uint8_t *y;
     int vec_bytes;            // widest aligned store the output rows allow: 16, 8, 4 or 1
     int epi;                  // EPI_* epilogue variant
-    // staged epilogue: the output tile (and the residual tile) pass through shared memory in column
-    // slabs of slab_w bytes per row, written / read by TMA with the matching swizzle
-    int slab_w;               // 16, 32, 64 or 128 bytes
-    int slab_chunks;          // slab_w / 16
-    int n_slabs;              // bn / slab_w
-    uint32_t swz_mask;        // 7, 3, 1 or 0: address bits 7.. XORed into the 16-byte chunk index
-    uint32_t out_bytes;       // TILE_M * bn
-    uint32_t res_off, out_off;   // byte offsets of the two residual / two output buffers behind the stages
+    // staged epilogue: every epilogue warp owns a 32-row x wbytes-column piece of the tile.  It writes the
+    // piece to its own swizzled staging region and stores it with one TMA instruction; the matching
+    // residual piece arrives by TMA, two tiles ahead.  No block-wide synchronisation is involved.
+    int wbytes;               // columns per warp: 16, 32 or 64
+    uint32_t wswz_mask;       // 3, 1 or 0: address bits 7.. XORed into the 16-byte chunk index
+    uint32_t wreg;            // bytes reserved per staging region (multiple of 1024)
+    uint32_t out_off, res_off, bias_off;   // byte offsets behind the stages: [warp][2] output regions,
+                                           // [warp][2] residual regions, int32 bias' of all padded columns
     F8Requant q;
     int *status;
 };
@@ -108,22 +107,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait.  Returns false when the kernel is aborting (this wait or another one ran out).
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                       int code, unsigned long long limit = WAIT_LIMIT_CYCLES) {
-    if (mbar_try_wait(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                            int code) {
     const unsigned long long t0 = clock64();
     unsigned spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
-            if ((unsigned long long)(clock64() - t0) > limit) {
+            if ((unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
                 *abort_flag = 1;
                 atomicCAS(status, 0, code);
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status, code);
 }
 
 __device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w,
@@ -303,13 +307,6 @@ __device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], const int
 
 enum { EPI_GENERIC = 0, EPI_U8 = 1, EPI_U8_RES = 2, EPI_S8 = 3, EPI_S8_RES = 4 };
 
-// Byte offset of 16-byte chunk `chunk` of row `row` inside a staging slab whose rows are slab_w bytes
-// long, in the layout the TMA uses for the matching swizzle mode (chunk index XOR address bits 7..9).
-__device__ __forceinline__ uint32_t slab_offset(int row, int chunk, int slab_w, uint32_t swz_mask) {
-    uint32_t off = (uint32_t)row * slab_w + chunk * 16;
-    return off ^ (((off >> 7) & swz_mask) << 4);
-}
-
 template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -322,11 +319,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     extern __shared__ uint8_t smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 8];
+    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+    __shared__ __align__(8) uint64_t res_bars[NUM_EPI_WARPS][2];   // per epilogue warp: residual piece has landed
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
-    __shared__ int epi_abort;
-    __shared__ __align__(16) int bias_stage[NUM_EPI_WARPS][64];   // per warp: bias of its columns, pre-shifted
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -334,25 +330,28 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const uint32_t empty_bar = smem_u32(&bars[MAX_STAGES]);
     const uint32_t tfull_bar = smem_u32(&bars[2 * MAX_STAGES]);
     const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + 2]);
-    const uint32_t rfull_bar = smem_u32(&bars[2 * MAX_STAGES + 4]);
-    const uint32_t rempty_bar = smem_u32(&bars[2 * MAX_STAGES + 6]);
     const uint32_t smem_base = smem_u32(smem);
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        epi_abort = 0;
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(full_bar + 8 * s, 2);       // one arrival per operand lane
             mbar_init(empty_bar + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
-            mbar_init(tempty_bar + 8 * a, 32 * NUM_EPI_WARPS);
-            mbar_init(rfull_bar + 8 * a, 1);
-            mbar_init(rempty_bar + 8 * a, 1);
+            mbar_init(tempty_bar + 8 * a, NUM_EPI_WARPS);
+            for (int w = 0; w < NUM_EPI_WARPS; ++w) mbar_init(smem_u32(&res_bars[w][a]), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (STAGED) {
+        // bias' = (bias << sh_acc) + 2^(s-1) for every (padded) output column, once per CTA
+        int *bias_all = (int *)(smem + p.bias_off);
+        const int rnd = 1 << (p.q.s - 1);
+        for (int i = threadIdx.x; i < p.n_tiles * p.bn; i += NUM_THREADS)
+            bias_all[i] = ((i < p.c_out && p.bias) ? (__ldg(p.bias + i) << p.q.sh_acc) : 0) + rnd;
     }
     if (warp == MMA_WARP) tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
     tc_fence_before();
@@ -365,71 +364,55 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     volatile int *abortp = &abort_flag;
 
     if (warp < NUM_PROD_WARPS) {
-        // ------------------------------------------------------------------ TMA producers
-        // k-iteration `it` (counted over all tiles of this CTA) belongs to producer warp it % prod_warps; the
-        // residual tiles all go through warp 0 so that they, too, are requested in order
-        if (lane == 0 && warp < p.prod_warps) {
-            uint32_t it = 0;
-            bool have_last = false;
-            uint32_t last_it = 0;           // this thread's most recent stage load (for the drain on abort)
-            int last_res = -1;              // ... and its most recent residual tile
-            int local = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
-                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
-                const int m0 = m_t * TILE_M;
-                if (RES && warp == 0) {
-                    // residual tile of this output tile -> staging buffer (local & 1), two tiles ahead of its use
-                    const int b = local & 1;
-                    if (!mbar_wait(rempty_bar + 8 * b, ((local >> 1) & 1) ^ 1, abortp, p.status, 106)) { ok = false; break; }
-                    const uint32_t rb = rfull_bar + 8 * b;
-                    mbar_expect_tx(rb, p.out_bytes);
-                    for (int sl = 0; sl < p.n_slabs; ++sl)
-                        tma_load_2d(smem_base + p.res_off + b * p.out_bytes + sl * (TILE_M * p.slab_w), &map_r, rb,
-                                    n_t * p.bn + sl * p.slab_w, m0);
-                    last_res = local;
-                }
-                const int ow = m0 % p.wo;
-                const int t1 = m0 / p.wo;
-                const int oh = t1 % p.ho;
-                const int img = t1 / p.ho;
-                const int base_w = ow * p.stride_w - p.pad_w;
-                const int base_h = oh * p.stride_h - p.pad_h;
-                for (int r = 0; ok && r < p.kh; ++r)
-                    for (int s = 0; ok && s < p.kw; ++s)
-                        for (int cc = 0; cc < p.c_chunks; ++cc, ++it) {
-                            if ((int)(it % (uint32_t)p.prod_warps) != warp) continue;
-                            const int stage = (int)(it % (uint32_t)p.stages);
-                            const uint32_t phase = (it / (uint32_t)p.stages) & 1;
-                            if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101)) {
-                                ok = false;
-                                break;
-                            }
-                            const uint32_t fb = full_bar + 8 * stage;
-                            const uint32_t a_dst = smem_base + stage * p.stage_bytes;
-                            mbar_expect_tx(fb, p.tx_bytes);
-                            tma_load_im2col(a_dst, &map_a, fb, cc * p.kb, base_w, base_h, img, (uint16_t)s,
-                                            (uint16_t)r);
-                            tma_load_3d(a_dst + p.a_bytes, &map_b, fb, cc * p.kb, r * p.kw + s, n_t * p.bn);
-                            have_last = true;
-                            last_it = it;
+        // ------------------------------------------------------------------ TMA producer warp
+        // The whole warp walks the k-iterations in order (no divergence, no divisions in the loop); the A
+        // load of the iteration that uses stage `st` is issued by lane 2*st and its B load by lane 2*st+1,
+        // so that consecutive loads sit in different per-thread TMA queues and overlap.
+        int stage = 0;
+        uint32_t phase = 0;
+        bool have_last = false;
+        uint32_t last_phase = 0;            // phase of this lane's most recent load (for the drain on abort)
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+            const int m0 = m_t * TILE_M;
+            const int ow = m0 % p.wo;
+            const int t1 = m0 / p.wo;
+            const int oh = t1 % p.ho;
+            const int img = t1 / p.ho;
+            const int base_w = ow * p.stride_w - p.pad_w;
+            const int base_h = oh * p.stride_h - p.pad_h;
+            const int n_base = n_t * p.bn;
+            int tap = 0;
+            for (int r = 0; ok && r < p.kh; ++r)
+                for (int s = 0; ok && s < p.kw; ++s, ++tap)
+                    for (int c0 = 0; c0 < p.c_chunks * p.kb; c0 += p.kb) {
+                        if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101))) {
+                            ok = false;
+                            break;
                         }
-            }
-            if (!ok) {
-                // Drain: loads of one thread are served in order, so waiting (bounded) for the most recent one
-                // covers everything this thread has in flight before the CTA's shared memory goes away.
-                if (have_last) {
-                    const unsigned long long t0 = clock64();
-                    while (!mbar_try_wait(full_bar + 8 * (last_it % (uint32_t)p.stages), (last_it / (uint32_t)p.stages) & 1) &&
-                           (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
+                        const uint32_t fb = full_bar + 8 * stage;
+                        const uint32_t a_dst = smem_base + stage * p.stage_bytes;
+                        if (lane == 2 * stage) {
+                            mbar_expect_tx(fb, p.tx_a);
+                            tma_load_im2col(a_dst, &map_a, fb, c0, base_w, base_h, img, (uint16_t)s, (uint16_t)r);
+                            have_last = true;
+                            last_phase = phase;
+                        } else if (lane == 2 * stage + 1) {
+                            mbar_expect_tx(fb, p.tx_b);
+                            tma_load_3d(a_dst + p.a_bytes, &map_b, fb, c0, tap, n_base);
+                            have_last = true;
+                            last_phase = phase;
+                        }
+                        if (++stage == p.stages) { stage = 0; phase ^= 1; }
                     }
-                }
-                if (last_res >= 0) {
-                    const unsigned long long t0 = clock64();
-                    while (!mbar_try_wait(rfull_bar + 8 * (last_res & 1), (last_res >> 1) & 1) &&
-                           (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
-                    }
-                }
+        }
+        if (!ok && have_last) {
+            // Drain: loads of one thread are served in order, so waiting (bounded) for the most recent one
+            // covers everything this lane has in flight before the CTA's shared memory goes away.
+            const unsigned long long t0 = clock64();
+            while (!mbar_try_wait(full_bar + 8 * (lane >> 1), last_phase) &&
+                   (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
             }
         }
     } else if (warp == MMA_WARP) {
@@ -442,6 +425,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             bool committed_any = false;
             int last_acc = 0;
             uint32_t last_acc_phase = 0;
+            const uint64_t a_desc0 = p.desc_hi | (uint64_t)((smem_base & 0x3ffffu) >> 4);
+            const uint32_t stage16 = p.stage_bytes >> 4, a16 = p.a_bytes >> 4;
+            const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
                 const uint32_t acc_phase = (local >> 1) & 1;
@@ -451,12 +437,15 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 for (int kc = 0; kc < k_iters; ++kc) {
                     if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, 103)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_base + stage * p.stage_bytes;
-                    const uint32_t b_addr = a_addr + p.a_bytes;
-                    const uint64_t a_desc = p.desc_hi | (uint64_t)((a_addr & 0x3ffffu) >> 4);
-                    const uint64_t b_desc = p.desc_hi | (uint64_t)((b_addr & 0x3ffffu) >> 4);
-                    for (int j = 0; j < p.kb / 32; ++j)   // 32 bytes of K per instruction: +2 in 16-byte units
-                        mma_i8(d_tmem, a_desc + 2 * j, b_desc + 2 * j, p.idesc, (kc | j) != 0 ? 1u : 0u);
+                    const uint64_t a_desc = a_desc0 + (uint64_t)(stage * stage16);
+                    const uint64_t b_desc = a_desc + a16;
+                    // 32 bytes of K per instruction: the descriptor start address advances by 2 (16-byte units)
+                    mma_i8(d_tmem, a_desc, b_desc, p.idesc, kc != 0 ? 1u : 0u);
+                    if (mmas >= 2) mma_i8(d_tmem, a_desc + 2, b_desc + 2, p.idesc, 1u);
+                    if (mmas == 4) {
+                        mma_i8(d_tmem, a_desc + 4, b_desc + 4, p.idesc, 1u);
+                        mma_i8(d_tmem, a_desc + 6, b_desc + 6, p.idesc, 1u);
+                    }
                     mma_commit(empty_bar + 8 * stage);    // frees the stage when these MMAs have read it
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
@@ -483,93 +472,121 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const int per_group = (chunks + 3) / 4;     // <= 4 chunks of 16 columns per warp
         const int ch_begin = min(group * per_group, chunks);
         const int nch = min(ch_begin + per_group, chunks) - ch_begin;
-        const int tile_row = quarter * 32 + lane;   // this thread's row of the tile
-        const bool issuer = ew == 0 && lane == 0;   // the thread that owns the bulk-store groups
-        int *bias_w = bias_stage[ew];
         const int mul_acc = 1 << p.q.sh_acc, mul_res = 1 << p.q.sh_res;
         int local = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
-            const int acc = local & 1;
-            const uint32_t acc_phase = (local >> 1) & 1;
-            const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
-            const int n0 = n_t * p.bn;
-            const size_t row = (size_t)m_t * TILE_M + tile_row;
-            const bool row_valid = row < (size_t)p.M;
-            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
-            if (STAGED) {
-                const int b = local & 1;
-                // bias of this warp's columns (+ rounding constant) -> shared memory, before the accumulator is ready
+        if (STAGED) {
+            const bool leader = lane == 0;           // owns this warp's bulk-store groups
+            const bool fetcher = lane == 1;          // requests this warp's residual pieces
+            const int *bias_all = (const int *)(smem + p.bias_off);
+            uint8_t *out_reg = smem + p.out_off + (uint32_t)(ew * 2) * p.wreg;
+            uint8_t *res_reg = smem + p.res_off + (uint32_t)(ew * 2) * p.wreg;
+            const uint32_t rbar = smem_u32(&res_bars[ew][0]);
+            const uint32_t piece_bytes = 32u * p.wbytes;
+            int res_pending[2] = {-1, -1};          // tile-sequence number whose residual piece is in flight
+            // chunk c of row `lane` inside a region
+            uint32_t so[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t off = (uint32_t)lane * p.wbytes + i * 16;
+                so[i] = off ^ (((off >> 7) & p.wswz_mask) << 4);
+            }
+            auto piece_exists = [&](int tile_id) {
+                const int nt = tile_id % p.n_tiles;
+                return nch > 0 && nt * p.bn + ch_begin * 16 < p.c_out;
+            };
+            auto request_residual = [&](int tile_id, int seq) {       // fetcher lane only
+                if (!piece_exists(tile_id)) return;
+                const int mt = tile_id / p.n_tiles, nt = tile_id - mt * p.n_tiles;
+                const uint32_t bar = rbar + 8 * (seq & 1);
+                mbar_expect_tx(bar, piece_bytes);
+                tma_load_2d(smem_u32(res_reg) + (seq & 1) * p.wreg, &map_r, bar, nt * p.bn + ch_begin * 16,
+                            mt * TILE_M + quarter * 32);
+                res_pending[seq & 1] = seq;
+            };
+            if (RES && fetcher) {
+                if ((int)blockIdx.x < total_tiles) request_residual(blockIdx.x, 0);
+                if ((int)(blockIdx.x + gridDim.x) < total_tiles) request_residual(blockIdx.x + gridDim.x, 1);
+            }
+            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+                const int acc = local & 1;
+                const uint32_t acc_phase = (local >> 1) & 1;
+                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+                const int n0 = n_t * p.bn;
                 const int c_first = n0 + ch_begin * 16;
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
-                __syncwarp();
-                if (lane < 16) {
-                    const int c0 = c_first + lane * 4;
-                    int4 bv = make_int4(0, 0, 0, 0);
-                    if (p.bias && lane * 4 < my_nch * 16) bv = __ldg((const int4 *)(p.bias + c0));
-                    const int rnd = 1 << (p.q.s - 1);        // rounding constant folded into the bias
-                    bv.x = (bv.x << p.q.sh_acc) + rnd; bv.y = (bv.y << p.q.sh_acc) + rnd;
-                    bv.z = (bv.z << p.q.sh_acc) + rnd; bv.w = (bv.w << p.q.sh_acc) + rnd;
-                    *(int4 *)(bias_w + lane * 4) = bv;
-                }
-                __syncwarp();
-                // A thread whose wait runs out keeps going through this tile (the kernel is aborting and the
-                // whole group leaves together at the next check) so that nobody is left alone at a barrier.
-                mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104);
-                if (RES) mbar_wait(rfull_bar + 8 * b, acc_phase, abortp, p.status, 107);
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
+                bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104);
+                if (RES && my_nch > 0) got = mbar_wait(rbar + 8 * acc, acc_phase, abortp, p.status, 107) && got;
+                if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tc_fence_after();
-                if (issuer) {
-                    // the store issued from this output buffer two tiles ago must have finished reading it
-                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    epi_abort = *abortp;
-                }
-                asm volatile("bar.sync 1, %0;" ::"n"(32 * NUM_EPI_WARPS) : "memory");
-                if (epi_abort) { ok = false; break; }
-                uint8_t *out_buf = smem + p.out_off + b * p.out_bytes;
-                const uint8_t *res_buf = smem + p.res_off + b * p.out_bytes;
+                // the store this warp issued from this region two tiles ago must have finished reading it
+                if (leader) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                __syncwarp();
+                uint8_t *out_buf = out_reg + acc * p.wreg;
+                const uint8_t *res_buf = res_reg + acc * p.wreg;
                 int va[16], vb[16];
                 if (my_nch > 0) tmem_ld16(t_addr, va);
 #pragma unroll
                 for (int i = 0; i < 4; i += 2) {
                     if (i < my_nch) {
-                        const int ch = ch_begin + i;
-                        const uint32_t so = (uint32_t)(ch / p.slab_chunks) * (TILE_M * p.slab_w) +
-                                            slab_offset(tile_row, ch % p.slab_chunks, p.slab_w, p.swz_mask);
                         uint4 rw = make_uint4(0, 0, 0, 0);
-                        if (RES) rw = *(const uint4 *)(res_buf + so);
+                        if (RES) rw = *(const uint4 *)(res_buf + so[i]);
                         tmem_ld_wait();
                         if (i + 1 < my_nch) tmem_ld16(t_addr + (i + 1) * 16, vb);
-                        const int4 *b4 = (const int4 *)(bias_w + i * 16);
-                        *(uint4 *)(out_buf + so) = epilogue_fast16<RES, SGN>(va, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s);
+                        const int4 *b4 = (const int4 *)(bias_all + c_first + i * 16);
+                        *(uint4 *)(out_buf + so[i]) = epilogue_fast16<RES, SGN>(va, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s);
                     }
                     if (i + 1 < my_nch) {
-                        const int ch = ch_begin + i + 1;
-                        const uint32_t so = (uint32_t)(ch / p.slab_chunks) * (TILE_M * p.slab_w) +
-                                            slab_offset(tile_row, ch % p.slab_chunks, p.slab_w, p.swz_mask);
                         uint4 rw = make_uint4(0, 0, 0, 0);
-                        if (RES) rw = *(const uint4 *)(res_buf + so);
+                        if (RES) rw = *(const uint4 *)(res_buf + so[i + 1]);
                         tmem_ld_wait();
                         if (i + 2 < my_nch) tmem_ld16(t_addr + (i + 2) * 16, va);
-                        const int4 *b4 = (const int4 *)(bias_w + (i + 1) * 16);
-                        *(uint4 *)(out_buf + so) = epilogue_fast16<RES, SGN>(vb, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s);
+                        const int4 *b4 = (const int4 *)(bias_all + c_first + (i + 1) * 16);
+                        *(uint4 *)(out_buf + so[i + 1]) = epilogue_fast16<RES, SGN>(vb, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s);
                     }
                 }
-                // the accumulator has been read: hand it back to the MMA warp
+                // the accumulator has been read; the writes above must be visible to the TMA
                 tc_fence_before();
-                mbar_arrive(tempty_bar + 8 * acc);
-                // make the generic-proxy writes visible to the TMA, then one thread stores the tile
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                asm volatile("bar.sync 2, %0;" ::"n"(32 * NUM_EPI_WARPS) : "memory");
-                if (issuer) {
-                    for (int sl = 0; sl < p.n_slabs; ++sl)
-                        if (n0 + sl * p.slab_w < p.c_out)
-                            tma_store_2d(&map_y, smem_u32(out_buf) + sl * (TILE_M * p.slab_w), n0 + sl * p.slab_w,
-                                         m_t * TILE_M);
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    if (RES) mbar_arrive(rempty_bar + 8 * b);     // everyone is past the barrier: residual buffer is free
+                __syncwarp();
+                if (leader) {
+                    mbar_arrive(tempty_bar + 8 * acc);            // hand the accumulator back to the MMA warp
+                    if (my_nch > 0) {
+                        tma_store_2d(&map_y, smem_u32(out_buf), c_first, m_t * TILE_M + quarter * 32);
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
                 }
-            } else {
-                if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104)) { ok = false; break; }
+                if (RES && fetcher) {
+                    res_pending[acc] = -1;
+                    const int next = tile + 2 * (int)gridDim.x;     // the tile that will use this region next
+                    if (next < total_tiles) request_residual(next, local + 2);
+                }
+            }
+            if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            if (fetcher) {
+                if (RES && !ok) {
+                    // aborting: give residual pieces that are still in flight time to land
+                    for (int b = 0; b < 2; ++b)
+                        if (res_pending[b] >= 0) {
+                            const unsigned long long t0 = clock64();
+                            while (!mbar_try_wait(rbar + 8 * b, (res_pending[b] >> 1) & 1) &&
+                                   (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
+                            }
+                        }
+                }
+            }
+        } else {
+            const int tile_row = quarter * 32 + lane;   // this thread's row of the tile
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+                const int acc = local & 1;
+                const uint32_t acc_phase = (local >> 1) & 1;
+                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+                const int n0 = n_t * p.bn;
+                const size_t row = (size_t)m_t * TILE_M + tile_row;
+                const bool row_valid = row < (size_t)p.M;
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
+                if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104))) { ok = false; break; }
                 tc_fence_after();
                 for (int i = 0; i < nch; ++i) {
                     const int co0 = n0 + (ch_begin + i) * 16;
@@ -580,10 +597,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     epilogue_chunk(p, v, row, co0, row_valid);
                 }
                 tc_fence_before();
-                mbar_arrive(tempty_bar + 8 * acc);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
             }
         }
-        if (STAGED && issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     tc_fence_before();
@@ -664,8 +681,8 @@ int choose_bn(int c_out) {
     return (c_out + 15) / 16 * 16;
 }
 
-// N tile of the staged epilogue: a power of two up to 128, or 256 (two 128-byte slabs) when no residual
-// buffers are needed; the TMA store clips columns beyond c_out.
+// N tile of the staged epilogue: a power of two up to 128, or 256 when no residual regions are needed
+// (the per-warp staging regions grow with the tile width); the TMA store clips columns beyond c_out.
 int choose_bn_staged(int c_out, bool has_res) {
     if (c_out > 128 && !has_res) return 256;
     int bn = 16;
@@ -731,15 +748,17 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.a_bytes = (uint32_t)(TILE_M * p.kb + 1023) / 1024 * 1024;
     const uint32_t b_bytes = (uint32_t)(p.bn * p.kb + 1023) / 1024 * 1024;
     p.stage_bytes = p.a_bytes + b_bytes;
-    p.tx_bytes = (uint32_t)((TILE_M + p.bn) * p.kb);
+    p.tx_a = (uint32_t)(TILE_M * p.kb);
+    p.tx_b = (uint32_t)(p.bn * p.kb);
     size_t staging = 0;
     if (staged) {
-        p.slab_w = p.bn < 128 ? p.bn : 128;
-        p.slab_chunks = p.slab_w / 16;
-        p.n_slabs = p.bn / p.slab_w;
-        p.swz_mask = p.slab_w == 128 ? 7u : (p.slab_w == 64 ? 3u : (p.slab_w == 32 ? 1u : 0u));
-        p.out_bytes = (uint32_t)(TILE_M * p.bn);
-        staging = (size_t)p.out_bytes * (q.has_res ? 4 : 2);
+        const int per_group = (p.bn / 16 + 3) / 4;
+        p.wbytes = per_group * 16;
+        p.wswz_mask = p.wbytes == 64 ? 3u : (p.wbytes == 32 ? 1u : 0u);
+        p.wreg = (uint32_t)(32 * p.wbytes + 1023) / 1024 * 1024;
+        const size_t regions = (size_t)NUM_EPI_WARPS * 2 * p.wreg;
+        const size_t bias_bytes = ((size_t)p.n_tiles * p.bn * 4 + 1023) / 1024 * 1024;
+        staging = regions * (q.has_res ? 2 : 1) + bias_bytes;
     }
     int stages = (int)((SMEM_LIMIT - 1024 - staging) / p.stage_bytes);
     if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -747,11 +766,10 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         *why = "stage does not fit";
         return cudaErrorInvalidValue;
     }
-    p.prod_warps = stages >= NUM_PROD_WARPS ? NUM_PROD_WARPS : stages;
-    stages -= stages % p.prod_warps;
     p.stages = stages;
-    p.res_off = (uint32_t)(p.stages * p.stage_bytes);
-    p.out_off = p.res_off + (q.has_res ? 2 * p.out_bytes : 0);
+    p.out_off = (uint32_t)(p.stages * p.stage_bytes);
+    p.res_off = p.out_off + (uint32_t)NUM_EPI_WARPS * 2 * p.wreg;
+    p.bias_off = p.res_off + (q.has_res ? (uint32_t)NUM_EPI_WARPS * 2 * p.wreg : 0u);
     // instruction descriptor: D = s32 (2 at bit 4), A format at bit 7 (0 = u8, 1 = s8), B = s8 at bit 10,
     // both operands K-major, N/8 at bit 17, M/16 at bit 24
     p.idesc = (2u << 4) | ((g.x_signed ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) |
@@ -797,17 +815,16 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
             return cudaErrorInvalidValue;
         }
     }
-    // output / residual [M, c_out] bytes, one box = one column slab of a tile
+    // output / residual [M, c_out] bytes, one box = the 32-row piece of one epilogue warp
     plan->map_y = plan->map_b;
     plan->map_r = plan->map_b;
     if (staged) {
         cuuint64_t dims[2] = {(cuuint64_t)g.c_out, (cuuint64_t)p.M};
         cuuint64_t strides[1] = {(cuuint64_t)g.c_out};
-        cuuint32_t box[2] = {(cuuint32_t)p.slab_w, (cuuint32_t)TILE_M};
+        cuuint32_t box[2] = {(cuuint32_t)p.wbytes, 32};
         cuuint32_t estr[2] = {1, 1};
-        const CUtensorMapSwizzle sw = p.slab_w == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
-                                      : (p.slab_w == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
-                                         : (p.slab_w == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE));
+        const CUtensorMapSwizzle sw = p.wbytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                      : (p.wbytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE);
         CUresult r = g_encode_tiled(&plan->map_y, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, y, dims, strides, box, estr,
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
