@@ -9,11 +9,12 @@
 //     in tensor memory, double buffered so the epilogue of tile i overlaps the main loop of tile i+1.
 //   * Sixteen epilogue warps read the accumulator with tcgen05.ld (one output pixel per thread, 16
 //     consecutive channels per load), add the bias, align and add the residual, apply the rounding
-//     shift and clip (Eq. 2 / signed form applied to Eq. 6).  Each warp writes its 32-row piece of the
-//     8-bit result to a private swizzled staging region and stores it with one TMA instruction; its
-//     piece of the residual tensor arrives the same way, two tiles ahead.  Global memory only sees
-//     full-sector accesses and the warps never synchronise with each other.  Shapes that do not fit
-//     this scheme (int32 output, c_out not a multiple of 16) use direct stores.
+//     shift and clip (Eq. 2 / signed form applied to Eq. 6).  The 8-bit result goes to a swizzled staging
+//     tile in shared memory; a mover thread stores finished tiles with one TMA instruction per 128-byte
+//     column slab and a fetcher thread brings in the residual tiles the same way, two tiles ahead.  All
+//     hand-offs are mbarriers, nobody waits at a block-wide barrier, and global memory only sees
+//     full-line accesses.  Shapes that do not fit this scheme (int32 output, c_out not a multiple of
+//     16) use direct stores.
 //   * Persistent CTAs (one per SM) walk the tile list; tiles that share an A tile are adjacent so that
 //     the activation tensor is read from HBM once and from L2 afterwards.
 //
@@ -39,9 +40,11 @@ constexpr int NUM_EPI_WARPS = 16;          // four warps per TMEM lane quarter, 
 // bytes per clock.  Loads issued by different threads (lanes of one warp included) overlap: every
 // (stage, operand) pair therefore has its own lane of the producer warp.
 constexpr int NUM_PROD_WARPS = 1;
-constexpr int MMA_WARP = NUM_PROD_WARPS;
-constexpr int FIRST_EPI_WARP = NUM_PROD_WARPS + 1;
-constexpr int NUM_THREADS = 32 * (NUM_PROD_WARPS + 1 + NUM_EPI_WARPS);   // producers, MMA issuer, epilogue
+constexpr int MMA_WARP = 1;
+constexpr int MOVER_WARP = 2;              // one thread stores finished output tiles
+constexpr int FETCH_WARP = 3;              // one thread fetches residual tiles
+constexpr int FIRST_EPI_WARP = 4;
+constexpr int NUM_THREADS = 32 * (FIRST_EPI_WARP + NUM_EPI_WARPS);   // producer, MMA issuer, mover, fetcher, epilogue
 constexpr int MAX_STAGES = 16;          // two producer lanes per stage
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
@@ -69,14 +72,16 @@ struct TcParams {
     uint8_t *y;
     int vec_bytes;            // widest aligned store the output rows allow: 16, 8, 4 or 1
     int epi;                  // EPI_* epilogue variant
-    // staged epilogue: every epilogue warp owns a 32-row x wbytes-column piece of the tile.  It writes the
-    // piece to its own swizzled staging region and stores it with one TMA instruction; the matching
-    // residual piece arrives by TMA, two tiles ahead.  No block-wide synchronisation is involved.
-    int wbytes;               // columns per warp: 16, 32 or 64
-    uint32_t wswz_mask;       // 3, 1 or 0: address bits 7.. XORed into the 16-byte chunk index
-    uint32_t wreg;            // bytes reserved per staging region (multiple of 1024)
-    uint32_t out_off, res_off, bias_off;   // byte offsets behind the stages: [warp][2] output regions,
-                                           // [warp][2] residual regions, int32 bias' of all padded columns
+    // staged epilogue: the output tile (and the residual tile) pass through shared memory in column
+    // slabs of slab_w bytes per row, written / read by TMA with the matching swizzle (few, large TMA
+    // operations: the TMA serves roughly one operation per hundred cycles whatever its size)
+    int slab_w;               // 16, 32, 64 or 128 bytes
+    int slab_chunks;          // slab_w / 16
+    int n_slabs;              // bn / slab_w
+    uint32_t swz_mask;        // 7, 3, 1 or 0: address bits 7.. XORed into the 16-byte chunk index
+    uint32_t out_bytes;       // TILE_M * bn
+    uint32_t out_off, res_off, bias_off;   // byte offsets behind the stages: two output tiles, two residual
+                                           // tiles, int32 bias' of all padded columns
     F8Requant q;
     int *status;
 };
@@ -320,7 +325,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
-    __shared__ __align__(8) uint64_t res_bars[NUM_EPI_WARPS][2];   // per epilogue warp: residual piece has landed
+    __shared__ __align__(8) uint64_t epi_bars[8];   // out_full[2], out_free[2], res_full[2], res_free[2]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -331,6 +336,8 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const uint32_t tfull_bar = smem_u32(&bars[2 * MAX_STAGES]);
     const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + 2]);
     const uint32_t smem_base = smem_u32(smem);
+    const uint32_t out_full = smem_u32(&epi_bars[0]), out_free = smem_u32(&epi_bars[2]);
+    const uint32_t res_full = smem_u32(&epi_bars[4]), res_free = smem_u32(&epi_bars[6]);
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -341,7 +348,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
             mbar_init(tempty_bar + 8 * a, NUM_EPI_WARPS);
-            for (int w = 0; w < NUM_EPI_WARPS; ++w) mbar_init(smem_u32(&res_bars[w][a]), 1);
+            mbar_init(smem_u32(&epi_bars[0 + a]), NUM_EPI_WARPS);   // out_full: every epilogue warp has written its part
+            mbar_init(smem_u32(&epi_bars[2 + a]), 1);               // out_free: the store has finished reading the tile
+            mbar_init(smem_u32(&epi_bars[4 + a]), 1);               // res_full: residual tile has landed (transaction count)
+            mbar_init(smem_u32(&epi_bars[6 + a]), NUM_EPI_WARPS);   // res_free: every epilogue warp has read its part
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -463,6 +473,54 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 }
             }
         }
+    } else if (warp == MOVER_WARP) {
+        // ------------------------------------------------------------------ output mover
+        if (STAGED && lane == 0) {
+            // stores: tile t leaves from output buffer t & 1 once all epilogue warps have written it
+            int local = 0;
+            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+                const int b = local & 1;
+                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+                if (!mbar_wait(out_full + 8 * b, (local >> 1) & 1, abortp, p.status, 108)) break;
+                const uint32_t src = smem_base + p.out_off + b * p.out_bytes;
+                for (int sl = 0; sl < p.n_slabs; ++sl)
+                    if (n_t * p.bn + sl * p.slab_w < p.c_out)
+                        tma_store_2d(&map_y, src + sl * (TILE_M * p.slab_w), n_t * p.bn + sl * p.slab_w, m_t * TILE_M);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                // the buffer is free again as soon as the store has read it (the next tile uses the other one)
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                mbar_arrive(out_free + 8 * b);
+            }
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        }
+    } else if (warp == FETCH_WARP) {
+        // ------------------------------------------------------------------ residual fetcher
+        if (RES && lane == 0) {
+            // residual tiles: up to two tiles ahead of the epilogue
+            int local = 0;
+            int last = -1;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+                const int b = local & 1;
+                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+                if (!mbar_wait(res_free + 8 * b, ((local >> 1) & 1) ^ 1, abortp, p.status, 106)) { ok = false; break; }
+                const uint32_t rb = res_full + 8 * b;
+                mbar_expect_tx(rb, p.out_bytes);
+                for (int sl = 0; sl < p.n_slabs; ++sl)
+                    tma_load_2d(smem_base + p.res_off + b * p.out_bytes + sl * (TILE_M * p.slab_w), &map_r, rb,
+                                n_t * p.bn + sl * p.slab_w, m_t * TILE_M);
+                last = local;
+            }
+            if (!ok && last >= 0) {
+                // aborting: give the loads that are still in flight time to land
+                for (int i = 0; i < 2 && last - i >= 0; ++i) {
+                    const unsigned long long t0 = clock64();
+                    while (!mbar_try_wait(res_full + 8 * ((last - i) & 1), ((last - i) >> 1) & 1) &&
+                           (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
+                    }
+                }
+            }
+        }
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 belong to this warp
@@ -476,55 +534,31 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         int local = 0;
         bool ok = true;
         if (STAGED) {
-            const bool leader = lane == 0;           // owns this warp's bulk-store groups
-            const bool fetcher = lane == 1;          // requests this warp's residual pieces
             const int *bias_all = (const int *)(smem + p.bias_off);
-            uint8_t *out_reg = smem + p.out_off + (uint32_t)(ew * 2) * p.wreg;
-            uint8_t *res_reg = smem + p.res_off + (uint32_t)(ew * 2) * p.wreg;
-            const uint32_t rbar = smem_u32(&res_bars[ew][0]);
-            const uint32_t piece_bytes = 32u * p.wbytes;
-            int res_pending[2] = {-1, -1};          // tile-sequence number whose residual piece is in flight
-            // chunk c of row `lane` inside a region
+            const int tile_row = quarter * 32 + lane;
+            // where this thread's 16-byte chunks live inside a staged tile (same for every tile)
             uint32_t so[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                uint32_t off = (uint32_t)lane * p.wbytes + i * 16;
-                so[i] = off ^ (((off >> 7) & p.wswz_mask) << 4);
-            }
-            auto piece_exists = [&](int tile_id) {
-                const int nt = tile_id % p.n_tiles;
-                return nch > 0 && nt * p.bn + ch_begin * 16 < p.c_out;
-            };
-            auto request_residual = [&](int tile_id, int seq) {       // fetcher lane only
-                if (!piece_exists(tile_id)) return;
-                const int mt = tile_id / p.n_tiles, nt = tile_id - mt * p.n_tiles;
-                const uint32_t bar = rbar + 8 * (seq & 1);
-                mbar_expect_tx(bar, piece_bytes);
-                tma_load_2d(smem_u32(res_reg) + (seq & 1) * p.wreg, &map_r, bar, nt * p.bn + ch_begin * 16,
-                            mt * TILE_M + quarter * 32);
-                res_pending[seq & 1] = seq;
-            };
-            if (RES && fetcher) {
-                if ((int)blockIdx.x < total_tiles) request_residual(blockIdx.x, 0);
-                if ((int)(blockIdx.x + gridDim.x) < total_tiles) request_residual(blockIdx.x + gridDim.x, 1);
+                const int ch = ch_begin + i;
+                uint32_t off = (uint32_t)tile_row * p.slab_w + (ch % p.slab_chunks) * 16;
+                off ^= ((off >> 7) & p.swz_mask) << 4;
+                so[i] = (uint32_t)(ch / p.slab_chunks) * (TILE_M * p.slab_w) + off;
             }
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
-                const int acc = local & 1;
+                const int acc = local & 1;                   // accumulator, output buffer and residual buffer in use
                 const uint32_t acc_phase = (local >> 1) & 1;
-                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
-                const int n0 = n_t * p.bn;
-                const int c_first = n0 + ch_begin * 16;
+                const int n_t = tile % p.n_tiles;
+                const int c_first = n_t * p.bn + ch_begin * 16;
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
                 bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104);
-                if (RES && my_nch > 0) got = mbar_wait(rbar + 8 * acc, acc_phase, abortp, p.status, 107) && got;
+                if (RES) got = mbar_wait(res_full + 8 * acc, acc_phase, abortp, p.status, 107) && got;
+                got = mbar_wait(out_free + 8 * acc, acc_phase ^ 1, abortp, p.status, 109) && got;
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tc_fence_after();
-                // the store this warp issued from this region two tiles ago must have finished reading it
-                if (leader) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                __syncwarp();
-                uint8_t *out_buf = out_reg + acc * p.wreg;
-                const uint8_t *res_buf = res_reg + acc * p.wreg;
+                uint8_t *out_buf = smem + p.out_off + acc * p.out_bytes;
+                const uint8_t *res_buf = smem + p.res_off + acc * p.out_bytes;
                 int va[16], vb[16];
                 if (my_nch > 0) tmem_ld16(t_addr, va);
 #pragma unroll
@@ -546,34 +580,15 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         *(uint4 *)(out_buf + so[i + 1]) = epilogue_fast16<RES, SGN>(vb, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s);
                     }
                 }
-                // the accumulator has been read; the writes above must be visible to the TMA
+                // accumulator and residual have been read, the output part is written: make the writes
+                // visible to the TMA and tell the MMA warp, the mover and the fetcher
                 tc_fence_before();
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
-                if (leader) {
-                    mbar_arrive(tempty_bar + 8 * acc);            // hand the accumulator back to the MMA warp
-                    if (my_nch > 0) {
-                        tma_store_2d(&map_y, smem_u32(out_buf), c_first, m_t * TILE_M + quarter * 32);
-                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    }
-                }
-                if (RES && fetcher) {
-                    res_pending[acc] = -1;
-                    const int next = tile + 2 * (int)gridDim.x;     // the tile that will use this region next
-                    if (next < total_tiles) request_residual(next, local + 2);
-                }
-            }
-            if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-            if (fetcher) {
-                if (RES && !ok) {
-                    // aborting: give residual pieces that are still in flight time to land
-                    for (int b = 0; b < 2; ++b)
-                        if (res_pending[b] >= 0) {
-                            const unsigned long long t0 = clock64();
-                            while (!mbar_try_wait(rbar + 8 * b, (res_pending[b] >> 1) & 1) &&
-                                   (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
-                            }
-                        }
+                if (lane == 0) {
+                    mbar_arrive(tempty_bar + 8 * acc);
+                    mbar_arrive(out_full + 8 * acc);
+                    if (RES) mbar_arrive(res_free + 8 * acc);
                 }
             }
         } else {
@@ -681,8 +696,8 @@ int choose_bn(int c_out) {
     return (c_out + 15) / 16 * 16;
 }
 
-// N tile of the staged epilogue: a power of two up to 128, or 256 when no residual regions are needed
-// (the per-warp staging regions grow with the tile width); the TMA store clips columns beyond c_out.
+// N tile of the staged epilogue: a power of two up to 128, or 256 (two 128-byte slabs) when no residual
+// buffers are needed; the TMA store clips columns beyond c_out.
 int choose_bn_staged(int c_out, bool has_res) {
     if (c_out > 128 && !has_res) return 256;
     int bn = 16;
@@ -752,13 +767,13 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.tx_b = (uint32_t)(p.bn * p.kb);
     size_t staging = 0;
     if (staged) {
-        const int per_group = (p.bn / 16 + 3) / 4;
-        p.wbytes = per_group * 16;
-        p.wswz_mask = p.wbytes == 64 ? 3u : (p.wbytes == 32 ? 1u : 0u);
-        p.wreg = (uint32_t)(32 * p.wbytes + 1023) / 1024 * 1024;
-        const size_t regions = (size_t)NUM_EPI_WARPS * 2 * p.wreg;
+        p.slab_w = p.bn < 128 ? p.bn : 128;
+        p.slab_chunks = p.slab_w / 16;
+        p.n_slabs = p.bn / p.slab_w;
+        p.swz_mask = p.slab_w == 128 ? 7u : (p.slab_w == 64 ? 3u : (p.slab_w == 32 ? 1u : 0u));
+        p.out_bytes = (uint32_t)(TILE_M * p.bn + 1023) / 1024 * 1024;
         const size_t bias_bytes = ((size_t)p.n_tiles * p.bn * 4 + 1023) / 1024 * 1024;
-        staging = regions * (q.has_res ? 2 : 1) + bias_bytes;
+        staging = (size_t)p.out_bytes * (q.has_res ? 4 : 2) + bias_bytes;
     }
     int stages = (int)((SMEM_LIMIT - 1024 - staging) / p.stage_bytes);
     if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -768,8 +783,8 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     }
     p.stages = stages;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
-    p.res_off = p.out_off + (uint32_t)NUM_EPI_WARPS * 2 * p.wreg;
-    p.bias_off = p.res_off + (q.has_res ? (uint32_t)NUM_EPI_WARPS * 2 * p.wreg : 0u);
+    p.res_off = p.out_off + 2 * p.out_bytes;
+    p.bias_off = p.res_off + (q.has_res ? 2 * p.out_bytes : 0u);
     // instruction descriptor: D = s32 (2 at bit 4), A format at bit 7 (0 = u8, 1 = s8), B = s8 at bit 10,
     // both operands K-major, N/8 at bit 17, M/16 at bit 24
     p.idesc = (2u << 4) | ((g.x_signed ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) |
@@ -815,16 +830,17 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
             return cudaErrorInvalidValue;
         }
     }
-    // output / residual [M, c_out] bytes, one box = the 32-row piece of one epilogue warp
+    // output / residual [M, c_out] bytes, one box = one column slab of a tile
     plan->map_y = plan->map_b;
     plan->map_r = plan->map_b;
     if (staged) {
         cuuint64_t dims[2] = {(cuuint64_t)g.c_out, (cuuint64_t)p.M};
         cuuint64_t strides[1] = {(cuuint64_t)g.c_out};
-        cuuint32_t box[2] = {(cuuint32_t)p.wbytes, 32};
+        cuuint32_t box[2] = {(cuuint32_t)p.slab_w, (cuuint32_t)TILE_M};
         cuuint32_t estr[2] = {1, 1};
-        const CUtensorMapSwizzle sw = p.wbytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
-                                      : (p.wbytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE);
+        const CUtensorMapSwizzle sw = p.slab_w == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                      : (p.slab_w == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                         : (p.slab_w == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE));
         CUresult r = g_encode_tiled(&plan->map_y, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, y, dims, strides, box, estr,
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
