@@ -185,6 +185,21 @@ def measured_peaks():
         return 6650.0, "fallback"
 
 
+def measured_traffic():
+    """DRAM bytes per step of the tensor-core conv kernel from the committed ncu summary, or None when the
+    kernel source has changed since those counters were taken."""
+    import hashlib
+    import re
+    try:
+        text = open(os.path.join(ROOT, "profiles", "dram_traffic_resnet50_b256.md")).read()
+        sha = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text).group(1)
+        traffic = int(re.search(r"traffic_bytes_per_step:\s*(\d+)", text).group(1))
+        src = open(os.path.join(ROOT, "paper_2202_05239_b200", "csrc", "f8_gemm_tc.cu"), "rb").read()
+        return traffic if hashlib.sha256(src).hexdigest() == sha else None
+    except (OSError, AttributeError, ValueError):
+        return None
+
+
 def run_ours(args):
     import torch
     from paper_2202_05239_b200 import api
@@ -298,7 +313,8 @@ def run_ours(args):
         "kernel": "f8_conv_gemm_tc_kernel",
         "bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
         "peak_source": f"{peak_kind} HBM copy bandwidth",
-        "traffic": None,
+        "traffic": measured_traffic(),
+        "traffic_note": "DRAM bytes of all launches of this kernel in one step (ncu, profiles/dram_traffic_resnet50_b256.md)",
         "launches_per_step": int(sum(tc_flags)), "kernel_ms_per_step": tc_ms,
         "algorithmic_bytes_per_step": tc_bytes,
         "tensor": {"achieved_tops": tc_ops / (tc_ms * 1e-3) / 1e12 if tc_ms > 0 else 0.0,
