@@ -192,6 +192,40 @@ void f8_debug_force_direct(int on);
  * the caller can time the launch and obtain the attainable INT8 rate of the device. */
 f8_status f8_mma_i8_probe(int iters, double *ops, void *cuda_stream);
 
+/* ---------------------------------------------------------------- a call that allocates nothing */
+
+/* Largest input, in bytes of its 8-bytes-per-pixel padded copy (n * h * wp * 8, wp about w + pad), that
+ * f8_stem_conv2d_fixed_static accepts: 40 images of 224 x 224 at once. */
+#define F8_STATIC_STEM_MAX_BYTES ((size_t)16 * 1024 * 1024)
+
+/* The paper has no counterpart to this entry point; it exists for callers that may not allocate
+ * device memory at the moment they need a result: code running under a framework that has reserved
+ * the whole device for its own pool, a real-time loop that must not take the allocator's lock, or a
+ * host that hands this library a fixed memory budget.  Every other entry point either takes a caller
+ * workspace or (f8_net_create, the first use of the status word) calls cudaMalloc.
+ *
+ * It computes the same thing as f8_conv2d_fixed for a few-channel first layer ("stem": c <= 8, even
+ * stride, kw <= 32, no residual, 8-bit output), on the tensor cores: the image is widened to 8 bytes
+ * per pixel, the weights are re-packed to match, and the convolution runs over that copy.  The copy,
+ * the packed weights and the kernel's status word live in one array that is part of the library image
+ * (about 16 MiB of device memory on every GPU that loads the library, until the process exits).  The
+ * call makes no cudaMalloc / cudaFree and calls no allocating routine; x, w_ohwi, bias and y are the
+ * caller's device buffers as in f8_conv2d_fixed.
+ *
+ *   - Inputs whose padded copy exceeds F8_STATIC_STEM_MAX_BYTES are rejected with F8_ERR_WORKSPACE;
+ *     inputs whose padded copy is below 128 KiB, or shapes outside the list above, with
+ *     F8_ERR_UNSUPPORTED (use f8_conv2d_fixed for those).
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls share the array and it keeps what the previous call left there.  Each call rewrites
+ *     every byte it later reads, so earlier contents never leak into a result, but two calls whose
+ *     GPU work overlaps (different streams, different host threads) race on it: serialise them.
+ *   - check_previous != 0 first synchronises the stream and returns F8_ERR_TIMEOUT if a kernel of an
+ *     earlier call on this device gave up on a bounded wait (f8_device_status does not see this
+ *     entry point's status word); with 0 the call never synchronises. */
+f8_status f8_stem_conv2d_fixed_static(const f8_conv_desc *desc, const void *x, const int8_t *w_ohwi,
+                                      const int32_t *bias, void *y, int check_previous, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -135,6 +135,21 @@ def f8_global_avgpool_fixed(n, h, w, c, x_dtype, fl_x, fl_y, x, y, stream=None):
     _check(_lib.f8_global_avgpool_fixed(n, h, w, c, x_dtype, fl_x, fl_y, _ptr(x), _ptr(y), _stream(stream)))
 
 
+_lib.f8_stem_conv2d_fixed_static.argtypes = [ctypes.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _ci, _vp]
+F8_STATIC_STEM_MAX_BYTES = 16 * 1024 * 1024
+
+
+def f8_stem_conv2d_fixed_static(desc: ConvDesc, x, w, bias, y, check_previous: bool = False, stream=None):
+    """First-layer convolution whose scratch memory is a fixed array inside the library: nothing is allocated.
+
+    For callers that cannot obtain device memory when they need the result (the device is owned by another
+    allocator, or allocation is forbidden on their path).  Same result as ``f8_conv2d_fixed``; calls share the
+    array, so do not let two of them overlap on the GPU.
+    """
+    _check(_lib.f8_stem_conv2d_fixed_static(ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(y),
+                                            1 if check_previous else 0, _stream(stream)))
+
+
 def f8_conv_workspace_bytes(desc: ConvDesc) -> int:
     return int(_lib.f8_conv_workspace_bytes(ctypes.byref(desc)))
 
@@ -164,7 +179,7 @@ def exported_symbols() -> List[str]:
     return ["f8_conv2d_fixed", "f8_dwconv_fixed", "f8_linear_fixed", "f8_maxpool_fixed", "f8_global_avgpool_fixed",
             "f8_conv_workspace_bytes", "f8_net_create", "f8_net_workspace_bytes", "f8_net_forward",
             "f8_net_last_launch_count", "f8_net_set_profiling", "f8_net_get_layer_ms", "f8_net_destroy", "f8_status_str", "f8_last_error", "f8_device_status",
-            "f8_mma_i8_probe"]
+            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static"]
 
 
 def run_layer(layer: "synth.Layer", x: torch.Tensor, residual: Optional[torch.Tensor] = None, params=None,

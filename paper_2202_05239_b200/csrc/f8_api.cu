@@ -148,6 +148,8 @@ f8_status run_dense(const F8ConvGeom &g, const F8Requant &q, const void *x, cons
 
 }   // namespace
 
+f8_status f8_set_error(f8_status s, const char *message) { return fail(s, "%s", message); }
+
 int *f8_status_word() {
     static int *words[64] = {nullptr};
     int dev = 0;

@@ -66,3 +66,6 @@ cudaError_t f8_tc_probe(int iters, double *ops, int *status_word, cudaStream_t s
 
 // Device status word (0 = fine); allocated once per process on first use.
 int *f8_status_word();
+
+// Records a message for f8_last_error() and returns `s` (for entry points defined outside f8_api.cu).
+f8_status f8_set_error(f8_status s, const char *message);
