@@ -698,8 +698,10 @@ int choose_bn(int c_out) {
 
 // N tile of the staged epilogue: a power of two up to 128, or 256 (two 128-byte slabs) when no residual
 // buffers are needed; the TMA store clips columns beyond c_out.
-int choose_bn_staged(int c_out, bool has_res) {
-    if (c_out > 128 && !has_res) return 256;
+int choose_bn_staged(int c_out, bool has_res, int kb) {
+    // with a residual the four staging tiles of a 256-wide tile leave room for the pipeline only when
+    // the K chunks are 64 bytes or less
+    if (c_out > 128 && (!has_res || kb <= 64)) return 256;
     int bn = 16;
     while (bn < c_out && bn < 128) bn *= 2;
     return bn;
@@ -752,12 +754,15 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.pad_h = g.pad_h;
     p.pad_w = g.pad_w;
     p.kb = choose_kb(g.c);
+    // residual layers are bound by the epilogue, not by the main loop: prefer 64-byte K chunks so that a
+    // 256-wide tile (half the tiles, half the A re-reads) still leaves room for the pipeline stages
+    if (q.has_res && g.c_out > 128 && p.kb == 128 && g.c <= 256) p.kb = 64;
     p.c_chunks = (g.c + p.kb - 1) / p.kb;
     p.epi = EPI_GENERIC;
     if (q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24 && g.c_out % 16 == 0)
         p.epi = q.y_kind == F8_U8 ? (q.has_res ? EPI_U8_RES : EPI_U8) : (q.has_res ? EPI_S8_RES : EPI_S8);
     const bool staged = p.epi != EPI_GENERIC;
-    p.bn = staged ? choose_bn_staged(g.c_out, q.has_res != 0) : choose_bn(g.c_out);
+    p.bn = staged ? choose_bn_staged(g.c_out, q.has_res != 0, p.kb) : choose_bn(g.c_out);
     p.m_tiles = (p.M + TILE_M - 1) / TILE_M;
     p.n_tiles = (g.c_out + p.bn - 1) / p.bn;
     p.a_bytes = (uint32_t)(TILE_M * p.kb + 1023) / 1024 * 1024;
