@@ -62,7 +62,9 @@ struct TcParams {
     int bn;                   // N tile, multiple of 16, <= 256
     int m_tiles, n_tiles;
     int stages;
-    uint32_t stage_bytes;     // A + B bytes of one stage (rounded to 1024)
+    int group;                // k-iterations per stage (1..4)
+    uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
+    uint32_t stage_bytes;     // group * sub_bytes
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
     uint32_t tx_a, tx_b;      // bytes the A / B load of a stage delivers
     uint32_t idesc;           // tcgen05 instruction descriptor
@@ -342,7 +344,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(full_bar + 8 * s, 2);       // one arrival per operand lane
+            mbar_init(full_bar + 8 * s, 1);       // one arrival (with the byte count of the whole group) per use
             mbar_init(empty_bar + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -375,10 +377,11 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 
     if (warp < NUM_PROD_WARPS) {
         // ------------------------------------------------------------------ TMA producer warp
-        // The whole warp walks the k-iterations in order (no divergence, no divisions in the loop); the A
-        // load of the iteration that uses stage `st` is issued by lane 2*st and its B load by lane 2*st+1,
-        // so that consecutive loads sit in different per-thread TMA queues and overlap.
-        int stage = 0;
+        // The whole warp walks the k-iterations in order (no divergence, no divisions in the loop).  A stage
+        // holds `group` consecutive k-iterations of one tile (fewer at the tile's end); sub-chunk j of stage
+        // st gets its A load from lane 2*(st*group + j) and its B load from the next lane, so that
+        // consecutive loads sit in different per-thread TMA queues and overlap.
+        int stage = 0, sub = 0;
         uint32_t phase = 0;
         bool have_last = false;
         uint32_t last_phase = 0;            // phase of this lane's most recent load (for the drain on abort)
@@ -394,34 +397,42 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int base_h = oh * p.stride_h - p.pad_h;
             const int n_base = n_t * p.bn;
             int tap = 0;
+            int left = k_iters;             // k-iterations of this tile not yet requested
             for (int r = 0; ok && r < p.kh; ++r)
                 for (int s = 0; ok && s < p.kw; ++s, ++tap)
                     for (int c0 = 0; c0 < p.c_chunks * p.kb; c0 += p.kb) {
-                        if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101))) {
-                            ok = false;
-                            break;
-                        }
                         const uint32_t fb = full_bar + 8 * stage;
-                        const uint32_t a_dst = smem_base + stage * p.stage_bytes;
-                        if (lane == 2 * stage) {
-                            mbar_expect_tx(fb, p.tx_a);
+                        if (sub == 0) {
+                            if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101))) {
+                                ok = false;
+                                break;
+                            }
+                            // one arrival per stage use; it announces the bytes of every load of the group
+                            if (lane == 2 * stage * p.group) mbar_expect_tx(fb, (uint32_t)min(left, p.group) * (p.tx_a + p.tx_b));
+                        }
+                        const uint32_t a_dst = smem_base + stage * p.stage_bytes + sub * p.sub_bytes;
+                        const int my = 2 * (stage * p.group + sub);
+                        if (lane == my) {
                             tma_load_im2col(a_dst, &map_a, fb, c0, base_w, base_h, img, (uint16_t)s, (uint16_t)r);
                             have_last = true;
                             last_phase = phase;
-                        } else if (lane == 2 * stage + 1) {
-                            mbar_expect_tx(fb, p.tx_b);
+                        } else if (lane == my + 1) {
                             tma_load_3d(a_dst + p.a_bytes, &map_b, fb, c0, tap, n_base);
                             have_last = true;
                             last_phase = phase;
                         }
-                        if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                        --left;
+                        if (++sub == p.group || left == 0) {
+                            sub = 0;
+                            if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                        }
                     }
         }
         if (!ok && have_last) {
             // Drain: loads of one thread are served in order, so waiting (bounded) for the most recent one
             // covers everything this lane has in flight before the CTA's shared memory goes away.
             const unsigned long long t0 = clock64();
-            while (!mbar_try_wait(full_bar + 8 * (lane >> 1), last_phase) &&
+            while (!mbar_try_wait(full_bar + 8 * ((lane >> 1) / p.group), last_phase) &&
                    (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
             }
         }
@@ -436,7 +447,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             int last_acc = 0;
             uint32_t last_acc_phase = 0;
             const uint64_t a_desc0 = p.desc_hi | (uint64_t)((smem_base & 0x3ffffu) >> 4);
-            const uint32_t stage16 = p.stage_bytes >> 4, a16 = p.a_bytes >> 4;
+            const uint32_t stage16 = p.stage_bytes >> 4, sub16 = p.sub_bytes >> 4, a16 = p.a_bytes >> 4;
             const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
@@ -444,17 +455,20 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, abortp, p.status, 102)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * 256;   // two 256-column accumulators
-                for (int kc = 0; kc < k_iters; ++kc) {
+                for (int kc = 0; kc < k_iters; kc += p.group) {
                     if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, 103)) { ok = false; break; }
                     tc_fence_after();
-                    const uint64_t a_desc = a_desc0 + (uint64_t)(stage * stage16);
-                    const uint64_t b_desc = a_desc + a16;
-                    // 32 bytes of K per instruction: the descriptor start address advances by 2 (16-byte units)
-                    mma_i8(d_tmem, a_desc, b_desc, p.idesc, kc != 0 ? 1u : 0u);
-                    if (mmas >= 2) mma_i8(d_tmem, a_desc + 2, b_desc + 2, p.idesc, 1u);
-                    if (mmas == 4) {
-                        mma_i8(d_tmem, a_desc + 4, b_desc + 4, p.idesc, 1u);
-                        mma_i8(d_tmem, a_desc + 6, b_desc + 6, p.idesc, 1u);
+                    uint64_t a_desc = a_desc0 + (uint64_t)(stage * stage16);
+                    const int subs = min(p.group, k_iters - kc);
+                    for (int j = 0; j < subs; ++j, a_desc += sub16) {
+                        const uint64_t b_desc = a_desc + a16;
+                        // 32 bytes of K per instruction: the descriptor start address advances by 2 (16-byte units)
+                        mma_i8(d_tmem, a_desc, b_desc, p.idesc, (kc | j) != 0 ? 1u : 0u);
+                        if (mmas >= 2) mma_i8(d_tmem, a_desc + 2, b_desc + 2, p.idesc, 1u);
+                        if (mmas == 4) {
+                            mma_i8(d_tmem, a_desc + 4, b_desc + 4, p.idesc, 1u);
+                            mma_i8(d_tmem, a_desc + 6, b_desc + 6, p.idesc, 1u);
+                        }
                     }
                     mma_commit(empty_bar + 8 * stage);    // frees the stage when these MMAs have read it
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
@@ -767,7 +781,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.n_tiles = (g.c_out + p.bn - 1) / p.bn;
     p.a_bytes = (uint32_t)(TILE_M * p.kb + 1023) / 1024 * 1024;
     const uint32_t b_bytes = (uint32_t)(p.bn * p.kb + 1023) / 1024 * 1024;
-    p.stage_bytes = p.a_bytes + b_bytes;
+    p.sub_bytes = p.a_bytes + b_bytes;
     p.tx_a = (uint32_t)(TILE_M * p.kb);
     p.tx_b = (uint32_t)(p.bn * p.kb);
     size_t staging = 0;
@@ -780,8 +794,17 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         const size_t bias_bytes = ((size_t)p.n_tiles * p.bn * 4 + 1023) / 1024 * 1024;
         staging = (size_t)p.out_bytes * (q.has_res ? 4 : 2) + bias_bytes;
     }
-    int stages = (int)((SMEM_LIMIT - 1024 - staging) / p.stage_bytes);
-    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    // k-iterations per stage: every stage use costs the MMA thread a wait, a fence and a commit (a few hundred
+    // cycles), so short K chunks are grouped -- as long as at least three stages and one lane per load remain
+    const int k_iters = g.kh * g.kw * p.c_chunks;
+    const size_t avail = SMEM_LIMIT - 1024 - staging;
+    int group = k_iters < 4 ? k_iters : 4;
+    if (const char *e = getenv("F8_TC_GROUP")) group = atoi(e) < group ? atoi(e) : group;
+    while (group > 1 && avail / ((size_t)group * p.sub_bytes) < 3) --group;
+    p.group = group;
+    p.stage_bytes = (uint32_t)group * p.sub_bytes;
+    int stages = (int)(avail / p.stage_bytes);
+    if (stages > MAX_STAGES / group) stages = MAX_STAGES / group;
     if (stages < 2) {
         *why = "stage does not fit";
         return cudaErrorInvalidValue;
