@@ -84,6 +84,7 @@ struct TcParams {
     uint32_t out_bytes;       // TILE_M * bn
     uint32_t out_off, res_off, bias_off;   // byte offsets behind the stages: two output tiles, two residual
                                            // tiles, int32 bias' of all padded columns
+    uint32_t ktab_off;        // table of k-iteration coordinates (8 bytes each)
     F8Requant q;
     int *status;
 };
@@ -358,6 +359,15 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    {
+        // coordinates of every k-iteration (filter tap and channel chunk), once per CTA
+        uint2 *ktab = (uint2 *)(smem + p.ktab_off);
+        for (int i = threadIdx.x; i < p.kh * p.kw * p.c_chunks; i += NUM_THREADS) {
+            const int tap = i / p.c_chunks, cc = i - tap * p.c_chunks;
+            const int r = tap / p.kw, sx = tap - r * p.kw;
+            ktab[i] = make_uint2((uint32_t)(cc * p.kb), ((uint32_t)tap << 16) | ((uint32_t)r << 8) | (uint32_t)sx);
+        }
+    }
     if (STAGED) {
         // bias' = (bias << sh_acc) + 2^(s-1) for every (padded) output column, once per CTA
         int *bias_all = (int *)(smem + p.bias_off);
@@ -377,14 +387,19 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 
     if (warp < NUM_PROD_WARPS) {
         // ------------------------------------------------------------------ TMA producer warp
-        // The whole warp walks the k-iterations in order (no divergence, no divisions in the loop).  A stage
-        // holds `group` consecutive k-iterations of one tile (fewer at the tile's end); sub-chunk j of stage
-        // st gets its A load from lane 2*(st*group + j) and its B load from the next lane, so that
-        // consecutive loads sit in different per-thread TMA queues and overlap.
-        int stage = 0, sub = 0;
+        // A stage holds `group` consecutive k-iterations of one tile (fewer at the tile's end).  The warp makes
+        // one pass per stage use: it waits for the stage, then lane (st*group + j) & 15 issues the activation
+        // load of sub-chunk j and lane 16 + that the weight load, each with the coordinates of its k-iteration
+        // from a table built at kernel start.  There is no per-k-iteration loop (a single warp executes a few
+        // hundred cycles of loop overhead per iteration, which used to bound layers with many short
+        // k-iterations), and consecutive loads sit in different per-thread TMA queues, so they overlap.
+        const uint2 *ktab = (const uint2 *)(smem + p.ktab_off);
+        const int half = lane >> 4, l16 = lane & 15;
+        int stage = 0;
         uint32_t phase = 0;
         bool have_last = false;
-        uint32_t last_phase = 0;            // phase of this lane's most recent load (for the drain on abort)
+        int last_stage = 0;
+        uint32_t last_phase = 0;            // stage / phase of this lane's most recent load (for the drain on abort)
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
             const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
@@ -396,43 +411,36 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int base_w = ow * p.stride_w - p.pad_w;
             const int base_h = oh * p.stride_h - p.pad_h;
             const int n_base = n_t * p.bn;
-            int tap = 0;
-            int left = k_iters;             // k-iterations of this tile not yet requested
-            for (int r = 0; ok && r < p.kh; ++r)
-                for (int s = 0; ok && s < p.kw; ++s, ++tap)
-                    for (int c0 = 0; c0 < p.c_chunks * p.kb; c0 += p.kb) {
-                        const uint32_t fb = full_bar + 8 * stage;
-                        if (sub == 0) {
-                            if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101))) {
-                                ok = false;
-                                break;
-                            }
-                            // one arrival per stage use; it announces the bytes of every load of the group
-                            if (lane == 2 * stage * p.group) mbar_expect_tx(fb, (uint32_t)min(left, p.group) * (p.tx_a + p.tx_b));
-                        }
-                        const uint32_t a_dst = smem_base + stage * p.stage_bytes + sub * p.sub_bytes;
-                        const int my = 2 * (stage * p.group + sub);
-                        if (lane == my) {
-                            tma_load_im2col(a_dst, &map_a, fb, c0, base_w, base_h, img, (uint16_t)s, (uint16_t)r);
-                            have_last = true;
-                            last_phase = phase;
-                        } else if (lane == my + 1) {
-                            tma_load_3d(a_dst + p.a_bytes, &map_b, fb, c0, tap, n_base);
-                            have_last = true;
-                            last_phase = phase;
-                        }
-                        --left;
-                        if (++sub == p.group || left == 0) {
-                            sub = 0;
-                            if (++stage == p.stages) { stage = 0; phase ^= 1; }
-                        }
-                    }
+            for (int kc = 0; kc < k_iters; kc += p.group) {
+                if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101))) {
+                    ok = false;
+                    break;
+                }
+                const int subs = min(p.group, k_iters - kc);
+                const uint32_t fb = full_bar + 8 * stage;
+                // one arrival per stage use; it announces the bytes of every load of the group
+                if (lane == 0) mbar_expect_tx(fb, (uint32_t)subs * (p.tx_a + p.tx_b));
+                const int j = (l16 - stage * p.group) & 15;
+                if (j < subs) {
+                    const uint2 e = ktab[kc + j];       // x: first channel of the chunk, y: tap << 16 | r << 8 | s
+                    const uint32_t dst = smem_base + stage * p.stage_bytes + j * p.sub_bytes;
+                    if (half == 0)
+                        tma_load_im2col(dst, &map_a, fb, (int)e.x, base_w, base_h, img, (uint16_t)(e.y & 0xff),
+                                        (uint16_t)((e.y >> 8) & 0xff));
+                    else
+                        tma_load_3d(dst + p.a_bytes, &map_b, fb, (int)e.x, (int)(e.y >> 16), n_base);
+                    have_last = true;
+                    last_stage = stage;
+                    last_phase = phase;
+                }
+                if (++stage == p.stages) { stage = 0; phase ^= 1; }
+            }
         }
         if (!ok && have_last) {
             // Drain: loads of one thread are served in order, so waiting (bounded) for the most recent one
             // covers everything this lane has in flight before the CTA's shared memory goes away.
             const unsigned long long t0 = clock64();
-            while (!mbar_try_wait(full_bar + 8 * ((lane >> 1) / p.group), last_phase) &&
+            while (!mbar_try_wait(full_bar + 8 * last_stage, last_phase) &&
                    (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
             }
         }
@@ -794,6 +802,12 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         const size_t bias_bytes = ((size_t)p.n_tiles * p.bn * 4 + 1023) / 1024 * 1024;
         staging = (size_t)p.out_bytes * (q.has_res ? 4 : 2) + bias_bytes;
     }
+    const size_t ktab_bytes = ((size_t)g.kh * g.kw * p.c_chunks * 8 + 1023) / 1024 * 1024;
+    if (ktab_bytes > 16 * 1024 || g.kh * g.kw > 0xffff) {
+        *why = "too many k-iterations for the coordinate table";
+        return cudaErrorInvalidValue;
+    }
+    staging += ktab_bytes;
     // k-iterations per stage: every stage use costs the MMA thread a wait, a fence and a commit (a few hundred
     // cycles), so short K chunks are grouped -- as long as at least three stages and one lane per load remain
     const int k_iters = g.kh * g.kw * p.c_chunks;
@@ -804,7 +818,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.group = group;
     p.stage_bytes = (uint32_t)group * p.sub_bytes;
     int stages = (int)(avail / p.stage_bytes);
-    if (stages > MAX_STAGES / group) stages = MAX_STAGES / group;
+    if (stages > 16 / group) stages = 16 / group;     // 16 lanes per operand
     if (stages < 2) {
         *why = "stage does not fit";
         return cudaErrorInvalidValue;
@@ -813,6 +827,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
     p.res_off = p.out_off + 2 * p.out_bytes;
     p.bias_off = p.res_off + (q.has_res ? 2 * p.out_bytes : 0u);
+    p.ktab_off = (uint32_t)(p.stages * p.stage_bytes + staging - ktab_bytes);
     // instruction descriptor: D = s32 (2 at bit 4), A format at bit 7 (0 = u8, 1 = s8), B = s8 at bit 10,
     // both operands K-major, N/8 at bit 17, M/16 at bit 24
     p.idesc = (2u << 4) | ((g.x_signed ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) |
