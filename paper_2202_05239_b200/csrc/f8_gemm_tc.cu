@@ -51,6 +51,14 @@ constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 G
 constexpr unsigned long long DRAIN_LIMIT_CYCLES = 200000000ull;
 constexpr size_t SMEM_LIMIT = 220 * 1024;     // dynamic shared memory budget (227 KiB per CTA minus static data)
 
+// Division by a run-time constant without a divide instruction (a 32-bit divide costs a lone thread well over a
+// hundred cycles): q = (n * mul) >> shift is exact for 0 <= n < 2^31 with mul = floor(2^shift / d) + 1,
+// shift = 31 + ceil(log2 d).
+struct FastDiv {
+    uint32_t mul, shift;
+};
+__device__ __forceinline__ int fast_div(int n, FastDiv d) { return (int)(((uint64_t)(uint32_t)n * d.mul) >> d.shift); }
+
 struct TcParams {
     int M;                    // total output pixels
     int ho, wo;
@@ -61,6 +69,7 @@ struct TcParams {
     int kb;                   // bytes (= int8 elements) of K per stage: 32, 64 or 128
     int bn;                   // N tile, multiple of 16, <= 256
     int m_tiles, n_tiles;
+    FastDiv div_n_tiles, div_wo, div_ho;
     int stages;
     int group;                // k-iterations per stage (1..4)
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
@@ -402,12 +411,12 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         uint32_t last_phase = 0;            // stage / phase of this lane's most recent load (for the drain on abort)
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-            const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+            const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
             const int m0 = m_t * TILE_M;
-            const int ow = m0 % p.wo;
-            const int t1 = m0 / p.wo;
-            const int oh = t1 % p.ho;
-            const int img = t1 / p.ho;
+            const int t1 = fast_div(m0, p.div_wo);
+            const int ow = m0 - t1 * p.wo;
+            const int img = fast_div(t1, p.div_ho);
+            const int oh = t1 - img * p.ho;
             const int base_w = ow * p.stride_w - p.pad_w;
             const int base_h = oh * p.stride_h - p.pad_h;
             const int n_base = n_t * p.bn;
@@ -502,7 +511,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             int local = 0;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
                 const int b = local & 1;
-                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+                const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
                 if (!mbar_wait(out_full + 8 * b, (local >> 1) & 1, abortp, p.status, 108)) break;
                 const uint32_t src = smem_base + p.out_off + b * p.out_bytes;
                 for (int sl = 0; sl < p.n_slabs; ++sl)
@@ -524,7 +533,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
                 const int b = local & 1;
-                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+                const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
                 if (!mbar_wait(res_free + 8 * b, ((local >> 1) & 1) ^ 1, abortp, p.status, 106)) { ok = false; break; }
                 const uint32_t rb = res_full + 8 * b;
                 mbar_expect_tx(rb, p.out_bytes);
@@ -570,7 +579,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
                 const int acc = local & 1;                   // accumulator, output buffer and residual buffer in use
                 const uint32_t acc_phase = (local >> 1) & 1;
-                const int n_t = tile % p.n_tiles;
+                const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
                 const int c_first = n_t * p.bn + ch_begin * 16;
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
@@ -618,7 +627,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
                 const uint32_t acc_phase = (local >> 1) & 1;
-                const int m_t = tile / p.n_tiles, n_t = tile - m_t * p.n_tiles;
+                const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
                 const int n0 = n_t * p.bn;
                 const size_t row = (size_t)m_t * TILE_M + tile_row;
                 const bool row_valid = row < (size_t)p.M;
@@ -711,6 +720,15 @@ bool load_driver_entry_points() {
     return true;
 }
 
+FastDiv make_fast_div(int d) {
+    uint32_t l = 0;
+    while ((1u << l) < (uint32_t)d) ++l;
+    FastDiv f;
+    f.shift = 31 + l;
+    f.mul = (uint32_t)(((uint64_t)1 << f.shift) / (uint32_t)d + 1);
+    return f;
+}
+
 int choose_kb(int c) { return c >= 96 ? 128 : (c >= 48 ? 64 : 32); }
 
 int choose_bn(int c_out) {
@@ -787,6 +805,9 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.bn = staged ? choose_bn_staged(g.c_out, q.has_res != 0, p.kb) : choose_bn(g.c_out);
     p.m_tiles = (p.M + TILE_M - 1) / TILE_M;
     p.n_tiles = (g.c_out + p.bn - 1) / p.bn;
+    p.div_n_tiles = make_fast_div(p.n_tiles);
+    p.div_wo = make_fast_div(g.wo);
+    p.div_ho = make_fast_div(g.ho);
     p.a_bytes = (uint32_t)(TILE_M * p.kb + 1023) / 1024 * 1024;
     const uint32_t b_bytes = (uint32_t)(p.bn * p.kb + 1023) / 1024 * 1024;
     p.sub_bytes = p.a_bytes + b_bytes;
