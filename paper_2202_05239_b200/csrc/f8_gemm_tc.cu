@@ -38,14 +38,16 @@ constexpr int NUM_EPI_WARPS = 16;          // four warps per TMEM lane quarter, 
 // The TMA serves the loads of one thread strictly one after the other, and one load occupies it for
 // several hundred cycles whatever the box size, so a single issuing thread caps a CTA at roughly ten
 // bytes per clock.  Loads issued by different threads (lanes of one warp included) overlap: every
-// (stage, operand) pair therefore has its own lane of the producer warp.
-constexpr int NUM_PROD_WARPS = 1;
+// (stage, sub-chunk) pair therefore has its own lane.  Issuing a TMA instruction also holds the issuing
+// warp for a few hundred cycles, so activations and weights are requested by two different warps.
+constexpr int A_PROD_WARP = 0;             // requests activation tiles
 constexpr int MMA_WARP = 1;
 constexpr int MOVER_WARP = 2;              // one thread stores finished output tiles
 constexpr int FETCH_WARP = 3;              // one thread fetches residual tiles
-constexpr int FIRST_EPI_WARP = 4;
-constexpr int NUM_THREADS = 32 * (FIRST_EPI_WARP + NUM_EPI_WARPS);   // producer, MMA issuer, mover, fetcher, epilogue
-constexpr int MAX_STAGES = 16;          // two producer lanes per stage
+constexpr int FIRST_EPI_WARP = 4;          // warps 4..19; warp & 3 is the TMEM lane quarter
+constexpr int B_PROD_WARP = FIRST_EPI_WARP + NUM_EPI_WARPS;   // requests weight tiles
+constexpr int NUM_THREADS = 32 * (B_PROD_WARP + 1);
+constexpr int MAX_STAGES = 16;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
 constexpr unsigned long long DRAIN_LIMIT_CYCLES = 200000000ull;
@@ -71,7 +73,7 @@ struct TcParams {
     int m_tiles, n_tiles;
     FastDiv div_n_tiles, div_wo, div_ho;
     int stages;
-    int group;                // k-iterations per stage (1..4)
+    int group;                // k-iterations per stage (1..8)
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
     uint32_t stage_bytes;     // group * sub_bytes
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
@@ -394,16 +396,16 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const int k_iters = p.kh * p.kw * p.c_chunks;
     volatile int *abortp = &abort_flag;
 
-    if (warp < NUM_PROD_WARPS) {
-        // ------------------------------------------------------------------ TMA producer warp
-        // A stage holds `group` consecutive k-iterations of one tile (fewer at the tile's end).  The warp makes
-        // one pass per stage use: it waits for the stage, then lane (st*group + j) & 15 issues the activation
-        // load of sub-chunk j and lane 16 + that the weight load, each with the coordinates of its k-iteration
-        // from a table built at kernel start.  There is no per-k-iteration loop (a single warp executes a few
-        // hundred cycles of loop overhead per iteration, which used to bound layers with many short
-        // k-iterations), and consecutive loads sit in different per-thread TMA queues, so they overlap.
+    if (warp == A_PROD_WARP || warp == B_PROD_WARP) {
+        // ------------------------------------------------------------------ TMA producer warps
+        // A stage holds `group` consecutive k-iterations of one tile (fewer at the tile's end).  Each producer
+        // warp makes one pass per stage use: it waits for the stage, then lane (st*group + j) & 31 issues the
+        // load of sub-chunk j with the coordinates of its k-iteration from a table built at kernel start.
+        // There is no per-k-iteration loop (a single warp spends a few hundred cycles of loop overhead per
+        // iteration, which used to bound layers with many short k-iterations), and consecutive loads sit in
+        // different per-thread TMA queues, so they overlap.
         const uint2 *ktab = (const uint2 *)(smem + p.ktab_off);
-        const int half = lane >> 4, l16 = lane & 15;
+        const int opnd = warp == A_PROD_WARP ? 0 : 1;
         int stage = 0;
         uint32_t phase = 0;
         bool have_last = false;
@@ -428,12 +430,12 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int subs = min(p.group, k_iters - kc);
                 const uint32_t fb = full_bar + 8 * stage;
                 // one arrival per stage use; it announces the bytes of every load of the group
-                if (lane == 0) mbar_expect_tx(fb, (uint32_t)subs * (p.tx_a + p.tx_b));
-                const int j = (l16 - stage * p.group) & 15;
+                if (opnd == 0 && lane == 0) mbar_expect_tx(fb, (uint32_t)subs * (p.tx_a + p.tx_b));
+                const int j = (lane - stage * p.group) & 31;
                 if (j < subs) {
                     const uint2 e = ktab[kc + j];       // x: first channel of the chunk, y: tap << 16 | r << 8 | s
                     const uint32_t dst = smem_base + stage * p.stage_bytes + j * p.sub_bytes;
-                    if (half == 0)
+                    if (opnd == 0)
                         tma_load_im2col(dst, &map_a, fb, (int)e.x, base_w, base_h, img, (uint16_t)(e.y & 0xff),
                                         (uint16_t)((e.y >> 8) & 0xff));
                     else
@@ -552,7 +554,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 }
             }
         }
-    } else {
+    } else if (warp >= FIRST_EPI_WARP && warp < FIRST_EPI_WARP + NUM_EPI_WARPS) {
         // ------------------------------------------------------------------ epilogue warps
         const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 belong to this warp
         const int ew = warp - FIRST_EPI_WARP;
@@ -833,13 +835,14 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // cycles), so short K chunks are grouped -- as long as at least three stages and one lane per load remain
     const int k_iters = g.kh * g.kw * p.c_chunks;
     const size_t avail = SMEM_LIMIT - 1024 - staging;
-    int group = k_iters < 4 ? k_iters : 4;
-    if (const char *e = getenv("F8_TC_GROUP")) group = atoi(e) < group ? atoi(e) : group;
+    const int uses = (k_iters + 7) / 8;                  // at most eight k-iterations per stage, evenly split
+    int group = (k_iters + uses - 1) / uses;
     while (group > 1 && avail / ((size_t)group * p.sub_bytes) < 3) --group;
     p.group = group;
     p.stage_bytes = (uint32_t)group * p.sub_bytes;
     int stages = (int)(avail / p.stage_bytes);
-    if (stages > 16 / group) stages = 16 / group;     // 16 lanes per operand
+    if (stages > 32 / group) stages = 32 / group;     // one lane per (stage, sub-chunk)
+    if (stages > MAX_STAGES) stages = MAX_STAGES;
     if (stages < 2) {
         *why = "stage does not fit";
         return cudaErrorInvalidValue;
