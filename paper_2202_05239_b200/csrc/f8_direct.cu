@@ -120,6 +120,85 @@ __global__ void __launch_bounds__(256) dwconv_vec4_kernel(F8ConvGeom g, F8Requan
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Depthwise 3x3, pad 1, stride S (1 or 2): the layers of MobileNet.  One thread owns 4 consecutive
+// channels and a strip of TW output pixels along W.  The nine filter taps of its channels stay in
+// registers and every input word (4 channels of one pixel) is loaded and unpacked once per filter row
+// and reused by all outputs of the strip that touch it, so the kernel does about one load and four
+// unpacks per eight multiply-accumulates instead of one load per multiply-accumulate.  Consecutive
+// threads take consecutive channel groups: loads and stores coalesce over the channel dimension.
+// Depthwise is not a contraction over channels, so this stays on the CUDA cores (IMAD); it is bound
+// by instruction issue, not by HBM.
+// ---------------------------------------------------------------------------------------
+template <int S, int TW, bool XS>
+__global__ void __launch_bounds__(128) dwconv3x3_strip_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
+                                                              const int8_t *__restrict__ w,
+                                                              const int32_t *__restrict__ bias,
+                                                              const void *__restrict__ res, void *__restrict__ y) {
+    constexpr int SPAN = (TW - 1) * S + 3;          // input pixels a strip touches along W
+    const int c4 = g.c >> 2;
+    const int strips = (g.wo + TW - 1) / TW;
+    const size_t total = (size_t)g.n * g.ho * strips * c4;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int cg = (int)(idx % c4);
+        size_t t = idx / c4;
+        const int strip = (int)(t % strips);
+        t /= strips;
+        const int oh = (int)(t % g.ho);
+        const int in = (int)(t / g.ho);
+        const int c0 = cg * 4;
+        const int ow0 = strip * TW;
+        int wt[9][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int k = 0; k < 9; ++k) wt[k][j] = (int)w[(size_t)(c0 + j) * 9 + k];
+        int acc[TW][4];
+        const int4 b = bias ? *(const int4 *)(bias + c0) : make_int4(0, 0, 0, 0);
+#pragma unroll
+        for (int o = 0; o < TW; ++o) { acc[o][0] = b.x; acc[o][1] = b.y; acc[o][2] = b.z; acc[o][3] = b.w; }
+        const int iw0 = ow0 * S - 1;
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+            const int ih = oh * S + r - 1;
+            if (ih < 0 || ih >= g.h) continue;
+            const uint8_t *row = x + (((size_t)in * g.h + ih) * g.w) * g.c + c0;
+#pragma unroll
+            for (int xx = 0; xx < SPAN; ++xx) {
+                const int iw = iw0 + xx;
+                uint32_t word = 0;
+                if (iw >= 0 && iw < g.w) word = __ldg((const uint32_t *)(row + (size_t)iw * g.c));
+                int v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] = XS ? (int)(int8_t)(word >> (8 * j)) : (int)((word >> (8 * j)) & 0xffu);
+#pragma unroll
+                for (int s = 0; s < 3; ++s) {
+                    // input column xx feeds output o through tap s when xx = o * S + s
+                    if ((xx - s) >= 0 && (xx - s) % S == 0 && (xx - s) / S < TW) {
+                        const int o = (xx - s) / S;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) acc[o][j] += v[j] * wt[r * 3 + s][j];
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 0; o < TW; ++o) {
+            const int ow = ow0 + o;
+            if (ow >= g.wo) break;
+            const size_t off = (((size_t)in * g.ho + oh) * g.wo + ow) * g.c + c0;
+            uint32_t rw = 0;
+            if (q.has_res) rw = *(const uint32_t *)((const uint8_t *)res + off);
+            int out[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) out[j] = f8_requant(acc[o][j], f8_byte(rw, j, q.r_signed), q);
+            if (q.y_kind == F8_S32) *(int4 *)((int32_t *)y + off) = make_int4(out[0], out[1], out[2], out[3]);
+            else *(uint32_t *)((uint8_t *)y + off) = f8_pack4(out[0], out[1], out[2], out[3]);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(256) dwconv_scalar_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
                                                             const int8_t *__restrict__ w,
                                                             const int32_t *__restrict__ bias,
@@ -305,7 +384,22 @@ cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void
                              const int32_t *bias, const void *res, void *y, cudaStream_t st) {
     const size_t total = (size_t)g.n * g.ho * g.wo * g.c;
     if (total == 0) return cudaSuccess;
-    if (g.c % 4 == 0)
+    const bool strip_ok = g.c % 4 == 0 && g.kh == 3 && g.kw == 3 && g.pad_h == 1 && g.pad_w == 1 &&
+                          g.stride_h == g.stride_w && (g.stride_h == 1 || g.stride_h == 2) &&
+                          (((uintptr_t)x | (uintptr_t)y | (uintptr_t)res | (uintptr_t)bias) & 15) == 0;
+    if (strip_ok) {
+        const int tw = g.stride_h == 1 ? 8 : 4;
+        const size_t threads = (size_t)g.n * g.ho * ((g.wo + tw - 1) / tw) * (g.c / 4);
+        const int grid = grid_for(threads, 128);
+        const uint8_t *xp = (const uint8_t *)x;
+        if (g.stride_h == 1) {
+            if (g.x_signed) dwconv3x3_strip_kernel<1, 8, true><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y);
+            else dwconv3x3_strip_kernel<1, 8, false><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y);
+        } else {
+            if (g.x_signed) dwconv3x3_strip_kernel<2, 4, true><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y);
+            else dwconv3x3_strip_kernel<2, 4, false><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y);
+        }
+    } else if (g.c % 4 == 0)
         dwconv_vec4_kernel<<<grid_for(total / 4, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
     else
         dwconv_scalar_kernel<<<grid_for(total, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);

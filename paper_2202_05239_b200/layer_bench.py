@@ -2,6 +2,7 @@
 
     python -m paper_2202_05239_b200.layer_bench --sweep            # the six CNN layer shapes at batch 32
     python -m paper_2202_05239_b200.layer_bench --h 56 --w 56 --c 64 --c-out 256 --k 1 --batch 32 --res
+    python -m paper_2202_05239_b200.layer_bench --net mobilenetv2 --batch 64     # per-layer times of a whole net
 
 Each layer is run over several copies of its tensors, rotated so that consecutive launches do not find
 their operands in L2 (the copies together exceed twice the L2 size).  Prints one JSON line per layer:
@@ -72,9 +73,43 @@ def custom_layer(args) -> synth.Layer:
                        args.k // 2, synth.U8, synth.U8, synth.U8, 5, flw, 5, 5, wgt, bias)
 
 
+def bench_net(name: str, batch: int, iters: int, warmup: int):
+    """Per-layer device times of a whole synthetic network (CUDA events recorded by f8_net_forward)."""
+    layers = synth.make_net(name, 0)
+    net = api.Net(layers, batch)
+    x = api.to_device(synth.draw_image(batch, 1))
+    for _ in range(warmup):
+        net.forward(x)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        net.forward(x)
+    e1.record()
+    torch.cuda.synchronize()
+    total_ms = e0.elapsed_time(e1) / iters
+    net.set_profiling(True)
+    acc = np.zeros(len(layers))
+    for _ in range(iters):
+        net.forward(x)
+        ms, tc = net.layer_ms()
+        acc += np.array(ms)
+    api.f8_device_status()
+    acc /= iters
+    for l, ms, on_tc in zip(layers, acc, tc):
+        byts = batch * l.bytes_per_image() + l.param_bytes()
+        print(json.dumps({"layer": l.name, "kind": synth.KIND_NAMES[l.kind], "shape": [l.h, l.w, l.c, l.c_out, l.kh, l.stride],
+                          "tensor_cores": bool(on_tc), "ms": round(float(ms), 5),
+                          "gbs": round(byts / (ms * 1e-3) / 1e9, 1) if ms > 0 else None,
+                          "tops": round(2 * batch * l.macs_per_image / (ms * 1e-3) / 1e12, 1) if ms > 0 else None}))
+    print(json.dumps({"net": name, "batch": batch, "ms_per_forward": total_ms, "images_per_s": batch / (total_ms * 1e-3),
+                      "launches": net.last_launch_count}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--net", default="", help="time every layer of a synthetic network: resnet18, resnet50, mobilenetv2")
     ap.add_argument("--h", type=int, default=56)
     ap.add_argument("--w", type=int, default=0)
     ap.add_argument("--c", type=int, default=64)
@@ -88,7 +123,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--warm-l2", action="store_true", help="reuse one buffer set (operands stay in L2)")
     args = ap.parse_args()
-    if args.sweep:
+    if args.net:
+        bench_net(args.net, args.batch, args.iters, args.warmup)
+    elif args.sweep:
         for i in range(len(synth.SWEEP_SHAPES)):
             layer, _ = synth.sweep_case(i, batch=1)
             print(json.dumps(bench_layer(layer, args.batch, False, args.iters, args.warmup, not args.warm_l2)), flush=True)
