@@ -130,48 +130,66 @@ __global__ void __launch_bounds__(256) dwconv_vec4_kernel(F8ConvGeom g, F8Requan
 // Depthwise is not a contraction over channels, so this stays on the CUDA cores (IMAD); it is bound
 // by instruction issue, not by HBM.
 // ---------------------------------------------------------------------------------------
-template <int S, int TW, bool XS>
+// Byte j of a word as a sign-extended int with one PRMT: selector nibble j picks the byte, nibble 8|j
+// replicates its sign bit (the intrinsic __byte_perm ignores that bit, hence the inline PTX).
+__device__ __forceinline__ int prmt_s8(uint32_t word, int j) {
+    int r;
+    const uint32_t sel = (uint32_t)(j | ((8 | j) << 4) | ((8 | j) << 8) | ((8 | j) << 12));
+    asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(word), "r"(sel));
+    return r;
+}
+
+// FAST: 8-bit output with shift 1..24 -> rounding constant folded into the bias, plain shift, saturating pack.
+template <int S, int TW, bool XS, bool FAST>
 __global__ void __launch_bounds__(128) dwconv3x3_strip_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
                                                               const int8_t *__restrict__ w,
                                                               const int32_t *__restrict__ bias,
-                                                              const void *__restrict__ res, void *__restrict__ y) {
+                                                              const void *__restrict__ res, void *__restrict__ y,
+                                                              int strips, int total) {
     constexpr int SPAN = (TW - 1) * S + 3;          // input pixels a strip touches along W
     const int c4 = g.c >> 2;
-    const int strips = (g.wo + TW - 1) / TW;
-    const size_t total = (size_t)g.n * g.ho * strips * c4;
-    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (size_t)gridDim.x * blockDim.x) {
-        const int cg = (int)(idx % c4);
-        size_t t = idx / c4;
-        const int strip = (int)(t % strips);
+    // all index arithmetic in 32 bits (the launcher checks that every offset fits)
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int cg = idx % c4;
+        int t = idx / c4;
+        const int strip = t % strips;
         t /= strips;
-        const int oh = (int)(t % g.ho);
-        const int in = (int)(t / g.ho);
+        const int oh = t % g.ho;
+        const int in = t / g.ho;
         const int c0 = cg * 4;
         const int ow0 = strip * TW;
         int wt[9][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j)
 #pragma unroll
-            for (int k = 0; k < 9; ++k) wt[k][j] = (int)w[(size_t)(c0 + j) * 9 + k];
+            for (int k = 0; k < 9; ++k) wt[k][j] = (int)w[(c0 + j) * 9 + k];
         int acc[TW][4];
-        const int4 b = bias ? *(const int4 *)(bias + c0) : make_int4(0, 0, 0, 0);
+        int4 b = bias ? *(const int4 *)(bias + c0) : make_int4(0, 0, 0, 0);
+        if (FAST) {
+            const int rnd = 1 << (q.s - 1);
+            b.x = (b.x << q.sh_acc) + rnd; b.y = (b.y << q.sh_acc) + rnd;
+            b.z = (b.z << q.sh_acc) + rnd; b.w = (b.w << q.sh_acc) + rnd;
+        }
 #pragma unroll
-        for (int o = 0; o < TW; ++o) { acc[o][0] = b.x; acc[o][1] = b.y; acc[o][2] = b.z; acc[o][3] = b.w; }
+        for (int o = 0; o < TW; ++o) { acc[o][0] = 0; acc[o][1] = 0; acc[o][2] = 0; acc[o][3] = 0; }
         const int iw0 = ow0 * S - 1;
 #pragma unroll
         for (int r = 0; r < 3; ++r) {
             const int ih = oh * S + r - 1;
             if (ih < 0 || ih >= g.h) continue;
-            const uint8_t *row = x + (((size_t)in * g.h + ih) * g.w) * g.c + c0;
+            const uint8_t *row = x + (size_t)((in * g.h + ih) * g.w) * g.c + c0;
+            uint32_t words[SPAN];
 #pragma unroll
             for (int xx = 0; xx < SPAN; ++xx) {
                 const int iw = iw0 + xx;
-                uint32_t word = 0;
-                if (iw >= 0 && iw < g.w) word = __ldg((const uint32_t *)(row + (size_t)iw * g.c));
+                words[xx] = (iw >= 0 && iw < g.w) ? __ldg((const uint32_t *)(row + iw * g.c)) : 0u;
+            }
+#pragma unroll
+            for (int xx = 0; xx < SPAN; ++xx) {
                 int v[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] = XS ? (int)(int8_t)(word >> (8 * j)) : (int)((word >> (8 * j)) & 0xffu);
+                for (int j = 0; j < 4; ++j)   // byte j as an int: one PRMT (selector 8|j replicates the sign bit)
+                    v[j] = XS ? prmt_s8(words[xx], j) : (int)__byte_perm(words[xx], 0, 0x4440 | j);
 #pragma unroll
                 for (int s = 0; s < 3; ++s) {
                     // input column xx feeds output o through tap s when xx = o * S + s
@@ -183,18 +201,40 @@ __global__ void __launch_bounds__(128) dwconv3x3_strip_kernel(F8ConvGeom g, F8Re
                 }
             }
         }
+        const int out_row = ((in * g.ho + oh) * g.wo) * g.c + c0;
+        const int bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
         for (int o = 0; o < TW; ++o) {
             const int ow = ow0 + o;
             if (ow >= g.wo) break;
-            const size_t off = (((size_t)in * g.ho + oh) * g.wo + ow) * g.c + c0;
+            const int off = out_row + ow * g.c;
             uint32_t rw = 0;
             if (q.has_res) rw = *(const uint32_t *)((const uint8_t *)res + off);
-            int out[4];
+            if (FAST) {
+                int tv[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) out[j] = f8_requant(acc[o][j], f8_byte(rw, j, q.r_signed), q);
-            if (q.y_kind == F8_S32) *(int4 *)((int32_t *)y + off) = make_int4(out[0], out[1], out[2], out[3]);
-            else *(uint32_t *)((uint8_t *)y + off) = f8_pack4(out[0], out[1], out[2], out[3]);
+                for (int j = 0; j < 4; ++j) {
+                    int v = (acc[o][j] << q.sh_acc) + bb[j];
+                    if (q.has_res) v += f8_byte(rw, j, q.r_signed) << q.sh_res;
+                    v >>= q.s;
+                    tv[j] = q.y_kind == F8_S8 ? max(v, -127) : v;
+                }
+                uint32_t hi2, word;
+                if (q.y_kind == F8_S8) {
+                    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+                    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+                } else {
+                    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+                    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+                }
+                *(uint32_t *)((uint8_t *)y + off) = word;
+            } else {
+                int out[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) out[j] = f8_requant(acc[o][j] + bb[j], f8_byte(rw, j, q.r_signed), q);
+                if (q.y_kind == F8_S32) *(int4 *)((int32_t *)y + off) = make_int4(out[0], out[1], out[2], out[3]);
+                else *(uint32_t *)((uint8_t *)y + off) = f8_pack4(out[0], out[1], out[2], out[3]);
+            }
         }
     }
 }
@@ -386,19 +426,25 @@ cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void
     if (total == 0) return cudaSuccess;
     const bool strip_ok = g.c % 4 == 0 && g.kh == 3 && g.kw == 3 && g.pad_h == 1 && g.pad_w == 1 &&
                           g.stride_h == g.stride_w && (g.stride_h == 1 || g.stride_h == 2) &&
-                          (((uintptr_t)x | (uintptr_t)y | (uintptr_t)res | (uintptr_t)bias) & 15) == 0;
+                          (((uintptr_t)x | (uintptr_t)y | (uintptr_t)res | (uintptr_t)bias) & 15) == 0 &&
+                          (size_t)g.n * g.h * g.w * g.c < (1u << 31) && total * (q.y_kind == F8_S32 ? 4 : 1) < (1u << 31);
     if (strip_ok) {
         const int tw = g.stride_h == 1 ? 8 : 4;
-        const size_t threads = (size_t)g.n * g.ho * ((g.wo + tw - 1) / tw) * (g.c / 4);
-        const int grid = grid_for(threads, 128);
+        const int strips = (g.wo + tw - 1) / tw;
+        const int threads = g.n * g.ho * strips * (g.c / 4);
+        const int grid = grid_for((size_t)threads, 128);
         const uint8_t *xp = (const uint8_t *)x;
+        const bool fast = q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24;
+#define F8_DW_LAUNCH(S_, TW_, XS_, FAST_) \
+    dwconv3x3_strip_kernel<S_, TW_, XS_, FAST_><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y, strips, threads)
         if (g.stride_h == 1) {
-            if (g.x_signed) dwconv3x3_strip_kernel<1, 8, true><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y);
-            else dwconv3x3_strip_kernel<1, 8, false><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y);
+            if (g.x_signed) { if (fast) F8_DW_LAUNCH(1, 8, true, true); else F8_DW_LAUNCH(1, 8, true, false); }
+            else { if (fast) F8_DW_LAUNCH(1, 8, false, true); else F8_DW_LAUNCH(1, 8, false, false); }
         } else {
-            if (g.x_signed) dwconv3x3_strip_kernel<2, 4, true><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y);
-            else dwconv3x3_strip_kernel<2, 4, false><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y);
+            if (g.x_signed) { if (fast) F8_DW_LAUNCH(2, 4, true, true); else F8_DW_LAUNCH(2, 4, true, false); }
+            else { if (fast) F8_DW_LAUNCH(2, 4, false, true); else F8_DW_LAUNCH(2, 4, false, false); }
         }
+#undef F8_DW_LAUNCH
     } else if (g.c % 4 == 0)
         dwconv_vec4_kernel<<<grid_for(total / 4, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
     else
