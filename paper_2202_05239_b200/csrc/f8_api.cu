@@ -319,6 +319,8 @@ struct Step {
 struct f8_net {
     std::vector<NetLayer> layers;
     std::vector<int> t_h, t_w, t_c, t_elem;     // per tensor: per-image shape and element size
+    std::vector<int> t_cp;                       // per tensor: channels as stored (intermediate 8-bit tensors are padded
+                                                 // to a multiple of 16 so that every dense layer can use the TMA path)
     int max_batch = 0;
     // cached execution plan
     int plan_batch = -1;
@@ -340,7 +342,7 @@ namespace {
 size_t round256(size_t v) { return (v + 255) / 256 * 256; }
 
 size_t tensor_bytes(const f8_net *net, int t, int batch) {
-    return (size_t)batch * net->t_h[t] * net->t_w[t] * net->t_c[t] * net->t_elem[t];
+    return (size_t)batch * net->t_h[t] * net->t_w[t] * net->t_cp[t] * net->t_elem[t];
 }
 
 // Assigns workspace offsets: tensors whose lifetimes do not overlap may share memory (first fit).
@@ -488,27 +490,59 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
                 return cleanup(fail(F8_ERR_ACC_BOUND, "layer %d channel %d: accumulator bound %lld exceeds int32", i, co, bound));
         }
     }
+    // Stored channel counts: intermediate 8-bit tensors whose channel count is not a multiple of 16 (24 in
+    // MobileNetV2) are padded with channels that are identically zero -- zero weights and bias produce them,
+    // zero weights consume them -- so the arithmetic of the real channels is untouched.
+    net->t_cp = net->t_c;
+    for (int t = 1; t < n_layers; ++t)
+        if (net->t_elem[t] == 1 && net->t_c[t] % 16 != 0) net->t_cp[t] = (net->t_c[t] + 15) / 16 * 16;
     // second pass (everything validated): upload the parameters
     for (int i = 0; i < n_layers; ++i) {
         NetLayer &L = net->layers[i];
         const f8_conv_desc &d = L.d.conv;
         const int kind = L.d.kind;
+        const int cp_in = net->t_cp[L.d.src], cp_out = net->t_cp[i + 1];
+        L.g.c = cp_in;
+        L.g.c_out = cp_out;
+        L.out_bytes_per_image = (size_t)net->t_h[i + 1] * net->t_w[i + 1] * cp_out * net->t_elem[i + 1];
         if (kind != F8_LAYER_CONV && kind != F8_LAYER_DWCONV && kind != F8_LAYER_LINEAR) continue;
         const int8_t *hw = host_weights[i];
         const int32_t *hb = host_bias ? host_bias[i] : nullptr;
-        const size_t wn = (size_t)d.kh * d.kw * (kind == F8_LAYER_DWCONV ? 1 : d.c) * d.c_out;
+        std::vector<int8_t> w_padded;
+        std::vector<int32_t> b_padded;
+        const int taps = d.kh * d.kw;
+        if (cp_in != d.c || cp_out != d.c_out) {
+            if (kind == F8_LAYER_DWCONV) {
+                w_padded.assign((size_t)cp_out * taps, 0);
+                memcpy(w_padded.data(), hw, (size_t)d.c * taps);
+            } else {
+                w_padded.assign((size_t)cp_out * taps * cp_in, 0);
+                for (int co = 0; co < d.c_out; ++co)
+                    for (int t = 0; t < taps; ++t)
+                        memcpy(&w_padded[((size_t)co * taps + t) * cp_in], &hw[((size_t)co * taps + t) * d.c], (size_t)d.c);
+            }
+            hw = w_padded.data();
+            if (hb) {
+                b_padded.assign((size_t)cp_out, 0);
+                memcpy(b_padded.data(), hb, 4 * (size_t)d.c_out);
+                hb = b_padded.data();
+            }
+        }
+        const size_t wn = (size_t)taps * (kind == F8_LAYER_DWCONV ? 1 : cp_in) * cp_out;
         cudaError_t e = cudaMalloc(&L.w, round256(wn));
         if (e == cudaSuccess) e = cudaMemcpy(L.w, hw, wn, cudaMemcpyHostToDevice);
         if (e == cudaSuccess && hb) {
-            e = cudaMalloc(&L.b, round256(4 * (size_t)d.c_out));
-            if (e == cudaSuccess) e = cudaMemcpy(L.b, hb, 4 * (size_t)d.c_out, cudaMemcpyHostToDevice);
+            e = cudaMalloc(&L.b, round256(4 * (size_t)cp_out));
+            if (e == cudaSuccess) e = cudaMemcpy(L.b, hb, 4 * (size_t)cp_out, cudaMemcpyHostToDevice);
         }
         if (e != cudaSuccess) return cleanup(cuda_fail(e, "parameter upload"));
+        hw = host_weights[i];     // the stem packing below reads the caller's layout
 
         // 3-channel (<= 8) stems with an even stride: widen pixels to 8 bytes so that the kw-tap window of an
         // output column is one contiguous, 16-byte aligned run of kw8 bytes; the layer then is a kh x 1
         // convolution over kw8 "channels" of an overlapping strided view, which the tensor-core path takes.
-        if (kind == F8_LAYER_CONV && d.c <= 8 && d.c % 16 != 0 && d.stride % 2 == 0 && d.kw * 8 <= 256) {
+        if (kind == F8_LAYER_CONV && cp_in == d.c && cp_out == d.c_out && d.c <= 8 && d.stride % 2 == 0 &&
+            d.kw * 8 <= 256) {
             L.packed = true;
             L.pack_left = d.pad;
             L.pack_kw8 = (d.kw * 8 + 31) / 32 * 32;
@@ -694,8 +728,14 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
             net->event_layer.push_back(stp.layer);
         }
         if (layer_dump && stp.kind >= 0 && layer_dump[stp.layer]) {
-            e = cudaMemcpyAsync(layer_dump[stp.layer], stp.y, (size_t)batch * L.out_bytes_per_image,
-                                cudaMemcpyDeviceToDevice, st);
+            const int c_true = net->t_c[stp.layer + 1], c_stored = net->t_cp[stp.layer + 1];
+            if (c_true == c_stored)
+                e = cudaMemcpyAsync(layer_dump[stp.layer], stp.y, (size_t)batch * L.out_bytes_per_image,
+                                    cudaMemcpyDeviceToDevice, st);
+            else   // drop the zero padding channels: one row per pixel
+                e = cudaMemcpy2DAsync(layer_dump[stp.layer], (size_t)c_true, stp.y, (size_t)c_stored, (size_t)c_true,
+                                      (size_t)batch * net->t_h[stp.layer + 1] * net->t_w[stp.layer + 1],
+                                      cudaMemcpyDeviceToDevice, st);
             if (e != cudaSuccess) return cuda_fail(e, "layer dump copy");
         }
     }

@@ -769,7 +769,8 @@ size_t f8_tc_plan_size() { return sizeof(F8TcPlan); }
 
 bool f8_tc_supported(const F8ConvGeom &g, size_t x_bytes) {
     if (g.c % 16 != 0) return false;                 // TMA strides are multiples of 16 bytes
-    if (x_bytes < 128 * 1024) return false;          // tiny tensors: latency bound, CUDA-core kernel
+    if (x_bytes < 128 * 1024) return false;          // im2col tensor maps of tensors below 128 KiB are avoided; such
+                                                     // problems are latency bound anyway: CUDA-core kernel
     if (g.kh > 255 || g.kw > 255) return false;
     if ((long long)g.n * g.ho * g.wo > 0x7fffff00ll) return false;
     return true;
