@@ -202,6 +202,46 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+
+// The K = 32 slices of one sub-chunk (kb / 32 of them), issued from one asm block.  A lone thread pays a few
+// cycles for every instruction it executes, and the tensor pipe is only kept busy when an MMA costs the
+// issuing thread no more than a handful of them: the shared-memory descriptors of the slices differ only
+// in their low words (start address, 16-byte units), so those are advanced with 32-bit adds inside the
+// block and the constant high word (SBO, version, swizzle mode) is attached by a register-pair move.
+#define F8_MMA_I8 "tcgen05.mma.cta_group::1.kind::i8 [%0], a, b, %4, "
+#define F8_MMA_NEXT(off) \
+    "add.u32 x, %1, " #off ";\n\tadd.u32 y, %2, " #off ";\n\tmov.b64 a, {x, %3};\n\tmov.b64 b, {y, %3};\n\t" F8_MMA_I8 "t;\n\t"
+template <int MMAS>
+__device__ __forceinline__ void mma_i8_sub(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                           uint32_t idesc, uint32_t accumulate) {
+    if (MMAS == 1)
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                     "mov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t" F8_MMA_I8 "p;\n\t}" ::"r"(d_tmem),
+                     "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+                     : "memory");
+    else if (MMAS == 2)
+        asm volatile("{\n\t.reg .pred p, t;\n\t.reg .b64 a, b;\n\t.reg .b32 x, y;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                     "setp.eq.b32 t, 0, 0;\n\tmov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t" F8_MMA_I8 "p;\n\t"
+                     F8_MMA_NEXT(2) "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+                     : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p, t;\n\t.reg .b64 a, b;\n\t.reg .b32 x, y;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                     "setp.eq.b32 t, 0, 0;\n\tmov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t" F8_MMA_I8 "p;\n\t"
+                     F8_MMA_NEXT(2) F8_MMA_NEXT(4) F8_MMA_NEXT(6) "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi),
+                     "r"(idesc), "r"(accumulate)
+                     : "memory");
+}
+
+// All sub-chunks of one stage use; `a_lo` is the low descriptor word of the stage's first A tile.
+template <int MMAS>
+__device__ __forceinline__ void mma_i8_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t a16, uint32_t sub16,
+                                             uint32_t desc_hi, uint32_t idesc, int subs, uint32_t accumulate_first) {
+    mma_i8_sub<MMAS>(d_tmem, a_lo, a_lo + a16, desc_hi, idesc, accumulate_first);
+    for (int j = 1; j < subs; ++j) {
+        a_lo += sub16;
+        mma_i8_sub<MMAS>(d_tmem, a_lo, a_lo + a16, desc_hi, idesc, 1u);
+    }
+}
 // mbarrier arrives once every tcgen05.mma issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
@@ -465,7 +505,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             bool committed_any = false;
             int last_acc = 0;
             uint32_t last_acc_phase = 0;
-            const uint64_t a_desc0 = p.desc_hi | (uint64_t)((smem_base & 0x3ffffu) >> 4);
+            // descriptor words: the low one holds the start address (16-byte units, 14 bits) and LBO
+            const uint32_t desc_lo0 = (uint32_t)p.desc_hi | ((smem_base & 0x3ffffu) >> 4);
+            const uint32_t desc_hi32 = (uint32_t)(p.desc_hi >> 32);
+            uint32_t stage_lo = desc_lo0;
             const uint32_t stage16 = p.stage_bytes >> 4, sub16 = p.sub_bytes >> 4, a16 = p.a_bytes >> 4;
             const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
@@ -477,20 +520,14 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 for (int kc = 0; kc < k_iters; kc += p.group) {
                     if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, 103)) { ok = false; break; }
                     tc_fence_after();
-                    uint64_t a_desc = a_desc0 + (uint64_t)(stage * stage16);
                     const int subs = min(p.group, k_iters - kc);
-                    for (int j = 0; j < subs; ++j, a_desc += sub16) {
-                        const uint64_t b_desc = a_desc + a16;
-                        // 32 bytes of K per instruction: the descriptor start address advances by 2 (16-byte units)
-                        mma_i8(d_tmem, a_desc, b_desc, p.idesc, (kc | j) != 0 ? 1u : 0u);
-                        if (mmas >= 2) mma_i8(d_tmem, a_desc + 2, b_desc + 2, p.idesc, 1u);
-                        if (mmas == 4) {
-                            mma_i8(d_tmem, a_desc + 4, b_desc + 4, p.idesc, 1u);
-                            mma_i8(d_tmem, a_desc + 6, b_desc + 6, p.idesc, 1u);
-                        }
-                    }
+                    const uint32_t first = kc != 0 ? 1u : 0u;      // the tile's first MMA overwrites the accumulator
+                    if (mmas == 4) mma_i8_stage<4>(d_tmem, stage_lo, a16, sub16, desc_hi32, p.idesc, subs, first);
+                    else if (mmas == 2) mma_i8_stage<2>(d_tmem, stage_lo, a16, sub16, desc_hi32, p.idesc, subs, first);
+                    else mma_i8_stage<1>(d_tmem, stage_lo, a16, sub16, desc_hi32, p.idesc, subs, first);
                     mma_commit(empty_bar + 8 * stage);    // frees the stage when these MMAs have read it
-                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                    stage_lo += stage16;
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; stage_lo = desc_lo0; }
                 }
                 if (!ok) break;
                 mma_commit(tfull_bar + 8 * acc);          // accumulator complete
