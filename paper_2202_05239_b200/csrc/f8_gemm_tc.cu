@@ -77,7 +77,11 @@ struct TcParams {
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
     uint32_t stage_bytes;     // group * sub_bytes
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
-    uint32_t tx_a, tx_b;      // bytes the A / B load of a stage delivers
+    uint32_t tx_a, tx_b;      // bytes the A / B load of a k-iteration delivers
+    uint32_t tx_sub;          // bytes a k-iteration adds to its stage's full barrier
+    int b_res;                // 1: the whole weight tensor stays in shared memory for the life of the CTA
+    uint32_t b_bytes;         // bytes of one B tile (rounded to 1024)
+    uint32_t bres_off;        // resident weights: tile (n_t, k-iteration) at bres_off + (n_t * k_iters + k) * b_bytes
     uint32_t idesc;           // tcgen05 instruction descriptor
     uint64_t desc_hi;         // constant upper part of the shared-memory matrix descriptors
     const int32_t *bias;
@@ -232,14 +236,16 @@ __device__ __forceinline__ void mma_i8_sub(uint32_t d_tmem, uint32_t a_lo, uint3
                      : "memory");
 }
 
-// All sub-chunks of one stage use; `a_lo` is the low descriptor word of the stage's first A tile.
+// All sub-chunks of one stage use; `a_lo` / `b_lo` are the low descriptor words of its first A / B tile.
 template <int MMAS>
-__device__ __forceinline__ void mma_i8_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t a16, uint32_t sub16,
-                                             uint32_t desc_hi, uint32_t idesc, int subs, uint32_t accumulate_first) {
-    mma_i8_sub<MMAS>(d_tmem, a_lo, a_lo + a16, desc_hi, idesc, accumulate_first);
+__device__ __forceinline__ void mma_i8_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_step,
+                                             uint32_t b_step, uint32_t desc_hi, uint32_t idesc, int subs,
+                                             uint32_t accumulate_first) {
+    mma_i8_sub<MMAS>(d_tmem, a_lo, b_lo, desc_hi, idesc, accumulate_first);
     for (int j = 1; j < subs; ++j) {
-        a_lo += sub16;
-        mma_i8_sub<MMAS>(d_tmem, a_lo, a_lo + a16, desc_hi, idesc, 1u);
+        a_lo += a_step;
+        b_lo += b_step;
+        mma_i8_sub<MMAS>(d_tmem, a_lo, b_lo, desc_hi, idesc, 1u);
     }
 }
 // mbarrier arrives once every tcgen05.mma issued so far by this thread has completed.
@@ -378,7 +384,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     extern __shared__ uint8_t smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 5];
     __shared__ __align__(8) uint64_t epi_bars[8];   // out_full[2], out_free[2], res_full[2], res_free[2]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -389,6 +395,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const uint32_t empty_bar = smem_u32(&bars[MAX_STAGES]);
     const uint32_t tfull_bar = smem_u32(&bars[2 * MAX_STAGES]);
     const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + 2]);
+    const uint32_t bres_bar = smem_u32(&bars[2 * MAX_STAGES + 4]);   // resident weights have landed
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t out_full = smem_u32(&epi_bars[0]), out_free = smem_u32(&epi_bars[2]);
     const uint32_t res_full = smem_u32(&epi_bars[4]), res_free = smem_u32(&epi_bars[6]);
@@ -399,6 +406,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             mbar_init(full_bar + 8 * s, 1);       // one arrival (with the byte count of the whole group) per use
             mbar_init(empty_bar + 8 * s, 1);
         }
+        mbar_init(bres_bar, 1);
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
             mbar_init(tempty_bar + 8 * a, NUM_EPI_WARPS);
@@ -446,6 +454,22 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // different per-thread TMA queues, so they overlap.
         const uint2 *ktab = (const uint2 *)(smem + p.ktab_off);
         const int opnd = warp == A_PROD_WARP ? 0 : 1;
+        if (opnd == 1 && p.b_res) {
+            // Resident weights: when all B tiles fit beside the pipeline, they are loaded once and every tile
+            // of this CTA reuses them; the stages then carry activations only (the weight re-reads are what
+            // saturates the L2 -> SM path of layers with few output channels).
+            const int n_loads = p.n_tiles * k_iters;
+            if (lane == 0) mbar_expect_tx(bres_bar, (uint32_t)n_loads * p.tx_b);
+            __syncwarp();
+            for (int i = lane; i < n_loads; i += 32) {
+                const int n_t = i / k_iters, k = i - n_t * k_iters;
+                const uint2 e = ktab[k];
+                tma_load_3d(smem_base + p.bres_off + (uint32_t)i * p.b_bytes, &map_b, bres_bar, (int)e.x, (int)(e.y >> 16),
+                            n_t * p.bn);
+            }
+            // the loads must have landed before this CTA's shared memory may go away
+            mbar_wait(bres_bar, 0, abortp, p.status, 107);
+        } else {
         int stage = 0;
         uint32_t phase = 0;
         bool have_last = false;
@@ -470,7 +494,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int subs = min(p.group, k_iters - kc);
                 const uint32_t fb = full_bar + 8 * stage;
                 // one arrival per stage use; it announces the bytes of every load of the group
-                if (opnd == 0 && lane == 0) mbar_expect_tx(fb, (uint32_t)subs * (p.tx_a + p.tx_b));
+                if (opnd == 0 && lane == 0) mbar_expect_tx(fb, (uint32_t)subs * p.tx_sub);
                 const int j = (lane - stage * p.group) & 31;
                 if (j < subs) {
                     const uint2 e = ktab[kc + j];       // x: first channel of the chunk, y: tap << 16 | r << 8 | s
@@ -495,6 +519,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                    (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
             }
         }
+        }
     } else if (warp == MMA_WARP) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
@@ -510,6 +535,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const uint32_t desc_hi32 = (uint32_t)(p.desc_hi >> 32);
             uint32_t stage_lo = desc_lo0;
             const uint32_t stage16 = p.stage_bytes >> 4, sub16 = p.sub_bytes >> 4, a16 = p.a_bytes >> 4;
+            const uint32_t b16 = p.b_bytes >> 4, bres_lo = desc_lo0 + (p.bres_off >> 4);
+            const uint32_t b_step = p.b_res ? b16 : sub16;
+            if (p.b_res && !mbar_wait(bres_bar, 0, abortp, p.status, 108)) ok = false;
             const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
@@ -517,14 +545,20 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, abortp, p.status, 102)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * 256;   // two 256-column accumulators
+                uint32_t b_tile_lo = 0;
+                if (p.b_res) {
+                    const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
+                    b_tile_lo = bres_lo + (uint32_t)(n_t * k_iters) * b16;
+                }
                 for (int kc = 0; kc < k_iters; kc += p.group) {
                     if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, 103)) { ok = false; break; }
                     tc_fence_after();
                     const int subs = min(p.group, k_iters - kc);
                     const uint32_t first = kc != 0 ? 1u : 0u;      // the tile's first MMA overwrites the accumulator
-                    if (mmas == 4) mma_i8_stage<4>(d_tmem, stage_lo, a16, sub16, desc_hi32, p.idesc, subs, first);
-                    else if (mmas == 2) mma_i8_stage<2>(d_tmem, stage_lo, a16, sub16, desc_hi32, p.idesc, subs, first);
-                    else mma_i8_stage<1>(d_tmem, stage_lo, a16, sub16, desc_hi32, p.idesc, subs, first);
+                    const uint32_t b_lo = p.b_res ? b_tile_lo + (uint32_t)kc * b16 : stage_lo + a16;
+                    if (mmas == 4) mma_i8_stage<4>(d_tmem, stage_lo, b_lo, sub16, b_step, desc_hi32, p.idesc, subs, first);
+                    else if (mmas == 2) mma_i8_stage<2>(d_tmem, stage_lo, b_lo, sub16, b_step, desc_hi32, p.idesc, subs, first);
+                    else mma_i8_stage<1>(d_tmem, stage_lo, b_lo, sub16, b_step, desc_hi32, p.idesc, subs, first);
                     mma_commit(empty_bar + 8 * stage);    // frees the stage when these MMAs have read it
                     stage_lo += stage16;
                     if (++stage == p.stages) { stage = 0; phase ^= 1; stage_lo = desc_lo0; }
@@ -850,6 +884,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.div_ho = make_fast_div(g.ho);
     p.a_bytes = (uint32_t)(TILE_M * p.kb + 1023) / 1024 * 1024;
     const uint32_t b_bytes = (uint32_t)(p.bn * p.kb + 1023) / 1024 * 1024;
+    p.b_bytes = b_bytes;
     p.sub_bytes = p.a_bytes + b_bytes;
     p.tx_a = (uint32_t)(TILE_M * p.kb);
     p.tx_b = (uint32_t)(p.bn * p.kb);
@@ -872,7 +907,15 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // k-iterations per stage: every stage use costs the MMA thread a wait, a fence and a commit (a few hundred
     // cycles), so short K chunks are grouped -- as long as at least three stages and one lane per load remain
     const int k_iters = g.kh * g.kw * p.c_chunks;
-    const size_t avail = SMEM_LIMIT - 1024 - staging;
+    size_t avail = SMEM_LIMIT - 1024 - staging;
+    // resident weights: one N tile, and at least 64 KiB left for the activation pipeline
+    const size_t b_all = (size_t)p.n_tiles * k_iters * b_bytes;
+    p.b_res = (p.n_tiles == 1 && b_all + 64 * 1024 <= avail && !getenv("F8_NO_BRES")) ? 1 : 0;
+    if (p.b_res) {
+        avail -= b_all;
+        p.sub_bytes = p.a_bytes;
+    }
+    p.tx_sub = p.tx_a + (p.b_res ? 0u : p.tx_b);
     const int uses = (k_iters + 7) / 8;                  // at most eight k-iterations per stage, evenly split
     int group = (k_iters + uses - 1) / uses;
     while (group > 1 && avail / ((size_t)group * p.sub_bytes) < 3) --group;
@@ -890,6 +933,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.res_off = p.out_off + 2 * p.out_bytes;
     p.bias_off = p.res_off + (q.has_res ? 2 * p.out_bytes : 0u);
     p.ktab_off = (uint32_t)(p.stages * p.stage_bytes + staging - ktab_bytes);
+    p.bres_off = (uint32_t)(p.stages * p.stage_bytes + staging);
     // instruction descriptor: D = s32 (2 at bit 4), A format at bit 7 (0 = u8, 1 = s8), B = s8 at bit 10,
     // both operands K-major, N/8 at bit 17, M/16 at bit 24
     p.idesc = (2u << 4) | ((g.x_signed ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) |
@@ -964,7 +1008,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     const int total_tiles = p.m_tiles * p.n_tiles;
     plan->grid = total_tiles < sms ? total_tiles : sms;
     // at least half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
-    plan->smem = (size_t)p.stages * p.stage_bytes + staging + 1024;
+    plan->smem = (size_t)p.stages * p.stage_bytes + staging + (p.b_res ? b_all : 0) + 1024;
     if (plan->smem < 120 * 1024) plan->smem = 120 * 1024;
     static bool attr_set = false;
     if (!attr_set) {
