@@ -131,7 +131,7 @@ f8_status run_dense(const F8ConvGeom &g, const F8Requant &q, const void *x, cons
         const char *why = "";
         cudaError_t e = f8_tc_plan_init(plan.get(), g, q, dense_view(x, g), w, bias, res, y, f8_status_word(), &why);
         if (e == cudaSuccess) {
-            e = f8_tc_launch(plan.get(), st);
+            e = f8_tc_launch(plan.get(), false, st);   // the caller's weights may come from earlier work in the stream
             if (e != cudaSuccess) return cuda_fail(e, "tensor-core conv launch");
             ++g_tc_launches;
             return F8_OK;
@@ -319,6 +319,7 @@ struct Step {
 struct f8_net {
     std::vector<NetLayer> layers;
     std::vector<int> t_h, t_w, t_c, t_elem;     // per tensor: per-image shape and element size
+    bool overlap_layers = getenv("F8NET_NO_OVERLAP") == nullptr;   // programmatic dependent launch between layers
     std::vector<int> t_cp;                       // per tensor: channels as stored (intermediate 8-bit tensors are padded
                                                  // to a multiple of 16 so that every dense layer can use the TMA path)
     int max_batch = 0;
@@ -707,7 +708,9 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                 break;
             case F8_LAYER_CONV:
             case F8_LAYER_LINEAR:
-                if (stp.use_tc) { e = f8_tc_launch(stp.plan.get(), st); ++g_tc_launches; }
+                // the net owns its weights (uploaded at creation), so a layer's prologue and weight loads may
+                // overlap the tail of the previous layer
+                if (stp.use_tc) { e = f8_tc_launch(stp.plan.get(), net->overlap_layers, st); ++g_tc_launches; }
                 else e = f8_launch_conv_direct(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st);
                 break;
             case F8_LAYER_DWCONV:

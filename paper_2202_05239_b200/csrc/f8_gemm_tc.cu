@@ -108,6 +108,13 @@ struct TcParams {
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// Programmatic dependent launch.  A grid launched with the programmatic-serialization attribute may start
+// while its predecessor in the stream is still running; grid_dependency_wait() returns once every
+// predecessor has completed and its writes are visible (at once for an ordinary launch).  Everything that
+// reads activations or writes the output sits behind it; the prologue and the weight loads do not.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
@@ -439,6 +446,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    // the next grid in the stream may be scheduled from here on: its CTAs take over an SM when this grid's
+    // CTA there has exited, and run their prologue while the rest of this grid finishes
+    grid_launch_dependents();
 
     const int total_tiles = p.m_tiles * p.n_tiles;
     const int k_iters = p.kh * p.kw * p.c_chunks;
@@ -470,6 +480,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             // the loads must have landed before this CTA's shared memory may go away
             mbar_wait(bres_bar, 0, abortp, p.status, 107);
         } else {
+        if (opnd == 0) grid_dependency_wait();      // activations come from the previous grid; weights do not
         int stage = 0;
         uint32_t phase = 0;
         bool have_last = false;
@@ -580,6 +591,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     } else if (warp == MOVER_WARP) {
         // ------------------------------------------------------------------ output mover
         if (STAGED && lane == 0) {
+            grid_dependency_wait();     // the output may overwrite a tensor the previous grid still reads
             // stores: tile t leaves from output buffer t & 1 once all epilogue warps have written it
             int local = 0;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
@@ -600,6 +612,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     } else if (warp == FETCH_WARP) {
         // ------------------------------------------------------------------ residual fetcher
         if (RES && lane == 0) {
+            grid_dependency_wait();
             // residual tiles: up to two tiles ahead of the epilogue
             int local = 0;
             int last = -1;
@@ -696,6 +709,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 }
             }
         } else {
+            grid_dependency_wait();     // direct stores (and residual reads) from these warps
             const int tile_row = quarter * 32 + lane;   // this thread's row of the tile
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
@@ -1036,16 +1050,32 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     return cudaSuccess;
 }
 
-cudaError_t f8_tc_launch(const F8TcPlan *plan, cudaStream_t st) {
+namespace {
+template <int EPI>
+cudaError_t launch_variant(const F8TcPlan *plan, bool overlap_previous, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)plan->grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = plan->smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_previous ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, f8_conv_gemm_tc_kernel<EPI>, plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p);
+}
+}   // namespace
+
+cudaError_t f8_tc_launch(const F8TcPlan *plan, bool overlap_previous, cudaStream_t st) {
     if (plan->p.M == 0) return cudaSuccess;
     switch (plan->p.epi) {
-        case EPI_U8: f8_conv_gemm_tc_kernel<EPI_U8><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
-        case EPI_U8_RES: f8_conv_gemm_tc_kernel<EPI_U8_RES><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
-        case EPI_S8: f8_conv_gemm_tc_kernel<EPI_S8><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
-        case EPI_S8_RES: f8_conv_gemm_tc_kernel<EPI_S8_RES><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
-        default: f8_conv_gemm_tc_kernel<EPI_GENERIC><<<plan->grid, NUM_THREADS, plan->smem, st>>>(plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p); break;
+        case EPI_U8: return launch_variant<EPI_U8>(plan, overlap_previous, st);
+        case EPI_U8_RES: return launch_variant<EPI_U8_RES>(plan, overlap_previous, st);
+        case EPI_S8: return launch_variant<EPI_S8>(plan, overlap_previous, st);
+        case EPI_S8_RES: return launch_variant<EPI_S8_RES>(plan, overlap_previous, st);
+        default: return launch_variant<EPI_GENERIC>(plan, overlap_previous, st);
     }
-    return cudaGetLastError();
 }
 
 cudaError_t f8_tc_probe(int iters, double *ops, int *status_word, cudaStream_t st) {

@@ -61,7 +61,9 @@ size_t f8_tc_plan_size();
 cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant &q, const F8TcTensorView &xv,
                             const int8_t *w /* [c_out][kh][kw][g.c] */, const int32_t *bias, const void *res,
                             void *y, int *status_word, const char **why);
-cudaError_t f8_tc_launch(const F8TcPlan *plan, cudaStream_t st);
+// overlap_previous: the grid may start before the preceding work of the stream has finished; only its weight
+// and bias reads then run early, so it is for callers whose weights no earlier work in the stream writes.
+cudaError_t f8_tc_launch(const F8TcPlan *plan, bool overlap_previous, cudaStream_t st);
 cudaError_t f8_tc_probe(int iters, double *ops, int *status_word, cudaStream_t st);
 
 // Device status word (0 = fine); allocated once per process on first use.

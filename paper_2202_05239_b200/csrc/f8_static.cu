@@ -146,7 +146,7 @@ extern "C" f8_status f8_stem_conv2d_fixed_static(const f8_conv_desc *d, const vo
     pack_stem_weights_kernel<<<(total_w + 255) / 256, 256, 0, st>>>(w, w_packed, d->c_out, d->kh, d->kw, d->c, kw8);
     e = cudaGetLastError();
     if (e == cudaSuccess) e = f8_launch_pack_stem(d->n, d->h, d->w, d->c, wp, d->pad, x, x_packed, st);
-    if (e == cudaSuccess) e = f8_tc_launch(plan, st);
+    if (e == cudaSuccess) e = f8_tc_launch(plan, false, st);
     if (e != cudaSuccess) return f8_set_error(F8_ERR_CUDA, cudaGetErrorString(e));
     return F8_OK;
 }
