@@ -704,24 +704,24 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         cudaError_t e = cudaSuccess;
         switch (stp.kind) {
             case -1:
-                e = f8_launch_pack_stem(batch, L.g.h, L.g.w, L.g.c, L.pack_wp, L.pack_left, stp.x, stp.y, st);
+                e = f8_launch_pack_stem(batch, L.g.h, L.g.w, L.g.c, L.pack_wp, L.pack_left, stp.x, stp.y, st, net->overlap_layers);
                 break;
             case F8_LAYER_CONV:
             case F8_LAYER_LINEAR:
                 // the net owns its weights (uploaded at creation), so a layer's prologue and weight loads may
                 // overlap the tail of the previous layer
                 if (stp.use_tc) { e = f8_tc_launch(stp.plan.get(), net->overlap_layers, st); ++g_tc_launches; }
-                else e = f8_launch_conv_direct(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st);
+                else e = f8_launch_conv_direct(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st, net->overlap_layers);
                 break;
             case F8_LAYER_DWCONV:
-                e = f8_launch_dwconv(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st);
+                e = f8_launch_dwconv(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st, net->overlap_layers);
                 break;
             case F8_LAYER_MAXPOOL:
                 e = f8_launch_maxpool(batch, L.g.h, L.g.w, L.g.c, L.d.conv.kh, L.d.conv.stride, L.d.conv.pad, L.g.x_signed,
-                                      stp.x, stp.y, st);
+                                      stp.x, stp.y, st, net->overlap_layers);
                 break;
             case F8_LAYER_GAP:
-                e = f8_launch_gap(batch, L.g.h, L.g.w, L.g.c, L.g.x_signed, L.q.s, stp.x, stp.y, st);
+                e = f8_launch_gap(batch, L.g.h, L.g.w, L.g.c, L.g.x_signed, L.q.s, stp.x, stp.y, st, net->overlap_layers);
                 break;
         }
         if (e != cudaSuccess) return cuda_fail(e, "layer launch");

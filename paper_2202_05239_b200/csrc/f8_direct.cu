@@ -5,6 +5,28 @@
 
 namespace {
 
+// Programmatic dependent launch (see the tensor-core kernel): every kernel here first waits for the grids
+// before it -- all of its inputs may come from them -- and then lets the grid after it start its prologue.
+__device__ __forceinline__ void grid_dependency_sync() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, int block, bool overlap_previous, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_previous ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+
 __device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {   // u8 x s8
     int d;
     asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
@@ -30,6 +52,7 @@ __global__ void __launch_bounds__(256) conv_direct_kernel(F8ConvGeom g, F8Requan
                                                           const int8_t *__restrict__ w,
                                                           const int32_t *__restrict__ bias,
                                                           const void *__restrict__ res, void *__restrict__ y) {
+    grid_dependency_sync();
     const size_t total = (size_t)g.n * g.ho * g.wo * g.c_out;
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (size_t)gridDim.x * blockDim.x) {
@@ -78,6 +101,7 @@ __global__ void __launch_bounds__(256) dwconv_vec4_kernel(F8ConvGeom g, F8Requan
                                                           const int8_t *__restrict__ w,
                                                           const int32_t *__restrict__ bias,
                                                           const void *__restrict__ res, void *__restrict__ y) {
+    grid_dependency_sync();
     const int c4 = g.c >> 2;
     const size_t total = (size_t)g.n * g.ho * g.wo * c4;
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
@@ -146,6 +170,7 @@ __global__ void __launch_bounds__(128) dwconv3x3_strip_kernel(F8ConvGeom g, F8Re
                                                               const int32_t *__restrict__ bias,
                                                               const void *__restrict__ res, void *__restrict__ y,
                                                               int strips, int total) {
+    grid_dependency_sync();
     constexpr int SPAN = (TW - 1) * S + 3;          // input pixels a strip touches along W
     const int c4 = g.c >> 2;
     // all index arithmetic in 32 bits (the launcher checks that every offset fits)
@@ -243,6 +268,7 @@ __global__ void __launch_bounds__(256) dwconv_scalar_kernel(F8ConvGeom g, F8Requ
                                                             const int8_t *__restrict__ w,
                                                             const int32_t *__restrict__ bias,
                                                             const void *__restrict__ res, void *__restrict__ y) {
+    grid_dependency_sync();
     const size_t total = (size_t)g.n * g.ho * g.wo * g.c;
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (size_t)gridDim.x * blockDim.x) {
@@ -279,6 +305,7 @@ template <int WORDS>   // WORDS 32-bit words (4 channels each) per thread: 4 -> 
 __global__ void __launch_bounds__(256) maxpool_kernel(int n, int h, int w, int c, int ho, int wo, int k, int stride,
                                                       int pad, int x_signed, const uint8_t *__restrict__ x,
                                                       uint8_t *__restrict__ y) {
+    grid_dependency_sync();
     const int cg = c / (4 * WORDS);
     const size_t total = (size_t)n * ho * wo * cg;
     const uint32_t identity = x_signed ? 0x80808080u : 0u;
@@ -324,6 +351,7 @@ __global__ void __launch_bounds__(256) maxpool_kernel(int n, int h, int w, int c
 __global__ void __launch_bounds__(256) maxpool_scalar_kernel(int n, int h, int w, int c, int ho, int wo, int k,
                                                              int stride, int pad, int x_signed,
                                                              const uint8_t *__restrict__ x, uint8_t *__restrict__ y) {
+    grid_dependency_sync();
     const size_t total = (size_t)n * ho * wo * c;
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (size_t)gridDim.x * blockDim.x) {
@@ -353,6 +381,7 @@ __global__ void __launch_bounds__(256) maxpool_scalar_kernel(int n, int h, int w
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) gap_kernel(int hw, int c, int x_signed, int s, const uint8_t *__restrict__ x,
                                                   uint8_t *__restrict__ y) {
+    grid_dependency_sync();
     const int in = blockIdx.y;
     const int ch = blockIdx.x * blockDim.x + threadIdx.x;
     if (ch >= c) return;
@@ -379,6 +408,7 @@ __global__ void __launch_bounds__(256) gap_kernel(int hw, int c, int x_signed, i
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) pack_stem_kernel(int n, int h, int w, int c, int wp, int left,
                                                         const uint8_t *__restrict__ x, uint2 *__restrict__ y) {
+    grid_dependency_sync();
     const size_t total = (size_t)n * h * wp;
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (size_t)gridDim.x * blockDim.x) {
@@ -409,19 +439,19 @@ inline int grid_for(size_t total, int block) {
 }   // namespace
 
 cudaError_t f8_launch_conv_direct(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
-                                  const int32_t *bias, const void *res, void *y, cudaStream_t st) {
+                                  const int32_t *bias, const void *res, void *y, cudaStream_t st, bool overlap_previous) {
     const size_t total = (size_t)g.n * g.ho * g.wo * g.c_out;
     if (total == 0) return cudaSuccess;
     const bool vec = (g.c % 4 == 0) && (((uintptr_t)x | (uintptr_t)w) % 4 == 0);
     if (vec)
-        conv_direct_kernel<true><<<grid_for(total, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
+        launch_k(conv_direct_kernel<true>, grid_for(total, 256), 256, overlap_previous, st, g, q, (const uint8_t *)x, w, bias, res, y);
     else
-        conv_direct_kernel<false><<<grid_for(total, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
+        launch_k(conv_direct_kernel<false>, grid_for(total, 256), 256, overlap_previous, st, g, q, (const uint8_t *)x, w, bias, res, y);
     return cudaGetLastError();
 }
 
 cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
-                             const int32_t *bias, const void *res, void *y, cudaStream_t st) {
+                             const int32_t *bias, const void *res, void *y, cudaStream_t st, bool overlap_previous) {
     const size_t total = (size_t)g.n * g.ho * g.wo * g.c;
     if (total == 0) return cudaSuccess;
     const bool strip_ok = g.c % 4 == 0 && g.kh == 3 && g.kw == 3 && g.pad_h == 1 && g.pad_w == 1 &&
@@ -436,7 +466,7 @@ cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void
         const uint8_t *xp = (const uint8_t *)x;
         const bool fast = q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24;
 #define F8_DW_LAUNCH(S_, TW_, XS_, FAST_) \
-    dwconv3x3_strip_kernel<S_, TW_, XS_, FAST_><<<grid, 128, 0, st>>>(g, q, xp, w, bias, res, y, strips, threads)
+    launch_k(dwconv3x3_strip_kernel<S_, TW_, XS_, FAST_>, grid, 128, overlap_previous, st, g, q, xp, w, bias, res, y, strips, threads)
         if (g.stride_h == 1) {
             if (g.x_signed) { if (fast) F8_DW_LAUNCH(1, 8, true, true); else F8_DW_LAUNCH(1, 8, true, false); }
             else { if (fast) F8_DW_LAUNCH(1, 8, false, true); else F8_DW_LAUNCH(1, 8, false, false); }
@@ -446,40 +476,41 @@ cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void
         }
 #undef F8_DW_LAUNCH
     } else if (g.c % 4 == 0)
-        dwconv_vec4_kernel<<<grid_for(total / 4, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
+        launch_k(dwconv_vec4_kernel, grid_for(total / 4, 256), 256, overlap_previous, st, g, q, (const uint8_t *)x, w, bias, res, y);
     else
-        dwconv_scalar_kernel<<<grid_for(total, 256), 256, 0, st>>>(g, q, (const uint8_t *)x, w, bias, res, y);
+        launch_k(dwconv_scalar_kernel, grid_for(total, 256), 256, overlap_previous, st, g, q, (const uint8_t *)x, w, bias, res, y);
     return cudaGetLastError();
 }
 
 cudaError_t f8_launch_maxpool(int n, int h, int w, int c, int k, int stride, int pad, int x_signed, const void *x,
-                              void *y, cudaStream_t st) {
+                              void *y, cudaStream_t st, bool overlap_previous) {
     const int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
     const size_t total = (size_t)n * ho * wo * c;
     if (total == 0) return cudaSuccess;
     if (c % 16 == 0)
-        maxpool_kernel<4><<<grid_for(total / 16, 256), 256, 0, st>>>(n, h, w, c, ho, wo, k, stride, pad, x_signed,
+        launch_k(maxpool_kernel<4>, grid_for(total / 16, 256), 256, overlap_previous, st, n, h, w, c, ho, wo, k, stride, pad, x_signed,
                                                                      (const uint8_t *)x, (uint8_t *)y);
     else if (c % 4 == 0)
-        maxpool_kernel<1><<<grid_for(total / 4, 256), 256, 0, st>>>(n, h, w, c, ho, wo, k, stride, pad, x_signed,
+        launch_k(maxpool_kernel<1>, grid_for(total / 4, 256), 256, overlap_previous, st, n, h, w, c, ho, wo, k, stride, pad, x_signed,
                                                                     (const uint8_t *)x, (uint8_t *)y);
     else
-        maxpool_scalar_kernel<<<grid_for(total, 256), 256, 0, st>>>(n, h, w, c, ho, wo, k, stride, pad, x_signed,
+        launch_k(maxpool_scalar_kernel, grid_for(total, 256), 256, overlap_previous, st, n, h, w, c, ho, wo, k, stride, pad, x_signed,
                                                                     (const uint8_t *)x, (uint8_t *)y);
     return cudaGetLastError();
 }
 
-cudaError_t f8_launch_gap(int n, int h, int w, int c, int x_signed, int s, const void *x, void *y, cudaStream_t st) {
+cudaError_t f8_launch_gap(int n, int h, int w, int c, int x_signed, int s, const void *x, void *y, cudaStream_t st,
+                          bool overlap_previous) {
     if (n == 0) return cudaSuccess;
     dim3 grid((c + 255) / 256, n);
-    gap_kernel<<<grid, 256, 0, st>>>(h * w, c, x_signed, s, (const uint8_t *)x, (uint8_t *)y);
+    launch_k(gap_kernel, grid, 256, overlap_previous, st, h * w, c, x_signed, s, (const uint8_t *)x, (uint8_t *)y);
     return cudaGetLastError();
 }
 
 cudaError_t f8_launch_pack_stem(int n, int h, int w, int c, int wp, int left, const void *x, void *y,
-                                cudaStream_t st) {
+                                cudaStream_t st, bool overlap_previous) {
     const size_t total = (size_t)n * h * wp;
     if (total == 0) return cudaSuccess;
-    pack_stem_kernel<<<grid_for(total, 256), 256, 0, st>>>(n, h, w, c, wp, left, (const uint8_t *)x, (uint2 *)y);
+    launch_k(pack_stem_kernel, grid_for(total, 256), 256, overlap_previous, st, n, h, w, c, wp, left, (const uint8_t *)x, (uint2 *)y);
     return cudaGetLastError();
 }

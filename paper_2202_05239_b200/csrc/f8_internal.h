@@ -32,17 +32,21 @@ struct F8ConvGeom {
 };
 
 // ---- CUDA-core kernels (f8_direct.cu) -------------------------------------------------
+// overlap_previous: launch with programmatic stream serialization (the kernel itself waits for the grids
+// before it prior to touching memory, so this is always safe; it lets launch latency overlap their tail).
 cudaError_t f8_launch_conv_direct(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
-                                  const int32_t *bias, const void *res, void *y, cudaStream_t st);
+                                  const int32_t *bias, const void *res, void *y, cudaStream_t st,
+                                  bool overlap_previous = false);
 cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
-                             const int32_t *bias, const void *res, void *y, cudaStream_t st);
+                             const int32_t *bias, const void *res, void *y, cudaStream_t st,
+                             bool overlap_previous = false);
 cudaError_t f8_launch_maxpool(int n, int h, int w, int c, int k, int stride, int pad, int x_signed,
-                              const void *x, void *y, cudaStream_t st);
+                              const void *x, void *y, cudaStream_t st, bool overlap_previous = false);
 cudaError_t f8_launch_gap(int n, int h, int w, int c, int x_signed, int s, const void *x, void *y,
-                          cudaStream_t st);
+                          cudaStream_t st, bool overlap_previous = false);
 // channel-padding pre-pass for 3-channel stems: [n,h,w,c] -> [n,h,wp,8] with `left` zero pixels in front
 cudaError_t f8_launch_pack_stem(int n, int h, int w, int c, int wp, int left, const void *x, void *y,
-                                cudaStream_t st);
+                                cudaStream_t st, bool overlap_previous = false);
 
 // ---- tensor-core implicit GEMM (f8_gemm_tc.cu) ----------------------------------------
 struct F8TcPlan;   // opaque: tensor maps + launch parameters of one conv launch
