@@ -101,6 +101,7 @@ struct TcParams {
                                            // tiles, int32 bias' of all padded columns
     uint32_t ktab_off;        // table of k-iteration coordinates (8 bytes each)
     F8Requant q;
+    int mul_acc, mul_res;     // 2^q.sh_acc, 2^q.sh_res (kept opaque to the compiler, see the epilogue)
     int *status;
 };
 
@@ -337,23 +338,36 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int (&ac
 //   y = clamp(t, lo, hi)                saturating pack; the signed quantizer additionally excludes -128
 // cvt.pack.sat packs two saturated values into the low half of d and moves the low half of c above
 // them: d = (c << 16) | (sat(a) << 8) | sat(b).
+// The integer ALU pipe (shifts, byte permutes, 3-input adds, packs) issues a warp instruction every other
+// cycle and is what bounds this code, so work is kept off it: the two scalings are multiply-adds whose
+// power-of-two factors arrive as opaque kernel parameters (the FMA pipe; a visible 1 << n would be turned
+// into shifts), a residual byte costs one PRMT whose selector (zero- or sign-extending) sits in a register,
+// and bias / residual / output go through explicit shared-space accesses.
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
 template <bool RES, bool SIGNED_OUT>
-__device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], const int4 *bias4, uint4 rw, int mul_acc,
-                                                 int mul_res, int r_signed, int s) {
+__device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], uint32_t bias_addr, uint4 rw, int mul_acc,
+                                                 int mul_res, const uint32_t (&rsel)[4], int s) {
     int t[16];
     const uint32_t rwords[4] = {rw.x, rw.y, rw.z, rw.w};
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
-        const int4 b = bias4[g];
-        const int bb[4] = {b.x, b.y, b.z, b.w};
+        const uint4 b = lds128(bias_addr + 16 * g);
+        const int bb[4] = {(int)b.x, (int)b.y, (int)b.z, (int)b.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const int j = 4 * g + k;
-            int v = RES ? acc[j] * mul_acc + bb[k] : acc[j] + bb[k];
+            int v = acc[j] * mul_acc + bb[k];
             if (RES) {
                 int r;
-                if (r_signed) asm("bfe.s32 %0, %1, %2, 8;" : "=r"(r) : "r"(rwords[g]), "r"(8 * k));
-                else asm("bfe.u32 %0, %1, %2, 8;" : "=r"(r) : "r"(rwords[g]), "r"(8 * k));
+                asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(rwords[g]), "r"(rsel[k]));
                 v += r * mul_res;
             }
             v >>= s;
@@ -647,12 +661,15 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const int per_group = (chunks + 3) / 4;     // <= 4 chunks of 16 columns per warp
         const int ch_begin = min(group * per_group, chunks);
         const int nch = min(ch_begin + per_group, chunks) - ch_begin;
-        const int mul_acc = 1 << p.q.sh_acc, mul_res = 1 << p.q.sh_res;
+        const int mul_acc = p.mul_acc, mul_res = p.mul_res;     // 2^sh_acc, 2^sh_res
         int local = 0;
         bool ok = true;
         if (STAGED) {
-            const int *bias_all = (const int *)(smem + p.bias_off);
             const int tile_row = quarter * 32 + lane;
+            // PRMT selectors that turn byte k of a residual word into an int (zero- or sign-extended)
+            uint32_t rsel[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) rsel[k] = p.q.r_signed ? (0x8880u | (0x1111u * k)) : (0x4440u | k);
             // where this thread's 16-byte chunks live inside a staged tile (same for every tile)
             uint32_t so[4];
 #pragma unroll
@@ -674,27 +691,26 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 got = mbar_wait(out_free + 8 * acc, acc_phase ^ 1, abortp, p.status, 109) && got;
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tc_fence_after();
-                uint8_t *out_buf = smem + p.out_off + acc * p.out_bytes;
-                const uint8_t *res_buf = smem + p.res_off + acc * p.out_bytes;
+                const uint32_t out_buf = smem_base + p.out_off + acc * p.out_bytes;
+                const uint32_t res_buf = smem_base + p.res_off + acc * p.out_bytes;
+                const uint32_t bias_s = smem_base + p.bias_off + 4 * c_first;
                 int va[16], vb[16];
                 if (my_nch > 0) tmem_ld16(t_addr, va);
 #pragma unroll
                 for (int i = 0; i < 4; i += 2) {
                     if (i < my_nch) {
                         uint4 rw = make_uint4(0, 0, 0, 0);
-                        if (RES) rw = *(const uint4 *)(res_buf + so[i]);
+                        if (RES) rw = lds128(res_buf + so[i]);
                         tmem_ld_wait();
                         if (i + 1 < my_nch) tmem_ld16(t_addr + (i + 1) * 16, vb);
-                        const int4 *b4 = (const int4 *)(bias_all + c_first + i * 16);
-                        *(uint4 *)(out_buf + so[i]) = epilogue_fast16<RES, SGN>(va, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s);
+                        sts128(out_buf + so[i], epilogue_fast16<RES, SGN>(va, bias_s + 64 * (i), rw, mul_acc, mul_res, rsel, p.q.s));
                     }
                     if (i + 1 < my_nch) {
                         uint4 rw = make_uint4(0, 0, 0, 0);
-                        if (RES) rw = *(const uint4 *)(res_buf + so[i + 1]);
+                        if (RES) rw = lds128(res_buf + so[i + 1]);
                         tmem_ld_wait();
                         if (i + 2 < my_nch) tmem_ld16(t_addr + (i + 2) * 16, va);
-                        const int4 *b4 = (const int4 *)(bias_all + c_first + (i + 1) * 16);
-                        *(uint4 *)(out_buf + so[i + 1]) = epilogue_fast16<RES, SGN>(vb, b4, rw, mul_acc, mul_res, p.q.r_signed, p.q.s);
+                        sts128(out_buf + so[i + 1], epilogue_fast16<RES, SGN>(vb, bias_s + 64 * (i + 1), rw, mul_acc, mul_res, rsel, p.q.s));
                     }
                 }
                 // accumulator and residual have been read, the output part is written: make the writes
@@ -957,6 +973,8 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.res = (const uint8_t *)res;
     p.y = (uint8_t *)y;
     p.q = q;
+    p.mul_acc = 1 << q.sh_acc;
+    p.mul_res = 1 << q.sh_res;
     p.status = status_word;
     const int ysz = q.y_kind == F8_S32 ? 4 : 1;
     const size_t row_bytes = (size_t)g.c_out * ysz;
