@@ -46,7 +46,10 @@ constexpr int MOVER_WARP = 2;              // one thread stores finished output 
 constexpr int FETCH_WARP = 3;              // one thread fetches residual tiles
 constexpr int FIRST_EPI_WARP = 4;          // warps 4..19; warp & 3 is the TMEM lane quarter
 constexpr int B_PROD_WARP = FIRST_EPI_WARP + NUM_EPI_WARPS;   // requests weight tiles
-constexpr int NUM_THREADS = 32 * (B_PROD_WARP + 1);
+// Issuing a tcgen05.mma costs its thread 70-100 cycles, more than the tensor pipe needs for a tile of up to
+// 128 columns; a second issuer (alternate tiles, the other accumulator) keeps the pipe fed for such layers.
+constexpr int MMA2_WARP = B_PROD_WARP + 1;
+constexpr int NUM_THREADS = 32 * (MMA2_WARP + 1);
 constexpr int MAX_STAGES = 16;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
@@ -74,6 +77,8 @@ struct TcParams {
     FastDiv div_n_tiles, div_wo, div_ho;
     int stages;
     int group;                // k-iterations per stage (1..8)
+    int uses;                 // stage uses per tile: ceil(k_iters / group)
+    int dual_issue;           // 1: two MMA-issuing threads (needs stages >= 2 * uses)
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
     uint32_t stage_bytes;     // group * sub_bytes
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
@@ -545,9 +550,15 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             }
         }
         }
-    } else if (warp == MMA_WARP) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+    } else if (warp == MMA_WARP || warp == MMA2_WARP) {
+        // ------------------------------------------------------------------ MMA issuers
+        // With two issuers, issuer q takes the CTA's tiles with (local & 1) == q, i.e. accumulator q, and steps
+        // over the stage uses of the other issuer's tiles.  A parity wait can only tell a phase from its
+        // neighbour, so an issuer must never wait on a stage whose previous use has not been filled yet: the
+        // plan enables the second issuer only when stages >= 2 * uses per tile, which guarantees that (the
+        // previous use of the stage then belongs to a tile this issuer, or the other one before it, is done with).
+        const int q_issuer = warp == MMA_WARP ? 0 : 1;
+        if (lane == 0 && (q_issuer == 0 || p.dual_issue)) {
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -566,6 +577,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
+                if (p.dual_issue && acc != q_issuer) {
+                    // the other issuer's tile: step over its stage uses
+                    stage += p.uses;
+                    while (stage >= p.stages) { stage -= p.stages; phase ^= 1; }
+                    stage_lo = desc_lo0 + (uint32_t)stage * stage16;
+                    continue;
+                }
                 const uint32_t acc_phase = (local >> 1) & 1;
                 if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, abortp, p.status, 102)) { ok = false; break; }
                 tc_fence_after();
@@ -959,6 +977,8 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         return cudaErrorInvalidValue;
     }
     p.stages = stages;
+    p.uses = (k_iters + group - 1) / group;
+    p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !getenv("F8_NO_DUAL")) ? 1 : 0;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
     p.res_off = p.out_off + 2 * p.out_bytes;
     p.bias_off = p.res_off + (q.has_res ? 2 * p.out_bytes : 0u);
