@@ -298,7 +298,9 @@ struct NetLayer {
     int32_t *b = nullptr;
     // stem packing (3-channel inputs on the tensor-core path)
     bool packed = false;
-    int pack_wp = 0, pack_left = 0, pack_kw8 = 0;
+    int pack_wp = 0, pack_left = 0, pack_kw8 = 0;   // pack_kw8: bytes of one window row (kw cells of 16 bytes, padded)
+    int pack_cpad = 8;     // bytes per pixel inside a cell (4 when c <= 4); a cell is two rows = 2 * pack_cpad bytes
+    int pack_hp = 0, pack_kh = 0, pack_top = 0, pack_bottom = 0;   // row pairs: count, taps, padding above / below
     int8_t *w_packed = nullptr;
     size_t out_bytes_per_image = 0;
 };
@@ -375,7 +377,7 @@ size_t assign_offsets(const f8_net *net, int batch, std::vector<size_t> *off, si
     *pack_off = top;
     size_t pack = 0;
     for (const NetLayer &l : net->layers)
-        if (l.packed) pack = std::max(pack, round256((size_t)batch * l.g.h * l.pack_wp * 8));
+        if (l.packed) pack = std::max(pack, round256((size_t)batch * l.pack_hp * l.pack_wp * 2 * l.pack_cpad));
     return top + pack;
 }
 
@@ -539,23 +541,38 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
         if (e != cudaSuccess) return cleanup(cuda_fail(e, "parameter upload"));
         hw = host_weights[i];     // the stem packing below reads the caller's layout
 
-        // 3-channel (<= 8) stems with an even stride: widen pixels to 8 bytes so that the kw-tap window of an
-        // output column is one contiguous, 16-byte aligned run of kw8 bytes; the layer then is a kh x 1
-        // convolution over kw8 "channels" of an overlapping strided view, which the tensor-core path takes.
-        if (kind == F8_LAYER_CONV && cp_in == d.c && cp_out == d.c_out && d.c <= 8 && d.stride % 2 == 0 &&
-            d.kw * 8 <= 256) {
+        // 3-channel (<= 8) stems with stride 2.  The image is re-packed into cells of 16 bytes that hold one
+        // pixel of two consecutive rows (8 bytes each), so that the kw-tap window of an output column over a
+        // row PAIR is one contiguous, 16-byte aligned run of kw16 bytes.  The layer then is a kh' x 1
+        // convolution with stride 1 over kw16 "channels" of an overlapping strided view (kh' row pairs cover
+        // the kh rows; taps that fall outside the filter get zero weights), which the tensor-core path takes
+        // with few, long TMA rows.  Kernel row r sits in pair j, half e with r = 2j + e + pad - 2*top.
+        if (kind == F8_LAYER_CONV && cp_in == d.c && cp_out == d.c_out && d.c <= 8 && d.stride == 2 &&
+            d.kw * 16 <= 256) {
             L.packed = true;
             L.pack_left = d.pad;
-            L.pack_kw8 = (d.kw * 8 + 31) / 32 * 32;
-            L.pack_wp = std::max(d.w + d.pad, (L.g.wo - 1) * d.stride + L.pack_kw8 / 8);
-            L.pack_wp = (L.pack_wp + 1) / 2 * 2;              // rows stay 16-byte multiples
-            std::vector<int8_t> wp((size_t)d.c_out * d.kh * L.pack_kw8, 0);
+            L.pack_cpad = d.c <= 4 ? 4 : 8;
+            const int cb = 2 * L.pack_cpad;                       // bytes per cell
+            L.pack_kw8 = (d.kw * cb + 31) / 32 * 32;
+            L.pack_wp = std::max(d.w + d.pad, (L.g.wo - 1) * d.stride + L.pack_kw8 / cb);
+            L.pack_wp = (L.pack_wp + 1) / 2 * 2;                  // rows of cells stay 16-byte multiples
+            L.pack_hp = (d.h + 1) / 2;
+            L.pack_top = (d.pad + 1) / 2;
+            L.pack_kh = (d.kh - 1 - d.pad >= 0 ? (d.kh - 1 - d.pad) / 2 : -((d.pad - d.kh + 2) / 2)) + L.pack_top + 1;
+            L.pack_bottom = L.g.ho - L.pack_hp - L.pack_top + L.pack_kh - 1;
+            std::vector<int8_t> wp((size_t)d.c_out * L.pack_kh * L.pack_kw8, 0);
             for (int co = 0; co < d.c_out; ++co)
-                for (int r = 0; r < d.kh; ++r)
-                    for (int s2 = 0; s2 < d.kw; ++s2)
-                        for (int ch = 0; ch < d.c; ++ch)
-                            wp[((size_t)co * d.kh + r) * L.pack_kw8 + s2 * 8 + ch] =
-                                hw[(((size_t)co * d.kh + r) * d.kw + s2) * d.c + ch];
+                for (int j = 0; j < L.pack_kh; ++j)
+                    for (int e2 = 0; e2 < 2; ++e2) {
+                        const int r = 2 * j + e2 + d.pad - 2 * L.pack_top;
+                        if (r < 0 || r >= d.kh) continue;
+                        for (int s2 = 0; s2 < d.kw; ++s2)
+                            for (int ch = 0; ch < d.c; ++ch)
+                                wp[((size_t)co * L.pack_kh + j) * L.pack_kw8 + s2 * cb + e2 * L.pack_cpad + ch] =
+                                    hw[(((size_t)co * d.kh + r) * d.kw + s2) * d.c + ch];
+                    }
+            if (L.pack_kh < 1 || L.pack_bottom < 0) L.packed = false;      // degenerate geometry: CUDA-core kernel
+            if (!L.packed) continue;
             e = cudaMalloc(&L.w_packed, round256(wp.size()));
             if (e == cudaSuccess) e = cudaMemcpy(L.w_packed, wp.data(), wp.size(), cudaMemcpyHostToDevice);
             if (e != cudaSuccess) return cleanup(cuda_fail(e, "packed stem weights upload"));
@@ -647,15 +664,18 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                 if (L.packed) {
                     F8ConvGeom pg = stp.g;
                     pg.c = L.pack_kw8; pg.kw = 1; pg.stride_w = 1; pg.pad_w = 0;
+                    pg.kh = L.pack_kh; pg.stride_h = 1; pg.pad_h = L.pack_top; pg.pad_h_end = L.pack_bottom;
+                    pg.h = L.pack_hp;
                     void *pbuf = (uint8_t *)workspace + net->pack_off;
-                    const size_t pbytes = (size_t)batch * L.g.h * L.pack_wp * 8;
+                    const uint64_t cb = 2 * (uint64_t)L.pack_cpad;
+                    const size_t pbytes = (size_t)batch * L.pack_hp * L.pack_wp * cb;
                     if (f8_tc_supported(pg, pbytes)) {
                         F8TcTensorView v;
                         v.base = pbuf;
-                        v.dim_c = L.pack_kw8; v.dim_w = L.g.wo; v.dim_h = L.g.h; v.dim_n = batch;
-                        v.stride_w = (uint64_t)L.g.stride_w * 8;
-                        v.stride_h = (uint64_t)L.pack_wp * 8;
-                        v.stride_n = (uint64_t)L.pack_wp * 8 * L.g.h;
+                        v.dim_c = L.pack_kw8; v.dim_w = L.g.wo; v.dim_h = L.pack_hp; v.dim_n = batch;
+                        v.stride_w = (uint64_t)L.g.stride_w * cb;
+                        v.stride_h = (uint64_t)L.pack_wp * cb;
+                        v.stride_n = (uint64_t)L.pack_wp * cb * L.pack_hp;
                         PlanPtr plan = alloc_plan();
                         if (plan && f8_tc_plan_init(plan.get(), pg, L.q, v, L.w_packed, L.b, stp.res, stp.y,
                                                     f8_status_word(), &why) == cudaSuccess) {
@@ -704,7 +724,8 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         cudaError_t e = cudaSuccess;
         switch (stp.kind) {
             case -1:
-                e = f8_launch_pack_stem(batch, L.g.h, L.g.w, L.g.c, L.pack_wp, L.pack_left, stp.x, stp.y, st, net->overlap_layers);
+                e = f8_launch_pack_stem_pairs(batch, L.g.h, L.g.w, L.g.c, L.pack_cpad, L.pack_hp, L.pack_wp, L.pack_left, stp.x, stp.y, st,
+                                              net->overlap_layers);
                 break;
             case F8_LAYER_CONV:
             case F8_LAYER_LINEAR:

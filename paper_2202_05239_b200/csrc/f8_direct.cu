@@ -428,6 +428,44 @@ __global__ void __launch_bounds__(256) pack_stem_kernel(int n, int h, int w, int
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Row-pair stem packing: [n,h,w,c] -> [n,hp,wp] cells of 2*CPAD bytes (CPAD = 4 for c <= 4, else 8); the cell
+// at column iw + left of pair p holds pixel iw of image row 2p (first CPAD bytes) and of row 2p+1 (last CPAD
+// bytes), channels first, zero filled.  One thread per cell.
+// ---------------------------------------------------------------------------------------
+template <int CPAD>
+__global__ void __launch_bounds__(256) pack_stem_pairs_kernel(int n, int h, int w, int c, int hp, int wp, int left,
+                                                              const uint8_t *__restrict__ x, uint32_t *__restrict__ y) {
+    grid_dependency_sync();
+    constexpr int WORDS = CPAD / 4;            // 32-bit words per pixel
+    const size_t total = (size_t)n * hp * wp;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int col = (int)(idx % wp);
+        const size_t np = idx / wp;            // n*hp + pair
+        const int pair = (int)(np % hp);
+        const size_t img = np / hp;
+        const int iw = col - left;
+        uint32_t word[2 * WORDS];
+#pragma unroll
+        for (int i = 0; i < 2 * WORDS; ++i) word[i] = 0;
+        if (iw >= 0 && iw < w) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int ih = 2 * pair + e;
+                if (ih < h) {
+                    const uint8_t *px = x + ((img * h + ih) * w + iw) * c;
+#pragma unroll
+                    for (int j = 0; j < CPAD; ++j)
+                        if (j < c) word[WORDS * e + (j >> 2)] |= (uint32_t)px[j] << (8 * (j & 3));
+                }
+            }
+        }
+        if (WORDS == 1) ((uint2 *)y)[idx] = make_uint2(word[0], word[1]);
+        else ((uint4 *)y)[idx] = make_uint4(word[0], word[1], word[2 * WORDS - 2], word[2 * WORDS - 1]);
+    }
+}
+
 inline int grid_for(size_t total, int block) {
     size_t blocks = (total + block - 1) / block;
     const size_t cap = 148 * 16;   // a few waves of a grid-stride loop on 148 SMs
@@ -512,5 +550,16 @@ cudaError_t f8_launch_pack_stem(int n, int h, int w, int c, int wp, int left, co
     const size_t total = (size_t)n * h * wp;
     if (total == 0) return cudaSuccess;
     launch_k(pack_stem_kernel, grid_for(total, 256), 256, overlap_previous, st, n, h, w, c, wp, left, (const uint8_t *)x, (uint2 *)y);
+    return cudaGetLastError();
+}
+
+cudaError_t f8_launch_pack_stem_pairs(int n, int h, int w, int c, int cpad, int hp, int wp, int left, const void *x,
+                                      void *y, cudaStream_t st, bool overlap_previous) {
+    const size_t total = (size_t)n * hp * wp;
+    if (total == 0) return cudaSuccess;
+    if (cpad == 4)
+        launch_k(pack_stem_pairs_kernel<4>, grid_for(total, 256), 256, overlap_previous, st, n, h, w, c, hp, wp, left, (const uint8_t *)x, (uint32_t *)y);
+    else
+        launch_k(pack_stem_pairs_kernel<8>, grid_for(total, 256), 256, overlap_previous, st, n, h, w, c, hp, wp, left, (const uint8_t *)x, (uint32_t *)y);
     return cudaGetLastError();
 }

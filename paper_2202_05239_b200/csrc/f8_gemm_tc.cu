@@ -967,6 +967,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     const int uses = (k_iters + 7) / 8;                  // at most eight k-iterations per stage, evenly split
     int group = (k_iters + uses - 1) / uses;
     while (group > 1 && avail / ((size_t)group * p.sub_bytes) < 3) --group;
+    group = (k_iters + (k_iters + group - 1) / group - 1) / ((k_iters + group - 1) / group);   // same uses, evenly split
     p.group = group;
     p.stage_bytes = (uint32_t)group * p.sub_bytes;
     int stages = (int)(avail / p.stage_bytes);
@@ -1006,7 +1007,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         cuuint64_t dims[4] = {xv.dim_c, xv.dim_w, xv.dim_h, xv.dim_n};
         cuuint64_t strides[3] = {xv.stride_w, xv.stride_h, xv.stride_n};
         int lower[2] = {-g.pad_w, -g.pad_h};
-        int upper[2] = {g.pad_w - (g.kw - 1), g.pad_h - (g.kh - 1)};
+        int upper[2] = {g.pad_w - (g.kw - 1), (g.pad_h_end >= 0 ? g.pad_h_end : g.pad_h) - (g.kh - 1)};
         cuuint32_t estr[4] = {1, (cuuint32_t)g.stride_w, (cuuint32_t)g.stride_h, 1};
         CUresult r = g_encode_im2col(&plan->map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(xv.base), dims,
                                      strides, lower, upper, (cuuint32_t)p.kb, (cuuint32_t)TILE_M, estr,

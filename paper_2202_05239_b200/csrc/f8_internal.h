@@ -29,6 +29,7 @@ struct F8ConvGeom {
     int stride_h, stride_w;
     int pad_h, pad_w;
     int x_signed;
+    int pad_h_end = -1;     // padding below the last row when it differs from pad_h (-1: symmetric)
 };
 
 // ---- CUDA-core kernels (f8_direct.cu) -------------------------------------------------
@@ -47,6 +48,11 @@ cudaError_t f8_launch_gap(int n, int h, int w, int c, int x_signed, int s, const
 // channel-padding pre-pass for 3-channel stems: [n,h,w,c] -> [n,h,wp,8] with `left` zero pixels in front
 cudaError_t f8_launch_pack_stem(int n, int h, int w, int c, int wp, int left, const void *x, void *y,
                                 cudaStream_t st, bool overlap_previous = false);
+
+// row-pair packing for stride-2 stems: [n,h,w,c<=8] -> [n,hp,wp] cells of 2*cpad bytes (cpad 4 or 8 >= c); the cell
+// at column iw + left of row pair p holds pixel iw of image rows 2p and 2p+1 (cpad bytes each, zero filled)
+cudaError_t f8_launch_pack_stem_pairs(int n, int h, int w, int c, int cpad, int hp, int wp, int left, const void *x,
+                                      void *y, cudaStream_t st, bool overlap_previous = false);
 
 // ---- tensor-core implicit GEMM (f8_gemm_tc.cu) ----------------------------------------
 struct F8TcPlan;   // opaque: tensor maps + launch parameters of one conv launch
