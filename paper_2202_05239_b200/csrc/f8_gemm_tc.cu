@@ -496,10 +496,14 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 tma_load_3d(smem_base + p.bres_off + (uint32_t)i * p.b_bytes, &map_b, bres_bar, (int)e.x, (int)(e.y >> 16),
                             n_t * p.bn);
             }
-            // the loads must have landed before this CTA's shared memory may go away
-            mbar_wait(bres_bar, 0, abortp, p.status, 107);
-        } else {
-        if (opnd == 0) grid_dependency_wait();      // activations come from the previous grid; weights do not
+        }
+        {
+        // With resident weights the weight warp has nothing left to request: it takes the odd sub-chunks of
+        // the activation loads off the activation warp (issuing a TMA instruction holds a warp for a few
+        // hundred cycles per participating lane, which otherwise bounds layers with short tiles).
+        const bool a_helper = opnd == 1 && p.b_res;
+        const int j_mask = p.b_res ? 1 : 0, j_want = a_helper ? 1 : 0;     // which sub-chunks this warp requests
+        if (opnd == 0 || a_helper) grid_dependency_wait();      // activations come from the previous grid; weights do not
         int stage = 0;
         uint32_t phase = 0;
         bool have_last = false;
@@ -526,10 +530,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 // one arrival per stage use; it announces the bytes of every load of the group
                 if (opnd == 0 && lane == 0) mbar_expect_tx(fb, (uint32_t)subs * p.tx_sub);
                 const int j = (lane - stage * p.group) & 31;
-                if (j < subs) {
+                if (j < subs && (j & j_mask) == j_want) {
                     const uint2 e = ktab[kc + j];       // x: first channel of the chunk, y: tap << 16 | r << 8 | s
                     const uint32_t dst = smem_base + stage * p.stage_bytes + j * p.sub_bytes;
-                    if (opnd == 0)
+                    if (opnd == 0 || a_helper)
                         tma_load_im2col(dst, &map_a, fb, (int)e.x, base_w, base_h, img, (uint16_t)(e.y & 0xff),
                                         (uint16_t)((e.y >> 8) & 0xff));
                     else
@@ -549,6 +553,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                    (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
             }
         }
+        // the resident weights must have landed before this CTA's shared memory may go away (they have, unless
+        // the kernel is aborting: the MMA issuers wait for them before their first instruction)
+        if (a_helper) mbar_wait(bres_bar, 0, abortp, p.status, 107);
         }
     } else if (warp == MMA_WARP || warp == MMA2_WARP) {
         // ------------------------------------------------------------------ MMA issuers
