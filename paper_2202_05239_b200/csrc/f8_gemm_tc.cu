@@ -960,7 +960,8 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     }
     staging += ktab_bytes;
     // k-iterations per stage: every stage use costs the MMA thread a wait, a fence and a commit (a few hundred
-    // cycles), so short K chunks are grouped -- as long as at least three stages and one lane per load remain
+    // cycles of a lone thread, as much as several MMAs), so K chunks are grouped -- as long as two stages and one
+    // lane per load remain; measured, fewer and larger stage uses beat a deeper ring of small ones
     const int k_iters = g.kh * g.kw * p.c_chunks;
     size_t avail = SMEM_LIMIT - 1024 - staging;
     // resident weights: one N tile, and at least 64 KiB left for the activation pipeline
@@ -973,7 +974,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.tx_sub = p.tx_a + (p.b_res ? 0u : p.tx_b);
     const int uses = (k_iters + 7) / 8;                  // at most eight k-iterations per stage, evenly split
     int group = (k_iters + uses - 1) / uses;
-    while (group > 1 && avail / ((size_t)group * p.sub_bytes) < 3) --group;
+    while (group > 1 && avail / ((size_t)group * p.sub_bytes) < 2) --group;
     group = (k_iters + (k_iters + group - 1) / group - 1) / ((k_iters + group - 1) / group);   // same uses, evenly split
     p.group = group;
     p.stage_bytes = (uint32_t)group * p.sub_bytes;
