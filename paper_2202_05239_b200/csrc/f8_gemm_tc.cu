@@ -53,6 +53,7 @@ constexpr int NUM_THREADS = 32 * (MMA2_WARP + 1);
 constexpr int MAX_STAGES = 16;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
+constexpr unsigned MIN_POLLS_BEFORE_TIMEOUT = 1u << 16;             // failed polls a wait needs before it may give up
 constexpr unsigned long long DRAIN_LIMIT_CYCLES = 200000000ull;
 constexpr size_t SMEM_LIMIT = 220 * 1024;     // dynamic shared memory budget (227 KiB per CTA minus static data)
 
@@ -151,7 +152,9 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
-            if ((unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
+            // both conditions: the cycle counter keeps running while the context is switched out (a profiler
+            // replaying the kernel does that for seconds), the poll count does not
+            if (spins >= MIN_POLLS_BEFORE_TIMEOUT && (unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
                 *abort_flag = 1;
                 atomicCAS(status, 0, code);
                 return false;
@@ -521,6 +524,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int base_h = oh * p.stride_h - p.pad_h;
             const int n_base = n_t * p.bn;
             for (int kc = 0; kc < k_iters; kc += p.group) {
+                if (a_helper && k_iters - kc < 2) {
+                    // A stage use without an odd sub-chunk: nothing to request, and nothing to wait for either.  A
+                    // warp that only polled here would not hold the pipeline back, could fall two phases behind
+                    // it, and a parity wait cannot tell a phase from the one two later.
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                    continue;
+                }
                 if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101))) {
                     ok = false;
                     break;
