@@ -291,3 +291,58 @@ class Net:
             self.close()
         except Exception:
             pass
+
+
+class HostPipeline:
+    """Forward passes from pinned host buffers with the copies overlapped: while the GPU runs batch i, the copy
+    engine uploads batch i+1 and downloads the logits of batch i-1.  Every slot has its own net (plans are cached per
+    set of buffer addresses), device input / output buffers and workspace; all arithmetic still runs in
+    f8_net_forward.  submit() returns at once; result `i` is in its host buffer after wait() (or once the event
+    submit() returns has completed)."""
+
+    def __init__(self, layers: Sequence["synth.Layer"], batch: int, depth: int = 2, device="cuda"):
+        self.batch = batch
+        self.depth = depth
+        self.nets = [Net(layers, batch) for _ in range(depth)]
+        first = layers[0]
+        in_dtype = torch_dtype(first.x_dtype)
+        self.x_dev = [torch.empty((batch, first.h, first.w, first.c), dtype=in_dtype, device=device) for _ in range(depth)]
+        self.y_dev = [torch.empty((batch,) + n.out_shape, dtype=n.out_dtype, device=device) for n in self.nets]
+        self.ws = [torch.empty(n.workspace_bytes(batch), dtype=torch.uint8, device=device) for n in self.nets]
+        self.up_stream = torch.cuda.Stream(device=device)        # host -> device copies
+        self.down_stream = torch.cuda.Stream(device=device)      # device -> host copies (the link is full duplex)
+        self.compute_stream = torch.cuda.Stream(device=device)
+        self.ev_in = [torch.cuda.Event() for _ in range(depth)]        # upload of the slot's input finished
+        self.ev_done = [torch.cuda.Event() for _ in range(depth)]      # forward pass of the slot finished
+        self.ev_out = [torch.cuda.Event() for _ in range(depth)]       # download of the slot's result finished
+        self.count = 0
+
+    def submit(self, x_host: torch.Tensor, y_host: torch.Tensor) -> "torch.cuda.Event":
+        b = self.count % self.depth
+        self.count += 1
+        with torch.cuda.stream(self.up_stream):
+            self.up_stream.wait_event(self.ev_done[b])        # the slot's previous forward pass has read its input
+            self.x_dev[b].copy_(x_host, non_blocking=True)
+            self.ev_in[b].record(self.up_stream)
+        self.compute_stream.wait_event(self.ev_in[b])
+        self.compute_stream.wait_event(self.ev_out[b])       # the slot's previous result has left its output buffer
+        self.nets[b].forward(self.x_dev[b], out=self.y_dev[b], workspace=self.ws[b], stream=self.compute_stream)
+        self.ev_done[b].record(self.compute_stream)
+        with torch.cuda.stream(self.down_stream):
+            self.down_stream.wait_event(self.ev_done[b])
+            y_host.copy_(self.y_dev[b], non_blocking=True)
+            self.ev_out[b].record(self.down_stream)
+        return self.ev_out[b]
+
+    def wait(self):
+        self.up_stream.synchronize()
+        self.compute_stream.synchronize()
+        self.down_stream.synchronize()
+
+    @property
+    def launches_per_step(self) -> int:
+        return self.nets[0].last_launch_count
+
+    def close(self):
+        for n in self.nets:
+            n.close()

@@ -348,6 +348,78 @@ __global__ void __launch_bounds__(256) maxpool_kernel(int n, int h, int w, int c
     }
 }
 
+// 3x3 / stride 2 / pad 1 max-pool, c % 16 == 0: a thread owns 16 channels of a block of 2 x 4 outputs.  It walks the
+// five input rows of the block once; per row it loads the nine columns once, takes the horizontal maxima of the four
+// windows and folds them into the one or two output rows the input row belongs to (5.6 loads per output instead
+// of 9).  Out-of-range taps contribute the identity of max (padding never wins).
+template <bool SIGNED>
+__global__ void __launch_bounds__(128) maxpool3x3s2_kernel(int n, int h, int w, int c, int ho, int wo,
+                                                           const uint8_t *__restrict__ x, uint8_t *__restrict__ y) {
+    grid_dependency_sync();
+    constexpr int TH = 2, TW = 4;
+    const int cg = c / 16;
+    const int wb = (wo + TW - 1) / TW, hb = (ho + TH - 1) / TH;
+    const size_t total = (size_t)n * hb * wb * cg;
+    const uint32_t ident = SIGNED ? 0x80808080u : 0u;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int g = (int)(idx % cg);
+        size_t t = idx / cg;
+        const int bw = (int)(t % wb);
+        t /= wb;
+        const int bh = (int)(t % hb);
+        const int img = (int)(t / hb);
+        const int oh0 = bh * TH, ow0 = bw * TW;
+        uint4 acc[TH][TW];
+#pragma unroll
+        for (int a = 0; a < TH; ++a)
+#pragma unroll
+            for (int b = 0; b < TW; ++b) acc[a][b] = make_uint4(ident, ident, ident, ident);
+#pragma unroll
+        for (int r = 0; r < 2 * TH + 1; ++r) {
+            const int ih = 2 * oh0 - 1 + r;
+            if (ih < 0 || ih >= h) continue;
+            const uint8_t *row = x + (((size_t)img * h + ih) * w) * c + g * 16;
+            uint4 v[2 * TW + 1];
+#pragma unroll
+            for (int j = 0; j < 2 * TW + 1; ++j) {
+                const int iw = 2 * ow0 - 1 + j;
+                v[j] = (iw >= 0 && iw < w) ? *(const uint4 *)(row + (size_t)iw * c) : make_uint4(ident, ident, ident, ident);
+            }
+#pragma unroll
+            for (int b = 0; b < TW; ++b) {
+                uint4 m;
+                if (SIGNED) {
+                    m.x = __vmaxs4(__vmaxs4(v[2 * b].x, v[2 * b + 1].x), v[2 * b + 2].x);
+                    m.y = __vmaxs4(__vmaxs4(v[2 * b].y, v[2 * b + 1].y), v[2 * b + 2].y);
+                    m.z = __vmaxs4(__vmaxs4(v[2 * b].z, v[2 * b + 1].z), v[2 * b + 2].z);
+                    m.w = __vmaxs4(__vmaxs4(v[2 * b].w, v[2 * b + 1].w), v[2 * b + 2].w);
+                } else {
+                    m.x = __vmaxu4(__vmaxu4(v[2 * b].x, v[2 * b + 1].x), v[2 * b + 2].x);
+                    m.y = __vmaxu4(__vmaxu4(v[2 * b].y, v[2 * b + 1].y), v[2 * b + 2].y);
+                    m.z = __vmaxu4(__vmaxu4(v[2 * b].z, v[2 * b + 1].z), v[2 * b + 2].z);
+                    m.w = __vmaxu4(__vmaxu4(v[2 * b].w, v[2 * b + 1].w), v[2 * b + 2].w);
+                }
+                // input row r of the block feeds output row a when r is one of 2a, 2a+1, 2a+2
+#pragma unroll
+                for (int a = 0; a < TH; ++a)
+                    if (r >= 2 * a && r <= 2 * a + 2) {
+                        acc[a][b].x = SIGNED ? __vmaxs4(acc[a][b].x, m.x) : __vmaxu4(acc[a][b].x, m.x);
+                        acc[a][b].y = SIGNED ? __vmaxs4(acc[a][b].y, m.y) : __vmaxu4(acc[a][b].y, m.y);
+                        acc[a][b].z = SIGNED ? __vmaxs4(acc[a][b].z, m.z) : __vmaxu4(acc[a][b].z, m.z);
+                        acc[a][b].w = SIGNED ? __vmaxs4(acc[a][b].w, m.w) : __vmaxu4(acc[a][b].w, m.w);
+                    }
+            }
+        }
+#pragma unroll
+        for (int a = 0; a < TH; ++a)
+#pragma unroll
+            for (int b = 0; b < TW; ++b)
+                if (oh0 + a < ho && ow0 + b < wo)
+                    *(uint4 *)(y + ((((size_t)img * ho + oh0 + a) * wo + ow0 + b) * c) + g * 16) = acc[a][b];
+    }
+}
+
 __global__ void __launch_bounds__(256) maxpool_scalar_kernel(int n, int h, int w, int c, int ho, int wo, int k,
                                                              int stride, int pad, int x_signed,
                                                              const uint8_t *__restrict__ x, uint8_t *__restrict__ y) {
@@ -525,7 +597,13 @@ cudaError_t f8_launch_maxpool(int n, int h, int w, int c, int k, int stride, int
     const int ho = (h + 2 * pad - k) / stride + 1, wo = (w + 2 * pad - k) / stride + 1;
     const size_t total = (size_t)n * ho * wo * c;
     if (total == 0) return cudaSuccess;
-    if (c % 16 == 0)
+    const size_t blocks8 = (size_t)n * ((ho + 1) / 2) * ((wo + 3) / 4) * (c / 16);
+    if (c % 16 == 0 && k == 3 && stride == 2 && pad == 1 && ((uintptr_t)x | (uintptr_t)y) % 16 == 0) {
+        if (x_signed)
+            launch_k(maxpool3x3s2_kernel<true>, grid_for(blocks8, 128), 128, overlap_previous, st, n, h, w, c, ho, wo, (const uint8_t *)x, (uint8_t *)y);
+        else
+            launch_k(maxpool3x3s2_kernel<false>, grid_for(blocks8, 128), 128, overlap_previous, st, n, h, w, c, ho, wo, (const uint8_t *)x, (uint8_t *)y);
+    } else if (c % 16 == 0)
         launch_k(maxpool_kernel<4>, grid_for(total / 16, 256), 256, overlap_previous, st, n, h, w, c, ho, wo, k, stride, pad, x_signed,
                                                                      (const uint8_t *)x, (uint8_t *)y);
     else if (c % 4 == 0)

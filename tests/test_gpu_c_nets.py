@@ -82,3 +82,22 @@ def test_workspace_too_small_is_rejected():
         net.forward(x, workspace=ws)
     assert e.value.status == 8
     net.close()
+
+
+def test_host_pipeline_matches_oracle(ref):
+    """Pipelined host-to-host forward passes (copies overlapped with compute, two slots): five different batches in
+    flight one after the other, every result equal to the oracle's logits."""
+    a = api()
+    batch, image = 3, 96
+    layers = synth.make_net("resnet18", 0, image=image)
+    pipe = a.HostPipeline(layers, batch, depth=2)
+    xs = [torch.from_numpy(synth.draw_image(batch, 10 + i, image, image)).pin_memory() for i in range(5)]
+    ys = [torch.empty((batch, 1000), dtype=torch.int32).pin_memory() for _ in range(5)]
+    for x, y in zip(xs, ys):
+        pipe.submit(x, y)
+    pipe.wait()
+    a.f8_device_status()
+    for i, (x, y) in enumerate(zip(xs, ys)):
+        want = ref.net_forward(layers, x.numpy(), keep_all=False)[-1]
+        assert np.array_equal(y.numpy(), want), f"batch {i}"
+    pipe.close()
