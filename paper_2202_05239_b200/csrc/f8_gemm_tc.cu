@@ -51,6 +51,7 @@ constexpr int B_PROD_WARP = FIRST_EPI_WARP + NUM_EPI_WARPS;   // requests weight
 constexpr int MMA2_WARP = B_PROD_WARP + 1;
 constexpr int NUM_THREADS = 32 * (MMA2_WARP + 1);
 constexpr int MAX_STAGES = 16;
+constexpr int MAX_RES_BUFS = 4;             // residual tiles in flight ahead of the epilogue (HBM latency is ~a tile time)
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
 constexpr unsigned MIN_POLLS_BEFORE_TIMEOUT = 1u << 16;             // failed polls a wait needs before it may give up
@@ -103,6 +104,7 @@ struct TcParams {
     int n_slabs;              // bn / slab_w
     uint32_t swz_mask;        // 7, 3, 1 or 0: address bits 7.. XORed into the 16-byte chunk index
     uint32_t out_bytes;       // TILE_M * bn
+    int res_bufs;             // residual tiles in flight (2..MAX_RES_BUFS)
     uint32_t out_off, res_off, bias_off;   // byte offsets behind the stages: two output tiles, two residual
                                            // tiles, int32 bias' of all padded columns
     uint32_t ktab_off;        // table of k-iteration coordinates (8 bytes each)
@@ -414,7 +416,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 5];
-    __shared__ __align__(8) uint64_t epi_bars[8];   // out_full[2], out_free[2], res_full[2], res_free[2]
+    __shared__ __align__(8) uint64_t epi_bars[4 + 2 * MAX_RES_BUFS];   // out_full[2], out_free[2], res_full[], res_free[]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -427,7 +429,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const uint32_t bres_bar = smem_u32(&bars[2 * MAX_STAGES + 4]);   // resident weights have landed
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t out_full = smem_u32(&epi_bars[0]), out_free = smem_u32(&epi_bars[2]);
-    const uint32_t res_full = smem_u32(&epi_bars[4]), res_free = smem_u32(&epi_bars[6]);
+    const uint32_t res_full = smem_u32(&epi_bars[4]), res_free = smem_u32(&epi_bars[4 + MAX_RES_BUFS]);
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -441,8 +443,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             mbar_init(tempty_bar + 8 * a, NUM_EPI_WARPS);
             mbar_init(smem_u32(&epi_bars[0 + a]), NUM_EPI_WARPS);   // out_full: every epilogue warp has written its part
             mbar_init(smem_u32(&epi_bars[2 + a]), 1);               // out_free: the store has finished reading the tile
-            mbar_init(smem_u32(&epi_bars[4 + a]), 1);               // res_full: residual tile has landed (transaction count)
-            mbar_init(smem_u32(&epi_bars[6 + a]), NUM_EPI_WARPS);   // res_free: every epilogue warp has read its part
+        }
+        for (int a = 0; a < MAX_RES_BUFS; ++a) {
+            mbar_init(res_full + 8 * a, 1);               // residual tile has landed (transaction count)
+            mbar_init(res_free + 8 * a, NUM_EPI_WARPS);   // every epilogue warp has read its part
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -662,26 +666,27 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // ------------------------------------------------------------------ residual fetcher
         if (RES && lane == 0) {
             grid_dependency_wait();
-            // residual tiles: up to two tiles ahead of the epilogue
+            // residual tiles: up to res_bufs tiles ahead of the epilogue
             int local = 0;
-            int last = -1;
+            int rb = 0;                 // buffer of this tile, and the parity of its current use
+            uint32_t rphase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
-                const int b = local & 1;
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
-                if (!mbar_wait(res_free + 8 * b, ((local >> 1) & 1) ^ 1, abortp, p.status, 106)) { ok = false; break; }
-                const uint32_t rb = res_full + 8 * b;
-                mbar_expect_tx(rb, p.out_bytes);
+                if (!mbar_wait(res_free + 8 * rb, rphase ^ 1, abortp, p.status, 106)) { ok = false; break; }
+                const uint32_t fb = res_full + 8 * rb;
+                mbar_expect_tx(fb, p.out_bytes);
                 for (int sl = 0; sl < p.n_slabs; ++sl)
-                    tma_load_2d(smem_base + p.res_off + b * p.out_bytes + sl * (TILE_M * p.slab_w), &map_r, rb,
+                    tma_load_2d(smem_base + p.res_off + rb * p.out_bytes + sl * (TILE_M * p.slab_w), &map_r, fb,
                                 n_t * p.bn + sl * p.slab_w, m_t * TILE_M);
-                last = local;
+                if (++rb == p.res_bufs) { rb = 0; rphase ^= 1; }
             }
-            if (!ok && last >= 0) {
-                // aborting: give the loads that are still in flight time to land
-                for (int i = 0; i < 2 && last - i >= 0; ++i) {
+            if (!ok && local > 0) {
+                // aborting: give the loads that are still in flight time to land (walk back over the buffers)
+                for (int i = 0; i < p.res_bufs && local - 1 - i >= 0; ++i) {
+                    const int l = local - 1 - i;
                     const unsigned long long t0 = clock64();
-                    while (!mbar_try_wait(res_full + 8 * ((last - i) & 1), ((last - i) >> 1) & 1) &&
+                    while (!mbar_try_wait(res_full + 8 * (l % p.res_bufs), (uint32_t)(l / p.res_bufs) & 1u) &&
                            (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
                     }
                 }
@@ -698,6 +703,8 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const int nch = min(ch_begin + per_group, chunks) - ch_begin;
         const int mul_acc = p.mul_acc, mul_res = p.mul_res;     // 2^sh_acc, 2^sh_res
         int local = 0;
+        int rb = 0;                 // residual buffer of the current tile and the parity of its use
+        uint32_t rphase = 0;
         bool ok = true;
         if (STAGED) {
             const int tile_row = quarter * 32 + lane;
@@ -722,12 +729,12 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
                 bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104);
-                if (RES) got = mbar_wait(res_full + 8 * acc, acc_phase, abortp, p.status, 107) && got;
+                if (RES) got = mbar_wait(res_full + 8 * rb, rphase, abortp, p.status, 107) && got;
                 got = mbar_wait(out_free + 8 * acc, acc_phase ^ 1, abortp, p.status, 109) && got;
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t out_buf = smem_base + p.out_off + acc * p.out_bytes;
-                const uint32_t res_buf = smem_base + p.res_off + acc * p.out_bytes;
+                const uint32_t res_buf = smem_base + p.res_off + rb * p.out_bytes;
                 const uint32_t bias_s = smem_base + p.bias_off + 4 * c_first;
                 int va[16], vb[16];
                 if (my_nch > 0) tmem_ld16(t_addr, va);
@@ -756,8 +763,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 if (lane == 0) {
                     mbar_arrive(tempty_bar + 8 * acc);
                     mbar_arrive(out_full + 8 * acc);
-                    if (RES) mbar_arrive(res_free + 8 * acc);
+                    if (RES) mbar_arrive(res_free + 8 * rb);
                 }
+                if (RES && ++rb == p.res_bufs) { rb = 0; rphase ^= 1; }
             }
         } else {
             grid_dependency_wait();     // direct stores (and residual reads) from these warps
@@ -961,7 +969,14 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         p.swz_mask = p.slab_w == 128 ? 7u : (p.slab_w == 64 ? 3u : (p.slab_w == 32 ? 1u : 0u));
         p.out_bytes = (uint32_t)(TILE_M * p.bn + 1023) / 1024 * 1024;
         const size_t bias_bytes = ((size_t)p.n_tiles * p.bn * 4 + 1023) / 1024 * 1024;
-        staging = (size_t)p.out_bytes * (q.has_res ? 4 : 2) + bias_bytes;
+        // a residual tile takes about as long to arrive from HBM as a tile takes to compute: keep three in flight
+        // where that does not cost pipeline depth, i.e. when the weights are resident anyway (one N tile) and 32 KiB
+        // remain for activation stages; measured, layers that lose stages to the third buffer get slower
+        p.res_bufs = 2;
+        const size_t weights = (size_t)g.kh * g.kw * p.c_chunks * b_bytes;
+        if (q.has_res && p.n_tiles == 1 && (size_t)p.out_bytes * 5 + bias_bytes + weights + 34 * 1024 <= SMEM_LIMIT - 1024)
+            p.res_bufs = 3;
+        staging = (size_t)p.out_bytes * (2 + (q.has_res ? p.res_bufs : 0)) + bias_bytes;
     }
     const size_t ktab_bytes = ((size_t)g.kh * g.kw * p.c_chunks * 8 + 1023) / 1024 * 1024;
     if (ktab_bytes > 16 * 1024 || g.kh * g.kw > 0xffff) {
@@ -974,9 +989,9 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // lane per load remain; measured, fewer and larger stage uses beat a deeper ring of small ones
     const int k_iters = g.kh * g.kw * p.c_chunks;
     size_t avail = SMEM_LIMIT - 1024 - staging;
-    // resident weights: one N tile, and at least 64 KiB left for the activation pipeline
+    // resident weights: one N tile, and at least 32 KiB left for the activation pipeline
     const size_t b_all = (size_t)p.n_tiles * k_iters * b_bytes;
-    p.b_res = (p.n_tiles == 1 && b_all + 64 * 1024 <= avail && !getenv("F8_NO_BRES")) ? 1 : 0;
+    p.b_res = (p.n_tiles == 1 && b_all + 32 * 1024 <= avail && !getenv("F8_NO_BRES")) ? 1 : 0;
     if (p.b_res) {
         avail -= b_all;
         p.sub_bytes = p.a_bytes;
@@ -1000,7 +1015,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !getenv("F8_NO_DUAL")) ? 1 : 0;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
     p.res_off = p.out_off + 2 * p.out_bytes;
-    p.bias_off = p.res_off + (q.has_res ? 2 * p.out_bytes : 0u);
+    p.bias_off = p.res_off + (q.has_res ? (uint32_t)p.res_bufs * p.out_bytes : 0u);
     p.ktab_off = (uint32_t)(p.stages * p.stage_bytes + staging - ktab_bytes);
     p.bres_off = (uint32_t)(p.stages * p.stage_bytes + staging);
     // instruction descriptor: D = s32 (2 at bit 4), A format at bit 7 (0 = u8, 1 = s8), B = s8 at bit 10,
