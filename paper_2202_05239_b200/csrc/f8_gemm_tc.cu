@@ -51,7 +51,8 @@ constexpr int B_PROD_WARP = FIRST_EPI_WARP + NUM_EPI_WARPS;   // requests weight
 constexpr int MMA2_WARP = B_PROD_WARP + 1;
 constexpr int NUM_THREADS = 32 * (MMA2_WARP + 1);
 constexpr int MAX_STAGES = 16;
-constexpr int MAX_RES_BUFS = 4;             // residual tiles in flight ahead of the epilogue (HBM latency is ~a tile time)
+constexpr int MAX_OUT_BUFS = 4;             // ring of staged output tiles; with a residual, the residual tile lands in the
+                                            // buffer first and the epilogue converts it in place
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
 constexpr unsigned MIN_POLLS_BEFORE_TIMEOUT = 1u << 16;             // failed polls a wait needs before it may give up
@@ -104,8 +105,8 @@ struct TcParams {
     int n_slabs;              // bn / slab_w
     uint32_t swz_mask;        // 7, 3, 1 or 0: address bits 7.. XORed into the 16-byte chunk index
     uint32_t out_bytes;       // TILE_M * bn
-    int res_bufs;             // residual tiles in flight (2..MAX_RES_BUFS)
-    uint32_t out_off, res_off, bias_off;   // byte offsets behind the stages: two output tiles, two residual
+    int out_bufs;             // staged output tiles in the ring (2..MAX_OUT_BUFS)
+    uint32_t out_off, bias_off;   // byte offsets behind the stages: two output tiles, two residual
                                            // tiles, int32 bias' of all padded columns
     uint32_t ktab_off;        // table of k-iteration coordinates (8 bytes each)
     F8Requant q;
@@ -416,7 +417,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 5];
-    __shared__ __align__(8) uint64_t epi_bars[4 + 2 * MAX_RES_BUFS];   // out_full[2], out_free[2], res_full[], res_free[]
+    __shared__ __align__(8) uint64_t epi_bars[3 * MAX_OUT_BUFS];   // out_full[], out_free[], res_full[]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -428,8 +429,8 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + 2]);
     const uint32_t bres_bar = smem_u32(&bars[2 * MAX_STAGES + 4]);   // resident weights have landed
     const uint32_t smem_base = smem_u32(smem);
-    const uint32_t out_full = smem_u32(&epi_bars[0]), out_free = smem_u32(&epi_bars[2]);
-    const uint32_t res_full = smem_u32(&epi_bars[4]), res_free = smem_u32(&epi_bars[4 + MAX_RES_BUFS]);
+    const uint32_t out_full = smem_u32(&epi_bars[0]), out_free = smem_u32(&epi_bars[MAX_OUT_BUFS]);
+    const uint32_t res_full = smem_u32(&epi_bars[2 * MAX_OUT_BUFS]);
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -441,12 +442,11 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
             mbar_init(tempty_bar + 8 * a, NUM_EPI_WARPS);
-            mbar_init(smem_u32(&epi_bars[0 + a]), NUM_EPI_WARPS);   // out_full: every epilogue warp has written its part
-            mbar_init(smem_u32(&epi_bars[2 + a]), 1);               // out_free: the store has finished reading the tile
         }
-        for (int a = 0; a < MAX_RES_BUFS; ++a) {
-            mbar_init(res_full + 8 * a, 1);               // residual tile has landed (transaction count)
-            mbar_init(res_free + 8 * a, NUM_EPI_WARPS);   // every epilogue warp has read its part
+        for (int a = 0; a < MAX_OUT_BUFS; ++a) {
+            mbar_init(out_full + 8 * a, NUM_EPI_WARPS);   // every epilogue warp has written its part of the tile
+            mbar_init(out_free + 8 * a, 1);               // the store has finished reading the tile
+            mbar_init(res_full + 8 * a, 1);               // the residual tile has landed in the buffer (transaction count)
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -645,20 +645,21 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // ------------------------------------------------------------------ output mover
         if (STAGED && lane == 0) {
             grid_dependency_wait();     // the output may overwrite a tensor the previous grid still reads
-            // stores: tile t leaves from output buffer t & 1 once all epilogue warps have written it
-            int local = 0;
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
-                const int b = local & 1;
+            // stores: a tile leaves from its buffer of the ring once all epilogue warps have written it
+            int b = 0;
+            uint32_t bphase = 0;
+            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
-                if (!mbar_wait(out_full + 8 * b, (local >> 1) & 1, abortp, p.status, 108)) break;
+                if (!mbar_wait(out_full + 8 * b, bphase, abortp, p.status, 108)) break;
                 const uint32_t src = smem_base + p.out_off + b * p.out_bytes;
                 for (int sl = 0; sl < p.n_slabs; ++sl)
                     if (n_t * p.bn + sl * p.slab_w < p.c_out)
                         tma_store_2d(&map_y, src + sl * (TILE_M * p.slab_w), n_t * p.bn + sl * p.slab_w, m_t * TILE_M);
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                // the buffer is free again as soon as the store has read it (the next tile uses the other one)
+                // the buffer is free again as soon as the store has read it (the next tiles use the others)
                 asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 mbar_arrive(out_free + 8 * b);
+                if (++b == p.out_bufs) { b = 0; bphase ^= 1; }
             }
             asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         }
@@ -666,27 +667,28 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // ------------------------------------------------------------------ residual fetcher
         if (RES && lane == 0) {
             grid_dependency_wait();
-            // residual tiles: up to res_bufs tiles ahead of the epilogue
+            // residual tiles go straight into the output ring (the epilogue converts them in place): a buffer is
+            // loaded as soon as the store of the tile that used it before has read it, up to out_bufs - 1 tiles ahead
             int local = 0;
-            int rb = 0;                 // buffer of this tile, and the parity of its current use
+            int rb = 0;
             uint32_t rphase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
-                if (!mbar_wait(res_free + 8 * rb, rphase ^ 1, abortp, p.status, 106)) { ok = false; break; }
+                if (!mbar_wait(out_free + 8 * rb, rphase ^ 1, abortp, p.status, 106)) { ok = false; break; }
                 const uint32_t fb = res_full + 8 * rb;
                 mbar_expect_tx(fb, p.out_bytes);
                 for (int sl = 0; sl < p.n_slabs; ++sl)
-                    tma_load_2d(smem_base + p.res_off + rb * p.out_bytes + sl * (TILE_M * p.slab_w), &map_r, fb,
+                    tma_load_2d(smem_base + p.out_off + rb * p.out_bytes + sl * (TILE_M * p.slab_w), &map_r, fb,
                                 n_t * p.bn + sl * p.slab_w, m_t * TILE_M);
-                if (++rb == p.res_bufs) { rb = 0; rphase ^= 1; }
+                if (++rb == p.out_bufs) { rb = 0; rphase ^= 1; }
             }
             if (!ok && local > 0) {
-                // aborting: give the loads that are still in flight time to land (walk back over the buffers)
-                for (int i = 0; i < p.res_bufs && local - 1 - i >= 0; ++i) {
+                // aborting: give the loads that are still in flight time to land (walk back over the ring)
+                for (int i = 0; i < p.out_bufs && local - 1 - i >= 0; ++i) {
                     const int l = local - 1 - i;
                     const unsigned long long t0 = clock64();
-                    while (!mbar_try_wait(res_full + 8 * (l % p.res_bufs), (uint32_t)(l / p.res_bufs) & 1u) &&
+                    while (!mbar_try_wait(res_full + 8 * (l % p.out_bufs), (uint32_t)(l / p.out_bufs) & 1u) &&
                            (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
                     }
                 }
@@ -703,8 +705,8 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const int nch = min(ch_begin + per_group, chunks) - ch_begin;
         const int mul_acc = p.mul_acc, mul_res = p.mul_res;     // 2^sh_acc, 2^sh_res
         int local = 0;
-        int rb = 0;                 // residual buffer of the current tile and the parity of its use
-        uint32_t rphase = 0;
+        int ob = 0;                 // buffer of the output ring for the current tile and the parity of its use
+        uint32_t ophase = 0;
         bool ok = true;
         if (STAGED) {
             const int tile_row = quarter * 32 + lane;
@@ -729,12 +731,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
                 bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104);
-                if (RES) got = mbar_wait(res_full + 8 * rb, rphase, abortp, p.status, 107) && got;
-                got = mbar_wait(out_free + 8 * acc, acc_phase ^ 1, abortp, p.status, 109) && got;
+                // the buffer holds the residual tile (which implies that its previous store has left), or is free
+                if (RES) got = mbar_wait(res_full + 8 * ob, ophase, abortp, p.status, 107) && got;
+                else got = mbar_wait(out_free + 8 * ob, ophase ^ 1, abortp, p.status, 109) && got;
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t out_buf = smem_base + p.out_off + acc * p.out_bytes;
-                const uint32_t res_buf = smem_base + p.res_off + rb * p.out_bytes;
+                const uint32_t out_buf = smem_base + p.out_off + ob * p.out_bytes;
+                const uint32_t res_buf = out_buf;       // in place: a thread reads and then overwrites its own 16 bytes
                 const uint32_t bias_s = smem_base + p.bias_off + 4 * c_first;
                 int va[16], vb[16];
                 if (my_nch > 0) tmem_ld16(t_addr, va);
@@ -762,10 +765,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(tempty_bar + 8 * acc);
-                    mbar_arrive(out_full + 8 * acc);
-                    if (RES) mbar_arrive(res_free + 8 * rb);
+                    mbar_arrive(out_full + 8 * ob);
                 }
-                if (RES && ++rb == p.res_bufs) { rb = 0; rphase ^= 1; }
+                if (++ob == p.out_bufs) { ob = 0; ophase ^= 1; }
             }
         } else {
             grid_dependency_wait();     // direct stores (and residual reads) from these warps
@@ -969,14 +971,14 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         p.swz_mask = p.slab_w == 128 ? 7u : (p.slab_w == 64 ? 3u : (p.slab_w == 32 ? 1u : 0u));
         p.out_bytes = (uint32_t)(TILE_M * p.bn + 1023) / 1024 * 1024;
         const size_t bias_bytes = ((size_t)p.n_tiles * p.bn * 4 + 1023) / 1024 * 1024;
-        // a residual tile takes about as long to arrive from HBM as a tile takes to compute: keep three in flight
-        // where that does not cost pipeline depth, i.e. when the weights are resident anyway (one N tile) and 32 KiB
-        // remain for activation stages; measured, layers that lose stages to the third buffer get slower
-        p.res_bufs = 2;
-        const size_t weights = (size_t)g.kh * g.kw * p.c_chunks * b_bytes;
-        if (q.has_res && p.n_tiles == 1 && (size_t)p.out_bytes * 5 + bias_bytes + weights + 34 * 1024 <= SMEM_LIMIT - 1024)
-            p.res_bufs = 3;
-        staging = (size_t)p.out_bytes * (2 + (q.has_res ? p.res_bufs : 0)) + bias_bytes;
+        // Output ring.  Without a residual two buffers overlap the epilogue of a tile with the store of the one
+        // before.  With a residual a buffer goes through load -> convert in place -> store, and a residual tile takes
+        // about as long to arrive from HBM as a tile takes to compute: three buffers (four when they are small).
+        p.out_bufs = !q.has_res ? 2 : (p.out_bytes <= 16 * 1024 ? 4 : 3);
+        if (getenv("F8_OUT_BUFS")) p.out_bufs = atoi(getenv("F8_OUT_BUFS"));
+        if (p.out_bufs < 2) p.out_bufs = 2;
+        if (p.out_bufs > MAX_OUT_BUFS) p.out_bufs = MAX_OUT_BUFS;
+        staging = (size_t)p.out_bytes * p.out_bufs + bias_bytes;
     }
     const size_t ktab_bytes = ((size_t)g.kh * g.kw * p.c_chunks * 8 + 1023) / 1024 * 1024;
     if (ktab_bytes > 16 * 1024 || g.kh * g.kw > 0xffff) {
@@ -1014,8 +1016,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.uses = (k_iters + group - 1) / group;
     p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !getenv("F8_NO_DUAL")) ? 1 : 0;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
-    p.res_off = p.out_off + 2 * p.out_bytes;
-    p.bias_off = p.res_off + (q.has_res ? (uint32_t)p.res_bufs * p.out_bytes : 0u);
+    p.bias_off = p.out_off + (uint32_t)p.out_bufs * p.out_bytes;
     p.ktab_off = (uint32_t)(p.stages * p.stage_bytes + staging - ktab_bytes);
     p.bres_off = (uint32_t)(p.stages * p.stage_bytes + staging);
     // instruction descriptor: D = s32 (2 at bit 4), A format at bit 7 (0 = u8, 1 = s8), B = s8 at bit 10,
