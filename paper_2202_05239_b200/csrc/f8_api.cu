@@ -195,12 +195,14 @@ f8_status f8_device_status(void) {
     if (!w) return fail(F8_ERR_CUDA, "no status word");
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
-    int v = 0;
-    e = cudaMemcpy(&v, w, sizeof(int), cudaMemcpyDeviceToHost);
+    int v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    e = cudaMemcpy(v, w, sizeof(v), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(e, "status read");
-    if (v != 0) {
-        cudaMemset(w, 0, sizeof(int));
-        return fail(F8_ERR_TIMEOUT, "a kernel abandoned a bounded wait (site %d)", v);
+    if (v[0] != 0) {
+        cudaMemset(w, 0, sizeof(v));
+        return fail(F8_ERR_TIMEOUT, "a kernel abandoned a bounded wait (site %d, layer %d, block %d, thread %d, barrier 0x%x, parity %d; "
+                    "%d polls, %.0f Mcycles, %.3f ms)",
+                    v[0] & 0xff, (v[0] >> 8) - 1, v[1], v[2], (unsigned)v[3], v[4], v[5], v[6] * 1.048576, v[7] * 1.024e-3);
     }
     return F8_OK;
 }
@@ -302,6 +304,7 @@ struct NetLayer {
     int pack_cpad = 8;     // bytes per pixel inside a cell (4 when c <= 4); a cell is two rows = 2 * pack_cpad bytes
     int pack_hp = 0, pack_kh = 0, pack_top = 0, pack_bottom = 0;   // row pairs: count, taps, padding above / below
     int8_t *w_packed = nullptr;
+    int8_t *w_core = nullptr;   // the same window weights as [K / 16][c_out][16] (core-matrix order) for the stem kernel
     size_t out_bytes_per_image = 0;
 };
 
@@ -312,6 +315,7 @@ struct Step {
     const void *res = nullptr;
     void *y = nullptr;
     bool use_tc = false;
+    bool fused_pool = false;  // kind -2: the stem kernel also computes the max pool that follows (layer + 1)
     PlanPtr plan;
     F8ConvGeom g;
 };
@@ -330,6 +334,7 @@ struct f8_net {
     const void *plan_x = nullptr;
     void *plan_y = nullptr, *plan_ws = nullptr;
     bool plan_force_direct = false;
+    bool plan_dump_first = false;                // the cached plan keeps the output of a fusable first layer
     std::vector<Step> steps;
     std::vector<size_t> t_off;                   // workspace offset per tensor
     size_t pack_off = 0;
@@ -386,6 +391,7 @@ void free_layers(f8_net *net) {
         if (l.w) cudaFree(l.w);
         if (l.b) cudaFree(l.b);
         if (l.w_packed) cudaFree(l.w_packed);
+        if (l.w_core) cudaFree(l.w_core);
     }
 }
 
@@ -576,6 +582,17 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
             e = cudaMalloc(&L.w_packed, round256(wp.size()));
             if (e == cudaSuccess) e = cudaMemcpy(L.w_packed, wp.data(), wp.size(), cudaMemcpyHostToDevice);
             if (e != cudaSuccess) return cleanup(cuda_fail(e, "packed stem weights upload"));
+            if (L.pack_cpad == 4) {
+                // core-matrix order for the stem kernel: 16 consecutive K bytes of one output channel are contiguous,
+                // then the output channels, then the K chunks
+                const size_t kb = (size_t)L.pack_kh * L.pack_kw8;
+                std::vector<int8_t> wc(kb * d.c_out, 0);
+                for (int co = 0; co < d.c_out; ++co)
+                    for (size_t k = 0; k < kb; ++k) wc[((k / 16) * d.c_out + co) * 16 + k % 16] = wp[(size_t)co * kb + k];
+                e = cudaMalloc(&L.w_core, round256(wc.size()));
+                if (e == cudaSuccess) e = cudaMemcpy(L.w_core, wc.data(), wc.size(), cudaMemcpyHostToDevice);
+                if (e != cudaSuccess) return cleanup(cuda_fail(e, "stem weights upload"));
+            }
         }
     }
     *out = net.release();
@@ -638,8 +655,13 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int nl = (int)net->layers.size();
 
+    // a first layer whose output is asked for cannot be fused with the pooling layer behind it
+    bool dump_fusable = false;
+    if (layer_dump)
+        for (int i = 0; i < nl; ++i)
+            if (net->layers[i].w_core && layer_dump[i]) dump_fusable = true;
     const bool replan = net->plan_batch != batch || net->plan_x != x || net->plan_y != y || net->plan_ws != workspace ||
-                        net->plan_force_direct != g_force_direct;
+                        net->plan_force_direct != g_force_direct || net->plan_dump_first != dump_fusable;
     if (replan) {
         net->steps.clear();
         net->plan_batch = -1;
@@ -649,8 +671,10 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
             if (t == nl) return y;
             return (uint8_t *)workspace + net->t_off[t];
         };
+        int skip_layer = -1;          // a pooling layer the stem kernel has taken over
         for (int i = 0; i < nl; ++i) {
             NetLayer &L = net->layers[i];
+            if (i == skip_layer) continue;
             Step stp;
             stp.kind = L.d.kind;
             stp.layer = i;
@@ -661,7 +685,25 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
             stp.g.n = batch;
             if ((L.d.kind == F8_LAYER_CONV || L.d.kind == F8_LAYER_LINEAR) && !g_force_direct) {
                 const char *why = "";
-                if (L.packed) {
+                if (L.packed && L.w_core && !getenv("F8_NO_STEM_KERNEL") &&
+                    f8_stem_tc_supported(stp.g, L.q, L.pack_kh, L.pack_kw8 / 32)) {
+                    // the stem kernel; it also takes the 3x3 / 2 / pad 1 max pool behind the layer when nothing else
+                    // reads the layer's output
+                    bool fuse = !dump_fusable && i + 1 < nl && !getenv("F8_NO_STEM_POOL_FUSION");
+                    if (fuse) {
+                        const NetLayer &P = net->layers[i + 1];
+                        fuse = P.d.kind == F8_LAYER_MAXPOOL && P.d.src == i + 1 && P.d.conv.kh == 3 && P.d.conv.kw == 3 &&
+                               P.d.conv.stride == 2 && P.d.conv.pad == 1;
+                        for (int l = i + 2; fuse && l < nl; ++l)
+                            if (net->layers[l].d.src == i + 1 || (net->layers[l].q.has_res && net->layers[l].d.res == i + 1)) fuse = false;
+                    }
+                    stp.kind = -2;
+                    stp.fused_pool = fuse;
+                    if (fuse) {
+                        stp.y = tensor_ptr(i + 2);
+                        skip_layer = i + 1;
+                    }
+                } else if (L.packed) {
                     F8ConvGeom pg = stp.g;
                     pg.c = L.pack_kw8; pg.kw = 1; pg.stride_w = 1; pg.pad_w = 0;
                     pg.kh = L.pack_kh; pg.stride_h = 1; pg.pad_h = L.pack_top; pg.pad_h_end = L.pack_bottom;
@@ -687,6 +729,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                             pre.g = stp.g;
                             net->steps.push_back(std::move(pre));
                             stp.use_tc = true;
+                            f8_tc_plan_set_tag(plan.get(), i + 1);
                             stp.plan = std::move(plan);
                         }
                     }
@@ -695,6 +738,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                     if (plan && f8_tc_plan_init(plan.get(), stp.g, L.q, dense_view(stp.x, stp.g), L.w, L.b, stp.res,
                                                 stp.y, f8_status_word(), &why) == cudaSuccess) {
                         stp.use_tc = true;
+                        f8_tc_plan_set_tag(plan.get(), i + 1);
                         stp.plan = std::move(plan);
                     }
                 }
@@ -706,6 +750,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         net->plan_y = y;
         net->plan_ws = workspace;
         net->plan_force_direct = g_force_direct;
+        net->plan_dump_first = dump_fusable;
     }
 
     int launches = 0;
@@ -723,6 +768,11 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         NetLayer &L = net->layers[stp.layer];
         cudaError_t e = cudaSuccess;
         switch (stp.kind) {
+            case -2:
+                e = f8_launch_stem_tc(stp.g, L.q, L.pack_kh, L.pack_top, L.pack_left, L.pack_kw8 / 32, stp.fused_pool ? 1 : 0, stp.x,
+                                      L.w_core, L.b, stp.y, f8_status_word(), stp.layer + 1, st, net->overlap_layers);
+                ++g_tc_launches;
+                break;
             case -1:
                 e = f8_launch_pack_stem_pairs(batch, L.g.h, L.g.w, L.g.c, L.pack_cpad, L.pack_hp, L.pack_wp, L.pack_left, stp.x, stp.y, st,
                                               net->overlap_layers);
@@ -749,16 +799,17 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         ++launches;
         if (prof) {
             cudaEventRecord(net->events[launches], st);
-            net->event_layer.push_back(stp.layer);
+            net->event_layer.push_back(stp.fused_pool ? stp.layer + 1 : stp.layer);
         }
-        if (layer_dump && stp.kind >= 0 && layer_dump[stp.layer]) {
-            const int c_true = net->t_c[stp.layer + 1], c_stored = net->t_cp[stp.layer + 1];
+        const int out_layer = stp.fused_pool ? stp.layer + 1 : stp.layer;      // the layer whose output this step wrote
+        if (layer_dump && stp.kind != -1 && layer_dump[out_layer]) {
+            const int c_true = net->t_c[out_layer + 1], c_stored = net->t_cp[out_layer + 1];
             if (c_true == c_stored)
-                e = cudaMemcpyAsync(layer_dump[stp.layer], stp.y, (size_t)batch * L.out_bytes_per_image,
+                e = cudaMemcpyAsync(layer_dump[out_layer], stp.y, (size_t)batch * net->layers[out_layer].out_bytes_per_image,
                                     cudaMemcpyDeviceToDevice, st);
             else   // drop the zero padding channels: one row per pixel
-                e = cudaMemcpy2DAsync(layer_dump[stp.layer], (size_t)c_true, stp.y, (size_t)c_stored, (size_t)c_true,
-                                      (size_t)batch * net->t_h[stp.layer + 1] * net->t_w[stp.layer + 1],
+                e = cudaMemcpy2DAsync(layer_dump[out_layer], (size_t)c_true, stp.y, (size_t)c_stored, (size_t)c_true,
+                                      (size_t)batch * net->t_h[out_layer + 1] * net->t_w[out_layer + 1],
                                       cudaMemcpyDeviceToDevice, st);
             if (e != cudaSuccess) return cuda_fail(e, "layer dump copy");
         }

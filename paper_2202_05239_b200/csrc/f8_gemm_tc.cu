@@ -30,6 +30,7 @@
 #include <algorithm>
 
 #include "f8_epilogue.cuh"
+#include "f8_tc_ptx.cuh"
 
 namespace {
 
@@ -54,9 +55,6 @@ constexpr int MAX_STAGES = 16;
 constexpr int MAX_OUT_BUFS = 4;             // ring of staged output tiles; with a residual, the residual tile lands in the
                                             // buffer first and the epilogue converts it in place
 constexpr int TMEM_COLS = 512;
-constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
-constexpr unsigned MIN_POLLS_BEFORE_TIMEOUT = 1u << 16;             // failed polls a wait needs before it may give up
-constexpr unsigned long long DRAIN_LIMIT_CYCLES = 200000000ull;
 constexpr size_t SMEM_LIMIT = 220 * 1024;     // dynamic shared memory budget (227 KiB per CTA minus static data)
 
 // Division by a run-time constant without a divide instruction (a 32-bit divide costs a lone thread well over a
@@ -112,187 +110,18 @@ struct TcParams {
     F8Requant q;
     int mul_acc, mul_res;     // 2^q.sh_acc, 2^q.sh_res (kept opaque to the compiler, see the epilogue)
     int *status;
+    // Windowed 3x3 (stride 1, pad 1, resident weights).  A tile is win_r whole output rows of one image; its M index runs
+    // over the rows of the zero-padded image (win_wp = W + 2 positions per row, the last two of each row are discarded).
+    // The padded input rows win_r + 2 rows tall are loaded ONCE per channel chunk as they lie in memory; the window of
+    // filter tap (r, s) is then the same shared-memory tile read from (r * win_wp + s) pixel rows further down, so the
+    // activations cross the L2 -> SM path once instead of nine times.
+    int win;
+    int win_r, win_wp, win_bands;
+    FastDiv div_bands;
+    uint32_t tx_win;          // bytes of one window load
+    uint32_t tx_res;          // bytes of one residual tile load
+    int tag;                  // caller's label of this launch (layer index + 1), reported with a timed-out wait
 };
-
-// ----------------------------------------------------------------------------- PTX wrappers
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// Programmatic dependent launch.  A grid launched with the programmatic-serialization attribute may start
-// while its predecessor in the stream is still running; grid_dependency_wait() returns once every
-// predecessor has completed and its writes are visible (at once for an ordinary launch).  Everything that
-// reads activations or writes the output sits behind it; the prologue and the weight loads do not.
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-// Bounded wait.  Returns false when the kernel is aborting (this wait or another one ran out).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                            int code) {
-    const unsigned long long t0 = clock64();
-    unsigned spins = 0;
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 63u) == 0) {
-            if (*abort_flag) return false;
-            // both conditions: the cycle counter keeps running while the context is switched out (a profiler
-            // replaying the kernel does that for seconds), the poll count does not
-            if (spins >= MIN_POLLS_BEFORE_TIMEOUT && (unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
-                *abort_flag = 1;
-                atomicCAS(status, 0, code);
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                          int code) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status, code);
-}
-
-__device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w,
-                                                int h, int n, uint16_t off_w, uint16_t off_h) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};" ::"r"(dst),
-        "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
-                                            int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
-        "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-        "l"(map), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-// shared -> global tile store; rows / columns outside the tensor are clipped by the hardware
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src),
-                 "r"(c0), "r"(c1)
-                 : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-
-// D[tmem] (+)= A[smem] * B[smem]^T, int8 operands, int32 accumulate.
-__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-// The K = 32 slices of one sub-chunk (kb / 32 of them), issued from one asm block.  A lone thread pays a few
-// cycles for every instruction it executes, and the tensor pipe is only kept busy when an MMA costs the
-// issuing thread no more than a handful of them: the shared-memory descriptors of the slices differ only
-// in their low words (start address, 16-byte units), so those are advanced with 32-bit adds inside the
-// block and the constant high word (SBO, version, swizzle mode) is attached by a register-pair move.
-#define F8_MMA_I8 "tcgen05.mma.cta_group::1.kind::i8 [%0], a, b, %4, "
-#define F8_MMA_NEXT(off) \
-    "add.u32 x, %1, " #off ";\n\tadd.u32 y, %2, " #off ";\n\tmov.b64 a, {x, %3};\n\tmov.b64 b, {y, %3};\n\t" F8_MMA_I8 "t;\n\t"
-template <int MMAS>
-__device__ __forceinline__ void mma_i8_sub(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
-                                           uint32_t idesc, uint32_t accumulate) {
-    if (MMAS == 1)
-        asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                     "mov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t" F8_MMA_I8 "p;\n\t}" ::"r"(d_tmem),
-                     "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
-                     : "memory");
-    else if (MMAS == 2)
-        asm volatile("{\n\t.reg .pred p, t;\n\t.reg .b64 a, b;\n\t.reg .b32 x, y;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                     "setp.eq.b32 t, 0, 0;\n\tmov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t" F8_MMA_I8 "p;\n\t"
-                     F8_MMA_NEXT(2) "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
-                     : "memory");
-    else
-        asm volatile("{\n\t.reg .pred p, t;\n\t.reg .b64 a, b;\n\t.reg .b32 x, y;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                     "setp.eq.b32 t, 0, 0;\n\tmov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t" F8_MMA_I8 "p;\n\t"
-                     F8_MMA_NEXT(2) F8_MMA_NEXT(4) F8_MMA_NEXT(6) "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi),
-                     "r"(idesc), "r"(accumulate)
-                     : "memory");
-}
-
-// All sub-chunks of one stage use; `a_lo` / `b_lo` are the low descriptor words of its first A / B tile.
-template <int MMAS>
-__device__ __forceinline__ void mma_i8_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_step,
-                                             uint32_t b_step, uint32_t desc_hi, uint32_t idesc, int subs,
-                                             uint32_t accumulate_first) {
-    mma_i8_sub<MMAS>(d_tmem, a_lo, b_lo, desc_hi, idesc, accumulate_first);
-    for (int j = 1; j < subs; ++j) {
-        a_lo += a_step;
-        b_lo += b_step;
-        mma_i8_sub<MMAS>(d_tmem, a_lo, b_lo, desc_hi, idesc, 1u);
-    }
-}
-// mbarrier arrives once every tcgen05.mma issued so far by this thread has completed.
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-                 : "memory");
-}
-
-// 16 consecutive accumulator columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
-        "%15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major tile whose rows are `kb` bytes long and swizzled with
-// the matching TMA mode: 8-row groups are 8*kb bytes apart (stride byte offset), the leading offset
-// is unused (1), descriptor version 1, layout code 2 / 4 / 6 for 128 / 64 / 32-byte swizzle.
-__host__ __device__ inline uint64_t smem_desc_hi(int kb) {
-    const uint64_t layout = kb == 128 ? 2 : (kb == 64 ? 4 : 6);
-    const uint64_t sbo = (uint64_t)(8 * kb) >> 4;
-    return ((uint64_t)1 << 16) | (sbo << 32) | ((uint64_t)1 << 46) | (layout << 61);
-}
 
 // ----------------------------------------------------------------------------- epilogue helpers
 
@@ -342,64 +171,6 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int (&ac
     }
 }
 
-// Branch-free epilogue for the common case (8-bit output, 1 <= s <= 24, c_out % 16 == 0).
-//   v = acc * 2^sh_acc + bias'          bias' = (bias << sh_acc) + 2^(s-1), staged in shared memory
-//   v += r << sh_res                    (RES only)
-//   t = v >> s                          = floor((acc' + 2^(s-1)) / 2^s), round half up
-//   y = clamp(t, lo, hi)                saturating pack; the signed quantizer additionally excludes -128
-// cvt.pack.sat packs two saturated values into the low half of d and moves the low half of c above
-// them: d = (c << 16) | (sat(a) << 8) | sat(b).
-// The integer ALU pipe (shifts, byte permutes, 3-input adds, packs) issues a warp instruction every other
-// cycle and is what bounds this code, so work is kept off it: the two scalings are multiply-adds whose
-// power-of-two factors arrive as opaque kernel parameters (the FMA pipe; a visible 1 << n would be turned
-// into shifts), a residual byte costs one PRMT whose selector (zero- or sign-extending) sits in a register,
-// and bias / residual / output go through explicit shared-space accesses.
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
-template <bool RES, bool SIGNED_OUT>
-__device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], uint32_t bias_addr, uint4 rw, int mul_acc,
-                                                 int mul_res, const uint32_t (&rsel)[4], int s) {
-    int t[16];
-    const uint32_t rwords[4] = {rw.x, rw.y, rw.z, rw.w};
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        const uint4 b = lds128(bias_addr + 16 * g);
-        const int bb[4] = {(int)b.x, (int)b.y, (int)b.z, (int)b.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int j = 4 * g + k;
-            int v = acc[j] * mul_acc + bb[k];
-            if (RES) {
-                int r;
-                asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(rwords[g]), "r"(rsel[k]));
-                v += r * mul_res;
-            }
-            v >>= s;
-            t[j] = SIGNED_OUT ? max(v, -127) : v;
-        }
-    }
-    uint32_t o[4];
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        uint32_t hi2;
-        if (SIGNED_OUT) {
-            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(t[4 * g + 3]), "r"(t[4 * g + 2]));
-            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(o[g]) : "r"(t[4 * g + 1]), "r"(t[4 * g]), "r"(hi2));
-        } else {
-            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(t[4 * g + 3]), "r"(t[4 * g + 2]));
-            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(o[g]) : "r"(t[4 * g + 1]), "r"(t[4 * g]), "r"(hi2));
-        }
-    }
-    return make_uint4(o[0], o[1], o[2], o[3]);
-}
-
 // ----------------------------------------------------------------------------- the kernel
 
 enum { EPI_GENERIC = 0, EPI_U8 = 1, EPI_U8_RES = 2, EPI_S8 = 3, EPI_S8_RES = 4 };
@@ -435,7 +206,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(full_bar + 8 * s, 1);       // one arrival (with the byte count of the whole group) per use
+            mbar_init(full_bar + 8 * s, p.win ? 1 : 2);   // per use: one arrival (with its byte count) per producer warp
             mbar_init(empty_bar + 8 * s, 1);
         }
         mbar_init(bres_bar, 1);
@@ -479,6 +250,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const int total_tiles = p.m_tiles * p.n_tiles;
     const int k_iters = p.kh * p.kw * p.c_chunks;
     volatile int *abortp = &abort_flag;
+    const int tagbits = p.tag << 8;     // status word of a timed-out wait: tag << 8 | site
 
     if (warp == A_PROD_WARP || warp == B_PROD_WARP) {
         // ------------------------------------------------------------------ TMA producer warps
@@ -517,6 +289,29 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         int last_stage = 0;
         uint32_t last_phase = 0;            // stage / phase of this lane's most recent load (for the drain on abort)
         bool ok = true;
+        if (p.win) {
+            // one load per (tile, channel chunk): the padded rows of the band, requested by the lane that owns the stage
+            for (int tile = blockIdx.x; ok && opnd == 0 && tile < total_tiles; tile += gridDim.x) {
+                const int m_t = fast_div(tile, p.div_n_tiles);
+                const int img = fast_div(m_t, p.div_bands);
+                const int y0 = (m_t - img * p.win_bands) * p.win_r;
+                for (int cc = 0; cc < p.c_chunks; ++cc) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, tagbits | 101))) {
+                        ok = false;
+                        break;
+                    }
+                    if (lane == (stage & 31)) {
+                        const uint32_t fb = full_bar + 8 * stage;
+                        mbar_expect_tx(fb, p.tx_win);
+                        tma_load_4d(smem_base + stage * p.stage_bytes, &map_a, fb, cc * p.kb, -1, y0 - 1, img);
+                        have_last = true;
+                        last_stage = stage;
+                        last_phase = phase;
+                    }
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                }
+            }
+        } else
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
             const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
             const int m0 = m_t * TILE_M;
@@ -528,21 +323,24 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int base_h = oh * p.stride_h - p.pad_h;
             const int n_base = n_t * p.bn;
             for (int kc = 0; kc < k_iters; kc += p.group) {
-                if (a_helper && k_iters - kc < 2) {
-                    // A stage use without an odd sub-chunk: nothing to request, and nothing to wait for either.  A
-                    // warp that only polled here would not hold the pipeline back, could fall two phases behind
-                    // it, and a parity wait cannot tell a phase from the one two later.
-                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
-                    continue;
-                }
-                if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, 101))) {
+                if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, tagbits | 101))) {
                     ok = false;
                     break;
                 }
                 const int subs = min(p.group, k_iters - kc);
                 const uint32_t fb = full_bar + 8 * stage;
-                // one arrival per stage use; it announces the bytes of every load of the group
-                if (opnd == 0 && lane == 0) mbar_expect_tx(fb, (uint32_t)subs * p.tx_sub);
+                // Two arrivals per stage use, one from each producer warp, and each announces the bytes of its own loads
+                // BEFORE it issues them: the barrier's byte count never runs ahead of what has been announced, and both
+                // warps are needed for every use, so neither can fall a barrier phase behind the pipeline (a parity wait
+                // cannot tell a phase from the one two later).  A helper without a load in this use just arrives.
+                if (lane == 0) {
+                    uint32_t bytes;
+                    if (opnd == 0) bytes = (uint32_t)(p.b_res ? (subs + 1) >> 1 : subs) * p.tx_a;
+                    else bytes = p.b_res ? (uint32_t)(subs >> 1) * p.tx_a : (uint32_t)subs * p.tx_b;
+                    if (bytes) mbar_expect_tx(fb, bytes);
+                    else mbar_arrive(fb);
+                }
+                __syncwarp();
                 const int j = (lane - stage * p.group) & 31;
                 if (j < subs && (j & j_mask) == j_want) {
                     const uint2 e = ktab[kc + j];       // x: first channel of the chunk, y: tap << 16 | r << 8 | s
@@ -569,7 +367,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         }
         // the resident weights must have landed before this CTA's shared memory may go away (they have, unless
         // the kernel is aborting: the MMA issuers wait for them before their first instruction)
-        if (a_helper) mbar_wait(bres_bar, 0, abortp, p.status, 107);
+        if (a_helper) mbar_wait(bres_bar, 0, abortp, p.status, tagbits | 110);
         }
     } else if (warp == MMA_WARP || warp == MMA2_WARP) {
         // ------------------------------------------------------------------ MMA issuers
@@ -594,7 +392,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const uint32_t stage16 = p.stage_bytes >> 4, sub16 = p.sub_bytes >> 4, a16 = p.a_bytes >> 4;
             const uint32_t b16 = p.b_bytes >> 4, bres_lo = desc_lo0 + (p.bres_off >> 4);
             const uint32_t b_step = p.b_res ? b16 : sub16;
-            if (p.b_res && !mbar_wait(bres_bar, 0, abortp, p.status, 108)) ok = false;
+            if (p.b_res && !mbar_wait(bres_bar, 0, abortp, p.status, tagbits | 111)) ok = false;
             const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
@@ -606,7 +404,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     continue;
                 }
                 const uint32_t acc_phase = (local >> 1) & 1;
-                if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, abortp, p.status, 102)) { ok = false; break; }
+                if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, abortp, p.status, tagbits | 102)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * 256;   // two 256-column accumulators
                 uint32_t b_tile_lo = 0;
@@ -614,8 +412,32 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
                     b_tile_lo = bres_lo + (uint32_t)(n_t * k_iters) * b16;
                 }
+                if (p.win) {
+                    // one stage use per channel chunk; the nine taps read the same tile at shifted row offsets
+                    const uint32_t kb16 = (uint32_t)p.kb >> 4;
+                    for (int cc = 0; cc < p.c_chunks; ++cc) {
+                        if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, tagbits | 103)) { ok = false; break; }
+                        tc_fence_after();
+                        uint32_t first = cc != 0 ? 1u : 0u;
+                        uint32_t b_lo = b_tile_lo + (uint32_t)cc * b16;
+                        for (int r = 0; r < 3; ++r) {
+                            uint32_t a_lo = stage_lo + (uint32_t)(r * p.win_wp) * kb16;
+                            for (int sx = 0; sx < 3; ++sx) {
+                                if (mmas == 4) mma_i8_sub<4>(d_tmem, a_lo, b_lo, desc_hi32, p.idesc, first);
+                                else if (mmas == 2) mma_i8_sub<2>(d_tmem, a_lo, b_lo, desc_hi32, p.idesc, first);
+                                else mma_i8_sub<1>(d_tmem, a_lo, b_lo, desc_hi32, p.idesc, first);
+                                first = 1u;
+                                a_lo += kb16;
+                                b_lo += (uint32_t)p.c_chunks * b16;
+                            }
+                        }
+                        mma_commit(empty_bar + 8 * stage);
+                        stage_lo += stage16;
+                        if (++stage == p.stages) { stage = 0; phase ^= 1; stage_lo = desc_lo0; }
+                    }
+                } else
                 for (int kc = 0; kc < k_iters; kc += p.group) {
-                    if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, 103)) { ok = false; break; }
+                    if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, tagbits | 103)) { ok = false; break; }
                     tc_fence_after();
                     const int subs = min(p.group, k_iters - kc);
                     const uint32_t first = kc != 0 ? 1u : 0u;      // the tile's first MMA overwrites the accumulator
@@ -650,8 +472,16 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             uint32_t bphase = 0;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
-                if (!mbar_wait(out_full + 8 * b, bphase, abortp, p.status, 108)) break;
+                if (!mbar_wait(out_full + 8 * b, bphase, abortp, p.status, tagbits | 108)) break;
                 const uint32_t src = smem_base + p.out_off + b * p.out_bytes;
+                if (p.win) {
+                    const int img = fast_div(m_t, p.div_bands);
+                    const int y0 = (m_t - img * p.win_bands) * p.win_r;
+                    // positions W and W + 1 of every row and rows below the image are clipped by the hardware
+                    for (int sl = 0; sl < p.n_slabs; ++sl)
+                        if (n_t * p.bn + sl * p.slab_w < p.c_out)
+                            tma_store_4d(&map_y, src + sl * (TILE_M * p.slab_w), n_t * p.bn + sl * p.slab_w, 0, y0, img);
+                } else
                 for (int sl = 0; sl < p.n_slabs; ++sl)
                     if (n_t * p.bn + sl * p.slab_w < p.c_out)
                         tma_store_2d(&map_y, src + sl * (TILE_M * p.slab_w), n_t * p.bn + sl * p.slab_w, m_t * TILE_M);
@@ -675,9 +505,16 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
-                if (!mbar_wait(out_free + 8 * rb, rphase ^ 1, abortp, p.status, 106)) { ok = false; break; }
+                if (!mbar_wait(out_free + 8 * rb, rphase ^ 1, abortp, p.status, tagbits | 106)) { ok = false; break; }
                 const uint32_t fb = res_full + 8 * rb;
-                mbar_expect_tx(fb, p.out_bytes);
+                mbar_expect_tx(fb, p.tx_res);
+                if (p.win) {
+                    const int img = fast_div(m_t, p.div_bands);
+                    const int y0 = (m_t - img * p.win_bands) * p.win_r;
+                    for (int sl = 0; sl < p.n_slabs; ++sl)
+                        tma_load_4d(smem_base + p.out_off + rb * p.out_bytes + sl * (TILE_M * p.slab_w), &map_r, fb,
+                                    n_t * p.bn + sl * p.slab_w, 0, y0, img);
+                } else
                 for (int sl = 0; sl < p.n_slabs; ++sl)
                     tma_load_2d(smem_base + p.out_off + rb * p.out_bytes + sl * (TILE_M * p.slab_w), &map_r, fb,
                                 n_t * p.bn + sl * p.slab_w, m_t * TILE_M);
@@ -730,10 +567,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int c_first = n_t * p.bn + ch_begin * 16;
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
-                bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104);
+                bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, tagbits | 104);
                 // the buffer holds the residual tile (which implies that its previous store has left), or is free
-                if (RES) got = mbar_wait(res_full + 8 * ob, ophase, abortp, p.status, 107) && got;
-                else got = mbar_wait(out_free + 8 * ob, ophase ^ 1, abortp, p.status, 109) && got;
+                if (RES) got = mbar_wait(res_full + 8 * ob, ophase, abortp, p.status, tagbits | 107) && got;
+                else got = mbar_wait(out_free + 8 * ob, ophase ^ 1, abortp, p.status, tagbits | 109) && got;
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t out_buf = smem_base + p.out_off + ob * p.out_bytes;
@@ -780,7 +617,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const size_t row = (size_t)m_t * TILE_M + tile_row;
                 const bool row_valid = row < (size_t)p.M;
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
-                if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, 104))) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, tagbits | 104))) { ok = false; break; }
                 tc_fence_after();
                 for (int i = 0; i < nch; ++i) {
                     const int co0 = n0 + (ch_begin + i) * 16;
@@ -912,6 +749,7 @@ struct F8TcPlan {
 };
 
 size_t f8_tc_plan_size() { return sizeof(F8TcPlan); }
+void f8_tc_plan_set_tag(F8TcPlan *plan, int tag) { plan->p.tag = tag; }
 
 bool f8_tc_supported(const F8ConvGeom &g, size_t x_bytes) {
     if (g.c % 16 != 0) return false;                 // TMA strides are multiples of 16 bytes
@@ -999,6 +837,50 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         p.sub_bytes = p.a_bytes;
     }
     p.tx_sub = p.tx_a + (p.b_res ? 0u : p.tx_b);
+    p.tx_res = p.out_bytes;
+    // Windowed mode for 3x3 / stride 1 / pad 1 layers whose weights can stay resident: whole padded rows are loaded once
+    // per tile and every filter tap reads them at a shifted row offset.  Worth it when whole rows fill most of a tile
+    // and the im2col loads are what bounds the layer: measured, 128-channel layers gain 1.8x (the resident weights
+    // leave room for two im2col stages only), 64-channel layers lose a little (their tiles are bound by per-tile
+    // costs, and whole-row tiles are 12.5 % more tiles).
+    p.win = 0;
+    if (staged && p.kb == 128 && g.kh == 3 && g.kw == 3 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 1 && g.pad_w == 1 &&
+        g.pad_h_end < 0 && p.n_tiles == 1 && g.w + 2 <= TILE_M && g.w == g.wo && g.h == g.ho && g.c % p.kb == 0 &&
+        !getenv("F8_NO_WIN")) {
+        const int wp = g.w + 2;
+        const int r = std::min(TILE_M / wp, g.ho);
+        const int bands = (g.ho + r - 1) / r;
+        const double fill = (double)g.ho * g.wo / ((double)bands * TILE_M);
+        const uint32_t box_bytes = (uint32_t)p.kb * wp * (r + 2);
+        const uint32_t win_stage = (box_bytes + 1023) / 1024 * 1024;
+        const size_t bias_bytes = ((size_t)p.n_tiles * p.bn * 4 + 1023) / 1024 * 1024;
+        int ob = p.out_bufs;
+        // at least two window stages beside the weights; give up output buffers before giving up the mode
+        while (ob > 1 && b_all + 2 * (size_t)win_stage + (size_t)p.out_bytes * ob + bias_bytes + ktab_bytes + 1024 > SMEM_LIMIT) --ob;
+        const bool fits = b_all + 2 * (size_t)win_stage + (size_t)p.out_bytes * ob + bias_bytes + ktab_bytes + 1024 <= SMEM_LIMIT;
+        if (fill >= 0.7 && fits) {
+            p.win = 1;
+            p.win_r = r;
+            p.win_wp = wp;
+            p.win_bands = bands;
+            p.div_bands = make_fast_div(bands);
+            p.tx_win = box_bytes;
+            p.tx_res = (uint32_t)p.bn * wp * r;
+            p.out_bufs = ob;
+            staging = (size_t)p.out_bytes * ob + bias_bytes + ktab_bytes;
+            p.b_res = 1;
+            p.m_tiles = g.n * bands;
+            p.sub_bytes = win_stage;
+        }
+    }
+    if (p.win) {
+        p.group = 1;
+        p.stage_bytes = p.sub_bytes;
+        int stages = (int)((SMEM_LIMIT - 1024 - staging - b_all) / p.stage_bytes);
+        if (stages > MAX_STAGES) stages = MAX_STAGES;
+        p.stages = stages;
+        p.uses = p.c_chunks;
+    } else {
     const int uses = (k_iters + 7) / 8;                  // at most eight k-iterations per stage, evenly split
     int group = (k_iters + uses - 1) / uses;
     while (group > 1 && avail / ((size_t)group * p.sub_bytes) < 2) --group;
@@ -1014,6 +896,8 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     }
     p.stages = stages;
     p.uses = (k_iters + group - 1) / group;
+    }
+    const int stages = p.stages;
     p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !getenv("F8_NO_DUAL")) ? 1 : 0;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
     p.bias_off = p.out_off + (uint32_t)p.out_bufs * p.out_bytes;
@@ -1035,6 +919,20 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     const size_t row_bytes = (size_t)g.c_out * ysz;
     p.vec_bytes = (row_bytes % 16 == 0) ? 16 : (row_bytes % 8 == 0 ? 8 : (row_bytes % 4 == 0 ? 4 : 1));
 
+    if (p.win) {
+        // A: the same tensor as plain tiles of win_r + 2 padded rows (coordinates -1 are zero filled)
+        cuuint64_t dims[4] = {xv.dim_c, xv.dim_w, xv.dim_h, xv.dim_n};
+        cuuint64_t strides[3] = {xv.stride_w, xv.stride_h, xv.stride_n};
+        cuuint32_t box[4] = {(cuuint32_t)p.kb, (cuuint32_t)p.win_wp, (cuuint32_t)(p.win_r + 2), 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        CUresult r = g_encode_tiled(&plan->map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(xv.base), dims, strides,
+                                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(p.kb),
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            *why = "cuTensorMapEncodeTiled rejected the activation tensor";
+            return cudaErrorInvalidValue;
+        }
+    } else
     // A: activation tensor (C, W, H, N) in im2col mode.  Corners follow the usual forward-convolution
     // rule: lower = -pad, upper = pad - (k - 1); the traversal stride is the convolution stride.
     {
@@ -1069,7 +967,27 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // output / residual [M, c_out] bytes, one box = one column slab of a tile
     plan->map_y = plan->map_b;
     plan->map_r = plan->map_b;
-    if (staged) {
+    if (staged && p.win) {
+        // output / residual as (C_out, W, H, N); one box = one column slab of win_r rows of W + 2 positions
+        cuuint64_t dims[4] = {(cuuint64_t)g.c_out, (cuuint64_t)g.wo, (cuuint64_t)g.ho, (cuuint64_t)g.n};
+        cuuint64_t strides[3] = {(cuuint64_t)g.c_out, (cuuint64_t)g.c_out * g.wo, (cuuint64_t)g.c_out * g.wo * g.ho};
+        cuuint32_t box[4] = {(cuuint32_t)p.slab_w, (cuuint32_t)p.win_wp, (cuuint32_t)p.win_r, 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        const CUtensorMapSwizzle sw = p.slab_w == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                      : (p.slab_w == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                         : (p.slab_w == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE));
+        CUresult r = g_encode_tiled(&plan->map_y, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, y, dims, strides, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r == CUDA_SUCCESS && q.has_res)
+            r = g_encode_tiled(&plan->map_r, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(res), dims, strides, box,
+                               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            *why = "cuTensorMapEncodeTiled rejected the output tensor";
+            return cudaErrorInvalidValue;
+        }
+    } else if (staged) {
         cuuint64_t dims[2] = {(cuuint64_t)g.c_out, (cuuint64_t)p.M};
         cuuint64_t strides[1] = {(cuuint64_t)g.c_out};
         cuuint32_t box[2] = {(cuuint32_t)p.slab_w, (cuuint32_t)TILE_M};

@@ -71,10 +71,20 @@ size_t f8_tc_plan_size();
 cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant &q, const F8TcTensorView &xv,
                             const int8_t *w /* [c_out][kh][kw][g.c] */, const int32_t *bias, const void *res,
                             void *y, int *status_word, const char **why);
+// Label reported (with the wait's site) when a bounded wait of this launch gives up; 0 = none.
+void f8_tc_plan_set_tag(F8TcPlan *plan, int tag);
 // overlap_previous: the grid may start before the preceding work of the stream has finished; only its weight
 // and bias reads then run early, so it is for callers whose weights no earlier work in the stream writes.
 cudaError_t f8_tc_launch(const F8TcPlan *plan, bool overlap_previous, cudaStream_t st);
 cudaError_t f8_tc_probe(int iters, double *ops, int *status_word, cudaStream_t st);
+
+// ---- first-layer kernel (f8_stem_tc.cu): stride-2 convolution over an image with <= 4 channels, optionally fused
+// with the 3x3 / 2 / pad 1 max pool behind it.  kh2 row pairs per window starting `top` pairs above the output row,
+// `left` zero cells in front of a row, `slices` 32-byte K slices per row pair; w_core is [K / 16][c_out][16].
+bool f8_stem_tc_supported(const F8ConvGeom &g, const F8Requant &q, int kh2, int slices);
+cudaError_t f8_launch_stem_tc(const F8ConvGeom &g, const F8Requant &q, int kh2, int top, int left, int slices, int pool,
+                              const void *x, const int8_t *w_core, const int32_t *bias, void *y, int *status_word, int tag,
+                              cudaStream_t st, bool overlap_previous);
 
 // Device status word (0 = fine); allocated once per process on first use.
 int *f8_status_word();
