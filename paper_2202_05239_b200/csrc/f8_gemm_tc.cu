@@ -791,6 +791,14 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     const bool staged = p.epi != EPI_GENERIC;
     p.bn = staged ? choose_bn_staged(g.c_out, q.has_res != 0, p.kb) : choose_bn(g.c_out);
     p.m_tiles = (p.M + TILE_M - 1) / TILE_M;
+    if (!staged) {
+        // few output pixels (a fully connected layer): narrower N tiles until every SM has one, the weights are
+        // what has to be streamed and each CTA then streams its own slice of them
+        int sm_count = 148, dev0 = 0;
+        cudaGetDevice(&dev0);
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev0);
+        while (p.bn > 32 && p.bn % 32 == 0 && (long long)p.m_tiles * ((g.c_out + p.bn - 1) / p.bn) < sm_count) p.bn /= 2;
+    }
     p.n_tiles = (g.c_out + p.bn - 1) / p.bn;
     p.div_n_tiles = make_fast_div(p.n_tiles);
     p.div_wo = make_fast_div(g.wo);
@@ -814,7 +822,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         // about as long to arrive from HBM as a tile takes to compute: three buffers (four when they are small).
         p.out_bufs = !q.has_res ? 2 : (p.out_bytes <= 16 * 1024 ? 4 : 3);
         if (getenv("F8_OUT_BUFS")) p.out_bufs = atoi(getenv("F8_OUT_BUFS"));
-        if (p.out_bufs < 2) p.out_bufs = 2;
+        if (p.out_bufs < 1) p.out_bufs = 1;
         if (p.out_bufs > MAX_OUT_BUFS) p.out_bufs = MAX_OUT_BUFS;
         staging = (size_t)p.out_bytes * p.out_bufs + bias_bytes;
     }
@@ -829,9 +837,11 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // lane per load remain; measured, fewer and larger stage uses beat a deeper ring of small ones
     const int k_iters = g.kh * g.kw * p.c_chunks;
     size_t avail = SMEM_LIMIT - 1024 - staging;
-    // resident weights: one N tile, and at least 32 KiB left for the activation pipeline
+    // resident weights: one N tile, and room left for at least four activation tiles in flight (with only two, a
+    // 3x3 layer of 128 channels waits on every im2col load: measured 62 us against 48 us with streamed weights)
     const size_t b_all = (size_t)p.n_tiles * k_iters * b_bytes;
-    p.b_res = (p.n_tiles == 1 && b_all + 32 * 1024 <= avail && !getenv("F8_NO_BRES")) ? 1 : 0;
+    p.b_res = (p.n_tiles == 1 && b_all + 4 * (size_t)p.a_bytes <= avail && b_all + 32 * 1024 <= avail &&
+               !getenv("F8_NO_BRES")) ? 1 : 0;
     if (p.b_res) {
         avail -= b_all;
         p.sub_bytes = p.a_bytes;

@@ -34,6 +34,11 @@ TC_CASES = [
     (33, 20, 16, 96, 1, 1, 0, 13, True, synth.U8, False),      # c = 16: half-empty 32-byte K chunk
     (20, 20, 64, 32, 5, 1, 2, 6, False, synth.U8, False),      # 5x5
     (31, 31, 64, 64, 3, 2, 0, 3, False, synth.U8, False),      # stride 2 without padding
+    (28, 28, 128, 128, 3, 1, 1, 2, False, synth.U8, False),    # windowed 3x3: four whole rows per tile
+    (28, 28, 128, 128, 3, 1, 1, 3, True, synth.S8, True),      # windowed 3x3 with residual, signed in / out
+    (30, 22, 128, 64, 3, 1, 1, 5, False, synth.U8, False),     # windowed 3x3: five rows of 24 positions, six bands
+    (14, 14, 128, 128, 3, 1, 1, 9, False, synth.U8, True),     # windowed 3x3: second band of an image is partial
+    (12, 40, 256, 32, 3, 1, 1, 3, True, synth.U8, False),      # windowed 3x3 with two channel chunks
 ]
 
 
