@@ -249,7 +249,28 @@ def run_ours(args):
         ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
         return ms, (sampler.stop() if rank == 0 else None)
 
+    incidents = []
+
+    def device_ok(where: str) -> bool:
+        """Reads the device status word; a kernel that gave up a bounded wait is recorded, not fatal the first time."""
+        try:
+            api.f8_device_status()
+            return True
+        except api.F8Error as exc:
+            incidents.append(f"{where}: {exc}")
+            if len(incidents) > 2:
+                raise
+            return False
+
+    def on_any_rank(flag: bool) -> bool:
+        """The ranks repeat a measurement together or not at all (it contains barriers)."""
+        return max_over_ranks(1.0 if flag else 0.0, world, dev) > 0.0
+
     elapsed_ms, clocks = timed_steps()
+    if on_any_rank(not device_ok("timed steps")):
+        elapsed_ms, clocks = timed_steps()      # that measurement contained a 2 s time-out: take it again
+        if on_any_rank(not device_ok("timed steps, second run")):
+            raise SystemExit("bench.py: bounded waits timed out twice: " + "; ".join(incidents))
     if rank == 0:
         throttled = bool(set(clocks["reasons"]) & {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"})
         stuck = (clocks["sm_mhz"] is not None and not clocks["reasons"] and clocks["sm_mhz"] < 0.8 * clocks["sm_max_mhz"])
@@ -276,16 +297,25 @@ def run_ours(args):
         pipe.submit(x_hosts[i & 1], out_hosts[i & 1])
     pipe.wait()
     torch.cuda.synchronize()
-    barrier(world)
+    device_ok("end-to-end warm-up")
     t_e0, t_e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_e0.record(pipe.up_stream)                  # before the first upload ...
-    for i in range(args.steps):
-        pipe.submit(x_hosts[i & 1], out_hosts[i & 1])
-    t_e1.record(pipe.down_stream)                # ... to after the last download
-    pipe.wait()
-    torch.cuda.synchronize()
-    barrier(world)
-    e2e_ms = max_over_ranks(t_e0.elapsed_time(t_e1), world, dev)
+
+    def timed_e2e():
+        barrier(world)
+        t_e0.record(pipe.up_stream)                  # before the first upload ...
+        for i in range(args.steps):
+            pipe.submit(x_hosts[i & 1], out_hosts[i & 1])
+        t_e1.record(pipe.down_stream)                # ... to after the last download
+        pipe.wait()
+        torch.cuda.synchronize()
+        barrier(world)
+        return max_over_ranks(t_e0.elapsed_time(t_e1), world, dev)
+
+    e2e_ms = timed_e2e()
+    if on_any_rank(not device_ok("end-to-end steps")):
+        e2e_ms = timed_e2e()
+        if on_any_rank(not device_ok("end-to-end steps, second run")):
+            raise SystemExit("bench.py: bounded waits timed out twice: " + "; ".join(incidents))
     e2e_value = whole_job_rate(BATCH, args.steps, world, e2e_ms)
     e2e_ok = bool(torch.equal(out_hosts[0], out.cpu()))      # same images as the device-resident run: same logits
     pipe.close()
@@ -312,7 +342,7 @@ def run_ours(args):
     e1.record(stream)
     torch.cuda.synchronize()
     probe_tops = ops / (e0.elapsed_time(e1) * 1e-3) / 1e12
-    api.f8_device_status()
+    device_ok("per-layer timing and probe")
 
     if rank != 0:
         return
@@ -378,6 +408,8 @@ def run_ours(args):
                     "logits_match_device_run": e2e_ok},
             "gpu_launches": int(launches),
             "roofline": roofline}
+    if incidents:
+        line["incidents"] = incidents       # bounded waits that gave up (each costs 2 s); the affected measurement was repeated
     if world == 1:
         line["cpu_baseline"] = cpu_baseline(layers)
     if args.layers:
