@@ -326,6 +326,7 @@ struct f8_net {
     std::vector<NetLayer> layers;
     std::vector<int> t_h, t_w, t_c, t_elem;     // per tensor: per-image shape and element size
     bool overlap_layers = getenv("F8NET_NO_OVERLAP") == nullptr;   // programmatic dependent launch between layers
+    bool sync_layers = getenv("F8NET_SYNC_LAYERS") != nullptr;     // synchronize after every launch (fault attribution)
     std::vector<int> t_cp;                       // per tensor: channels as stored (intermediate 8-bit tensors are padded
                                                  // to a multiple of 16 so that every dense layer can use the TMA path)
     int max_batch = 0;
@@ -795,7 +796,11 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                 e = f8_launch_gap(batch, L.g.h, L.g.w, L.g.c, L.g.x_signed, L.q.s, stp.x, stp.y, st, net->overlap_layers);
                 break;
         }
-        if (e != cudaSuccess) return cuda_fail(e, "layer launch");
+        if (e != cudaSuccess) return fail(F8_ERR_CUDA, "launch of layer %d: %s", stp.layer, cudaGetErrorString(e));
+        if (net->sync_layers) {     // debugging aid: a device-side fault is then reported with the layer that raised it
+            e = cudaStreamSynchronize(st);
+            if (e != cudaSuccess) return fail(F8_ERR_CUDA, "layer %d failed on the device: %s", stp.layer, cudaGetErrorString(e));
+        }
         ++launches;
         if (prof) {
             cudaEventRecord(net->events[launches], st);

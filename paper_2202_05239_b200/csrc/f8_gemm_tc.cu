@@ -55,6 +55,7 @@ constexpr int MAX_STAGES = 16;
 constexpr int MAX_OUT_BUFS = 4;             // ring of staged output tiles; with a residual, the residual tile lands in the
                                             // buffer first and the epilogue converts it in place
 constexpr int TMEM_COLS = 512;
+constexpr int MAX_ACC = 8;                  // accumulators of 64 columns; 4 of 128 or 2 of 256 for wider tiles
 constexpr size_t SMEM_LIMIT = 220 * 1024;     // dynamic shared memory budget (227 KiB per CTA minus static data)
 
 // Division by a run-time constant without a divide instruction (a 32-bit divide costs a lone thread well over a
@@ -80,6 +81,7 @@ struct TcParams {
     int group;                // k-iterations per stage (1..8)
     int uses;                 // stage uses per tile: ceil(k_iters / group)
     int dual_issue;           // 1: two MMA-issuing threads (needs stages >= 2 * uses)
+    int acc_log2;             // accumulators in tensor memory: 2, 4 or 8 (1 << acc_log2), 512 / count columns apart
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
     uint32_t stage_bytes;     // group * sub_bytes
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
@@ -187,7 +189,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     extern __shared__ uint8_t smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 5];
+    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 2 * MAX_ACC + 1];
     __shared__ __align__(8) uint64_t epi_bars[3 * MAX_OUT_BUFS];   // out_full[], out_free[], res_full[]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -197,8 +199,8 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const uint32_t full_bar = smem_u32(&bars[0]);
     const uint32_t empty_bar = smem_u32(&bars[MAX_STAGES]);
     const uint32_t tfull_bar = smem_u32(&bars[2 * MAX_STAGES]);
-    const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + 2]);
-    const uint32_t bres_bar = smem_u32(&bars[2 * MAX_STAGES + 4]);   // resident weights have landed
+    const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + MAX_ACC]);
+    const uint32_t bres_bar = smem_u32(&bars[2 * MAX_STAGES + 2 * MAX_ACC]);   // resident weights have landed
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t out_full = smem_u32(&epi_bars[0]), out_free = smem_u32(&epi_bars[MAX_OUT_BUFS]);
     const uint32_t res_full = smem_u32(&epi_bars[2 * MAX_OUT_BUFS]);
@@ -210,7 +212,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             mbar_init(empty_bar + 8 * s, 1);
         }
         mbar_init(bres_bar, 1);
-        for (int a = 0; a < 2; ++a) {
+        for (int a = 0; a < MAX_ACC; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
             mbar_init(tempty_bar + 8 * a, NUM_EPI_WARPS);
         }
@@ -395,18 +397,17 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             if (p.b_res && !mbar_wait(bres_bar, 0, abortp, p.status, tagbits | 111)) ok = false;
             const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
-                const int acc = local & 1;
-                if (p.dual_issue && acc != q_issuer) {
+                const int acc = local & ((1 << p.acc_log2) - 1);
+                if (p.dual_issue && (local & 1) != q_issuer) {
                     // the other issuer's tile: step over its stage uses
                     stage += p.uses;
                     while (stage >= p.stages) { stage -= p.stages; phase ^= 1; }
                     stage_lo = desc_lo0 + (uint32_t)stage * stage16;
                     continue;
                 }
-                const uint32_t acc_phase = (local >> 1) & 1;
+                const uint32_t acc_phase = (local >> p.acc_log2) & 1;
                 if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, abortp, p.status, tagbits | 102)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * 256;   // two 256-column accumulators
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * (TMEM_COLS >> p.acc_log2);
                 uint32_t b_tile_lo = 0;
                 if (p.b_res) {
                     const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
@@ -561,12 +562,12 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 so[i] = (uint32_t)(ch / p.slab_chunks) * (TILE_M * p.slab_w) + off;
             }
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
-                const int acc = local & 1;                   // accumulator, output buffer and residual buffer in use
-                const uint32_t acc_phase = (local >> 1) & 1;
+                const int acc = local & ((1 << p.acc_log2) - 1);
+                const uint32_t acc_phase = (local >> p.acc_log2) & 1;
                 const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
                 const int c_first = n_t * p.bn + ch_begin * 16;
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
-                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * (TMEM_COLS >> p.acc_log2) + ch_begin * 16;
                 bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, tagbits | 104);
                 // the buffer holds the residual tile (which implies that its previous store has left), or is free
                 if (RES) got = mbar_wait(res_full + 8 * ob, ophase, abortp, p.status, tagbits | 107) && got;
@@ -610,13 +611,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             grid_dependency_wait();     // direct stores (and residual reads) from these warps
             const int tile_row = quarter * 32 + lane;   // this thread's row of the tile
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
-                const int acc = local & 1;
-                const uint32_t acc_phase = (local >> 1) & 1;
+                const int acc = local & ((1 << p.acc_log2) - 1);
+                const uint32_t acc_phase = (local >> p.acc_log2) & 1;
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
                 const int n0 = n_t * p.bn;
                 const size_t row = (size_t)m_t * TILE_M + tile_row;
                 const bool row_valid = row < (size_t)p.M;
-                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * (TMEM_COLS >> p.acc_log2) + ch_begin * 16;
                 if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, tagbits | 104))) { ok = false; break; }
                 tc_fence_after();
                 for (int i = 0; i < nch; ++i) {
@@ -909,6 +910,12 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     }
     const int stages = p.stages;
     p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !getenv("F8_NO_DUAL")) ? 1 : 0;
+    // Narrow tiles leave room for more accumulators.  The chain "accumulator free -> issue -> commit -> epilogue ->
+    // accumulator free" costs about 2500 cycles whatever the tile (per-role timestamps), and only more tiles in flight
+    // hide it: 8 accumulators of 64 columns, 4 of 128, else 2 of 256.
+    p.acc_log2 = p.bn <= 64 ? 3 : (p.bn <= 128 ? 2 : 1);
+    if (getenv("F8_ACC_LOG2")) p.acc_log2 = std::max(1, std::min(3, atoi(getenv("F8_ACC_LOG2"))));
+    if ((TMEM_COLS >> p.acc_log2) < p.bn) p.acc_log2 = 1;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
     p.bias_off = p.out_off + (uint32_t)p.out_bufs * p.out_bytes;
     p.ktab_off = (uint32_t)(p.stages * p.stage_bytes + staging - ktab_bytes);
