@@ -170,6 +170,41 @@ f8_status f8_net_get_layer_ms(f8_net *net, float *ms, int *on_tensor_cores);
 
 void f8_net_destroy(f8_net *net);
 
+/* ---------------------------------------------------------------- weight compile step */
+
+/* One Conv-BN block's parameters turned into what the layer entry points above consume (Sec. 4.2 - 4.3):
+ *
+ *     W_eff[i, j] = (gamma_i / sigma_i) * (eta_in / eta_out) * W[i, j]         effective weight, Eq. 6
+ *     b_eff[i]    = (beta_i - (gamma_i / sigma_i) * mu_i) / eta_out             effective bias, Eq. 6
+ *     FL_w        = floor(log2(40 / std(W_eff))), clamped to [fl_w_min, fl_w_max]   Eq. 1, signed branch
+ *     w_q         = round(clip(W_eff * 2^FL_w, -127, 127))                      signed fix_quant (appendix), WL = 8
+ *     bias_q      = round(b_eff * 2^(fl_x + FL_w)), saturated to int32          accumulator format
+ *
+ * gamma, beta: BatchNorm weight and bias; sigma, mu: its running standard deviation and mean (sigma is the
+ * standard deviation itself, already including any epsilon); eta_in / eta_out: the fix scaling factors of Eq. 5,
+ * eta_fix = 2^FL * alpha / 255, of this block's input quantiser and of the next block's.  std is the population
+ * standard deviation over the whole tensor; round is round half up.  All arithmetic is float64 with one IEEE
+ * operation per step in the order written, so the integer codes are reproducible.
+ *
+ * w [c_out, k] fp32 (k = kh * kw * c_in in the layout the convolution will use, e.g. OHWI), gamma / sigma /
+ * beta / mu [c_out] fp32, w_q [c_out, k] int8, bias_q [c_out] int32, fl_w one int -- all DEVICE pointers; the
+ * chosen fractional length is written to *fl_w on the device (read it back after the stream has finished).
+ * workspace: at least f8_fold_workspace_bytes() bytes of device memory, 8-byte aligned; its contents need not be
+ * initialised and are overwritten.  Three kernels are enqueued on the stream; nothing is synchronised.
+ * Errors: F8_ERR_NULL, F8_ERR_SHAPE (extents, non-positive eta), F8_ERR_FL_RANGE, F8_ERR_WORKSPACE,
+ * F8_ERR_ALIGN; nothing is launched when validation fails. */
+typedef struct {
+    int c_out, k;
+    int fl_x;                   /* fractional length of the block's input activations, 0..8 */
+    int fl_w_min, fl_w_max;     /* accepted range of the weight format, inside [-8, 24] (the paper: 0..7) */
+    double eta_in, eta_out;
+} f8_fold_desc;
+
+size_t f8_fold_workspace_bytes(const f8_fold_desc *desc);
+f8_status f8_fold_quantize_fixed(const f8_fold_desc *desc, const float *w, const float *gamma, const float *sigma,
+                                 const float *beta, const float *mu, int8_t *w_q, int32_t *bias_q, int *fl_w,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* ---------------------------------------------------------------- diagnostics */
 
 const char *f8_status_str(f8_status s);

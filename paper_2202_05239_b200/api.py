@@ -150,6 +150,27 @@ def f8_stem_conv2d_fixed_static(desc: ConvDesc, x, w, bias, y, check_previous: b
                                             1 if check_previous else 0, _stream(stream)))
 
 
+class FoldDesc(ctypes.Structure):
+    _fields_ = [("c_out", ctypes.c_int), ("k", ctypes.c_int), ("fl_x", ctypes.c_int), ("fl_w_min", ctypes.c_int),
+                ("fl_w_max", ctypes.c_int), ("eta_in", ctypes.c_double), ("eta_out", ctypes.c_double)]
+
+
+_lib.f8_fold_workspace_bytes.argtypes = [ctypes.POINTER(FoldDesc)]
+_lib.f8_fold_workspace_bytes.restype = _sz
+_lib.f8_fold_quantize_fixed.argtypes = [ctypes.POINTER(FoldDesc)] + [_vp] * 9 + [_sz, _vp]
+
+
+def f8_fold_workspace_bytes(desc: FoldDesc) -> int:
+    return int(_lib.f8_fold_workspace_bytes(ctypes.byref(desc)))
+
+
+def f8_fold_quantize_fixed(desc: FoldDesc, w, gamma, sigma, beta, mu, w_q, bias_q, fl_w, workspace, stream=None):
+    """Eq. 6 + Eq. 1 + signed quantiser for one Conv-BN block; every tensor on the device, fl_w a 1-element int32."""
+    _check(_lib.f8_fold_quantize_fixed(ctypes.byref(desc), _ptr(w), _ptr(gamma), _ptr(sigma), _ptr(beta), _ptr(mu),
+                                       _ptr(w_q), _ptr(bias_q), _ptr(fl_w), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
 def f8_conv_workspace_bytes(desc: ConvDesc) -> int:
     return int(_lib.f8_conv_workspace_bytes(ctypes.byref(desc)))
 
@@ -179,7 +200,7 @@ def exported_symbols() -> List[str]:
     return ["f8_conv2d_fixed", "f8_dwconv_fixed", "f8_linear_fixed", "f8_maxpool_fixed", "f8_global_avgpool_fixed",
             "f8_conv_workspace_bytes", "f8_net_create", "f8_net_workspace_bytes", "f8_net_forward",
             "f8_net_last_launch_count", "f8_net_set_profiling", "f8_net_get_layer_ms", "f8_net_destroy", "f8_status_str", "f8_last_error", "f8_device_status",
-            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static"]
+            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static", "f8_fold_quantize_fixed", "f8_fold_workspace_bytes"]
 
 
 def run_layer(layer: "synth.Layer", x: torch.Tensor, residual: Optional[torch.Tensor] = None, params=None,

@@ -106,8 +106,36 @@ def bench_net(name: str, batch: int, iters: int, warmup: int):
                       "launches": net.last_launch_count}), flush=True)
 
 
+def bench_fold(c_out: int, k: int, iters: int, warmup: int):
+    """Device time of the weight compile step (f8_fold_quantize_fixed) on one [c_out, k] fp32 tensor.  Algorithmic
+    bytes: 4 read + 1 written per weight (the fp32 tensor has to be read twice -- statistics, then quantisation --
+    unless it stays in L2, so DRAM traffic can be up to 9 bytes per weight)."""
+    rng = np.random.default_rng(2)
+    d = api.FoldDesc(c_out, k, 5, 0, 24, 0.11, 0.07)
+    w = torch.from_numpy(rng.normal(0, 0.05, (c_out, k)).astype(np.float32)).cuda()
+    vec = [torch.from_numpy(rng.uniform(0.5, 1.5, c_out).astype(np.float32)).cuda() for _ in range(4)]
+    w_q = torch.empty((c_out, k), dtype=torch.int8, device="cuda")
+    b_q = torch.empty(c_out, dtype=torch.int32, device="cuda")
+    fl = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(api.f8_fold_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+    for _ in range(warmup):
+        api.f8_fold_quantize_fixed(d, w, *vec, w_q, b_q, fl, ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        api.f8_fold_quantize_fixed(d, w, *vec, w_q, b_q, fl, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    n = c_out * k
+    print(json.dumps({"op": "fold_quantize", "c_out": c_out, "k": k, "ms": ms, "fl_w": int(fl.item()),
+                      "algorithmic_gbs": 5.0 * n / (ms * 1e-3) / 1e9, "weights_per_s": n / (ms * 1e-3)}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--fold", action="store_true", help="time the weight compile step on a [c-out, k * k * c] tensor")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--net", default="", help="time every layer of a synthetic network: resnet18, resnet50, mobilenetv2")
     ap.add_argument("--h", type=int, default=56)
@@ -123,6 +151,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--warm-l2", action="store_true", help="reuse one buffer set (operands stay in L2)")
     args = ap.parse_args()
+    if args.fold:
+        bench_fold(args.c_out, args.k * args.k * args.c, args.iters, args.warmup)
+        return
     if args.net:
         bench_net(args.net, args.batch, args.iters, args.warmup)
     elif args.sweep:

@@ -93,3 +93,27 @@ def test_net_create_validates_graph_and_accumulator_bound(lib):
     with pytest.raises(api.F8Error) as e:
         api.Net(layers, 1)
     assert e.value.status == 7
+
+
+@pytest.mark.parametrize("kw,status", [
+    (dict(c_out=0), 2), (dict(k=-3), 2), (dict(fl_x=9), 4), (dict(fl_w_min=5, fl_w_max=4), 4), (dict(fl_w_max=30), 4),
+    (dict(eta_out=0.0), 2), (dict(eta_in=float("nan")), 2),
+])
+def test_fold_validation_rejects_without_launching(lib, kw, status):
+    from paper_2202_05239_b200 import api
+    base = dict(c_out=8, k=16, fl_x=4, fl_w_min=0, fl_w_max=7, eta_in=0.5, eta_out=0.25)
+    base.update(kw)
+    d = api.FoldDesc(**base)
+    fake = ctypes.c_void_p(0x1000)       # never dereferenced: validation fails first
+    st = api._lib.f8_fold_quantize_fixed(ctypes.byref(d), *([fake] * 9), 1 << 20, None)
+    assert st == status, api._lib.f8_last_error()
+
+
+def test_fold_workspace_and_null_are_reported(lib):
+    from paper_2202_05239_b200 import api
+    d = api.FoldDesc(8, 16, 4, 0, 7, 0.5, 0.25)
+    fake = ctypes.c_void_p(0x1000)
+    assert api._lib.f8_fold_quantize_fixed(ctypes.byref(d), *([fake] * 8), None, 0, None) == 8
+    assert api._lib.f8_fold_quantize_fixed(ctypes.byref(d), *([fake] * 9), 16, None) == 8
+    assert api._lib.f8_fold_quantize_fixed(ctypes.byref(d), None, *([fake] * 8), 1 << 20, None) == 1
+    assert api._lib.f8_fold_workspace_bytes(ctypes.byref(d)) >= 16384
