@@ -190,7 +190,7 @@ void f8_net_destroy(f8_net *net);
  * beta / mu [c_out] fp32, w_q [c_out, k] int8, bias_q [c_out] int32, fl_w one int -- all DEVICE pointers; the
  * chosen fractional length is written to *fl_w on the device (read it back after the stream has finished).
  * workspace: at least f8_fold_workspace_bytes() bytes of device memory, 8-byte aligned; its contents need not be
- * initialised and are overwritten.  Three kernels are enqueued on the stream; nothing is synchronised.
+ * initialised and are overwritten.  Four kernels are enqueued on the stream; nothing is synchronised.
  * Errors: F8_ERR_NULL, F8_ERR_SHAPE (extents, non-positive eta), F8_ERR_FL_RANGE, F8_ERR_WORKSPACE,
  * F8_ERR_ALIGN; nothing is launched when validation fails. */
 typedef struct {

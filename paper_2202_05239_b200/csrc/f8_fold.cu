@@ -13,7 +13,7 @@
 // powers of two is exact, and floor(log2(r)) is taken from the exponent of r.  Only the summation order of the
 // variance is free; it is fixed too (per-block partial sums reduced in index order), so results are reproducible.
 //
-// The work is three small launches: partial sums -> format and bias -> quantised weights.  It is bound by memory
+// The work is four small launches: row scales -> partial sums -> format and bias -> quantised weights.  It is bound by memory
 // traffic: the fp32 weights are read twice and one byte per weight is written.
 #include <math.h>
 
@@ -22,7 +22,7 @@
 namespace {
 
 constexpr int FOLD_THREADS = 256;
-constexpr int FOLD_CHUNK = 2048;         // weights of one row handled by one block iteration
+constexpr int FOLD_CHUNK = 4096;         // weights of one row handled by one block iteration
 constexpr int FOLD_MAX_BLOCKS = 1024;
 
 struct FoldParams {
@@ -32,16 +32,21 @@ struct FoldParams {
     double ratio;                         // eta_in / eta_out
     double eta_out;
     int fl_x, fl_min, fl_max;
+    int vec4;                             // k % 4 == 0 and w 16-byte, w_q 4-byte aligned: four weights per thread and access
     const float *w, *gamma, *sigma, *beta, *mu;
     int8_t *w_q;
     int32_t *b_q;
     int *fl_w;
     double *partial;                      // [blocks][2], then [2]: mean, std
+    double *scale;                        // [c_out]: (gamma / sigma) * ratio, written by the first launch
 };
 
-__device__ __forceinline__ double row_scale(const FoldParams &p, int row) {
-    return __dmul_rn(__ddiv_rn((double)__ldg(p.gamma + row), (double)__ldg(p.sigma + row)), p.ratio);
+__global__ void __launch_bounds__(FOLD_THREADS) fold_scale_kernel(const FoldParams p) {
+    const int i = blockIdx.x * FOLD_THREADS + threadIdx.x;
+    if (i < p.c_out) p.scale[i] = __dmul_rn(__ddiv_rn((double)__ldg(p.gamma + i), (double)__ldg(p.sigma + i)), p.ratio);
 }
+
+__device__ __forceinline__ double row_scale(const FoldParams &p, int row) { return p.scale[row]; }
 
 __global__ void __launch_bounds__(FOLD_THREADS) fold_stats_kernel(const FoldParams p) {
     double s1 = 0.0, s2 = 0.0;
@@ -50,6 +55,15 @@ __global__ void __launch_bounds__(FOLD_THREADS) fold_stats_kernel(const FoldPara
         const double sc = row_scale(p, row);
         const float *wr = p.w + (size_t)row * p.k;
         const int j1 = min(p.k, (chunk + 1) * FOLD_CHUNK);
+        if (p.vec4) {       // rows are multiples of four weights and 16-byte aligned: one 16-byte load per thread
+            for (int j = chunk * FOLD_CHUNK + 4 * threadIdx.x; j < j1; j += 4 * FOLD_THREADS) {
+                const float4 f = __ldg((const float4 *)(wr + j));
+                const double v0 = __dmul_rn(sc, (double)f.x), v1 = __dmul_rn(sc, (double)f.y);
+                const double v2 = __dmul_rn(sc, (double)f.z), v3 = __dmul_rn(sc, (double)f.w);
+                s1 += (v0 + v1) + (v2 + v3);
+                s2 += (v0 * v0 + v1 * v1) + (v2 * v2 + v3 * v3);
+            }
+        } else
         for (int j = chunk * FOLD_CHUNK + threadIdx.x; j < j1; j += FOLD_THREADS) {
             const double v = __dmul_rn(sc, (double)__ldg(wr + j));
             s1 += v;
@@ -122,14 +136,29 @@ __global__ void __launch_bounds__(FOLD_THREADS) fold_format_kernel(const FoldPar
 
 __global__ void __launch_bounds__(FOLD_THREADS) fold_quant_kernel(const FoldParams p) {
     const int fl = *p.fl_w;
+    const double pow2 = scalbn(1.0, fl);          // multiplying by a power of two is exact
     for (long long item = blockIdx.x; item < p.items; item += gridDim.x) {
         const int row = (int)(item / p.chunks_per_row), chunk = (int)(item - (long long)row * p.chunks_per_row);
         const double sc = row_scale(p, row);
         const float *wr = p.w + (size_t)row * p.k;
         int8_t *qr = p.w_q + (size_t)row * p.k;
         const int j1 = min(p.k, (chunk + 1) * FOLD_CHUNK);
+        if (p.vec4) {
+            for (int j = chunk * FOLD_CHUNK + 4 * threadIdx.x; j < j1; j += 4 * FOLD_THREADS) {
+                const float4 f = __ldg((const float4 *)(wr + j));
+                const float in[4] = {f.x, f.y, f.z, f.w};
+                uint32_t packed = 0;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const double v = __dmul_rn(__dmul_rn(sc, (double)in[t]), pow2);
+                    const int q = (int)floor(__dadd_rn(fmin(fmax(v, -127.0), 127.0), 0.5));
+                    packed |= (uint32_t)(q & 0xff) << (8 * t);
+                }
+                *(uint32_t *)(qr + j) = packed;
+            }
+        } else
         for (int j = chunk * FOLD_CHUNK + threadIdx.x; j < j1; j += FOLD_THREADS) {
-            const double v = scalbn(__dmul_rn(sc, (double)__ldg(wr + j)), fl);
+            const double v = __dmul_rn(__dmul_rn(sc, (double)__ldg(wr + j)), pow2);
             qr[j] = (int8_t)(int)floor(__dadd_rn(fmin(fmax(v, -127.0), 127.0), 0.5));
         }
     }
@@ -141,7 +170,9 @@ int fold_blocks(long long items) { return (int)std::min<long long>(items, FOLD_M
 
 extern "C" {
 
-size_t f8_fold_workspace_bytes(const f8_fold_desc *) { return (size_t)(2 * FOLD_MAX_BLOCKS + 2) * sizeof(double); }
+size_t f8_fold_workspace_bytes(const f8_fold_desc *d) {
+    return (size_t)(2 * FOLD_MAX_BLOCKS + 2 + (d && d->c_out > 0 ? d->c_out : 0)) * sizeof(double);
+}
 
 f8_status f8_fold_quantize_fixed(const f8_fold_desc *d, const float *w, const float *gamma, const float *sigma,
                                  const float *beta, const float *mu, int8_t *w_q, int32_t *bias_q, int *fl_w,
@@ -162,10 +193,13 @@ f8_status f8_fold_quantize_fixed(const f8_fold_desc *d, const float *w, const fl
     p.ratio = d->eta_in / d->eta_out;
     p.eta_out = d->eta_out;
     p.fl_x = d->fl_x; p.fl_min = d->fl_w_min; p.fl_max = d->fl_w_max;
+    p.vec4 = (d->k % 4 == 0 && ((uintptr_t)w & 15) == 0 && ((uintptr_t)w_q & 3) == 0) ? 1 : 0;
     p.w = w; p.gamma = gamma; p.sigma = sigma; p.beta = beta; p.mu = mu;
     p.w_q = w_q; p.b_q = bias_q; p.fl_w = fl_w; p.partial = (double *)workspace;
+    p.scale = p.partial + 2 * FOLD_MAX_BLOCKS + 2;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int blocks = fold_blocks(p.items);
+    fold_scale_kernel<<<(d->c_out + FOLD_THREADS - 1) / FOLD_THREADS, FOLD_THREADS, 0, st>>>(p);
     fold_stats_kernel<<<blocks, FOLD_THREADS, 0, st>>>(p);
     fold_format_kernel<<<1, FOLD_THREADS, 0, st>>>(p, blocks);
     fold_quant_kernel<<<blocks, FOLD_THREADS, 0, st>>>(p);
