@@ -205,6 +205,20 @@ f8_status f8_fold_quantize_fixed(const f8_fold_desc *desc, const float *w, const
                                  const float *beta, const float *mu, int8_t *w_q, int32_t *bias_q, int *fl_w,
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* ---------------------------------------------------------------- statistical study of the formats */
+
+/* The experiment of Sec. 3.3 (Fig. 2, Fig. 3; appendix "More Details for Statistical Analysis") on a caller-given
+ * sample x [n] fp32 (DEVICE): relative quantisation error  err[FL] = sum (q_FL(x') - x')^2 / sum x'^2  for every
+ * 8-bit format -- unsigned, Eq. 2, FL = 0..8, with x' = max(x, 0) (the sample "processed by ReLU"), or signed
+ * (appendix), FL = 0..7, x' = x -- and the format with the smallest error (the smaller FL on a tie), which Eq. 1
+ * approximates from the standard deviation.  err: 9 doubles on the DEVICE (err[8] = -1 for the signed study),
+ * best_fl: one int on the DEVICE.  float64 arithmetic, fixed summation order.  workspace: at least
+ * f8_format_study_workspace_bytes() bytes of device memory, 8-byte aligned, contents irrelevant.  Two kernels are
+ * enqueued; nothing is synchronised.  Errors: F8_ERR_NULL, F8_ERR_SHAPE (n <= 0), F8_ERR_WORKSPACE, F8_ERR_ALIGN. */
+size_t f8_format_study_workspace_bytes(void);
+f8_status f8_format_study_fixed(const float *x, long long n, int is_unsigned, double *err, int *best_fl,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* ---------------------------------------------------------------- diagnostics */
 
 const char *f8_status_str(f8_status s);

@@ -171,6 +171,20 @@ def f8_fold_quantize_fixed(desc: FoldDesc, w, gamma, sigma, beta, mu, w_q, bias_
                                        workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
+_lib.f8_format_study_workspace_bytes.restype = _sz
+_lib.f8_format_study_fixed.argtypes = [_vp, ctypes.c_longlong, _ci, _vp, _vp, _vp, _sz, _vp]
+
+
+def f8_format_study_workspace_bytes() -> int:
+    return int(_lib.f8_format_study_workspace_bytes())
+
+
+def f8_format_study_fixed(x, unsigned: bool, err, best_fl, workspace, stream=None):
+    """Sec. 3.3's experiment on the device sample x (fp32): err (9 float64) and best_fl (1 int32) are device tensors."""
+    _check(_lib.f8_format_study_fixed(_ptr(x), x.numel(), 1 if unsigned else 0, _ptr(err), _ptr(best_fl), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
 def f8_conv_workspace_bytes(desc: ConvDesc) -> int:
     return int(_lib.f8_conv_workspace_bytes(ctypes.byref(desc)))
 
@@ -200,7 +214,7 @@ def exported_symbols() -> List[str]:
     return ["f8_conv2d_fixed", "f8_dwconv_fixed", "f8_linear_fixed", "f8_maxpool_fixed", "f8_global_avgpool_fixed",
             "f8_conv_workspace_bytes", "f8_net_create", "f8_net_workspace_bytes", "f8_net_forward",
             "f8_net_last_launch_count", "f8_net_set_profiling", "f8_net_get_layer_ms", "f8_net_destroy", "f8_status_str", "f8_last_error", "f8_device_status",
-            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static", "f8_fold_quantize_fixed", "f8_fold_workspace_bytes"]
+            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static", "f8_fold_quantize_fixed", "f8_fold_workspace_bytes", "f8_format_study_fixed", "f8_format_study_workspace_bytes"]
 
 
 def run_layer(layer: "synth.Layer", x: torch.Tensor, residual: Optional[torch.Tensor] = None, params=None,

@@ -471,6 +471,19 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 last_acc = acc;
                 last_acc_phase = acc_phase;
             }
+            if (ok && local > 0) {
+                // The commits that free the last stage uses arrive on barriers nobody waits for any more (the producers
+                // are done).  Such an arrival must not land after this CTA has gone: the next kernel's CTA takes over
+                // the SM at once and keeps its own barriers at the same shared-memory addresses.  So every issuer waits
+                // for the last arrival on each stage that came from one of its own tiles.
+                const int uses_tile = p.win ? p.c_chunks : p.uses;
+                const int total_uses = local * uses_tile;
+                for (int g = max(0, total_uses - p.stages); g < total_uses; ++g) {
+                    const int t_of_g = g / uses_tile;
+                    if (p.dual_issue && (t_of_g & 1) != q_issuer) continue;
+                    mbar_wait(empty_bar + 8 * (g % p.stages), (uint32_t)(g / p.stages) & 1u, abortp, p.status, tagbits | 112);
+                }
+            }
             if (!ok && committed_any) {
                 // let the tensor pipe finish what was issued before TMEM is released
                 const unsigned long long t0 = clock64();
