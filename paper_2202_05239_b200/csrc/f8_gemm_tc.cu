@@ -50,17 +50,11 @@ constexpr int B_PROD_WARP = FIRST_EPI_WARP + NUM_EPI_WARPS;   // requests weight
 // Issuing a tcgen05.mma costs its thread 70-100 cycles, more than the tensor pipe needs for a tile of up to
 // 128 columns; a second issuer (alternate tiles, the other accumulator) keeps the pipe fed for such layers.
 constexpr int MMA2_WARP = B_PROD_WARP + 1;
-// A producer warp spends roughly a thousand cycles per stage use (wait for the stage, announce, issue, loop), and with
-// streamed weights the few stages that fit make the ring latency bound: a second pair of producer warps takes every
-// other stage use.
-constexpr int A2_PROD_WARP = MMA2_WARP + 1;
-constexpr int B2_PROD_WARP = MMA2_WARP + 2;
-constexpr int NUM_THREADS = 32 * (B2_PROD_WARP + 1);
+constexpr int NUM_THREADS = 32 * (MMA2_WARP + 1);
 constexpr int MAX_STAGES = 16;
 constexpr int MAX_OUT_BUFS = 4;             // ring of staged output tiles; with a residual, the residual tile lands in the
                                             // buffer first and the epilogue converts it in place
 constexpr int TMEM_COLS = 512;
-constexpr int MAX_ACC = 8;                  // accumulators of 64 columns; 4 of 128 or 2 of 256 for wider tiles
 constexpr size_t SMEM_LIMIT = 220 * 1024;     // dynamic shared memory budget (227 KiB per CTA minus static data)
 
 // Division by a run-time constant without a divide instruction (a 32-bit divide costs a lone thread well over a
@@ -86,9 +80,6 @@ struct TcParams {
     int group;                // k-iterations per stage (1..8)
     int uses;                 // stage uses per tile: ceil(k_iters / group)
     int dual_issue;           // 1: two MMA-issuing threads (needs stages >= 2 * uses)
-    int alt;                  // 1: two pairs of producer warps, pair h takes the stage uses of parity h (streamed weights,
-                              // one MMA issuer: fills may then complete out of order, the consumer is in order)
-    int acc_log2;             // accumulators in tensor memory: 2, 4 or 8 (1 << acc_log2), 512 / count columns apart
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
     uint32_t stage_bytes;     // group * sub_bytes
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
@@ -196,7 +187,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     extern __shared__ uint8_t smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 2 * MAX_ACC + 1];
+    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 5];
     __shared__ __align__(8) uint64_t epi_bars[3 * MAX_OUT_BUFS];   // out_full[], out_free[], res_full[]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -206,8 +197,8 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const uint32_t full_bar = smem_u32(&bars[0]);
     const uint32_t empty_bar = smem_u32(&bars[MAX_STAGES]);
     const uint32_t tfull_bar = smem_u32(&bars[2 * MAX_STAGES]);
-    const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + MAX_ACC]);
-    const uint32_t bres_bar = smem_u32(&bars[2 * MAX_STAGES + 2 * MAX_ACC]);   // resident weights have landed
+    const uint32_t tempty_bar = smem_u32(&bars[2 * MAX_STAGES + 2]);
+    const uint32_t bres_bar = smem_u32(&bars[2 * MAX_STAGES + 4]);   // resident weights have landed
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t out_full = smem_u32(&epi_bars[0]), out_free = smem_u32(&epi_bars[MAX_OUT_BUFS]);
     const uint32_t res_full = smem_u32(&epi_bars[2 * MAX_OUT_BUFS]);
@@ -219,7 +210,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             mbar_init(empty_bar + 8 * s, 1);
         }
         mbar_init(bres_bar, 1);
-        for (int a = 0; a < MAX_ACC; ++a) {
+        for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
             mbar_init(tempty_bar + 8 * a, NUM_EPI_WARPS);
         }
@@ -261,7 +252,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     volatile int *abortp = &abort_flag;
     const int tagbits = p.tag << 8;     // status word of a timed-out wait: tag << 8 | site
 
-    if (warp == A_PROD_WARP || warp == B_PROD_WARP || ((warp == A2_PROD_WARP || warp == B2_PROD_WARP) && p.alt)) {
+    if (warp == A_PROD_WARP || warp == B_PROD_WARP) {
         // ------------------------------------------------------------------ TMA producer warps
         // A stage holds `group` consecutive k-iterations of one tile (fewer at the tile's end).  Each producer
         // warp makes one pass per stage use: it waits for the stage, then lane (st*group + j) & 31 issues the
@@ -270,9 +261,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // iteration, which used to bound layers with many short k-iterations), and consecutive loads sit in
         // different per-thread TMA queues, so they overlap.
         const uint2 *ktab = (const uint2 *)(smem + p.ktab_off);
-        const int opnd = (warp == A_PROD_WARP || warp == A2_PROD_WARP) ? 0 : 1;
-        const int half = (warp == A2_PROD_WARP || warp == B2_PROD_WARP) ? 1 : 0;      // which uses this warp takes (p.alt)
-        int use_idx = 0;
+        const int opnd = warp == A_PROD_WARP ? 0 : 1;
         if (opnd == 1 && p.b_res) {
             // Resident weights: when all B tiles fit beside the pipeline, they are loaded once and every tile
             // of this CTA reuses them; the stages then carry activations only (the weight re-reads are what
@@ -333,13 +322,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int base_w = ow * p.stride_w - p.pad_w;
             const int base_h = oh * p.stride_h - p.pad_h;
             const int n_base = n_t * p.bn;
-            for (int kc = 0; kc < k_iters; kc += p.group, ++use_idx) {
-                if (p.alt && (use_idx & 1) != half) {
-                    // the other pair's use.  This warp waits only for the stages of its own uses, and the single,
-                    // in-order MMA issuer cannot pass one of those without it: it never falls a barrier phase behind.
-                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
-                    continue;
-                }
+            for (int kc = 0; kc < k_iters; kc += p.group) {
                 if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, tagbits | 101))) {
                     ok = false;
                     break;
@@ -412,17 +395,18 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             if (p.b_res && !mbar_wait(bres_bar, 0, abortp, p.status, tagbits | 111)) ok = false;
             const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
-                const int acc = local & ((1 << p.acc_log2) - 1);
-                if (p.dual_issue && (local & 1) != q_issuer) {
+                const int acc = local & 1;
+                if (p.dual_issue && acc != q_issuer) {
                     // the other issuer's tile: step over its stage uses
                     stage += p.uses;
                     while (stage >= p.stages) { stage -= p.stages; phase ^= 1; }
                     stage_lo = desc_lo0 + (uint32_t)stage * stage16;
                     continue;
                 }
-                const uint32_t acc_phase = (local >> p.acc_log2) & 1;
+                const uint32_t acc_phase = (local >> 1) & 1;
                 if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, abortp, p.status, tagbits | 102)) { ok = false; break; }
-                const uint32_t d_tmem = tmem_base + (uint32_t)acc * (TMEM_COLS >> p.acc_log2);
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * 256;   // two 256-column accumulators
                 uint32_t b_tile_lo = 0;
                 if (p.b_res) {
                     const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
@@ -590,12 +574,12 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 so[i] = (uint32_t)(ch / p.slab_chunks) * (TILE_M * p.slab_w) + off;
             }
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
-                const int acc = local & ((1 << p.acc_log2) - 1);
-                const uint32_t acc_phase = (local >> p.acc_log2) & 1;
+                const int acc = local & 1;                   // accumulator, output buffer and residual buffer in use
+                const uint32_t acc_phase = (local >> 1) & 1;
                 const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
                 const int c_first = n_t * p.bn + ch_begin * 16;
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
-                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * (TMEM_COLS >> p.acc_log2) + ch_begin * 16;
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
                 bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, tagbits | 104);
                 // the buffer holds the residual tile (which implies that its previous store has left), or is free
                 if (RES) got = mbar_wait(res_full + 8 * ob, ophase, abortp, p.status, tagbits | 107) && got;
@@ -639,13 +623,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             grid_dependency_wait();     // direct stores (and residual reads) from these warps
             const int tile_row = quarter * 32 + lane;   // this thread's row of the tile
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
-                const int acc = local & ((1 << p.acc_log2) - 1);
-                const uint32_t acc_phase = (local >> p.acc_log2) & 1;
+                const int acc = local & 1;
+                const uint32_t acc_phase = (local >> 1) & 1;
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
                 const int n0 = n_t * p.bn;
                 const size_t row = (size_t)m_t * TILE_M + tile_row;
                 const bool row_valid = row < (size_t)p.M;
-                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * (TMEM_COLS >> p.acc_log2) + ch_begin * 16;
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
                 if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, tagbits | 104))) { ok = false; break; }
                 tc_fence_after();
                 for (int i = 0; i < nch; ++i) {
@@ -938,13 +922,6 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     }
     const int stages = p.stages;
     p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !getenv("F8_NO_DUAL")) ? 1 : 0;
-    // Narrow tiles leave room for more accumulators.  The chain "accumulator free -> issue -> commit -> epilogue ->
-    // accumulator free" costs about 2500 cycles whatever the tile (per-role timestamps), and only more tiles in flight
-    // hide it: 8 accumulators of 64 columns, 4 of 128, else 2 of 256.
-    p.alt = (!p.b_res && !p.dual_issue && !p.win && p.stages >= 2 && !getenv("F8_NO_ALT")) ? 1 : 0;
-    p.acc_log2 = p.bn <= 64 ? 3 : (p.bn <= 128 ? 2 : 1);
-    if (getenv("F8_ACC_LOG2")) p.acc_log2 = std::max(1, std::min(3, atoi(getenv("F8_ACC_LOG2"))));
-    if ((TMEM_COLS >> p.acc_log2) < p.bn) p.acc_log2 = 1;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
     p.bias_off = p.out_off + (uint32_t)p.out_bufs * p.out_bytes;
     p.ktab_off = (uint32_t)(p.stages * p.stage_bytes + staging - ktab_bytes);
@@ -1058,7 +1035,6 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int total_tiles = p.m_tiles * p.n_tiles;
     plan->grid = total_tiles < sms ? total_tiles : sms;
-    if (getenv("F8_MAX_GRID")) plan->grid = std::max(1, std::min(plan->grid, atoi(getenv("F8_MAX_GRID"))));   // experiments
     // at least half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
     plan->smem = (size_t)p.stages * p.stage_bytes + staging + (p.b_res ? b_all : 0) + 1024;
     if (plan->smem < 120 * 1024) plan->smem = 120 * 1024;
