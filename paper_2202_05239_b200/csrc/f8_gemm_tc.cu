@@ -50,7 +50,12 @@ constexpr int B_PROD_WARP = FIRST_EPI_WARP + NUM_EPI_WARPS;   // requests weight
 // Issuing a tcgen05.mma costs its thread 70-100 cycles, more than the tensor pipe needs for a tile of up to
 // 128 columns; a second issuer (alternate tiles, the other accumulator) keeps the pipe fed for such layers.
 constexpr int MMA2_WARP = B_PROD_WARP + 1;
-constexpr int NUM_THREADS = 32 * (MMA2_WARP + 1);
+// A producer warp spends roughly a thousand cycles per stage use (wait for the stage, announce, issue, loop), and with
+// streamed weights the few stages that fit make the ring latency bound: a second pair of producer warps takes every
+// other stage use.
+constexpr int A2_PROD_WARP = MMA2_WARP + 1;
+constexpr int B2_PROD_WARP = MMA2_WARP + 2;
+constexpr int NUM_THREADS = 32 * (B2_PROD_WARP + 1);
 constexpr int MAX_STAGES = 16;
 constexpr int MAX_OUT_BUFS = 4;             // ring of staged output tiles; with a residual, the residual tile lands in the
                                             // buffer first and the epilogue converts it in place
@@ -80,6 +85,8 @@ struct TcParams {
     int group;                // k-iterations per stage (1..8)
     int uses;                 // stage uses per tile: ceil(k_iters / group)
     int dual_issue;           // 1: two MMA-issuing threads (needs stages >= 2 * uses)
+    int alt;                  // 1: two pairs of producer warps, pair h takes the stage uses of parity h (streamed weights,
+                              // one MMA issuer: fills may then complete out of order, the consumer is in order)
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
     uint32_t stage_bytes;     // group * sub_bytes
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
@@ -252,7 +259,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     volatile int *abortp = &abort_flag;
     const int tagbits = p.tag << 8;     // status word of a timed-out wait: tag << 8 | site
 
-    if (warp == A_PROD_WARP || warp == B_PROD_WARP) {
+    if (warp == A_PROD_WARP || warp == B_PROD_WARP || ((warp == A2_PROD_WARP || warp == B2_PROD_WARP) && p.alt)) {
         // ------------------------------------------------------------------ TMA producer warps
         // A stage holds `group` consecutive k-iterations of one tile (fewer at the tile's end).  Each producer
         // warp makes one pass per stage use: it waits for the stage, then lane (st*group + j) & 31 issues the
@@ -261,7 +268,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // iteration, which used to bound layers with many short k-iterations), and consecutive loads sit in
         // different per-thread TMA queues, so they overlap.
         const uint2 *ktab = (const uint2 *)(smem + p.ktab_off);
-        const int opnd = warp == A_PROD_WARP ? 0 : 1;
+        const int opnd = (warp == A_PROD_WARP || warp == A2_PROD_WARP) ? 0 : 1;
+        const int half = (warp == A2_PROD_WARP || warp == B2_PROD_WARP) ? 1 : 0;      // which uses this warp takes (p.alt)
+        int use_idx = 0;
         if (opnd == 1 && p.b_res) {
             // Resident weights: when all B tiles fit beside the pipeline, they are loaded once and every tile
             // of this CTA reuses them; the stages then carry activations only (the weight re-reads are what
@@ -322,7 +331,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int base_w = ow * p.stride_w - p.pad_w;
             const int base_h = oh * p.stride_h - p.pad_h;
             const int n_base = n_t * p.bn;
-            for (int kc = 0; kc < k_iters; kc += p.group) {
+            for (int kc = 0; kc < k_iters; kc += p.group, ++use_idx) {
+                if (p.alt && (use_idx & 1) != half) {
+                    // the other pair's use.  This warp waits only for the stages of its own uses, and the single,
+                    // in-order MMA issuer cannot pass one of those without it: it never falls a barrier phase behind.
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                    continue;
+                }
                 if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, tagbits | 101))) {
                     ok = false;
                     break;
@@ -922,6 +937,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     }
     const int stages = p.stages;
     p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !getenv("F8_NO_DUAL")) ? 1 : 0;
+    p.alt = (!p.b_res && !p.dual_issue && !p.win && p.stages >= 2 && !getenv("F8_NO_ALT")) ? 1 : 0;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
     p.bias_off = p.out_off + (uint32_t)p.out_bufs * p.out_bytes;
     p.ktab_off = (uint32_t)(p.stages * p.stage_bytes + staging - ktab_bytes);
