@@ -72,6 +72,37 @@ def test_resnet50_full_batch_sampled_images(ref):
     net.close()
 
 
+def test_resnet50_many_back_to_back_passes():
+    """Long runs: several hundred forward passes queued without synchronising (each layer's prologue overlaps the tail of
+    the one before, across passes too), then the pipelined host-to-host path.  Barrier-protocol mistakes that a single
+    pass never meets show up here as a device fault, a timed-out wait or different bits."""
+    a = api()
+    batch = 256
+    layers = synth.make_net("resnet50", 0)
+    x_host = torch.from_numpy(synth.draw_image(batch, 3)).pin_memory()
+    x = x_host.cuda()
+    net = a.Net(layers, batch)
+    out = torch.empty((batch, 1000), dtype=torch.int32, device="cuda")
+    ws = torch.empty(net.workspace_bytes(batch), dtype=torch.uint8, device="cuda")
+    net.forward(x, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    first = out.clone()
+    for _ in range(500):
+        net.forward(x, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    a.f8_device_status()
+    assert torch.equal(out, first)
+    pipe = a.HostPipeline(layers, batch, depth=2)
+    ys = [torch.empty((batch, 1000), dtype=torch.int32).pin_memory() for _ in range(2)]
+    for i in range(300):
+        pipe.submit(x_host, ys[i & 1])
+    pipe.wait()
+    a.f8_device_status()
+    assert torch.equal(ys[0], first.cpu()) and torch.equal(ys[1], first.cpu())
+    pipe.close()
+    net.close()
+
+
 def test_workspace_too_small_is_rejected():
     a = api()
     layers = synth.make_net("resnet18", 0, image=64)
