@@ -85,6 +85,7 @@ struct TcParams {
     int group;                // k-iterations per stage (1..8)
     int uses;                 // stage uses per tile: ceil(k_iters / group)
     int dual_issue;           // 1: two MMA-issuing threads (needs stages >= 2 * uses)
+    int a_plain;              // 1: pointwise layer on a small tensor: activations read as a plain [M, C] matrix (tiled map)
     int alt;                  // 1: two pairs of producer warps, pair h takes the stage uses of parity h (streamed weights,
                               // one MMA issuer: fills may then complete out of order, the consumer is in order)
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
@@ -360,7 +361,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 if (j < subs && (j & j_mask) == j_want) {
                     const uint2 e = ktab[kc + j];       // x: first channel of the chunk, y: tap << 16 | r << 8 | s
                     const uint32_t dst = smem_base + stage * p.stage_bytes + j * p.sub_bytes;
-                    if (opnd == 0 || a_helper)
+                    if ((opnd == 0 || a_helper) && p.a_plain)
+                        tma_load_2d(dst, &map_a, fb, (int)e.x, m0);
+                    else if (opnd == 0 || a_helper)
                         tma_load_im2col(dst, &map_a, fb, (int)e.x, base_w, base_h, img, (uint16_t)(e.y & 0xff),
                                         (uint16_t)((e.y >> 8) & 0xff));
                     else
@@ -781,8 +784,11 @@ void f8_tc_plan_set_tag(F8TcPlan *plan, int tag) { plan->p.tag = tag; }
 
 bool f8_tc_supported(const F8ConvGeom &g, size_t x_bytes) {
     if (g.c % 16 != 0) return false;                 // TMA strides are multiples of 16 bytes
-    if (x_bytes < 128 * 1024) return false;          // im2col tensor maps of tensors below 128 KiB are avoided; such
-                                                     // problems are latency bound anyway: CUDA-core kernel
+    // im2col tensor maps of tensors below 128 KiB are avoided.  A pointwise layer (1x1, stride 1, no padding) needs no
+    // im2col: its activations are a plain [pixels, channels] matrix read through a tiled map, whatever their size;
+    // other small problems go to the CUDA-core kernel.
+    const bool pointwise = g.kh == 1 && g.kw == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 && g.pad_w == 0;
+    if (x_bytes < 128 * 1024 && !(pointwise && x_bytes >= 4096)) return false;
     if (g.kh > 255 || g.kw > 255) return false;
     if ((long long)g.n * g.ho * g.wo > 0x7fffff00ll) return false;
     return true;
@@ -958,7 +964,23 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     const size_t row_bytes = (size_t)g.c_out * ysz;
     p.vec_bytes = (row_bytes % 16 == 0) ? 16 : (row_bytes % 8 == 0 ? 8 : (row_bytes % 4 == 0 ? 4 : 1));
 
-    if (p.win) {
+    const bool dense_x = xv.stride_w == xv.dim_c && xv.stride_h == xv.dim_c * xv.dim_w && xv.stride_n == xv.dim_c * xv.dim_w * xv.dim_h;
+    p.a_plain = (g.kh == 1 && g.kw == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 && g.pad_w == 0 && dense_x &&
+                 xv.dim_c * xv.dim_w * xv.dim_h * xv.dim_n < 128 * 1024) ? 1 : 0;
+    if (p.a_plain) {
+        // A: [M, C] bytes, box = 128 pixels x kb channels; rows past the last pixel are zero filled
+        cuuint64_t dims[2] = {xv.dim_c, (cuuint64_t)p.M};
+        cuuint64_t strides[1] = {xv.dim_c};
+        cuuint32_t box[2] = {(cuuint32_t)p.kb, (cuuint32_t)TILE_M};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = g_encode_tiled(&plan->map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(xv.base), dims, strides,
+                                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(p.kb),
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            *why = "cuTensorMapEncodeTiled rejected the activation matrix";
+            return cudaErrorInvalidValue;
+        }
+    } else if (p.win) {
         // A: the same tensor as plain tiles of win_r + 2 padded rows (coordinates -1 are zero filled)
         cuuint64_t dims[4] = {xv.dim_c, xv.dim_w, xv.dim_h, xv.dim_n};
         cuuint64_t strides[3] = {xv.stride_w, xv.stride_h, xv.stride_n};

@@ -54,6 +54,28 @@ def test_tensor_core_conv(ref, case):
     check_layer(ref, layer, x, res, expect_tc=True)
 
 
+# pointwise layers on tensors below 128 KiB: activations are read as a plain matrix (no im2col map)
+# (h, w, c, c_out, n, x_signed, y_dtype, res)
+SMALL_POINTWISE = [
+    (1, 1, 1280, 1000, 64, False, synth.S32, False),    # a fully connected layer at batch 64 (80 KB)
+    (7, 7, 160, 960, 1, True, synth.U8, False),          # batch-1 inference: 7.8 KB, one ragged M tile
+    (7, 7, 960, 160, 2, False, synth.S8, True),          # 94 KB, residual, eight K chunks
+    (3, 5, 320, 48, 9, False, synth.U8, False),          # 135 pixels: two M tiles, the second nearly empty
+]
+
+
+@pytest.mark.parametrize("case", range(len(SMALL_POINTWISE)))
+def test_small_pointwise_on_tensor_cores(ref, case):
+    h, w, c, c_out, n, xs, y_dtype, with_res = SMALL_POINTWISE[case]
+    rng = np.random.default_rng(700 + case)
+    layer = random_conv_layer(rng, h=h, w=w, c=c, c_out=c_out, k=1, stride=1, pad=0, x_signed=xs, y_dtype=y_dtype,
+                              with_res=with_res)
+    x = random_input(rng, n, layer)
+    assert 4096 <= x.size < 128 * 1024
+    res = random_residual(rng, n, layer) if with_res else None
+    check_layer(ref, layer, x, res, expect_tc=True)
+
+
 def test_extreme_operands_on_tensor_cores(ref):
     """-128 weights against 255 / -128 activations: the signedness selection of the MMA must be right."""
     rng = np.random.default_rng(5)
