@@ -170,6 +170,19 @@ f8_status f8_net_get_layer_ms(f8_net *net, float *ms, int *on_tensor_cores);
 
 void f8_net_destroy(f8_net *net);
 
+/* ---------------------------------------------------------------- one 32-bit value, several consumers */
+
+/* A value with several consumers is "stored in 32-bit" and quantised once per consumer with that consumer's own
+ * fractional length (Sec. 4.3, "Clipping-Level Sharing and Private Fractional Length"; appendix "Private Fractional
+ * Lengths Enabling Different Clipping-Levels": the cost is only some bit shifting).  acc [n] int32 in format fa
+ * (for instance the F8_S32 output of f8_conv2d_fixed, fa = fl_x + fl_w) ->
+ *     y1[i] = clip(rshift_round(acc[i], fa - fl_y1))    and, when y2 != NULL,    y2[i] = clip(rshift_round(acc[i], fa - fl_y2))
+ * with the unsigned clip [0, 255] (Eq. 2; also the ReLU) for F8_U8 and [-127, 127] (appendix) for F8_S8; a negative
+ * shift multiplies.  All pointers DEVICE; y1 / y2 [n] bytes.  Errors: F8_ERR_NULL, F8_ERR_SHAPE (n < 0),
+ * F8_ERR_DTYPE, F8_ERR_FL_RANGE, F8_ERR_SHIFT_RANGE (fa - fl outside [-8, 31]), F8_ERR_ALIGN (acc not 4-byte aligned). */
+f8_status f8_requantize_dual_fixed(long long n, const int32_t *acc, int fa, void *y1, int y1_dtype, int fl_y1,
+                                   void *y2, int y2_dtype, int fl_y2, void *cuda_stream);
+
 /* ---------------------------------------------------------------- weight compile step */
 
 /* One Conv-BN block's parameters turned into what the layer entry points above consume (Sec. 4.2 - 4.3):

@@ -185,6 +185,15 @@ def f8_format_study_fixed(x, unsigned: bool, err, best_fl, workspace, stream=Non
                                       workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
+_lib.f8_requantize_dual_fixed.argtypes = [ctypes.c_longlong, _vp, _ci, _vp, _ci, _ci, _vp, _ci, _ci, _vp]
+
+
+def f8_requantize_dual_fixed(acc, fa, y1, y1_dtype, fl_y1, y2=None, y2_dtype=F8_U8, fl_y2=0, stream=None):
+    """int32 tensor in format fa -> one or two 8-bit tensors, each with its own fractional length (Sec. 4.3)."""
+    _check(_lib.f8_requantize_dual_fixed(acc.numel(), _ptr(acc), fa, _ptr(y1), y1_dtype, fl_y1, _ptr(y2), y2_dtype, fl_y2,
+                                         _stream(stream)))
+
+
 def f8_conv_workspace_bytes(desc: ConvDesc) -> int:
     return int(_lib.f8_conv_workspace_bytes(ctypes.byref(desc)))
 
@@ -214,7 +223,7 @@ def exported_symbols() -> List[str]:
     return ["f8_conv2d_fixed", "f8_dwconv_fixed", "f8_linear_fixed", "f8_maxpool_fixed", "f8_global_avgpool_fixed",
             "f8_conv_workspace_bytes", "f8_net_create", "f8_net_workspace_bytes", "f8_net_forward",
             "f8_net_last_launch_count", "f8_net_set_profiling", "f8_net_get_layer_ms", "f8_net_destroy", "f8_status_str", "f8_last_error", "f8_device_status",
-            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static", "f8_fold_quantize_fixed", "f8_fold_workspace_bytes", "f8_format_study_fixed", "f8_format_study_workspace_bytes"]
+            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static", "f8_fold_quantize_fixed", "f8_fold_workspace_bytes", "f8_format_study_fixed", "f8_format_study_workspace_bytes", "f8_requantize_dual_fixed"]
 
 
 def run_layer(layer: "synth.Layer", x: torch.Tensor, residual: Optional[torch.Tensor] = None, params=None,
