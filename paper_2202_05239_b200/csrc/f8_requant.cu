@@ -20,7 +20,19 @@ __global__ void __launch_bounds__(256) requant_dual_kernel(const int32_t *__rest
     const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (vec) {
         const long long n4 = n >> 2;
-        for (long long i = i0; i < n4; i += stride) {
+        long long i = i0;
+        // four independent 16-byte loads in flight per thread
+        for (; i + 3 * stride < n4; i += 4 * stride) {
+            int4 a[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) a[u] = __ldg((const int4 *)acc + i + u * stride);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                ((uint32_t *)y1)[i + u * stride] = requant4(a[u], q1);
+                if (y2) ((uint32_t *)y2)[i + u * stride] = requant4(a[u], q2);
+            }
+        }
+        for (; i < n4; i += stride) {
             const int4 a = __ldg((const int4 *)acc + i);
             ((uint32_t *)y1)[i] = requant4(a, q1);
             if (y2) ((uint32_t *)y2)[i] = requant4(a, q2);

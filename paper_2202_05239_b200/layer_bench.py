@@ -133,8 +133,27 @@ def bench_fold(c_out: int, k: int, iters: int, warmup: int):
                       "algorithmic_gbs": 5.0 * n / (ms * 1e-3) / 1e9, "weights_per_s": n / (ms * 1e-3)}), flush=True)
 
 
+def bench_requant(n: int, iters: int, warmup: int):
+    """Device time of f8_requantize_dual_fixed on n int32 values (4 bytes read, 2 written per element)."""
+    acc = torch.randint(-(1 << 18), 1 << 18, (n,), dtype=torch.int32, device="cuda")
+    y1 = torch.empty(n, dtype=torch.uint8, device="cuda")
+    y2 = torch.empty(n, dtype=torch.int8, device="cuda")
+    for _ in range(warmup):
+        api.f8_requantize_dual_fixed(acc, 12, y1, synth.U8, 4, y2, synth.S8, 5)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        api.f8_requantize_dual_fixed(acc, 12, y1, synth.U8, 4, y2, synth.S8, 5)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    print(json.dumps({"op": "requantize_dual", "n": n, "ms": ms, "algorithmic_gbs": 6.0 * n / (ms * 1e-3) / 1e9}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--requant", type=int, default=0, help="time the dual requantisation on this many int32 values")
     ap.add_argument("--fold", action="store_true", help="time the weight compile step on a [c-out, k * k * c] tensor")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--net", default="", help="time every layer of a synthetic network: resnet18, resnet50, mobilenetv2")
@@ -151,6 +170,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--warm-l2", action="store_true", help="reuse one buffer set (operands stay in L2)")
     args = ap.parse_args()
+    if args.requant:
+        bench_requant(args.requant, args.iters, args.warmup)
+        return
     if args.fold:
         bench_fold(args.c_out, args.k * args.k * args.c, args.iters, args.warmup)
         return
