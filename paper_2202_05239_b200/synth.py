@@ -367,7 +367,22 @@ def mobilenetv2(seed: int = 0, image: int = 224) -> List[Layer]:
     return b.layers
 
 
-NETS = {"resnet18": resnet18, "resnet50": resnet50, "mobilenetv2": mobilenetv2}
+def mobilenetv1(seed: int = 0, image: int = 224) -> List[Layer]:
+    """13 depthwise-separable blocks (3x3 depthwise + 1x1 pointwise, ReLU after both, no shortcuts), widths and strides of the
+    public MobileNet architecture at width multiplier 1."""
+    b = _NetBuilder(seed, 1, image, image, 3)
+    t = b.conv("stem", 0, 32, 3, 2, True)
+    cfg = [(64, 1), (128, 2), (128, 1), (256, 2), (256, 1), (512, 2), (512, 1), (512, 1), (512, 1), (512, 1), (512, 1),
+           (1024, 2), (1024, 1)]
+    for bi, (c_out, stride) in enumerate(cfg):
+        t = b.conv(f"b{bi}.dw", t, b.stats[t].c, 3, stride, True, depthwise=True)
+        t = b.conv(f"b{bi}.pw", t, c_out, 1, 1, True)
+    t = b.gap("gap", t)
+    b.linear("fc", t, 1000)
+    return b.layers
+
+
+NETS = {"resnet18": resnet18, "resnet50": resnet50, "mobilenetv2": mobilenetv2, "mobilenetv1": mobilenetv1}
 
 
 def make_net(name: str, seed: int = 0, image: int = 224) -> List[Layer]:

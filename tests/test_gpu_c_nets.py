@@ -39,13 +39,13 @@ def _compare_net(ref, name, batch, image, force_direct=False, seed=0):
     net.close()
 
 
-@pytest.mark.parametrize("name", ["resnet18", "resnet50", "mobilenetv2"])
+@pytest.mark.parametrize("name", ["resnet18", "resnet50", "mobilenetv2", "mobilenetv1"])
 def test_net_parity_cuda_core_path(ref, name):
     _compare_net(ref, name, 2, 64, force_direct=True)
 
 
 @pytest.mark.parametrize("name,batch,image", [("resnet18", 3, 224), ("resnet50", 2, 224), ("mobilenetv2", 3, 224),
-                                              ("resnet50", 1, 224), ("resnet18", 5, 96)])
+                                              ("resnet50", 1, 224), ("resnet18", 5, 96), ("mobilenetv1", 3, 224)])
 def test_net_parity(ref, name, batch, image):
     _compare_net(ref, name, batch, image)
 

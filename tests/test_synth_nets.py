@@ -5,7 +5,7 @@ import pytest
 from paper_2202_05239_b200 import synth
 
 
-@pytest.mark.parametrize("name,n_layers,gmac", [("resnet18", 23, 1.814), ("resnet50", 56, 4.089), ("mobilenetv2", 54, 0.3008)])
+@pytest.mark.parametrize("name,n_layers,gmac", [("resnet18", 23, 1.814), ("resnet50", 56, 4.089), ("mobilenetv2", 54, 0.3008), ("mobilenetv1", 29, 0.5688)])
 def test_shapes_and_macs(name, n_layers, gmac):
     layers = synth.make_net(name, 0)
     assert len(layers) == n_layers
@@ -29,7 +29,7 @@ def test_generators_are_seeded():
     assert np.array_equal(synth.draw_image(2, 5), synth.draw_image(2, 5))
 
 
-@pytest.mark.parametrize("name", ["resnet18", "resnet50", "mobilenetv2"])
+@pytest.mark.parametrize("name", ["resnet18", "resnet50", "mobilenetv2", "mobilenetv1"])
 def test_activations_are_not_degenerate(ref, name):
     """The analytic FL choice keeps every layer's codes spread out (neither all zero nor all clipped)."""
     layers = synth.make_net(name, 0, image=96)
