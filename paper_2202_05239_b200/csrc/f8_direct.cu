@@ -1,6 +1,8 @@
 // CUDA-core kernels: generic direct convolution (any shape), depthwise convolution, pooling and the
 // stem packing pre-pass.  Depthwise and pooling layers are not dense contractions: they are bound by
 // HBM traffic, so these kernels are organised around wide, coalesced NHWC accesses.
+#include <stdlib.h>
+
 #include "f8_epilogue.cuh"
 
 namespace {
@@ -260,6 +262,151 @@ __global__ void __launch_bounds__(128) dwconv3x3_strip_kernel(F8ConvGeom g, F8Re
                 if (q.y_kind == F8_S32) *(int4 *)((int32_t *)y + off) = make_int4(out[0], out[1], out[2], out[3]);
                 else *(uint32_t *)((uint8_t *)y + off) = f8_pack4(out[0], out[1], out[2], out[3]);
             }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Depthwise 3x3, pad 1, stride 1, walking down the image.  One thread owns 4 consecutive channels, a strip of 4 output
+// columns and a band of output rows.  It keeps the accumulators of the three output rows that are open (an input row
+// feeds the output rows above, at and below it), so every input word is loaded and unpacked ONCE and the filter taps
+// are loaded once per band: about 15 instructions per output instead of the 36 of the strip kernel, whose threads
+// re-read and re-unpack every input row three times and re-load the taps for every output row.
+// ---------------------------------------------------------------------------------------
+constexpr int DW_WALK_COLS = 4;     // output columns per thread
+constexpr int DW_WALK_SPAN = 6;     // input columns they touch
+
+template <bool XS>
+__device__ __forceinline__ void dw_walk_unpack(const uint32_t (&words)[DW_WALK_SPAN], int (&v)[DW_WALK_SPAN][4]) {
+#pragma unroll
+    for (int xx = 0; xx < DW_WALK_SPAN; ++xx)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[xx][j] = XS ? prmt_s8(words[xx], j) : (int)__byte_perm(words[xx], 0, 0x4440 | j);
+}
+
+// input row `ih` (already unpacked) into the three open output rows: slot (K + 1 - r) mod 3 holds output row ih + 1 - r
+template <int K>
+__device__ __forceinline__ void dw_walk_accumulate(const int (&v)[DW_WALK_SPAN][4], const int (&wt)[9][4],
+                                                   int (&acc)[3][DW_WALK_COLS][4]) {
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        constexpr int dummy = 0;
+        (void)dummy;
+        const int slot = (K + 1 - r + 3) % 3;
+#pragma unroll
+        for (int o = 0; o < DW_WALK_COLS; ++o)
+#pragma unroll
+            for (int sx = 0; sx < 3; ++sx)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[slot][o][j] += v[o + sx][j] * wt[r * 3 + sx][j];
+    }
+}
+
+template <bool XS, bool SIGNED_OUT>
+__global__ void __launch_bounds__(128) dwconv3x3_walk_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
+                                                             const int8_t *__restrict__ w,
+                                                             const int32_t *__restrict__ bias, uint8_t *__restrict__ y,
+                                                             int strips, int bands, int band_rows, int total) {
+    grid_dependency_sync();
+    const int c4 = g.c >> 2;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int cg = idx % c4;
+        int t = idx / c4;
+        const int strip = t % strips;
+        t /= strips;
+        const int band = t % bands;
+        const int in = t / bands;
+        const int c0 = cg * 4;
+        const int ow0 = strip * DW_WALK_COLS;
+        const int oh0 = band * band_rows, oh1 = min(g.ho, oh0 + band_rows);
+        int wt[9][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int k = 0; k < 9; ++k) wt[k][j] = (int)w[(c0 + j) * 9 + k];
+        int4 b = bias ? *(const int4 *)(bias + c0) : make_int4(0, 0, 0, 0);
+        const int rnd = 1 << (q.s - 1);
+        const int bb[4] = {b.x + rnd, b.y + rnd, b.z + rnd, b.w + rnd};
+        int acc[3][DW_WALK_COLS][4];
+#pragma unroll
+        for (int a = 0; a < 3; ++a)
+#pragma unroll
+            for (int o = 0; o < DW_WALK_COLS; ++o)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[a][o][j] = 0;
+        // column offsets (bytes) of the six input columns; columns outside the image read as zero
+        const int iw0 = ow0 - 1;
+        bool col_ok[DW_WALK_SPAN];
+#pragma unroll
+        for (int xx = 0; xx < DW_WALK_SPAN; ++xx) col_ok[xx] = iw0 + xx >= 0 && iw0 + xx < g.w;
+        const int row_stride = g.w * g.c;
+        const uint8_t *img = x + (size_t)in * g.h * row_stride + c0 + iw0 * g.c;
+
+        auto load_row = [&](int ih, uint32_t (&words)[DW_WALK_SPAN]) {
+            const bool row_ok = ih >= 0 && ih < g.h;
+            const uint8_t *rp = img + (size_t)ih * row_stride;
+#pragma unroll
+            for (int xx = 0; xx < DW_WALK_SPAN; ++xx)
+                words[xx] = (row_ok && col_ok[xx]) ? __ldg((const uint32_t *)(rp + xx * g.c)) : 0u;
+        };
+        // output row `oh` is complete: shift, clip, pack, store; then its slot starts the next open row
+        auto emit = [&](int oh, int (&a)[DW_WALK_COLS][4]) {
+            if (oh >= oh0 && oh < oh1) {
+                uint8_t *out = y + ((size_t)(in * g.ho + oh) * g.wo + ow0) * g.c + c0;
+#pragma unroll
+                for (int o = 0; o < DW_WALK_COLS; ++o) {
+                    if (ow0 + o < g.wo) {
+                        int tv[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int vv = (a[o][j] + bb[j]) >> q.s;
+                            tv[j] = SIGNED_OUT ? max(vv, -127) : vv;
+                        }
+                        uint32_t hi2, word;
+                        if (SIGNED_OUT) {
+                            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+                            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+                        } else {
+                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+                        }
+                        *(uint32_t *)(out + o * g.c) = word;
+                    }
+                }
+            }
+#pragma unroll
+            for (int o = 0; o < DW_WALK_COLS; ++o)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) a[o][j] = 0;
+        };
+
+        // input rows oh0 - 1 .. oh1, three per trip so that the slots are compile-time; the next row's words are
+        // requested before the current row is used
+        uint32_t cur[DW_WALK_SPAN], nxt[DW_WALK_SPAN];
+        int ih = oh0 - 1;
+        load_row(ih, cur);
+        while (ih <= oh1) {
+            int v[DW_WALK_SPAN][4];
+            // K = 0: input row ih feeds slots 1 (row ih + 1), 0 (row ih), 2 (row ih - 1, now complete)
+            load_row(ih + 1, nxt);
+            dw_walk_unpack<XS>(cur, v);
+            dw_walk_accumulate<0>(v, wt, acc);
+            emit(ih - 1, acc[2]);
+            if (++ih > oh1) break;
+            // K = 1: slots 2 (row ih + 1), 1 (row ih), 0 (row ih - 1)
+            load_row(ih + 1, cur);
+            dw_walk_unpack<XS>(nxt, v);
+            dw_walk_accumulate<1>(v, wt, acc);
+            emit(ih - 1, acc[0]);
+            if (++ih > oh1) break;
+            // K = 2: slots 0 (row ih + 1), 2 (row ih), 1 (row ih - 1)
+            load_row(ih + 1, nxt);
+            dw_walk_unpack<XS>(cur, v);
+            dw_walk_accumulate<2>(v, wt, acc);
+            emit(ih - 1, acc[1]);
+            if (++ih > oh1) break;
+#pragma unroll
+            for (int xx = 0; xx < DW_WALK_SPAN; ++xx) cur[xx] = nxt[xx];
         }
     }
 }
@@ -568,7 +715,27 @@ cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void
                           g.stride_h == g.stride_w && (g.stride_h == 1 || g.stride_h == 2) &&
                           (((uintptr_t)x | (uintptr_t)y | (uintptr_t)res | (uintptr_t)bias) & 15) == 0 &&
                           (size_t)g.n * g.h * g.w * g.c < (1u << 31) && total * (q.y_kind == F8_S32 ? 4 : 1) < (1u << 31);
-    if (strip_ok) {
+    const bool walk_ok = strip_ok && g.stride_h == 1 && !q.has_res && q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24 &&
+                         q.sh_acc == 0 && !getenv("F8_NO_DW_WALK");
+    if (walk_ok) {
+        const int strips = (g.wo + DW_WALK_COLS - 1) / DW_WALK_COLS;
+        // bands of output rows: long enough to amortise the two extra input rows and the tap loads, short enough to
+        // give every SM several blocks
+        int band_rows = g.ho;
+        while (band_rows > 8 && (long long)g.n * ((g.ho + band_rows - 1) / band_rows) * strips * (g.c / 4) < 148 * 128 * 8)
+            band_rows = (band_rows + 1) / 2;
+        const int bands = (g.ho + band_rows - 1) / band_rows;
+        const int threads = g.n * bands * strips * (g.c / 4);
+        const int grid = grid_for((size_t)threads, 128);
+        const uint8_t *xp = (const uint8_t *)x;
+        if (g.x_signed) {
+            if (q.y_kind == F8_S8) launch_k(dwconv3x3_walk_kernel<true, true>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads);
+            else launch_k(dwconv3x3_walk_kernel<true, false>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads);
+        } else {
+            if (q.y_kind == F8_S8) launch_k(dwconv3x3_walk_kernel<false, true>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads);
+            else launch_k(dwconv3x3_walk_kernel<false, false>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads);
+        }
+    } else if (strip_ok) {
         const int tw = g.stride_h == 1 ? 8 : 4;
         const int strips = (g.wo + tw - 1) / tw;
         const int threads = g.n * g.ho * strips * (g.c / 4);
