@@ -298,7 +298,11 @@ __device__ __forceinline__ void dw_walk_accumulate(const int (&v)[DW_WALK_SPAN][
 #pragma unroll
             for (int sx = 0; sx < 3; ++sx)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[slot][o][j] += v[o + sx][j] * wt[r * 3 + sx][j];
+                for (int j = 0; j < 4; ++j) {
+                    // the top tap row opens output row ih + 1: its first product starts the sum
+                    if (r == 0 && sx == 0) acc[slot][o][j] = v[o][j] * wt[0][j];
+                    else acc[slot][o][j] += v[o + sx][j] * wt[r * 3 + sx][j];
+                }
     }
 }
 
@@ -349,7 +353,7 @@ __global__ void __launch_bounds__(128) dwconv3x3_walk_kernel(F8ConvGeom g, F8Req
             for (int xx = 0; xx < DW_WALK_SPAN; ++xx)
                 words[xx] = (row_ok && col_ok[xx]) ? __ldg((const uint32_t *)(rp + xx * g.c)) : 0u;
         };
-        // output row `oh` is complete: shift, clip, pack, store; then its slot starts the next open row
+        // output row `oh` is complete: shift, clip, pack, store (its slot is re-opened by the next top-tap products)
         auto emit = [&](int oh, int (&a)[DW_WALK_COLS][4]) {
             if (oh >= oh0 && oh < oh1) {
                 uint8_t *out = y + ((size_t)(in * g.ho + oh) * g.wo + ow0) * g.c + c0;
@@ -374,10 +378,6 @@ __global__ void __launch_bounds__(128) dwconv3x3_walk_kernel(F8ConvGeom g, F8Req
                     }
                 }
             }
-#pragma unroll
-            for (int o = 0; o < DW_WALK_COLS; ++o)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) a[o][j] = 0;
         };
 
         // input rows oh0 - 1 .. oh1, three per trip so that the slots are compile-time; the next row's words are
