@@ -267,16 +267,14 @@ __global__ void __launch_bounds__(128) dwconv3x3_strip_kernel(F8ConvGeom g, F8Re
 }
 
 // ---------------------------------------------------------------------------------------
-// Depthwise 3x3, pad 1, stride 1, walking down the image.  One thread owns 4 consecutive channels, a strip of 4 output
-// columns and a band of output rows.  It keeps the accumulators of the three output rows that are open (an input row
+// Depthwise 3x3, pad 1, stride 1, walking down the image.  One thread owns 4 consecutive channels, a strip of 2 (or 4)
+// output columns and a band of output rows.  It keeps the accumulators of the three output rows that are open (an input row
 // feeds the output rows above, at and below it), so every input word is loaded and unpacked ONCE and the filter taps
 // are loaded once per band: about 15 instructions per output instead of the 36 of the strip kernel, whose threads
 // re-read and re-unpack every input row three times and re-load the taps for every output row.
 // ---------------------------------------------------------------------------------------
-constexpr int DW_WALK_COLS = 4;     // output columns per thread
-constexpr int DW_WALK_SPAN = 6;     // input columns they touch
 
-template <bool XS>
+template <bool XS, int DW_WALK_SPAN>
 __device__ __forceinline__ void dw_walk_unpack(const uint32_t (&words)[DW_WALK_SPAN], int (&v)[DW_WALK_SPAN][4]) {
 #pragma unroll
     for (int xx = 0; xx < DW_WALK_SPAN; ++xx)
@@ -285,8 +283,8 @@ __device__ __forceinline__ void dw_walk_unpack(const uint32_t (&words)[DW_WALK_S
 }
 
 // input row `ih` (already unpacked) into the three open output rows: slot (K + 1 - r) mod 3 holds output row ih + 1 - r
-template <int K>
-__device__ __forceinline__ void dw_walk_accumulate(const int (&v)[DW_WALK_SPAN][4], const int (&wt)[9][4],
+template <int K, int DW_WALK_COLS>
+__device__ __forceinline__ void dw_walk_accumulate(const int (&v)[DW_WALK_COLS + 2][4], const int (&wt)[9][4],
                                                    int (&acc)[3][DW_WALK_COLS][4]) {
 #pragma unroll
     for (int r = 0; r < 3; ++r) {
@@ -306,12 +304,14 @@ __device__ __forceinline__ void dw_walk_accumulate(const int (&v)[DW_WALK_SPAN][
     }
 }
 
-template <bool XS, bool SIGNED_OUT>
+// DW_WALK_COLS output columns per thread (4: fewest instructions; 2: half the registers, more warps per SM)
+template <bool XS, bool SIGNED_OUT, int DW_WALK_COLS>
 __global__ void __launch_bounds__(128) dwconv3x3_walk_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
                                                              const int8_t *__restrict__ w,
                                                              const int32_t *__restrict__ bias, uint8_t *__restrict__ y,
                                                              int strips, int bands, int band_rows, int total) {
     grid_dependency_sync();
+    constexpr int DW_WALK_SPAN = DW_WALK_COLS + 2;
     const int c4 = g.c >> 2;
     for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
         const int cg = idx % c4;
@@ -389,20 +389,20 @@ __global__ void __launch_bounds__(128) dwconv3x3_walk_kernel(F8ConvGeom g, F8Req
             int v[DW_WALK_SPAN][4];
             // K = 0: input row ih feeds slots 1 (row ih + 1), 0 (row ih), 2 (row ih - 1, now complete)
             load_row(ih + 1, nxt);
-            dw_walk_unpack<XS>(cur, v);
-            dw_walk_accumulate<0>(v, wt, acc);
+            dw_walk_unpack<XS, DW_WALK_SPAN>(cur, v);
+            dw_walk_accumulate<0, DW_WALK_COLS>(v, wt, acc);
             emit(ih - 1, acc[2]);
             if (++ih > oh1) break;
             // K = 1: slots 2 (row ih + 1), 1 (row ih), 0 (row ih - 1)
             load_row(ih + 1, cur);
-            dw_walk_unpack<XS>(nxt, v);
-            dw_walk_accumulate<1>(v, wt, acc);
+            dw_walk_unpack<XS, DW_WALK_SPAN>(nxt, v);
+            dw_walk_accumulate<1, DW_WALK_COLS>(v, wt, acc);
             emit(ih - 1, acc[0]);
             if (++ih > oh1) break;
             // K = 2: slots 0 (row ih + 1), 2 (row ih), 1 (row ih - 1)
             load_row(ih + 1, nxt);
-            dw_walk_unpack<XS>(cur, v);
-            dw_walk_accumulate<2>(v, wt, acc);
+            dw_walk_unpack<XS, DW_WALK_SPAN>(cur, v);
+            dw_walk_accumulate<2, DW_WALK_COLS>(v, wt, acc);
             emit(ih - 1, acc[1]);
             if (++ih > oh1) break;
 #pragma unroll
@@ -718,7 +718,10 @@ cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void
     const bool walk_ok = strip_ok && g.stride_h == 1 && !q.has_res && q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24 &&
                          q.sh_acc == 0 && !getenv("F8_NO_DW_WALK");
     if (walk_ok) {
-        const int strips = (g.wo + DW_WALK_COLS - 1) / DW_WALK_COLS;
+        // two columns per thread measured slightly ahead of four (96 against 128 registers: 20 against 16 warps per SM)
+        const int cols = getenv("F8_DW_COLS") ? atoi(getenv("F8_DW_COLS")) : 2;
+        const int wcols = cols == 4 ? 4 : 2;
+        const int strips = (g.wo + wcols - 1) / wcols;
         // bands of output rows: long enough to amortise the two extra input rows and the tap loads, short enough to
         // give every SM several blocks
         int band_rows = g.ho;
@@ -728,13 +731,17 @@ cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void
         const int threads = g.n * bands * strips * (g.c / 4);
         const int grid = grid_for((size_t)threads, 128);
         const uint8_t *xp = (const uint8_t *)x;
-        if (g.x_signed) {
-            if (q.y_kind == F8_S8) launch_k(dwconv3x3_walk_kernel<true, true>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads);
-            else launch_k(dwconv3x3_walk_kernel<true, false>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads);
+#define F8_DW_WALK(XS_, SO_, C_) \
+    launch_k(dwconv3x3_walk_kernel<XS_, SO_, C_>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads)
+        const bool so = q.y_kind == F8_S8;
+        if (wcols == 2) {
+            if (g.x_signed) { if (so) F8_DW_WALK(true, true, 2); else F8_DW_WALK(true, false, 2); }
+            else { if (so) F8_DW_WALK(false, true, 2); else F8_DW_WALK(false, false, 2); }
         } else {
-            if (q.y_kind == F8_S8) launch_k(dwconv3x3_walk_kernel<false, true>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads);
-            else launch_k(dwconv3x3_walk_kernel<false, false>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads);
+            if (g.x_signed) { if (so) F8_DW_WALK(true, true, 4); else F8_DW_WALK(true, false, 4); }
+            else { if (so) F8_DW_WALK(false, true, 4); else F8_DW_WALK(false, false, 4); }
         }
+#undef F8_DW_WALK
     } else if (strip_ok) {
         const int tw = g.stride_h == 1 ? 8 : 4;
         const int strips = (g.wo + tw - 1) / tw;
