@@ -170,6 +170,30 @@ f8_status f8_net_get_layer_ms(f8_net *net, float *ms, int *on_tensor_cores);
 
 void f8_net_destroy(f8_net *net);
 
+/* ---------------------------------------------------------------- forward passes from host buffers */
+
+/* The same forward pass for callers whose images and results live in HOST memory (the end-to-end path).  The
+ * object owns `depth` slots, each with its own network object, device input / output buffers and workspace
+ * (allocated here, on the current device), and three streams: while the GPU computes pass i, the copy engines
+ * upload the input of pass i + 1 and download the result of pass i - 1.  Every step of the arithmetic still runs
+ * in f8_net_forward.
+ *   f8_net_forward_host   host_x: [batch, h, w, c] network input, host_y: the last layer's output, both in HOST
+ *                         memory (page-locked memory is needed for the copies to overlap; pageable memory works but
+ *                         serialises them).  One cudaMemcpyAsync each way per call.  Returns at once; host_x may be
+ *                         reused and host_y read after f8_net_host_wait (or after `depth` further calls).
+ *   f8_net_host_wait      blocks until everything submitted so far has finished.
+ *   f8_net_host_streams   the three streams (cudaStream_t as void*), so that a caller can record its own events
+ *                         around a run of calls.
+ * Errors as f8_net_create / f8_net_forward; F8_ERR_SHAPE for depth outside 1..8. */
+typedef struct f8_net_host f8_net_host;
+f8_status f8_net_host_create(const f8_layer_desc *layers, int n_layers, const int8_t *const *host_weights,
+                             const int32_t *const *host_bias, int batch, int depth, f8_net_host **out);
+f8_status f8_net_forward_host(f8_net_host *pipe, const void *host_x, void *host_y);
+f8_status f8_net_host_wait(f8_net_host *pipe);
+f8_status f8_net_host_streams(f8_net_host *pipe, void **upload, void **compute, void **download);
+int f8_net_host_launches_per_pass(const f8_net_host *pipe);
+void f8_net_host_destroy(f8_net_host *pipe);
+
 /* ---------------------------------------------------------------- one 32-bit value, several consumers */
 
 /* A value with several consumers is "stored in 32-bit" and quantised once per consumer with that consumer's own
@@ -247,6 +271,47 @@ long long f8_tc_launch_count(void);
 
 /* Test hook: non-zero routes every dense layer to the CUDA-core kernel (same results). */
 void f8_debug_force_direct(int on);
+
+/* Test hook: switches planning choices off so that the alternative code paths can be checked against
+ * the oracle (results never change; the default, 0, is the fastest plan).  Process-wide; takes effect for
+ * plans made after the call (f8_net objects plan again when the mask has changed).
+ *   F8_PLAN_OFF_RESIDENT_WEIGHTS  weights are streamed through the pipeline even where they would fit in shared memory
+ *   F8_PLAN_OFF_WINDOWED          3x3 stride-1 layers gather their taps by im2col instead of reading whole padded rows
+ *   F8_PLAN_OFF_DUAL_ISSUE        one MMA-issuing thread per CTA
+ *   F8_PLAN_OFF_ALT_PRODUCERS     one pair of TMA producer warps
+ *   F8_PLAN_OFF_PAIRS             no two-CTA tiles (tcgen05 cta_group::2)
+ *   F8_PLAN_OFF_DW_WALK           depthwise 3x3 stride-1 layers take the strip kernel
+ *   F8_PLAN_OFF_STEM_KERNEL       first layers take the packed-row-pair GEMM instead of the first-layer kernel
+ *   F8_PLAN_OFF_STEM_POOL_FUSION  the max pool behind a first layer runs as its own kernel
+ *   F8_PLAN_OFF_LAYER_OVERLAP     f8_net_forward launches without programmatic dependent launch
+ *   F8_PLAN_OFF_MICRO_BATCH       f8_net_forward runs every layer over the whole batch
+ *   F8_PLAN_SYNC_LAYERS           f8_net_forward synchronises after every launch, so that a device fault is
+ *                                 reported with the layer that raised it */
+enum {
+    F8_PLAN_OFF_RESIDENT_WEIGHTS = 1, F8_PLAN_OFF_WINDOWED = 2, F8_PLAN_OFF_DUAL_ISSUE = 4, F8_PLAN_OFF_ALT_PRODUCERS = 8,
+    F8_PLAN_OFF_PAIRS = 16, F8_PLAN_OFF_DW_WALK = 32, F8_PLAN_OFF_STEM_KERNEL = 64, F8_PLAN_OFF_STEM_POOL_FUSION = 128,
+    F8_PLAN_OFF_LAYER_OVERLAP = 256, F8_PLAN_OFF_MICRO_BATCH = 512, F8_PLAN_SYNC_LAYERS = 1024
+};
+void f8_debug_plan_options(unsigned off_mask);
+
+/* What the most recent tensor-core plan of this process decided (n <= 10 ints are written, the count is returned):
+ * [0] flags below, [1] epilogue variant (0 generic, 1 u8, 2 u8 + residual, 3 s8, 4 s8 + residual), [2] N tile,
+ * [3] K bytes per chunk, [4] pipeline stages, [5] K chunks per stage, [6] M tiles, [7] N tiles, [8] CTAs launched,
+ * [9] staged output buffers.  Lets a test assert which path a case took and how many tiles each CTA walked. */
+enum {
+    F8_PLAN_RESIDENT_WEIGHTS = 1, F8_PLAN_WINDOWED = 2, F8_PLAN_DUAL_ISSUE = 4, F8_PLAN_ALT_PRODUCERS = 8,
+    F8_PLAN_PLAIN_MATRIX = 16, F8_PLAN_STAGED_EPILOGUE = 32, F8_PLAN_PAIRS = 64
+};
+int f8_debug_last_plan(int *info, int n);
+
+/* Bound of every in-kernel barrier wait, in milliseconds at the maximum SM clock (0 restores the default of
+ * about two seconds).  Process-wide; for kernels launched after the call. */
+void f8_debug_set_wait_limit_ms(double ms);
+
+/* Failure-detection check that harms nothing: one thread of a one-block kernel waits, with the given bound, on a
+ * barrier that nothing will ever arrive at.  The wait runs out, the kernel records it in the device status word
+ * (site 199) and returns normally; the next f8_device_status() reports F8_ERR_TIMEOUT. */
+f8_status f8_debug_wait_timeout_probe(double limit_ms, void *cuda_stream);
 
 /* Tensor-core probe: every SM issues `iters` back-to-back tcgen05.mma kind::i8
  * 128 x 256 x 32 instructions on resident shared-memory tiles (no global traffic).

@@ -219,18 +219,82 @@ def f8_debug_force_direct(on: bool):
     _lib.f8_debug_force_direct(1 if on else 0)
 
 
+_lib.f8_debug_plan_options.argtypes = [ctypes.c_uint]
+_lib.f8_debug_plan_options.restype = None
+_lib.f8_debug_last_plan.argtypes = [ctypes.POINTER(ctypes.c_int), _ci]
+_lib.f8_debug_set_wait_limit_ms.argtypes = [ctypes.c_double]
+_lib.f8_debug_set_wait_limit_ms.restype = None
+_lib.f8_debug_wait_timeout_probe.argtypes = [ctypes.c_double, _vp]
+
+# f8_debug_plan_options bits (planning choices switched off) and f8_debug_last_plan flags
+PLAN_OFF_RESIDENT_WEIGHTS, PLAN_OFF_WINDOWED, PLAN_OFF_DUAL_ISSUE, PLAN_OFF_ALT_PRODUCERS = 1, 2, 4, 8
+PLAN_OFF_PAIRS, PLAN_OFF_DW_WALK, PLAN_OFF_STEM_KERNEL, PLAN_OFF_STEM_POOL_FUSION = 16, 32, 64, 128
+PLAN_OFF_LAYER_OVERLAP, PLAN_OFF_MICRO_BATCH, PLAN_SYNC_LAYERS = 256, 512, 1024
+PLAN_RESIDENT_WEIGHTS, PLAN_WINDOWED, PLAN_DUAL_ISSUE, PLAN_ALT_PRODUCERS = 1, 2, 4, 8
+PLAN_PLAIN_MATRIX, PLAN_STAGED_EPILOGUE, PLAN_PAIRS = 16, 32, 64
+
+
+def f8_debug_plan_options(off_mask: int):
+    _lib.f8_debug_plan_options(off_mask)
+
+
+def f8_debug_last_plan() -> dict:
+    """What the most recent tensor-core plan decided (which code path a layer takes, how many tiles per CTA)."""
+    v = (ctypes.c_int * 10)()
+    _lib.f8_debug_last_plan(v, 10)
+    keys = ("flags", "epilogue", "bn", "kb", "stages", "group", "m_tiles", "n_tiles", "ctas", "out_bufs")
+    return dict(zip(keys, [int(x) for x in v]))
+
+
+def f8_debug_set_wait_limit_ms(ms: float):
+    _lib.f8_debug_set_wait_limit_ms(ms)
+
+
+def f8_debug_wait_timeout_probe(limit_ms: float, stream=None):
+    _check(_lib.f8_debug_wait_timeout_probe(limit_ms, _stream(stream)))
+
+
 def exported_symbols() -> List[str]:
     return ["f8_conv2d_fixed", "f8_dwconv_fixed", "f8_linear_fixed", "f8_maxpool_fixed", "f8_global_avgpool_fixed",
             "f8_conv_workspace_bytes", "f8_net_create", "f8_net_workspace_bytes", "f8_net_forward",
             "f8_net_last_launch_count", "f8_net_set_profiling", "f8_net_get_layer_ms", "f8_net_destroy", "f8_status_str", "f8_last_error", "f8_device_status",
-            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static", "f8_fold_quantize_fixed", "f8_fold_workspace_bytes", "f8_format_study_fixed", "f8_format_study_workspace_bytes", "f8_requantize_dual_fixed"]
+            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static", "f8_fold_quantize_fixed", "f8_fold_workspace_bytes", "f8_format_study_fixed", "f8_format_study_workspace_bytes", "f8_requantize_dual_fixed",
+            "f8_tc_launch_count", "f8_debug_force_direct", "f8_debug_plan_options", "f8_debug_last_plan",
+            "f8_debug_set_wait_limit_ms", "f8_debug_wait_timeout_probe"]
+
+
+def layer_output_shape(layer: "synth.Layer", n: int):
+    if layer.kind in (synth.CONV, synth.DWCONV):
+        return (n, layer.ho, layer.wo, layer.c_out)
+    if layer.kind == synth.MAXPOOL:
+        return (n, layer.ho, layer.wo, layer.c)
+    if layer.kind == synth.GAP:
+        return (n, layer.c)
+    return (n, layer.c_out)
 
 
 def run_layer(layer: "synth.Layer", x: torch.Tensor, residual: Optional[torch.Tensor] = None, params=None,
-              stream=None) -> torch.Tensor:
-    """One generated layer through the single-layer entry points; returns a new output tensor."""
+              stream=None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """One generated layer through the single-layer entry points; returns the output tensor (`out` if given)."""
     n = x.shape[0]
     w, b = params if params is not None else (to_device(layer.weight), to_device(layer.bias))
+    if out is not None:
+        y = out
+        if layer.kind in (synth.CONV, synth.DWCONV):
+            fn = f8_conv2d_fixed if layer.kind == synth.CONV else f8_dwconv_fixed
+            fn(conv_desc(layer, n), x, w, b, residual, y, stream=stream)
+        elif layer.kind == synth.LINEAR:
+            f8_linear_fixed(n, layer.c, layer.c_out, layer.x_dtype, layer.y_dtype, layer.fl_x, layer.fl_w, layer.fl_y,
+                            x, w, b, y, stream=stream)
+        elif layer.kind == synth.MAXPOOL:
+            f8_maxpool_fixed(n, layer.h, layer.w, layer.c, layer.kh, layer.stride, layer.pad, layer.x_dtype, x, y,
+                             stream=stream)
+        elif layer.kind == synth.GAP:
+            f8_global_avgpool_fixed(n, layer.h, layer.w, layer.c, layer.x_dtype, layer.fl_x, layer.fl_y, x, y,
+                                    stream=stream)
+        else:
+            raise ValueError(layer.kind)
+        return y
     if layer.kind in (synth.CONV, synth.DWCONV):
         y = torch.empty((n, layer.ho, layer.wo, layer.c_out), dtype=torch_dtype(layer.y_dtype), device=x.device)
         fn = f8_conv2d_fixed if layer.kind == synth.CONV else f8_dwconv_fixed
@@ -259,20 +323,7 @@ class Net:
         self.layers = list(layers)
         self.max_batch = max_batch
         n = len(self.layers)
-        descs = (LayerDesc * n)()
-        wptrs = (_vp * n)()
-        bptrs = (_vp * n)()
-        self._keep = []
-        for i, l in enumerate(self.layers):
-            descs[i] = LayerDesc(l.kind, l.src, l.res, conv_desc(l, 1))
-            if l.weight is not None:
-                w = np.ascontiguousarray(l.weight, dtype=np.int8)
-                self._keep.append(w)
-                wptrs[i] = w.ctypes.data
-            if l.bias is not None:
-                b = np.ascontiguousarray(l.bias, dtype=np.int32)
-                self._keep.append(b)
-                bptrs[i] = b.ctypes.data
+        descs, wptrs, bptrs, self._keep = _layer_tables(self.layers)
         handle = _vp()
         _check(_lib.f8_net_create(descs, n, wptrs, bptrs, max_batch, ctypes.byref(handle)))
         self._h = handle
@@ -337,56 +388,78 @@ class Net:
             pass
 
 
+def _layer_tables(layers):
+    """ctypes tables f8_net_create / f8_net_host_create take: descriptors, host weight and bias pointers (+ the arrays
+    that must stay alive while the call runs)."""
+    n = len(layers)
+    descs = (LayerDesc * n)()
+    wptrs = (_vp * n)()
+    bptrs = (_vp * n)()
+    keep = []
+    for i, l in enumerate(layers):
+        descs[i] = LayerDesc(l.kind, l.src, l.res, conv_desc(l, 1))
+        if l.weight is not None:
+            w = np.ascontiguousarray(l.weight, dtype=np.int8)
+            keep.append(w)
+            wptrs[i] = w.ctypes.data
+        if l.bias is not None:
+            b = np.ascontiguousarray(l.bias, dtype=np.int32)
+            keep.append(b)
+            bptrs[i] = b.ctypes.data
+    return descs, wptrs, bptrs, keep
+
+
+_lib.f8_net_host_create.argtypes = [ctypes.POINTER(LayerDesc), _ci, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _ci, _ci,
+                                    ctypes.POINTER(_vp)]
+_lib.f8_net_forward_host.argtypes = [_vp, _vp, _vp]
+_lib.f8_net_host_wait.argtypes = [_vp]
+_lib.f8_net_host_streams.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]
+_lib.f8_net_host_launches_per_pass.argtypes = [_vp]
+_lib.f8_net_host_destroy.argtypes = [_vp]
+_lib.f8_net_host_destroy.restype = None
+
+
 class HostPipeline:
-    """Forward passes from pinned host buffers with the copies overlapped: while the GPU runs batch i, the copy
-    engine uploads batch i+1 and downloads the logits of batch i-1.  Every slot has its own net (plans are cached per
-    set of buffer addresses), device input / output buffers and workspace; all arithmetic still runs in
-    f8_net_forward.  submit() returns at once; result `i` is in its host buffer after wait() (or once the event
-    submit() returns has completed)."""
+    """Forward passes from (pinned) host buffers through ``f8_net_forward_host``: while the GPU runs batch i, the copy
+    engines upload batch i+1 and download the logits of batch i-1.  Slots, device buffers, streams and events all
+    belong to the library object; this class only passes host pointers.  submit() returns at once; result `i` is in
+    its host buffer after wait()."""
 
     def __init__(self, layers: Sequence["synth.Layer"], batch: int, depth: int = 2, device="cuda"):
         self.batch = batch
         self.depth = depth
-        self.nets = [Net(layers, batch) for _ in range(depth)]
-        first = layers[0]
-        in_dtype = torch_dtype(first.x_dtype)
-        self.x_dev = [torch.empty((batch, first.h, first.w, first.c), dtype=in_dtype, device=device) for _ in range(depth)]
-        self.y_dev = [torch.empty((batch,) + n.out_shape, dtype=n.out_dtype, device=device) for n in self.nets]
-        self.ws = [torch.empty(n.workspace_bytes(batch), dtype=torch.uint8, device=device) for n in self.nets]
-        self.up_stream = torch.cuda.Stream(device=device)        # host -> device copies
-        self.down_stream = torch.cuda.Stream(device=device)      # device -> host copies (the link is full duplex)
-        self.compute_stream = torch.cuda.Stream(device=device)
-        self.ev_in = [torch.cuda.Event() for _ in range(depth)]        # upload of the slot's input finished
-        self.ev_done = [torch.cuda.Event() for _ in range(depth)]      # forward pass of the slot finished
-        self.ev_out = [torch.cuda.Event() for _ in range(depth)]       # download of the slot's result finished
-        self.count = 0
+        dev = torch.device(device)
+        with torch.cuda.device(dev if dev.index is not None else torch.cuda.current_device()):
+            descs, wptrs, bptrs, keep = _layer_tables(list(layers))
+            handle = _vp()
+            _check(_lib.f8_net_host_create(descs, len(layers), wptrs, bptrs, batch, depth, ctypes.byref(handle)))
+            self._h = handle
+            up, comp, down = _vp(), _vp(), _vp()
+            _check(_lib.f8_net_host_streams(self._h, ctypes.byref(up), ctypes.byref(comp), ctypes.byref(down)))
+            self.up_stream = torch.cuda.ExternalStream(up.value)
+            self.compute_stream = torch.cuda.ExternalStream(comp.value)
+            self.down_stream = torch.cuda.ExternalStream(down.value)
+        del keep
 
-    def submit(self, x_host: torch.Tensor, y_host: torch.Tensor) -> "torch.cuda.Event":
-        b = self.count % self.depth
-        self.count += 1
-        with torch.cuda.stream(self.up_stream):
-            self.up_stream.wait_event(self.ev_done[b])        # the slot's previous forward pass has read its input
-            self.x_dev[b].copy_(x_host, non_blocking=True)
-            self.ev_in[b].record(self.up_stream)
-        self.compute_stream.wait_event(self.ev_in[b])
-        self.compute_stream.wait_event(self.ev_out[b])       # the slot's previous result has left its output buffer
-        self.nets[b].forward(self.x_dev[b], out=self.y_dev[b], workspace=self.ws[b], stream=self.compute_stream)
-        self.ev_done[b].record(self.compute_stream)
-        with torch.cuda.stream(self.down_stream):
-            self.down_stream.wait_event(self.ev_done[b])
-            y_host.copy_(self.y_dev[b], non_blocking=True)
-            self.ev_out[b].record(self.down_stream)
-        return self.ev_out[b]
+    def submit(self, x_host: torch.Tensor, y_host: torch.Tensor):
+        if x_host.is_cuda or y_host.is_cuda or not x_host.is_contiguous() or not y_host.is_contiguous():
+            raise ValueError("submit() takes contiguous host tensors")
+        _check(_lib.f8_net_forward_host(self._h, ctypes.c_void_p(x_host.data_ptr()), ctypes.c_void_p(y_host.data_ptr())))
 
     def wait(self):
-        self.up_stream.synchronize()
-        self.compute_stream.synchronize()
-        self.down_stream.synchronize()
+        _check(_lib.f8_net_host_wait(self._h))
 
     @property
     def launches_per_step(self) -> int:
-        return self.nets[0].last_launch_count
+        return int(_lib.f8_net_host_launches_per_pass(self._h))
 
     def close(self):
-        for n in self.nets:
-            n.close()
+        if self._h:
+            _lib.f8_net_host_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

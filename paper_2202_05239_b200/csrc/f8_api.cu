@@ -18,6 +18,9 @@ namespace {
 thread_local char g_err[512] = "";
 bool g_force_direct = false;
 long long g_tc_launches = 0;
+unsigned g_plan_off = 0;                      // F8_PLAN_OFF_* bits (test hook)
+unsigned long long g_wait_limit_cycles = 0;   // 0: the kernels' default
+int g_last_plan[10] = {0};
 
 f8_status fail(f8_status s, const char *fmt, ...) {
     va_list ap;
@@ -138,7 +141,6 @@ f8_status run_dense(const F8ConvGeom &g, const F8Requant &q, const void *x, cons
         }
         if (e != cudaErrorInvalidValue && e != cudaErrorNotSupported) return cuda_fail(e, why);
         // the tensor map could not be encoded for this shape: take the CUDA-core kernel
-        if (getenv("F8NET_VERBOSE")) fprintf(stderr, "f8net: tensor-core plan rejected (%s: %s), using the CUDA-core kernel\n", why, cudaGetErrorString(e));
         (void)cudaGetLastError();
     }
     cudaError_t e = f8_launch_conv_direct(g, q, x, w, bias, res, y, st);
@@ -149,6 +151,10 @@ f8_status run_dense(const F8ConvGeom &g, const F8Requant &q, const void *x, cons
 }   // namespace
 
 f8_status f8_set_error(f8_status s, const char *message) { return fail(s, "%s", message); }
+
+unsigned f8_plan_options_off() { return g_plan_off; }
+unsigned long long f8_wait_limit_cycles() { return g_wait_limit_cycles; }
+int *f8_last_plan_info() { return g_last_plan; }
 
 int *f8_status_word() {
     static int *words[64] = {nullptr};
@@ -189,6 +195,35 @@ long long f8_tc_launch_count(void) { return g_tc_launches; }
 
 // Test hook: non-zero routes every dense layer to the CUDA-core kernel.
 void f8_debug_force_direct(int on) { g_force_direct = on != 0; }
+
+void f8_debug_plan_options(unsigned off_mask) { g_plan_off = off_mask; }
+
+int f8_debug_last_plan(int *info, int n) {
+    if (!info || n <= 0) return 0;
+    const int m = n < 10 ? n : 10;
+    for (int i = 0; i < m; ++i) info[i] = g_last_plan[i];
+    return m;
+}
+
+void f8_debug_set_wait_limit_ms(double ms) {
+    int dev = 0, khz = 1965000;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev);
+    g_wait_limit_cycles = ms > 0 ? (unsigned long long)(ms * (double)khz) : 0ull;
+    if (ms > 0 && g_wait_limit_cycles == 0) g_wait_limit_cycles = 1;
+}
+
+f8_status f8_debug_wait_timeout_probe(double limit_ms, void *cuda_stream) {
+    if (!(limit_ms > 0) || limit_ms > 100.0) return fail(F8_ERR_SHAPE, "limit_ms must be in (0, 100]");
+    int *w = f8_status_word();
+    if (!w) return fail(F8_ERR_CUDA, "no status word");
+    int dev = 0, khz = 1965000;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev);
+    unsigned long long cycles = (unsigned long long)(limit_ms * (double)khz);
+    if (cycles == 0) cycles = 1;
+    cudaError_t e = f8_tc_wait_probe(cycles, w, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "wait probe launch");
+    return F8_OK;
+}
 
 f8_status f8_device_status(void) {
     int *w = f8_status_word();
@@ -325,8 +360,9 @@ struct Step {
 struct f8_net {
     std::vector<NetLayer> layers;
     std::vector<int> t_h, t_w, t_c, t_elem;     // per tensor: per-image shape and element size
-    bool overlap_layers = getenv("F8NET_NO_OVERLAP") == nullptr;   // programmatic dependent launch between layers
-    bool sync_layers = getenv("F8NET_SYNC_LAYERS") != nullptr;     // synchronize after every launch (fault attribution)
+    bool overlap_layers = true;                  // programmatic dependent launch between layers
+    bool sync_layers = false;                    // synchronize after every launch (fault attribution)
+    unsigned plan_options = 0;                   // F8_PLAN_OFF_* mask the cached plan was made under
     std::vector<int> t_cp;                       // per tensor: channels as stored (intermediate 8-bit tensors are padded
                                                  // to a multiple of 16 so that every dense layer can use the TMA path)
     int max_batch = 0;
@@ -344,6 +380,12 @@ struct f8_net {
     bool profiling = false;
     std::vector<cudaEvent_t> events;             // steps + 1 events of the last profiled forward
     std::vector<int> event_layer;                // layer each step belongs to
+    // Host copy of the device status word: every pass ends with an asynchronous copy of the word into this pinned
+    // buffer, and the next call looks at it once the copy has completed -- a kernel that gave up a bounded wait is
+    // then reported by f8_net_forward itself, without a synchronisation.
+    int *host_status = nullptr;
+    cudaEvent_t status_ev = nullptr;
+    bool status_pending = false;
 };
 
 namespace {
@@ -596,6 +638,13 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
             }
         }
     }
+    if (cudaHostAlloc((void **)&net->host_status, 64, cudaHostAllocDefault) != cudaSuccess ||
+        cudaEventCreateWithFlags(&net->status_ev, cudaEventDisableTiming) != cudaSuccess) {
+        if (net->host_status) cudaFreeHost(net->host_status);
+        (void)cudaGetLastError();
+        return cleanup(fail(F8_ERR_CUDA, "could not create the status mirror"));
+    }
+    memset(net->host_status, 0, 64);
     *out = net.release();
     return F8_OK;
 }
@@ -639,6 +688,8 @@ f8_status f8_net_get_layer_ms(f8_net *net, float *ms, int *on_tensor_cores) {
 void f8_net_destroy(f8_net *net) {
     if (!net) return;
     for (cudaEvent_t ev : net->events) cudaEventDestroy(ev);
+    if (net->status_ev) cudaEventDestroy(net->status_ev);
+    if (net->host_status) cudaFreeHost(net->host_status);
     free_layers(net);
     delete net;
 }
@@ -655,6 +706,21 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         return fail(F8_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, workspace_bytes);
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int nl = (int)net->layers.size();
+    if (net->status_pending) {
+        const cudaError_t q = cudaEventQuery(net->status_ev);
+        if (q == cudaSuccess) {
+            net->status_pending = false;
+            const int v = net->host_status[0];
+            if (v != 0) {
+                net->host_status[0] = 0;
+                return fail(F8_ERR_TIMEOUT, "a kernel abandoned a bounded wait before or during the previous pass (site %d, layer %d): "
+                            "its output is incomplete; f8_device_status() gives the details and clears the record",
+                            v & 0xff, (v >> 8) - 1);
+            }
+        } else {
+            (void)cudaGetLastError();       // "not ready" is not an error
+        }
+    }
 
     // a first layer whose output is asked for cannot be fused with the pooling layer behind it
     bool dump_fusable = false;
@@ -662,7 +728,10 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         for (int i = 0; i < nl; ++i)
             if (net->layers[i].w_core && layer_dump[i]) dump_fusable = true;
     const bool replan = net->plan_batch != batch || net->plan_x != x || net->plan_y != y || net->plan_ws != workspace ||
-                        net->plan_force_direct != g_force_direct || net->plan_dump_first != dump_fusable;
+                        net->plan_force_direct != g_force_direct || net->plan_dump_first != dump_fusable ||
+                        net->plan_options != g_plan_off;
+    net->overlap_layers = !(g_plan_off & F8_PLAN_OFF_LAYER_OVERLAP);
+    net->sync_layers = (g_plan_off & F8_PLAN_SYNC_LAYERS) != 0;
     if (replan) {
         net->steps.clear();
         net->plan_batch = -1;
@@ -686,11 +755,11 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
             stp.g.n = batch;
             if ((L.d.kind == F8_LAYER_CONV || L.d.kind == F8_LAYER_LINEAR) && !g_force_direct) {
                 const char *why = "";
-                if (L.packed && L.w_core && !getenv("F8_NO_STEM_KERNEL") &&
+                if (L.packed && L.w_core && !(g_plan_off & F8_PLAN_OFF_STEM_KERNEL) &&
                     f8_stem_tc_supported(stp.g, L.q, L.pack_kh, L.pack_kw8 / 32)) {
                     // the stem kernel; it also takes the 3x3 / 2 / pad 1 max pool behind the layer when nothing else
                     // reads the layer's output
-                    bool fuse = !dump_fusable && i + 1 < nl && !getenv("F8_NO_STEM_POOL_FUSION");
+                    bool fuse = !dump_fusable && i + 1 < nl && !(g_plan_off & F8_PLAN_OFF_STEM_POOL_FUSION);
                     if (fuse) {
                         const NetLayer &P = net->layers[i + 1];
                         fuse = P.d.kind == F8_LAYER_MAXPOOL && P.d.src == i + 1 && P.d.conv.kh == 3 && P.d.conv.kw == 3 &&
@@ -752,6 +821,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         net->plan_ws = workspace;
         net->plan_force_direct = g_force_direct;
         net->plan_dump_first = dump_fusable;
+        net->plan_options = g_plan_off;
     }
 
     int launches = 0;
@@ -820,7 +890,134 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         }
     }
     net->last_launches = launches;
+    if (int *word = f8_status_word()) {
+        if (cudaMemcpyAsync(net->host_status, word, sizeof(int), cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+            cudaEventRecord(net->status_ev, st) == cudaSuccess)
+            net->status_pending = true;
+        else
+            (void)cudaGetLastError();
+    }
     return F8_OK;
 }
 
 }   // extern "C"
+
+// ===========================================================================================
+// Forward passes from host buffers: copies of neighbouring passes overlap the compute
+// ===========================================================================================
+
+struct f8_net_host {
+    int depth = 0, batch = 0;
+    size_t x_bytes = 0, y_bytes = 0, ws_bytes = 0;
+    std::vector<f8_net *> nets;                  // one per slot: execution plans are cached per set of buffer addresses
+    std::vector<void *> x_dev, y_dev, ws;
+    cudaStream_t up = nullptr, compute = nullptr, down = nullptr;
+    std::vector<cudaEvent_t> ev_in, ev_done, ev_out;
+    long long count = 0;
+};
+
+extern "C" {
+
+void f8_net_host_destroy(f8_net_host *p) {
+    if (!p) return;
+    if (p->up) cudaStreamSynchronize(p->up);
+    if (p->compute) cudaStreamSynchronize(p->compute);
+    if (p->down) cudaStreamSynchronize(p->down);
+    for (f8_net *n : p->nets) f8_net_destroy(n);
+    for (void *b : p->x_dev) cudaFree(b);
+    for (void *b : p->y_dev) cudaFree(b);
+    for (void *b : p->ws) cudaFree(b);
+    for (cudaEvent_t e : p->ev_in) cudaEventDestroy(e);
+    for (cudaEvent_t e : p->ev_done) cudaEventDestroy(e);
+    for (cudaEvent_t e : p->ev_out) cudaEventDestroy(e);
+    if (p->up) cudaStreamDestroy(p->up);
+    if (p->compute) cudaStreamDestroy(p->compute);
+    if (p->down) cudaStreamDestroy(p->down);
+    delete p;
+}
+
+f8_status f8_net_host_create(const f8_layer_desc *layers, int n_layers, const int8_t *const *host_weights,
+                             const int32_t *const *host_bias, int batch, int depth, f8_net_host **out) {
+    if (!out) return fail(F8_ERR_NULL, "out is NULL");
+    if (batch <= 0 || depth < 1 || depth > 8) return fail(F8_ERR_SHAPE, "batch must be positive and depth in 1..8");
+    std::unique_ptr<f8_net_host, void (*)(f8_net_host *)> p(new (std::nothrow) f8_net_host, f8_net_host_destroy);
+    if (!p) return fail(F8_ERR_CUDA, "out of host memory");
+    p->depth = depth;
+    p->batch = batch;
+    for (int i = 0; i < depth; ++i) {
+        f8_net *n = nullptr;
+        const f8_status s = f8_net_create(layers, n_layers, host_weights, host_bias, batch, &n);
+        if (s != F8_OK) return s;
+        p->nets.push_back(n);
+    }
+    const f8_net *n0 = p->nets[0];
+    const int nl = (int)n0->layers.size();
+    p->x_bytes = (size_t)batch * n0->t_h[0] * n0->t_w[0] * n0->t_c[0];
+    p->y_bytes = (size_t)batch * n0->t_h[nl] * n0->t_w[nl] * n0->t_c[nl] * n0->t_elem[nl];
+    p->ws_bytes = f8_net_workspace_bytes(n0, batch);
+    cudaError_t e = cudaStreamCreateWithFlags(&p->up, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->compute, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->down, cudaStreamNonBlocking);
+    for (int i = 0; i < depth && e == cudaSuccess; ++i) {
+        void *b = nullptr;
+        e = cudaMalloc(&b, round256(p->x_bytes));
+        if (e == cudaSuccess) { p->x_dev.push_back(b); e = cudaMalloc(&b, round256(p->y_bytes)); }
+        if (e == cudaSuccess) { p->y_dev.push_back(b); e = cudaMalloc(&b, round256(p->ws_bytes)); }
+        if (e == cudaSuccess) p->ws.push_back(b);
+        cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+        for (int k = 0; k < 3 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ev[k], cudaEventDisableTiming);
+        if (ev[0]) p->ev_in.push_back(ev[0]);
+        if (ev[1]) p->ev_done.push_back(ev[1]);
+        if (ev[2]) p->ev_out.push_back(ev[2]);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "host pipeline set-up");
+    *out = p.release();
+    return F8_OK;
+}
+
+f8_status f8_net_forward_host(f8_net_host *p, const void *host_x, void *host_y) {
+    if (!p) return fail(F8_ERR_NULL, "pipeline is NULL");
+    if (!host_x || !host_y) return fail(F8_ERR_NULL, "host_x and host_y must not be NULL");
+    const int b = (int)(p->count % p->depth);
+    // upload: once the slot's previous forward pass has read its input
+    cudaError_t e = cudaStreamWaitEvent(p->up, p->ev_done[b], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(p->x_dev[b], host_x, p->x_bytes, cudaMemcpyHostToDevice, p->up);
+    if (e == cudaSuccess) e = cudaEventRecord(p->ev_in[b], p->up);
+    // forward pass: once the input is there and the slot's previous result has left its output buffer
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(p->compute, p->ev_in[b], 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(p->compute, p->ev_out[b], 0);
+    if (e != cudaSuccess) return cuda_fail(e, "host pipeline upload");
+    const f8_status s = f8_net_forward(p->nets[b], p->batch, p->x_dev[b], p->y_dev[b], p->ws[b], round256(p->ws_bytes), nullptr,
+                                       p->compute);
+    if (s != F8_OK) return s;
+    e = cudaEventRecord(p->ev_done[b], p->compute);
+    // download
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(p->down, p->ev_done[b], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(host_y, p->y_dev[b], p->y_bytes, cudaMemcpyDeviceToHost, p->down);
+    if (e == cudaSuccess) e = cudaEventRecord(p->ev_out[b], p->down);
+    if (e != cudaSuccess) return cuda_fail(e, "host pipeline download");
+    ++p->count;
+    return F8_OK;
+}
+
+f8_status f8_net_host_wait(f8_net_host *p) {
+    if (!p) return fail(F8_ERR_NULL, "pipeline is NULL");
+    cudaError_t e = cudaStreamSynchronize(p->up);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(p->compute);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(p->down);
+    if (e != cudaSuccess) return cuda_fail(e, "host pipeline wait");
+    return F8_OK;
+}
+
+f8_status f8_net_host_streams(f8_net_host *p, void **upload, void **compute, void **download) {
+    if (!p) return fail(F8_ERR_NULL, "pipeline is NULL");
+    if (upload) *upload = p->up;
+    if (compute) *compute = p->compute;
+    if (download) *download = p->down;
+    return F8_OK;
+}
+
+int f8_net_host_launches_per_pass(const f8_net_host *p) { return p && !p->nets.empty() ? p->nets[0]->last_launches : 0; }
+
+}   // extern "C"
+

@@ -1,8 +1,6 @@
 // CUDA-core kernels: generic direct convolution (any shape), depthwise convolution, pooling and the
 // stem packing pre-pass.  Depthwise and pooling layers are not dense contractions: they are bound by
 // HBM traffic, so these kernels are organised around wide, coalesced NHWC accesses.
-#include <stdlib.h>
-
 #include "f8_epilogue.cuh"
 
 namespace {
@@ -716,11 +714,10 @@ cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void
                           (((uintptr_t)x | (uintptr_t)y | (uintptr_t)res | (uintptr_t)bias) & 15) == 0 &&
                           (size_t)g.n * g.h * g.w * g.c < (1u << 31) && total * (q.y_kind == F8_S32 ? 4 : 1) < (1u << 31);
     const bool walk_ok = strip_ok && g.stride_h == 1 && !q.has_res && q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24 &&
-                         q.sh_acc == 0 && !getenv("F8_NO_DW_WALK");
+                         q.sh_acc == 0 && !(f8_plan_options_off() & F8_PLAN_OFF_DW_WALK);
     if (walk_ok) {
         // two columns per thread measured slightly ahead of four (96 against 128 registers: 20 against 16 warps per SM)
-        const int cols = getenv("F8_DW_COLS") ? atoi(getenv("F8_DW_COLS")) : 2;
-        const int wcols = cols == 4 ? 4 : 2;
+        const int wcols = 2;
         const int strips = (g.wo + wcols - 1) / wcols;
         // bands of output rows: long enough to amortise the two extra input rows and the tap loads, short enough to
         // give every SM several blocks

@@ -60,7 +60,16 @@ constexpr int MAX_STAGES = 16;
 constexpr int MAX_OUT_BUFS = 4;             // ring of staged output tiles; with a residual, the residual tile lands in the
                                             // buffer first and the epilogue converts it in place
 constexpr int TMEM_COLS = 512;
-constexpr size_t SMEM_LIMIT = 220 * 1024;     // dynamic shared memory budget (227 KiB per CTA minus static data)
+constexpr size_t SMEM_LIMIT = 220 * 1024;     // shared memory budget of stages, staging and resident weights
+constexpr uint32_t CONTROL_BYTES = 1024;      // control block in front of them (plus up to 1023 bytes of alignment slack)
+
+struct TcControl {
+    uint64_t bars[2 * MAX_STAGES + 5];        // full[], empty[], tfull[2], tempty[2], bres
+    uint64_t epi_bars[3 * MAX_OUT_BUFS];      // out_full[], out_free[], res_full[]
+    uint32_t tmem_base_slot;
+    int abort_flag;
+};
+static_assert(sizeof(TcControl) <= CONTROL_BYTES, "control block does not fit its slot");
 
 // Division by a run-time constant without a divide instruction (a 32-bit divide costs a lone thread well over a
 // hundred cycles): q = (n * mul) >> shift is exact for 0 <= n < 2^31 with mul = floor(2^shift / d) + 1,
@@ -129,6 +138,7 @@ struct TcParams {
     uint32_t tx_win;          // bytes of one window load
     uint32_t tx_res;          // bytes of one residual tile load
     int tag;                  // caller's label of this launch (layer index + 1), reported with a timed-out wait
+    unsigned long long wait_limit;   // bound of every mbarrier wait in SM cycles (0: the default, about two seconds)
 };
 
 // ----------------------------------------------------------------------------- epilogue helpers
@@ -194,11 +204,16 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 
     extern __shared__ uint8_t smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 5];
-    __shared__ __align__(8) uint64_t epi_bars[3 * MAX_OUT_BUFS];   // out_full[], out_free[], res_full[]
-    __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
+    uint8_t *smem_aligned = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // Barriers, the tensor-memory address and the abort flag live in the first KiB of the aligned buffer: the same
+    // place in every instantiation of this kernel (the kernel has no static shared memory of its own, so the
+    // compiler lays nothing out).  Everything else follows behind it.
+    TcControl &ctl = *(TcControl *)smem_aligned;
+    uint8_t *smem = smem_aligned + CONTROL_BYTES;
+    uint64_t *const bars = ctl.bars;
+    uint64_t *const epi_bars = ctl.epi_bars;         // out_full[], out_free[], res_full[]
+    uint32_t &tmem_base_slot = ctl.tmem_base_slot;
+    int &abort_flag = ctl.abort_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -257,7 +272,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 
     const int total_tiles = p.m_tiles * p.n_tiles;
     const int k_iters = p.kh * p.kw * p.c_chunks;
-    volatile int *abortp = &abort_flag;
+    const WaitCtx wc = make_wait_ctx(&abort_flag, p.status, p.wait_limit);
     const int tagbits = p.tag << 8;     // status word of a timed-out wait: tag << 8 | site
 
     if (warp == A_PROD_WARP || warp == B_PROD_WARP || ((warp == A2_PROD_WARP || warp == B2_PROD_WARP) && p.alt)) {
@@ -306,7 +321,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int img = fast_div(m_t, p.div_bands);
                 const int y0 = (m_t - img * p.win_bands) * p.win_r;
                 for (int cc = 0; cc < p.c_chunks; ++cc) {
-                    if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, tagbits | 101))) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, wc, tagbits | 101))) {
                         ok = false;
                         break;
                     }
@@ -339,7 +354,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
                     continue;
                 }
-                if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, abortp, p.status, tagbits | 101))) {
+                if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, wc, tagbits | 101))) {
                     ok = false;
                     break;
                 }
@@ -385,7 +400,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         }
         // the resident weights must have landed before this CTA's shared memory may go away (they have, unless
         // the kernel is aborting: the MMA issuers wait for them before their first instruction)
-        if (a_helper) mbar_wait(bres_bar, 0, abortp, p.status, tagbits | 110);
+        if (a_helper) mbar_wait(bres_bar, 0, wc, tagbits | 110);
         }
     } else if (warp == MMA_WARP || warp == MMA2_WARP) {
         // ------------------------------------------------------------------ MMA issuers
@@ -410,7 +425,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const uint32_t stage16 = p.stage_bytes >> 4, sub16 = p.sub_bytes >> 4, a16 = p.a_bytes >> 4;
             const uint32_t b16 = p.b_bytes >> 4, bres_lo = desc_lo0 + (p.bres_off >> 4);
             const uint32_t b_step = p.b_res ? b16 : sub16;
-            if (p.b_res && !mbar_wait(bres_bar, 0, abortp, p.status, tagbits | 111)) ok = false;
+            if (p.b_res && !mbar_wait(bres_bar, 0, wc, tagbits | 111)) ok = false;
             const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
@@ -422,7 +437,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     continue;
                 }
                 const uint32_t acc_phase = (local >> 1) & 1;
-                if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, abortp, p.status, tagbits | 102)) { ok = false; break; }
+                if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1, wc, tagbits | 102)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * 256;   // two 256-column accumulators
                 uint32_t b_tile_lo = 0;
@@ -434,7 +449,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     // one stage use per channel chunk; the nine taps read the same tile at shifted row offsets
                     const uint32_t kb16 = (uint32_t)p.kb >> 4;
                     for (int cc = 0; cc < p.c_chunks; ++cc) {
-                        if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, tagbits | 103)) { ok = false; break; }
+                        if (!mbar_wait(full_bar + 8 * stage, phase, wc, tagbits | 103)) { ok = false; break; }
                         tc_fence_after();
                         uint32_t first = cc != 0 ? 1u : 0u;
                         uint32_t b_lo = b_tile_lo + (uint32_t)cc * b16;
@@ -455,7 +470,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     }
                 } else
                 for (int kc = 0; kc < k_iters; kc += p.group) {
-                    if (!mbar_wait(full_bar + 8 * stage, phase, abortp, p.status, tagbits | 103)) { ok = false; break; }
+                    if (!mbar_wait(full_bar + 8 * stage, phase, wc, tagbits | 103)) { ok = false; break; }
                     tc_fence_after();
                     const int subs = min(p.group, k_iters - kc);
                     const uint32_t first = kc != 0 ? 1u : 0u;      // the tile's first MMA overwrites the accumulator
@@ -483,7 +498,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 for (int g = max(0, total_uses - p.stages); g < total_uses; ++g) {
                     const int t_of_g = g / uses_tile;
                     if (p.dual_issue && (t_of_g & 1) != q_issuer) continue;
-                    mbar_wait(empty_bar + 8 * (g % p.stages), (uint32_t)(g / p.stages) & 1u, abortp, p.status, tagbits | 112);
+                    mbar_wait(empty_bar + 8 * (g % p.stages), (uint32_t)(g / p.stages) & 1u, wc, tagbits | 112);
                 }
             }
             if (!ok && committed_any) {
@@ -503,7 +518,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             uint32_t bphase = 0;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
-                if (!mbar_wait(out_full + 8 * b, bphase, abortp, p.status, tagbits | 108)) break;
+                if (!mbar_wait(out_full + 8 * b, bphase, wc, tagbits | 108)) break;
                 const uint32_t src = smem_base + p.out_off + b * p.out_bytes;
                 if (p.win) {
                     const int img = fast_div(m_t, p.div_bands);
@@ -536,7 +551,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
-                if (!mbar_wait(out_free + 8 * rb, rphase ^ 1, abortp, p.status, tagbits | 106)) { ok = false; break; }
+                if (!mbar_wait(out_free + 8 * rb, rphase ^ 1, wc, tagbits | 106)) { ok = false; break; }
                 const uint32_t fb = res_full + 8 * rb;
                 mbar_expect_tx(fb, p.tx_res);
                 if (p.win) {
@@ -598,10 +613,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int c_first = n_t * p.bn + ch_begin * 16;
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
-                bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, tagbits | 104);
+                bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, wc, tagbits | 104);
                 // the buffer holds the residual tile (which implies that its previous store has left), or is free
-                if (RES) got = mbar_wait(res_full + 8 * ob, ophase, abortp, p.status, tagbits | 107) && got;
-                else got = mbar_wait(out_free + 8 * ob, ophase ^ 1, abortp, p.status, tagbits | 109) && got;
+                if (RES) got = mbar_wait(res_full + 8 * ob, ophase, wc, tagbits | 107) && got;
+                else got = mbar_wait(out_free + 8 * ob, ophase ^ 1, wc, tagbits | 109) && got;
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t out_buf = smem_base + p.out_off + ob * p.out_bytes;
@@ -648,7 +663,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const size_t row = (size_t)m_t * TILE_M + tile_row;
                 const bool row_valid = row < (size_t)p.M;
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
-                if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar + 8 * acc, acc_phase, abortp, p.status, tagbits | 104))) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar + 8 * acc, acc_phase, wc, tagbits | 104))) { ok = false; break; }
                 tc_fence_after();
                 for (int i = 0; i < nch; ++i) {
                     const int co0 = n0 + (ch_begin + i) * 16;
@@ -705,13 +720,28 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) f8_mma_probe_kernel(int iters,
         for (int i = 0; i < iters; ++i)
             mma_i8(tmem_base + (i & 1) * 256, a_desc + 2 * (i & 3), b_desc + 2 * (i & 3), idesc, i > 1 ? 1u : 0u);
         mma_commit(smem_u32(&bar));
-        mbar_wait(smem_u32(&bar), 0, &abort_flag, status, 105);
+        mbar_wait(smem_u32(&bar), 0, make_wait_ctx(&abort_flag, status, 0), 105);
     }
     tc_fence_before();
     __syncthreads();
     if (warp == MMA_WARP) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ----------------------------------------------------------------------------- time-out probe
+
+// The time-out path of the bounded waits, exercised without harming anything: a barrier with one expected arrival that
+// nobody makes.  The wait gives up after `limit_cycles`, records itself in the status word and the kernel returns.
+__global__ void __launch_bounds__(32, 1) f8_wait_probe_kernel(unsigned long long limit_cycles, int *status) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(smem_u32(&bar), 0, make_wait_ctx(&abort_flag, status, limit_cycles), 199);
     }
 }
 
@@ -855,9 +885,6 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         // before.  With a residual a buffer goes through load -> convert in place -> store, and a residual tile takes
         // about as long to arrive from HBM as a tile takes to compute: three buffers (four when they are small).
         p.out_bufs = !q.has_res ? 2 : (p.out_bytes <= 16 * 1024 ? 4 : 3);
-        if (getenv("F8_OUT_BUFS")) p.out_bufs = atoi(getenv("F8_OUT_BUFS"));
-        if (p.out_bufs < 1) p.out_bufs = 1;
-        if (p.out_bufs > MAX_OUT_BUFS) p.out_bufs = MAX_OUT_BUFS;
         staging = (size_t)p.out_bytes * p.out_bufs + bias_bytes;
     }
     const size_t ktab_bytes = ((size_t)g.kh * g.kw * p.c_chunks * 8 + 1023) / 1024 * 1024;
@@ -874,8 +901,9 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // resident weights: one N tile, and room left for at least four activation tiles in flight (with only two, a
     // 3x3 layer of 128 channels waits on every im2col load: measured 62 us against 48 us with streamed weights)
     const size_t b_all = (size_t)p.n_tiles * k_iters * b_bytes;
+    const unsigned off = f8_plan_options_off();
     p.b_res = (p.n_tiles == 1 && b_all + 4 * (size_t)p.a_bytes <= avail && b_all + 32 * 1024 <= avail &&
-               !getenv("F8_NO_BRES")) ? 1 : 0;
+               !(off & F8_PLAN_OFF_RESIDENT_WEIGHTS)) ? 1 : 0;
     if (p.b_res) {
         avail -= b_all;
         p.sub_bytes = p.a_bytes;
@@ -890,7 +918,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.win = 0;
     if (staged && p.kb == 128 && g.kh == 3 && g.kw == 3 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 1 && g.pad_w == 1 &&
         g.pad_h_end < 0 && p.n_tiles == 1 && g.w + 2 <= TILE_M && g.w == g.wo && g.h == g.ho && g.c % p.kb == 0 &&
-        !getenv("F8_NO_WIN")) {
+        !(off & (F8_PLAN_OFF_WINDOWED | F8_PLAN_OFF_RESIDENT_WEIGHTS))) {
         const int wp = g.w + 2;
         const int r = std::min(TILE_M / wp, g.ho);
         const int bands = (g.ho + r - 1) / r;
@@ -942,8 +970,8 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.uses = (k_iters + group - 1) / group;
     }
     const int stages = p.stages;
-    p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !getenv("F8_NO_DUAL")) ? 1 : 0;
-    p.alt = (!p.b_res && !p.dual_issue && !p.win && p.stages >= 2 && !getenv("F8_NO_ALT")) ? 1 : 0;
+    p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !(off & F8_PLAN_OFF_DUAL_ISSUE)) ? 1 : 0;
+    p.alt = (!p.b_res && !p.dual_issue && !p.win && p.stages >= 2 && !(off & F8_PLAN_OFF_ALT_PRODUCERS)) ? 1 : 0;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
     p.bias_off = p.out_off + (uint32_t)p.out_bufs * p.out_bytes;
     p.ktab_off = (uint32_t)(p.stages * p.stage_bytes + staging - ktab_bytes);
@@ -1074,30 +1102,35 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     const int total_tiles = p.m_tiles * p.n_tiles;
     plan->grid = total_tiles < sms ? total_tiles : sms;
     // at least half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
-    plan->smem = (size_t)p.stages * p.stage_bytes + staging + (p.b_res ? b_all : 0) + 1024;
+    plan->smem = (size_t)p.stages * p.stage_bytes + staging + (p.b_res ? b_all : 0) + 1024 + CONTROL_BYTES;
     if (plan->smem < 120 * 1024) plan->smem = 120 * 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        const int bytes = (int)SMEM_LIMIT;
+    p.wait_limit = f8_wait_limit_cycles();
+    // what the plan decided, for tests that must know which code path a case exercises
+    {
+        int *info = f8_last_plan_info();
+        info[0] = (p.b_res ? F8_PLAN_RESIDENT_WEIGHTS : 0) | (p.win ? F8_PLAN_WINDOWED : 0) | (p.dual_issue ? F8_PLAN_DUAL_ISSUE : 0) |
+                  (p.alt ? F8_PLAN_ALT_PRODUCERS : 0) | (p.a_plain ? F8_PLAN_PLAIN_MATRIX : 0) | (staged ? F8_PLAN_STAGED_EPILOGUE : 0);
+        info[1] = p.epi; info[2] = p.bn; info[3] = p.kb; info[4] = p.stages; info[5] = p.group;
+        info[6] = p.m_tiles; info[7] = p.n_tiles; info[8] = plan->grid; info[9] = staged ? p.out_bufs : 0;
+    }
+    // the opt-in to large dynamic shared memory is a per-device attribute of each kernel
+    static bool attr_set[64] = {false};
+    if (dev < 0 || dev >= 64) {
+        *why = "device index out of range";
+        return cudaErrorInvalidDevice;
+    }
+    if (!attr_set[dev]) {
+        const int bytes = (int)(SMEM_LIMIT + CONTROL_BYTES);
         cudaError_t e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_GENERIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e != cudaSuccess) {
-            if (getenv("F8NET_VERBOSE")) {
-                cudaFuncAttributes fa;
-                int optin = 0, dev2 = 0;
-                cudaGetDevice(&dev2);
-                cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev2);
-                if (cudaFuncGetAttributes(&fa, f8_conv_gemm_tc_kernel<EPI_U8>) == cudaSuccess)
-                    fprintf(stderr, "f8net: static smem %zu, regs %d, max threads %d, local %zu, optin %d, asked %d\n",
-                            fa.sharedSizeBytes, fa.numRegs, fa.maxThreadsPerBlock, fa.localSizeBytes, optin, bytes);
-            }
             *why = "cudaFuncSetAttribute(MaxDynamicSharedMemorySize) failed";
             return e;
         }
-        attr_set = true;
+        attr_set[dev] = true;
     }
     return cudaSuccess;
 }
@@ -1128,6 +1161,13 @@ cudaError_t f8_tc_launch(const F8TcPlan *plan, bool overlap_previous, cudaStream
         case EPI_S8_RES: return launch_variant<EPI_S8_RES>(plan, overlap_previous, st);
         default: return launch_variant<EPI_GENERIC>(plan, overlap_previous, st);
     }
+}
+
+cudaError_t f8_tc_wait_probe(unsigned long long limit_cycles, int *status_word, cudaStream_t st) {
+    // never the unbounded default: a probe waits a hundred milliseconds at most
+    if (limit_cycles == 0 || limit_cycles > 250000000ull) limit_cycles = 250000000ull;
+    f8_wait_probe_kernel<<<1, 32, 0, st>>>(limit_cycles, status_word);
+    return cudaGetLastError();
 }
 
 cudaError_t f8_tc_probe(int iters, double *ops, int *status_word, cudaStream_t st) {

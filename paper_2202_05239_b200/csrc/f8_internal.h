@@ -77,6 +77,8 @@ void f8_tc_plan_set_tag(F8TcPlan *plan, int tag);
 // and bias reads then run early, so it is for callers whose weights no earlier work in the stream writes.
 cudaError_t f8_tc_launch(const F8TcPlan *plan, bool overlap_previous, cudaStream_t st);
 cudaError_t f8_tc_probe(int iters, double *ops, int *status_word, cudaStream_t st);
+// One thread waits `limit_cycles` on a barrier nothing arrives at, records the time-out (site 199) and returns.
+cudaError_t f8_tc_wait_probe(unsigned long long limit_cycles, int *status_word, cudaStream_t st);
 
 // ---- first-layer kernel (f8_stem_tc.cu): stride-2 convolution over an image with <= 4 channels, optionally fused
 // with the 3x3 / 2 / pad 1 max pool behind it.  kh2 row pairs per window starting `top` pairs above the output row,
@@ -86,8 +88,14 @@ cudaError_t f8_launch_stem_tc(const F8ConvGeom &g, const F8Requant &q, int kh2, 
                               const void *x, const int8_t *w_core, const int32_t *bias, void *y, int *status_word, int tag,
                               cudaStream_t st, bool overlap_previous);
 
-// Device status word (0 = fine); allocated once per process on first use.
+// Device status word (0 = fine); allocated once per device on first use.
 int *f8_status_word();
+
+// Planning choices switched off by f8_debug_plan_options (F8_PLAN_OFF_* bits), the bound of in-kernel waits in SM
+// cycles (0 = default) and the record of the last tensor-core plan (10 ints, see f8_debug_last_plan).
+unsigned f8_plan_options_off();
+unsigned long long f8_wait_limit_cycles();
+int *f8_last_plan_info();
 
 // Records a message for f8_last_error() and returns `s` (for entry points defined outside f8_api.cu).
 f8_status f8_set_error(f8_status s, const char *message);

@@ -60,6 +60,7 @@ struct StemParams {
     uint8_t *y;
     int *status;
     int tag;
+    unsigned long long wait_limit;   // bound of the accumulator wait in SM cycles (0: the default)
 };
 
 __device__ __forceinline__ uint32_t ldg32(const uint8_t *p) { return __ldg((const uint32_t *)p); }
@@ -128,6 +129,7 @@ __global__ void __launch_bounds__(STEM_THREADS, 3) f8_stem_tc_kernel(const StemP
     grid_dependency_wait();        // the image / the output buffer may belong to earlier work in the stream
 
     volatile int *abortp = &abort_flag;
+    const WaitCtx wc = make_wait_ctx(&abort_flag, p.status, p.wait_limit);
     const int tagbits = p.tag << 8;
     const long long total = grid_units_total;
     const int u_begin = (int)(total * blockIdx.x / gridDim.x), u_end = (int)(total * (blockIdx.x + 1) / gridDim.x);
@@ -264,7 +266,7 @@ __global__ void __launch_bounds__(STEM_THREADS, 3) f8_stem_tc_kernel(const StemP
                 bool got = false;
 #pragma unroll 1
                 for (int t = 0; t < 4 && !got; ++t) got = mbar_try_wait_hint(smem_u32(&acc_bar[k & 1]), (uint32_t)(k >> 1) & 1u, 4000u);
-                if (!got) got = mbar_wait(smem_u32(&acc_bar[k & 1]), (uint32_t)(k >> 1) & 1u, abortp, p.status, tagbits | 120);
+                if (!got) got = mbar_wait(smem_u32(&acc_bar[k & 1]), (uint32_t)(k >> 1) & 1u, wc, tagbits | 120);
                 if (__all_sync(0xffffffffu, got)) {
                     tc_fence_after();
                     const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((k & 1) * p.acc_cols);
@@ -417,6 +419,7 @@ cudaError_t f8_launch_stem_tc(const F8ConvGeom &g, const F8Requant &q, int kh2, 
     p.signed_out = q.y_kind == F8_S8 ? 1 : 0;
     p.x_signed = g.x_signed;
     p.x = (const uint8_t *)x; p.wk = w_core; p.bias = bias; p.y = (uint8_t *)y; p.status = status_word; p.tag = tag;
+    p.wait_limit = f8_wait_limit_cycles();
 
     const bool fast = ((uintptr_t)x & 3) == 0 && ((size_t)g.n * g.h * g.w * g.c) % 4 == 0;
     const bool sgn = p.signed_out != 0;

@@ -8,9 +8,27 @@
 
 namespace {
 
-constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
+constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;   // default bound of a wait: ~2 s at 2 GHz
 constexpr unsigned MIN_POLLS_BEFORE_TIMEOUT = 1u << 16;             // failed polls a wait needs before it may give up
 constexpr unsigned long long DRAIN_LIMIT_CYCLES = 200000000ull;
+
+// What a bounded wait needs besides the barrier: where to raise the CTA's abort flag, where to record the wait
+// that gave up, and how long to try.  limit_cycles is a launch parameter (0 = the default above).
+struct WaitCtx {
+    volatile int *abort_flag;
+    int *status;
+    unsigned long long limit_cycles;
+    unsigned min_polls;
+};
+__device__ __forceinline__ WaitCtx make_wait_ctx(volatile int *abort_flag, int *status, unsigned long long limit_cycles) {
+    WaitCtx c;
+    c.abort_flag = abort_flag;
+    c.status = status;
+    c.limit_cycles = limit_cycles ? limit_cycles : WAIT_LIMIT_CYCLES;
+    // a short limit is a test of the time-out path itself: it must not wait for the poll count of a real run
+    c.min_polls = limit_cycles && limit_cycles < (1ull << 28) ? 256u : MIN_POLLS_BEFORE_TIMEOUT;
+    return c;
+}
 
 // ----------------------------------------------------------------------------- PTX wrappers
 
@@ -58,8 +76,9 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity
 }
 
 // Bounded wait.  Returns false when the kernel is aborting (this wait or another one ran out).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                            int code) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtx &wc, int code) {
+    volatile int *abort_flag = wc.abort_flag;
+    int *status = wc.status;
     const unsigned long long t0 = clock64();
     unsigned long long g0 = 0;
     unsigned spins = 0;
@@ -67,11 +86,11 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
             // wall clock of a wait that is already long (reading it costs the warp a microsecond or so)
-            if (spins == 4096u) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0));
+            if (spins == 4096u || (spins == 64u && wc.min_polls < 4096u)) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0));
             if (*abort_flag) return false;
             // both conditions: the cycle counter keeps running while the context is switched out (a profiler
             // replaying the kernel does that for seconds), the poll count does not
-            if (spins >= MIN_POLLS_BEFORE_TIMEOUT && (unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
+            if (spins >= wc.min_polls && (unsigned long long)(clock64() - t0) > wc.limit_cycles) {
                 *abort_flag = 1;
                 if (atomicCAS(status, 0, code) == 0) {
                     // the first wait to give up leaves a description: CTA, thread, barrier address, parity
@@ -84,18 +103,17 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
                     const unsigned long long dc = clock64() - t0, dg = g1 - g0;
                     status[5] = (int)spins;
                     status[6] = (int)(dc >> 20);       // SM cycles / 2^20
-                    status[7] = (int)(dg >> 10);       // wall-clock microseconds (ns / 1024) since the 4096th poll
+                    status[7] = (int)(dg >> 10);       // wall-clock microseconds (ns / 1024) since the 4096th poll (the 64th under a short test limit)
                 }
                 return false;
             }
         }
     }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                          int code) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx &wc, int code) {
     if (mbar_try_wait(bar, parity)) return true;
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status, code);
+    return mbar_wait_slow(bar, parity, wc, code);
 }
 
 __device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w,

@@ -49,20 +49,58 @@ def random_residual(rng, n, layer):
     return rng.integers(0, 256, size=shape).astype(np.uint8)
 
 
-def check_layer(ref, layer, x, res=None, force_direct=False, expect_tc=None):
-    """Runs one layer on the GPU through the C ABI and on the oracle; asserts bit-exact equality."""
+GUARD = 4096          # bytes of poison on either side of every output buffer
+POISON = 0xA5
+
+
+class Guarded:
+    """An output tensor inside a poison-filled allocation: `t` is the tensor the kernel writes, `intact()` says whether
+    the bands in front of and behind it still hold the poison (a stand-in for a memory checker: an out-of-bounds
+    store next to an output shows up here).  The tensor itself starts out poisoned too, so an element a kernel
+    forgot to write is very unlikely to compare equal."""
+
+    def __init__(self, shape, dtype, device="cuda"):
+        self.nbytes = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        pad = (-self.nbytes) % 256
+        self.raw = torch.full((GUARD + self.nbytes + pad + GUARD,), POISON, dtype=torch.uint8, device=device)
+        self.t = self.raw[GUARD:GUARD + self.nbytes].view(dtype).view(shape)
+
+    def intact(self) -> bool:
+        head, tail = self.raw[:GUARD], self.raw[GUARD + self.nbytes:]
+        return bool((head == POISON).all().item()) and bool((tail == POISON).all().item())
+
+
+def assert_equal_arrays(got, want, what=""):
+    bad = np.argwhere(got != want)
+    assert bad.shape[0] == 0, (f"{what}{bad.shape[0]} of {want.size} elements differ; first at {bad[0]}: "
+                               f"got {got[tuple(bad[0])]} want {want[tuple(bad[0])]}")
+
+
+def check_layer(ref, layer, x, res=None, force_direct=False, expect_tc=None, plan_off=0, expect_flags=0,
+                forbid_flags=0, min_tiles_per_cta=0):
+    """Runs one layer on the GPU through the C ABI and on the oracle; asserts bit-exact equality and that nothing
+    next to the output buffer was touched.  plan_off switches planning choices off (the alternative code paths);
+    expect_flags / forbid_flags / min_tiles_per_cta assert what the tensor-core plan decided."""
     a = api()
     want = ref.run_layer(layer, x, res)
     a.f8_debug_force_direct(force_direct)
+    a.f8_debug_plan_options(plan_off)
     before = a.f8_tc_launch_count()
+    out = Guarded(a.layer_output_shape(layer, x.shape[0]), a.torch_dtype(layer.y_dtype))
     try:
-        got = a.run_layer(layer, a.to_device(x), a.to_device(res) if res is not None else None)
+        got = a.run_layer(layer, a.to_device(x), a.to_device(res) if res is not None else None, out=out.t)
         torch.cuda.synchronize()
         a.f8_device_status()
     finally:
         a.f8_debug_force_direct(False)
+        a.f8_debug_plan_options(0)
     if expect_tc is not None:
         assert (a.f8_tc_launch_count() - before == 1) == expect_tc, "layer did not take the expected path"
-    got = got.cpu().numpy().reshape(want.shape)
-    bad = np.argwhere(got != want)
-    assert bad.shape[0] == 0, f"{bad.shape[0]} of {want.size} elements differ; first at {bad[0]}: got {got[tuple(bad[0])]} want {want[tuple(bad[0])]}"
+    if expect_flags or forbid_flags or min_tiles_per_cta:
+        plan = a.f8_debug_last_plan()
+        assert plan["flags"] & expect_flags == expect_flags, f"plan {plan} lacks flags {expect_flags}"
+        assert plan["flags"] & forbid_flags == 0, f"plan {plan} has one of the flags {forbid_flags}"
+        tiles = plan["m_tiles"] * plan["n_tiles"]
+        assert tiles >= min_tiles_per_cta * plan["ctas"], f"plan {plan}: fewer than {min_tiles_per_cta} tiles per CTA"
+    assert out.intact(), "the kernel wrote outside its output buffer"
+    assert_equal_arrays(got.cpu().numpy().reshape(want.shape), want)

@@ -91,9 +91,56 @@ def test_extreme_operands_on_tensor_cores(ref):
 
 @pytest.mark.parametrize("index", range(6))
 def test_layer_sweep_shapes(ref, index):
-    """The CNN layer-shape sweep at a batch the oracle finishes in seconds."""
-    layer, x = synth.sweep_case(index, batch=6, seed=0)
+    """The CNN layer-shape sweep at its stated batch of 32 (the oracle needs a fraction of a second per layer)."""
+    layer, x = synth.sweep_case(index, batch=32, seed=0)
     check_layer(ref, layer, x, expect_tc=True)
+
+
+# Cases in which every CTA walks several tiles: the accumulator double buffer, the stage ring, the output ring and the
+# second issuer's tile alternation all wrap around.  One case per plan mode and epilogue variant; the mode is asserted.
+#   (h, w, c, c_out, k, stride, n, x_signed, y_dtype, res, plan_off, expect, forbid)
+def _modes():
+    from paper_2202_05239_b200 import api as a
+    RW, WIN, DUAL, ALT, STAGED = (a.PLAN_RESIDENT_WEIGHTS, a.PLAN_WINDOWED, a.PLAN_DUAL_ISSUE, a.PLAN_ALT_PRODUCERS,
+                                  a.PLAN_STAGED_EPILOGUE)
+    return [
+        # resident weights, two issuers, u8
+        (56, 56, 64, 64, 1, 1, 32, False, synth.U8, False, 0, RW | DUAL | STAGED, WIN),
+        # resident weights, 256-wide tile, residual, u8 and s8 outputs
+        (56, 56, 64, 256, 1, 1, 32, False, synth.U8, True, 0, RW | STAGED, 0),
+        (56, 56, 64, 256, 1, 1, 32, True, synth.S8, True, 0, RW | STAGED, 0),
+        # signed output without residual, resident weights, 3x3 through im2col, two issuers
+        (56, 56, 64, 64, 3, 1, 32, False, synth.S8, False, 0, RW | DUAL | STAGED, WIN),
+        # streamed weights, two N tiles, second producer pair
+        (28, 28, 512, 512, 1, 1, 50, False, synth.U8, False, 0, ALT | STAGED, RW),
+        # the same without the second producer pair
+        (28, 28, 512, 512, 1, 1, 50, False, synth.U8, False, a.PLAN_OFF_ALT_PRODUCERS, STAGED, RW | ALT),
+        # K-heavy 3x3 through im2col, streamed weights
+        (14, 14, 256, 256, 3, 1, 400, False, synth.U8, False, 0, STAGED, RW),
+        # windowed 3x3 with residual
+        (28, 28, 128, 128, 3, 1, 100, False, synth.U8, True, 0, WIN | RW | STAGED, 0),
+        # the same layer through im2col (windowed mode off), then with streamed weights as well
+        (28, 28, 128, 128, 3, 1, 100, False, synth.U8, True, a.PLAN_OFF_WINDOWED, STAGED, WIN),
+        (28, 28, 128, 128, 3, 1, 100, False, synth.U8, True, a.PLAN_OFF_RESIDENT_WEIGHTS, STAGED, WIN | RW),
+        # one issuer where two are the default
+        (56, 56, 64, 64, 1, 1, 32, False, synth.U8, False, a.PLAN_OFF_DUAL_ISSUE, RW | STAGED, DUAL),
+        # int32 output: generic epilogue with direct stores, many tiles
+        (56, 56, 256, 64, 1, 1, 32, False, synth.S32, False, 0, 0, STAGED),
+        # stride 2 with residual and streamed weights
+        (56, 56, 128, 128, 3, 2, 100, False, synth.U8, True, 0, STAGED, 0),
+    ]
+
+
+@pytest.mark.parametrize("case", range(13))
+def test_many_tiles_per_cta_in_every_plan_mode(ref, case):
+    h, w, c, c_out, k, stride, n, xs, y_dtype, with_res, off, expect, forbid = _modes()[case]
+    rng = np.random.default_rng(900 + case)
+    layer = random_conv_layer(rng, h=h, w=w, c=c, c_out=c_out, k=k, stride=stride, pad=k // 2, x_signed=xs,
+                              y_dtype=y_dtype, with_res=with_res)
+    x = random_input(rng, n, layer)
+    res = random_residual(rng, n, layer) if with_res else None
+    check_layer(ref, layer, x, res, expect_tc=True, plan_off=off, expect_flags=expect, forbid_flags=forbid,
+                min_tiles_per_cta=4)
 
 
 def test_linear_on_tensor_cores(ref):

@@ -4,31 +4,43 @@ import pytest
 import torch
 
 from paper_2202_05239_b200 import synth
-from gpu_util import api
+from gpu_util import api, Guarded, assert_equal_arrays
 
 pytestmark = pytest.mark.gpu
 
 
-def _compare_net(ref, name, batch, image, force_direct=False, seed=0):
+def _layer_shape(l, batch):
+    return (batch, l.c_out) if l.kind in (synth.LINEAR, synth.GAP) else (batch, l.ho, l.wo, l.c_out)
+
+
+def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0):
+    """Every layer's output against the oracle.  The dump buffers, the network output and the workspace sit between
+    poisoned guard bands that must come back untouched."""
     a = api()
     layers = synth.make_net(name, seed, image=image)
     x = synth.draw_image(batch, seed + 1, image, image)
     want = ref.net_forward(layers, x)
     a.f8_debug_force_direct(force_direct)
+    a.f8_debug_plan_options(plan_off)
     before = a.f8_tc_launch_count()
     try:
         net = a.Net(layers, batch)
-        dump = [net.layer_output(i, batch) for i in range(len(layers))]
-        out = net.forward(a.to_device(x), dump=dump)
+        guards = [Guarded(_layer_shape(l, batch), a.torch_dtype(l.y_dtype)) for l in layers]
+        dump = [g.t for g in guards]
+        out = Guarded((batch,) + net.out_shape, net.out_dtype)
+        ws = Guarded((net.workspace_bytes(batch),), torch.uint8)
+        net.forward(a.to_device(x), out=out.t, workspace=ws.t, dump=dump)
         torch.cuda.synchronize()
         a.f8_device_status()
     finally:
         a.f8_debug_force_direct(False)
+        a.f8_debug_plan_options(0)
     for i, l in enumerate(layers):
         got = dump[i].cpu().numpy().reshape(want[i + 1].shape)
-        bad = int((got != want[i + 1]).sum())
-        assert bad == 0, f"{name} layer {i} ({l.name}): {bad} of {got.size} elements differ"
-    assert np.array_equal(out.cpu().numpy(), want[-1])
+        assert_equal_arrays(got, want[i + 1], f"{name} layer {i} ({l.name}): ")
+        assert guards[i].intact(), f"{name} layer {i} ({l.name}): bytes next to the dump buffer were overwritten"
+    assert np.array_equal(out.t.cpu().numpy(), want[-1])
+    assert out.intact() and ws.intact(), "bytes next to the output or the workspace were overwritten"
     assert net.last_launch_count >= len(layers)
     tc = a.f8_tc_launch_count() - before
     if force_direct:
@@ -45,9 +57,60 @@ def test_net_parity_cuda_core_path(ref, name):
 
 
 @pytest.mark.parametrize("name,batch,image", [("resnet18", 3, 224), ("resnet50", 2, 224), ("mobilenetv2", 3, 224),
-                                              ("resnet50", 1, 224), ("resnet18", 5, 96), ("mobilenetv1", 3, 224)])
+                                              ("resnet50", 1, 224), ("resnet18", 5, 96), ("mobilenetv1", 3, 224),
+                                              ("mobilenetv2", 1, 224), ("resnet18", 1, 224), ("mobilenetv1", 1, 224)])
 def test_net_parity(ref, name, batch, image):
     _compare_net(ref, name, batch, image)
+
+
+@pytest.mark.parametrize("name", ["resnet50", "resnet18", "mobilenetv2", "mobilenetv1"])
+def test_net_parity_batch_64_every_layer(ref, name):
+    """Throughput batches: at 64 images every CTA of the tensor-core kernel walks many tiles in the early stages."""
+    _compare_net(ref, name, 64, 224)
+
+
+def _off_masks():
+    from paper_2202_05239_b200 import api as a
+    return [a.PLAN_OFF_STEM_KERNEL, a.PLAN_OFF_STEM_POOL_FUSION, a.PLAN_OFF_LAYER_OVERLAP, a.PLAN_OFF_MICRO_BATCH,
+            a.PLAN_OFF_DUAL_ISSUE | a.PLAN_OFF_ALT_PRODUCERS, a.PLAN_OFF_RESIDENT_WEIGHTS, a.PLAN_OFF_PAIRS,
+            a.PLAN_SYNC_LAYERS]
+
+
+@pytest.mark.parametrize("case", range(8))
+def test_net_parity_with_planning_choices_switched_off(ref, case):
+    """The alternative code paths behind f8_debug_plan_options give the same bits."""
+    _compare_net(ref, "resnet50", 4, 224, plan_off=_off_masks()[case])
+
+
+def test_mobilenet_parity_with_the_strip_kernel(ref):
+    a = api()
+    _compare_net(ref, "mobilenetv1", 3, 224, plan_off=a.PLAN_OFF_DW_WALK)
+
+
+def _sampled_full_batch(ref, name, batch, samples):
+    """The timed configuration: one full-batch launch with every layer dumped; images are independent, so the oracle
+    checks a sample of them one by one, every layer."""
+    a = api()
+    layers = synth.make_net(name, 0)
+    x = synth.draw_image(batch, 1)
+    net = a.Net(layers, batch)
+    dump = [net.layer_output(i, batch) for i in range(len(layers))]
+    out = net.forward(a.to_device(x), dump=dump)
+    torch.cuda.synchronize()
+    a.f8_device_status()
+    for i in samples:
+        want = ref.net_forward(layers, x[i:i + 1])
+        for li, l in enumerate(layers):
+            got = dump[li][i:i + 1].cpu().numpy().reshape(want[li + 1].shape)
+            assert_equal_arrays(got, want[li + 1], f"{name} image {i} layer {li} ({l.name}): ")
+        assert np.array_equal(out[i:i + 1].cpu().numpy(), want[-1])
+    del dump
+    net.close()
+
+
+@pytest.mark.parametrize("name,batch", [("resnet18", 256), ("resnet50", 256), ("mobilenetv1", 256)])
+def test_full_batch_sampled_images_every_layer(ref, name, batch):
+    _sampled_full_batch(ref, name, batch, (0, 101, 255))
 
 
 def test_resnet50_full_batch_sampled_images(ref):

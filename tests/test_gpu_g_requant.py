@@ -10,14 +10,13 @@ from gpu_util import api
 pytestmark = pytest.mark.gpu
 
 
-def _want(ref, acc, s, lo, hi):
-    # the oracle's scalar definition on a sample, and the same definition in int64 numpy on everything
-    a = acc.astype(np.int64)
-    t = ((a + (1 << (s - 1))) >> s) if s > 0 else (a << (-s))
-    y = np.clip(t, lo, hi)
-    for i in np.linspace(0, acc.size - 1, 50).astype(int):
-        assert ref.shift_round_clip(int(acc.flat[i]), s, lo, hi) == int(y.flat[i])
-    return y
+def _want(ref, acc, fa, fl, dtype):
+    """Every element through the oracle's own quantiser: a fully connected layer with a zero input and zero weights
+    hands each int32 value, as the bias in accumulator format fa, to the oracle's rounding shift + clip."""
+    n = acc.size
+    y = ref.linear(np.zeros((1, 1), dtype=np.uint8), np.zeros((n, 1), dtype=np.int8), np.ascontiguousarray(acc),
+                   fl_x=0, fl_w=fa, fl_y=fl, y_dtype=dtype)
+    return y.reshape(n).astype(np.int64)
 
 
 @pytest.mark.parametrize("n,fa,fl1,d1,fl2,d2", [
@@ -37,10 +36,9 @@ def test_requantize_dual(ref, n, fa, fl1, d1, fl2, d2):
     y2 = torch.empty(n, dtype=a.torch_dtype(d2), device="cuda") if d2 is not None else None
     a.f8_requantize_dual_fixed(accd, fa, y1, d1, fl1, y2, d2 if d2 is not None else 0, fl2 if fl2 is not None else 0)
     torch.cuda.synchronize()
-    lohi = {synth.U8: (0, 255), synth.S8: (-127, 127)}
-    assert np.array_equal(y1.cpu().numpy().astype(np.int64), _want(ref, acc, fa - fl1, *lohi[d1]))
+    assert np.array_equal(y1.cpu().numpy().astype(np.int64), _want(ref, acc, fa, fl1, d1))
     if y2 is not None:
-        assert np.array_equal(y2.cpu().numpy().astype(np.int64), _want(ref, acc, fa - fl2, *lohi[d2]))
+        assert np.array_equal(y2.cpu().numpy().astype(np.int64), _want(ref, acc, fa, fl2, d2))
 
 
 def test_private_formats_versus_realigning_one_tensor(ref):
