@@ -150,6 +150,84 @@ int f8ref_conv2d(int n, int h, int w, int ci, int co, int kh, int kw, int stride
 }
 
 /*
+ * Sibling consumers of one 32-bit value (Sec. 4.3 "Clipping-Level Sharing and Private Fractional Length", Fig. 4;
+ * appendix "Private Fractional Lengths Enabling Different Clipping-Levels").  The paper keeps the sum of a layer
+ * in 32 bits and quantizes it once per child layer with that child's own fractional length; a shortcut stays in
+ * 32 bits until it is added.  For one output element:
+ *
+ *     acc  = sum_taps x*w + bias                              format FA = FLx + FLw
+ *     F    = max(FA, FLr)          v = acc * 2^(F-FA) + r * 2^(F-FLr)        (r: 8-bit code or 32-bit value)
+ *     child k (k = 1, 2):  kind 0: clip(round(v * 2^(FLk - F)), 0, 255)      Eq. 2
+ *                          kind 1: clip(round(v * 2^(FLk - F)), -127, 127)   signed form
+ *                          kind 2: v itself, int32 in format F
+ *                          kind 3: max(v, 0), int32 in format F  (the value behind a ReLU, still unrounded:
+ *                                  reading -- the paper says such values "are stored in 32-bit" and only
+ *                                  "quantized into 8-bit for multiplication"; it does not spell the clip out)
+ * Same loop nest as f8ref_conv2d; res_kind 0 u8, 1 s8, 2 int32; y2 may be NULL.
+ */
+static int finish_child(int64_t v, int f, int kind, int fl, void *y, size_t yi)
+{
+    if (kind == 2) ((int32_t *)y)[yi] = (int32_t)v;
+    else if (kind == 3) ((int32_t *)y)[yi] = (int32_t)(v > 0 ? v : 0);
+    else if (kind == 0) ((uint8_t *)y)[yi] = (uint8_t)f8ref_shift_round_clip(v, f - fl, 0, 255);
+    else if (kind == 1) ((int8_t *)y)[yi] = (int8_t)f8ref_shift_round_clip(v, f - fl, -127, 127);
+    else return F8REF_ERR_ARG;
+    return F8REF_OK;
+}
+
+int f8ref_conv2d_siblings(int n, int h, int w, int ci, int co, int kh, int kw, int stride, int pad,
+                          int x_signed, int fl_x, int fl_w,
+                          const void *x, const int8_t *wgt, const int32_t *bias,
+                          const void *res, int res_kind, int fl_r,
+                          void *y1, int y1_kind, int fl_y1, void *y2, int y2_kind, int fl_y2)
+{
+    if (n < 0 || h <= 0 || w <= 0 || ci <= 0 || co <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0)
+        return F8REF_ERR_ARG;
+    if (!y1 || (res && (res_kind < 0 || res_kind > 2))) return F8REF_ERR_ARG;
+    const int ho = (h + 2 * pad - kh) / stride + 1;
+    const int wo = (w + 2 * pad - kw) / stride + 1;
+    if (ho <= 0 || wo <= 0) return F8REF_ERR_ARG;
+    int status = F8REF_OK;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int in = 0; in < n; ++in)
+        for (int oh = 0; oh < ho; ++oh)
+            for (int ow = 0; ow < wo; ++ow)
+                for (int oc = 0; oc < co; ++oc) {
+                    int64_t acc = 0;
+                    for (int r = 0; r < kh; ++r)
+                        for (int s = 0; s < kw; ++s) {
+                            const int ih = oh * stride + r - pad;
+                            const int iw = ow * stride + s - pad;
+                            if (ih < 0 || ih >= h || iw < 0 || iw >= w) continue;
+                            for (int c = 0; c < ci; ++c) {
+                                const size_t xi = (((size_t)in * h + ih) * w + iw) * ci + c;
+                                const size_t wi = (((size_t)oc * kh + r) * kw + s) * ci + c;
+                                acc += load8(x, xi, x_signed) * (int64_t)wgt[wi];
+                            }
+                        }
+                    if (bias) acc += bias[oc];
+                    const size_t yi = (((size_t)in * ho + oh) * wo + ow) * co + oc;
+                    int st = F8REF_OK;
+                    int f = fl_x + fl_w;
+                    int64_t v = acc;
+                    if (acc > INT32_MAX || acc < INT32_MIN) st = F8REF_ERR_ACC_RANGE;
+                    if (res) {
+                        const int64_t rv = res_kind == 2 ? (int64_t)((const int32_t *)res)[yi] : load8(res, yi, res_kind == 1);
+                        f = f > fl_r ? f : fl_r;
+                        v = acc * ((int64_t)1 << (f - (fl_x + fl_w))) + rv * ((int64_t)1 << (f - fl_r));
+                        if (v > INT32_MAX || v < INT32_MIN) st = F8REF_ERR_ACC_RANGE;
+                    }
+                    if (st == F8REF_OK) st = finish_child(v, f, y1_kind, fl_y1, y1, yi);
+                    if (st == F8REF_OK && y2) st = finish_child(v, f, y2_kind, fl_y2, y2, yi);
+                    if (st != F8REF_OK) {
+#pragma omp atomic write
+                        status = st;
+                    }
+                }
+    return status;
+}
+
+/*
  * Depthwise convolution layer: one kh x kw filter per channel (MobileNet's
  * depthwise layers).  wgt : [c, kh, kw] s8.  Everything else as f8ref_conv2d.
  */

@@ -88,6 +88,30 @@ def conv2d(x, w, bias, *, stride, pad, fl_x, fl_w, fl_y, y_dtype, residual=None,
     return y
 
 
+S32_RELU = 3      # output kind of conv2d_siblings only: the 32-bit value behind a ReLU, max(v, 0), unrounded
+_NP_OUT = {U8: np.uint8, S8: np.int8, S32: np.int32, S32_RELU: np.int32}
+
+
+def conv2d_siblings(x, w, bias, *, stride, pad, fl_x, fl_w, y1_kind, fl_y1, y2_kind=None, fl_y2=0, residual=None, fl_r=0):
+    """One accumulator, one output per child layer, each with its private fractional length (Sec. 4.3); the shortcut
+    may be an 8-bit tensor or an int32 tensor in format fl_r.  Returns (y1, y2) with y2 None when not asked for."""
+    n, h, wd, ci = x.shape
+    co, kh, kw, ci2 = w.shape
+    assert ci2 == ci and w.dtype == np.int8
+    ho, wo = (h + 2 * pad - kh) // stride + 1, (wd + 2 * pad - kw) // stride + 1
+    y1 = np.empty((n, ho, wo, co), dtype=_NP_OUT[y1_kind])
+    y2 = np.empty((n, ho, wo, co), dtype=_NP_OUT[y2_kind]) if y2_kind is not None else None
+    res_kind = 0
+    if residual is not None:
+        assert residual.shape == y1.shape and residual.flags["C_CONTIGUOUS"]
+        res_kind = 2 if residual.dtype == np.int32 else _dtype_code(residual)
+    st = lib().f8ref_conv2d_siblings(n, h, wd, ci, co, kh, kw, stride, pad, _dtype_code(x), fl_x, fl_w,
+                                     _ptr(x), _ptr(w), _ptr(bias), _ptr(residual), res_kind, fl_r,
+                                     _ptr(y1), y1_kind, fl_y1, _ptr(y2), y2_kind if y2_kind is not None else 0, fl_y2)
+    _check(st, "conv2d_siblings")
+    return y1, y2
+
+
 def dwconv(x, w, bias, *, stride, pad, fl_x, fl_w, fl_y, y_dtype, residual=None, fl_r=0):
     n, h, wd, c = x.shape
     c2, kh, kw = w.shape
