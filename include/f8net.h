@@ -66,7 +66,9 @@ typedef enum {
     F8_ERR_TIMEOUT = 11       /* a kernel gave up on a bounded wait (see f8_device_status) */
 } f8_status;
 
-typedef enum { F8_U8 = 0, F8_S8 = 1, F8_S32 = 2 } f8_dtype;
+typedef enum { F8_U8 = 0, F8_S8 = 1, F8_S32 = 2,
+               F8_S32_RELU = 3      /* output of the sibling entry points only: int32, max(value, 0) */
+} f8_dtype;
 
 /*
  * One convolution-shaped layer (Eq. 6).  Input x is [n, h, w, c]; the output is
@@ -97,6 +99,20 @@ f8_status f8_conv2d_fixed(const f8_conv_desc *desc, const void *x, const int8_t 
                           const void *residual, void *y, void *workspace, size_t workspace_bytes,
                           void *cuda_stream);
 
+/* One 32-bit sum, several consumers (Sec. 4.3 "Clipping-Level Sharing and Private Fractional Length", Fig. 4;
+ * appendix "Private Fractional Lengths Enabling Different Clipping-Levels").  The paper keeps a layer's sum in
+ * 32 bits and quantizes it once per child layer with that child's own fractional length, and keeps a shortcut in
+ * 32 bits until it is added.  This call is f8_conv2d_fixed with
+ *   - a second output y2 (NULL: none) of dtype y2_dtype with its private fl_y2, produced from the same sum;
+ *   - desc->r_dtype == F8_S32 allowed: the residual is an int32 tensor in format fl_r (0..31);
+ *   - F8_S32_RELU allowed for y_dtype / y2_dtype: the sum behind a ReLU, max(v, 0), unrounded, int32 in the format
+ *     F = max(fl_x + fl_w, fl_r) of the aligned sum (F8_S32: the sum itself).
+ * Both 8-bit outputs equal what two f8_conv2d_fixed calls with fl_y and fl_y2 would give.  Precondition as for every
+ * layer: the aligned sum fits int32.  Runs with direct stores (not the staged TMA epilogue); same validation errors. */
+f8_status f8_conv2d_siblings_fixed(const f8_conv_desc *desc, int y2_dtype, int fl_y2, const void *x,
+                                   const int8_t *w_ohwi, const int32_t *bias, const void *residual, void *y, void *y2,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Depthwise convolution (one kh x kw filter per channel; MobileNet layers of Sec. 5),
  * c_out must equal c.  w_chw [c, kh, kw] int8.  Everything else as f8_conv2d_fixed. */
 f8_status f8_dwconv_fixed(const f8_conv_desc *desc, const void *x, const int8_t *w_chw, const int32_t *bias,
@@ -125,12 +141,22 @@ size_t f8_conv_workspace_bytes(const f8_conv_desc *desc);
 /* ---------------------------------------------------------------- whole networks */
 
 typedef enum { F8_LAYER_CONV = 0, F8_LAYER_DWCONV = 1, F8_LAYER_MAXPOOL = 2, F8_LAYER_GAP = 3,
-               F8_LAYER_LINEAR = 4 } f8_layer_kind;
+               F8_LAYER_LINEAR = 4,
+               F8_LAYER_SIBLING = 5     /* a second consumer's view of the previous layer's 32-bit sum */
+} f8_layer_kind;
 
 /* Tensor 0 is the network input; layer i writes tensor i + 1.  src / res name tensors
  * (res = -1: no residual).  conv.n is ignored (the batch is given per call); for
  * F8_LAYER_LINEAR conv.c = inputs and conv.c_out = outputs; for pooling layers only the
- * geometry, x_dtype and fl_x / fl_y are read. */
+ * geometry, x_dtype and fl_x / fl_y are read.
+ *
+ * Sibling consumers (Sec. 4.3, Fig. 4): an F8_LAYER_SIBLING layer i must directly follow a dense convolution
+ * (layer i - 1) and name that layer's output tensor as src (src = i).  Its tensor i + 1 is the SAME 32-bit sum
+ * quantised with this layer's own conv.y_dtype / conv.fl_y (F8_U8, F8_S8, or F8_S32 / F8_S32_RELU to keep it in
+ * 32 bits, e.g. as the shortcut of the next block); the other fields are ignored.  Both tensors are written by
+ * one launch.  Dense convolutions inside a network may name an int32 tensor as their residual (r_dtype F8_S32,
+ * fl_r = the format that tensor was produced in: fl_x + fl_w of its producer, or max(fl_x + fl_w, fl_r) if the
+ * producer had a residual itself). */
 typedef struct {
     int kind;
     int src;
@@ -154,7 +180,12 @@ size_t f8_net_workspace_bytes(const f8_net *net, int batch);
 /* One forward pass (the fixed-point inference path end to end).  x: [batch, h, w, c] network
  * input; y: the last layer's output ([batch, out] int32 logits for a net ending in a linear
  * layer).  layer_dump: NULL, or an array of n_layers device pointers; a non-NULL entry i
- * receives a copy of layer i's output (for parity checks). */
+ * receives a copy of layer i's output (for parity checks).
+ * Schedule: layers run one after the other over the whole batch, except that a run of layers with equal output
+ * size whose tensors do not fit the L2 cache at the full batch may be executed depth-first over micro-batches
+ * (images are independent, so no result changes): tensors inside the run then hold one micro-batch and stay in
+ * the cache between producer and consumer.  Status: if a kernel of an earlier pass on this object gave up a bounded
+ * wait, the call returns F8_ERR_TIMEOUT before enqueuing anything (see f8_device_status). */
 f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *workspace,
                          size_t workspace_bytes, void *const *layer_dump, void *cuda_stream);
 
@@ -293,6 +324,15 @@ enum {
     F8_PLAN_OFF_LAYER_OVERLAP = 256, F8_PLAN_OFF_MICRO_BATCH = 512, F8_PLAN_SYNC_LAYERS = 1024
 };
 void f8_debug_plan_options(unsigned off_mask);
+
+/* Test hook for the micro-batch schedule of f8_net_forward.  By default a run of layers whose tensors exceed the L2
+ * cache at the full batch is executed depth-first over micro-batches sized to the cache, provided every dense layer
+ * of the run still has a few tiles per SM (see f8_net_forward).  images > 0 forces that micro-batch for every run of
+ * three or more layers with equal output size (whatever the sizes); 0 restores the rule.  f8_net_micro_batching
+ * reports what the last forward pass of a network did: the number of micro-batched runs (return value) and the
+ * smallest micro-batch (*images). */
+void f8_debug_set_micro_batch(int images);
+int f8_net_micro_batching(const f8_net *net, int *images);
 
 /* What the most recent tensor-core plan of this process decided (n <= 10 ints are written, the count is returned):
  * [0] flags below, [1] epilogue variant (0 generic, 1 u8, 2 u8 + residual, 3 s8, 4 s8 + residual), [2] N tile,

@@ -22,7 +22,7 @@ _LIB = os.path.join(_HERE, "libf8ref.so")
 _lib = None
 
 # dtype / layer-kind codes of the layer descriptions: defined once, by the input generator
-from paper_2202_05239_b200.synth import U8, S8, S32, CONV, DWCONV, MAXPOOL, GAP, LINEAR  # noqa: E402
+from paper_2202_05239_b200.synth import U8, S8, S32, CONV, DWCONV, MAXPOOL, GAP, LINEAR, SIBLING  # noqa: E402
 
 
 def build(force: bool = False) -> str:
@@ -170,6 +170,21 @@ def run_layer(layer, x: np.ndarray, residual: Optional[np.ndarray] = None) -> np
     raise ValueError(f"unknown layer kind {layer.kind}")
 
 
+def run_layer_with_sibling(layer, sibling, x: np.ndarray, residual: Optional[np.ndarray] = None):
+    """A dense convolution whose 32-bit sum has a second consumer (`sibling`: a SIBLING layer description, or None),
+    or whose shortcut / output stays in 32 bits (Sec. 4.3): returns (output, sibling output or None)."""
+    assert layer.kind == CONV
+    return conv2d_siblings(np.ascontiguousarray(x), layer.weight, layer.bias, stride=layer.stride, pad=layer.pad,
+                           fl_x=layer.fl_x, fl_w=layer.fl_w, y1_kind=layer.y_dtype, fl_y1=layer.fl_y,
+                           y2_kind=sibling.y_dtype if sibling is not None else None,
+                           fl_y2=sibling.fl_y if sibling is not None else 0, residual=residual, fl_r=layer.fl_r)
+
+
+def _needs_sibling_form(layer, nxt) -> bool:
+    return layer.kind == CONV and ((nxt is not None and nxt.kind == SIBLING) or layer.y_dtype == S32_RELU or
+                                   (layer.res >= 0 and layer.r_dtype == S32))
+
+
 def net_forward(layers: Sequence, image: np.ndarray, keep_all: bool = True) -> List[np.ndarray]:
     """Run a layer list; returns every tensor (tensor 0 = image, layer i -> tensor i+1).
 
@@ -182,9 +197,18 @@ def net_forward(layers: Sequence, image: np.ndarray, keep_all: bool = True) -> L
         if l.res >= 0:
             last_use[l.res] = i
     tensors: List[Optional[np.ndarray]] = [np.ascontiguousarray(image)]
+    pending = None            # the output of a sibling layer, computed together with its parent
     for i, l in enumerate(layers):
         r = tensors[l.res] if l.res >= 0 else None
-        tensors.append(run_layer(l, tensors[l.src], r))
+        nxt = layers[i + 1] if i + 1 < len(layers) else None
+        if l.kind == SIBLING:
+            tensors.append(pending)
+            pending = None
+        elif _needs_sibling_form(l, nxt):
+            y, pending = run_layer_with_sibling(l, nxt if nxt is not None and nxt.kind == SIBLING else None, tensors[l.src], r)
+            tensors.append(y)
+        else:
+            tensors.append(run_layer(l, tensors[l.src], r))
         if not keep_all:
             for t in {l.src, l.res}:
                 if t >= 0 and last_use.get(t, -1) <= i:

@@ -27,7 +27,7 @@ if not os.path.exists(_LIB_PATH):
 _lib = ctypes.CDLL(_LIB_PATH)
 
 F8_OK = 0
-F8_U8, F8_S8, F8_S32 = 0, 1, 2
+F8_U8, F8_S8, F8_S32, F8_S32_RELU = 0, 1, 2, 3
 STATUS_NAMES = ["F8_OK", "F8_ERR_NULL", "F8_ERR_SHAPE", "F8_ERR_DTYPE", "F8_ERR_FL_RANGE", "F8_ERR_SHIFT_RANGE",
                 "F8_ERR_ALIGN", "F8_ERR_ACC_BOUND", "F8_ERR_WORKSPACE", "F8_ERR_UNSUPPORTED", "F8_ERR_CUDA",
                 "F8_ERR_TIMEOUT"]
@@ -99,7 +99,7 @@ def conv_desc(layer: "synth.Layer", n: int) -> ConvDesc:
                     layer.x_dtype, layer.y_dtype, layer.r_dtype, layer.fl_x, layer.fl_w, layer.fl_y, layer.fl_r)
 
 
-_TORCH_DTYPE = {F8_U8: torch.uint8, F8_S8: torch.int8, F8_S32: torch.int32}
+_TORCH_DTYPE = {F8_U8: torch.uint8, F8_S8: torch.int8, F8_S32: torch.int32, F8_S32_RELU: torch.int32}
 
 
 def torch_dtype(code: int) -> torch.dtype:
@@ -115,6 +115,16 @@ def to_device(a: Optional[np.ndarray], device="cuda") -> Optional[torch.Tensor]:
 def f8_conv2d_fixed(desc: ConvDesc, x, w, bias, residual, y, workspace=None, stream=None):
     _check(_lib.f8_conv2d_fixed(ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y),
                                 _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+_lib.f8_conv2d_siblings_fixed.argtypes = [ctypes.POINTER(ConvDesc), _ci, _ci, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+
+
+def f8_conv2d_siblings_fixed(desc: ConvDesc, y2_dtype, fl_y2, x, w, bias, residual, y, y2, workspace=None, stream=None):
+    """One 32-bit sum, one output per consumer with its private fractional length; 32-bit shortcuts allowed (Sec. 4.3)."""
+    _check(_lib.f8_conv2d_siblings_fixed(ctypes.byref(desc), y2_dtype, fl_y2, _ptr(x), _ptr(w), _ptr(bias), _ptr(residual),
+                                         _ptr(y), _ptr(y2), _ptr(workspace),
+                                         workspace.numel() if workspace is not None else 0, _stream(stream)))
 
 
 def f8_dwconv_fixed(desc: ConvDesc, x, w, bias, residual, y, workspace=None, stream=None):
@@ -236,6 +246,16 @@ PLAN_PLAIN_MATRIX, PLAN_STAGED_EPILOGUE, PLAN_PAIRS = 16, 32, 64
 
 def f8_debug_plan_options(off_mask: int):
     _lib.f8_debug_plan_options(off_mask)
+
+
+_lib.f8_debug_set_micro_batch.argtypes = [_ci]
+_lib.f8_debug_set_micro_batch.restype = None
+_lib.f8_net_micro_batching.argtypes = [_vp, ctypes.POINTER(_ci)]
+
+
+def f8_debug_set_micro_batch(images: int):
+    """Forces the micro-batch of f8_net_forward's depth-first runs (0: the library's own rule)."""
+    _lib.f8_debug_set_micro_batch(images)
 
 
 def f8_debug_last_plan() -> dict:
@@ -375,6 +395,12 @@ class Net:
     @property
     def last_launch_count(self) -> int:
         return int(_lib.f8_net_last_launch_count(self._h))
+
+    def micro_batching(self):
+        """(number of runs of layers the last forward pass executed depth-first over micro-batches, smallest micro-batch)."""
+        images = _ci(0)
+        runs = int(_lib.f8_net_micro_batching(self._h, ctypes.byref(images)))
+        return runs, int(images.value)
 
     def close(self):
         if self._h:

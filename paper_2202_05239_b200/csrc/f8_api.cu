@@ -21,6 +21,7 @@ long long g_tc_launches = 0;
 unsigned g_plan_off = 0;                      // F8_PLAN_OFF_* bits (test hook)
 unsigned long long g_wait_limit_cycles = 0;   // 0: the kernels' default
 int g_last_plan[10] = {0};
+int g_micro_batch = 0;                        // test hook: > 0 forces this micro-batch in every eligible run of layers
 
 f8_status fail(f8_status s, const char *fmt, ...) {
     va_list ap;
@@ -43,7 +44,8 @@ int ceil_log2(long long v) {
 }
 
 // Validates one conv-shaped descriptor and derives geometry + requantisation parameters.
-f8_status check_conv(const f8_conv_desc *d, bool depthwise, bool has_res, F8ConvGeom *g, F8Requant *q) {
+f8_status check_conv(const f8_conv_desc *d, bool depthwise, bool has_res, F8ConvGeom *g, F8Requant *q,
+                     bool siblings = false /* accept a 32-bit shortcut and the F8_S32_RELU output */) {
     if (!d) return fail(F8_ERR_NULL, "descriptor is NULL");
     if (d->n < 0 || d->h <= 0 || d->w <= 0 || d->c <= 0 || d->c_out <= 0 || d->kh <= 0 || d->kw <= 0 ||
         d->stride <= 0 || d->pad < 0)
@@ -56,7 +58,7 @@ f8_status check_conv(const f8_conv_desc *d, bool depthwise, bool has_res, F8Conv
     if ((long long)d->n * ho * wo * d->c_out >= (1ll << 40) || (long long)d->n * d->h * d->w * d->c >= (1ll << 40))
         return fail(F8_ERR_SHAPE, "tensor too large");
     if (d->x_dtype != F8_U8 && d->x_dtype != F8_S8) return fail(F8_ERR_DTYPE, "x_dtype must be F8_U8 or F8_S8");
-    if (d->y_dtype != F8_U8 && d->y_dtype != F8_S8 && d->y_dtype != F8_S32)
+    if (d->y_dtype != F8_U8 && d->y_dtype != F8_S8 && d->y_dtype != F8_S32 && !(siblings && d->y_dtype == F8_S32_RELU))
         return fail(F8_ERR_DTYPE, "y_dtype must be F8_U8, F8_S8 or F8_S32");
     if (d->fl_x < 0 || d->fl_x > (d->x_dtype == F8_U8 ? 8 : 7))
         return fail(F8_ERR_FL_RANGE, "fl_x = %d outside the 8-bit format range", d->fl_x);
@@ -65,10 +67,13 @@ f8_status check_conv(const f8_conv_desc *d, bool depthwise, bool has_res, F8Conv
     q->sh_acc = q->sh_res = 0;
     q->has_res = has_res ? 1 : 0;
     q->r_signed = 0;
+    q->r_s32 = 0;
     if (has_res) {
-        if (d->r_dtype != F8_U8 && d->r_dtype != F8_S8) return fail(F8_ERR_DTYPE, "r_dtype must be F8_U8 or F8_S8");
-        if (d->fl_r < 0 || d->fl_r > (d->r_dtype == F8_U8 ? 8 : 7))
-            return fail(F8_ERR_FL_RANGE, "fl_r = %d outside the 8-bit format range", d->fl_r);
+        const bool r32 = siblings && d->r_dtype == F8_S32;
+        if (d->r_dtype != F8_U8 && d->r_dtype != F8_S8 && !r32) return fail(F8_ERR_DTYPE, "r_dtype must be F8_U8 or F8_S8");
+        if (d->fl_r < 0 || d->fl_r > (r32 ? 31 : (d->r_dtype == F8_U8 ? 8 : 7)))
+            return fail(F8_ERR_FL_RANGE, "fl_r = %d outside the accepted range", d->fl_r);
+        q->r_s32 = r32 ? 1 : 0;
         const int f = std::max(fa, d->fl_r);
         q->sh_acc = f - fa;
         q->sh_res = f - d->fl_r;
@@ -78,7 +83,7 @@ f8_status check_conv(const f8_conv_desc *d, bool depthwise, bool has_res, F8Conv
         fa = f;
     }
     q->y_kind = d->y_dtype;
-    if (d->y_dtype == F8_S32) {
+    if (d->y_dtype == F8_S32 || d->y_dtype == F8_S32_RELU) {
         q->s = 0;
         q->lo = q->hi = 0;
     } else {
@@ -124,15 +129,35 @@ PlanPtr alloc_plan() {
     return PlanPtr((F8TcPlan *)p);
 }
 
+// The second consumer of a layer's sum: its quantizer relative to the format F of the aligned sum.
+f8_status make_sibling(const f8_conv_desc *d, const F8Requant &q, int y2_dtype, int fl_y2, void *y2, F8Sibling *sib) {
+    if (y2_dtype != F8_U8 && y2_dtype != F8_S8 && y2_dtype != F8_S32 && y2_dtype != F8_S32_RELU)
+        return fail(F8_ERR_DTYPE, "y2_dtype must be F8_U8, F8_S8, F8_S32 or F8_S32_RELU");
+    sib->y2 = y2;
+    sib->y_kind = y2_dtype;
+    sib->s = 0;
+    sib->lo = sib->hi = 0;
+    if (y2_dtype == F8_U8 || y2_dtype == F8_S8) {
+        if (fl_y2 < 0 || fl_y2 > (y2_dtype == F8_U8 ? 8 : 7))
+            return fail(F8_ERR_FL_RANGE, "fl_y2 = %d outside the 8-bit format range", fl_y2);
+        const int f = d->fl_x + d->fl_w + q.sh_acc;        // format of the aligned sum
+        sib->s = f - fl_y2;
+        if (sib->s < -8 || sib->s > 31) return fail(F8_ERR_SHIFT_RANGE, "requantisation shift %d of the second output outside [-8, 31]", sib->s);
+        sib->lo = y2_dtype == F8_U8 ? 0 : -127;
+        sib->hi = y2_dtype == F8_U8 ? 255 : 127;
+    }
+    return F8_OK;
+}
+
 f8_status run_dense(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w, const int32_t *bias,
-                    const void *res, void *y, cudaStream_t st) {
+                    const void *res, void *y, cudaStream_t st, const F8Sibling *sib = nullptr) {
     if (g.n == 0) return F8_OK;
     const size_t x_bytes = (size_t)g.n * g.h * g.w * g.c;
     if (!g_force_direct && f8_tc_supported(g, x_bytes)) {
         PlanPtr plan = alloc_plan();
         if (!plan) return fail(F8_ERR_CUDA, "out of host memory");
         const char *why = "";
-        cudaError_t e = f8_tc_plan_init(plan.get(), g, q, dense_view(x, g), w, bias, res, y, f8_status_word(), &why);
+        cudaError_t e = f8_tc_plan_init(plan.get(), g, q, dense_view(x, g), w, bias, res, y, f8_status_word(), &why, sib);
         if (e == cudaSuccess) {
             e = f8_tc_launch(plan.get(), false, st);   // the caller's weights may come from earlier work in the stream
             if (e != cudaSuccess) return cuda_fail(e, "tensor-core conv launch");
@@ -143,7 +168,7 @@ f8_status run_dense(const F8ConvGeom &g, const F8Requant &q, const void *x, cons
         // the tensor map could not be encoded for this shape: take the CUDA-core kernel
         (void)cudaGetLastError();
     }
-    cudaError_t e = f8_launch_conv_direct(g, q, x, w, bias, res, y, st);
+    cudaError_t e = f8_launch_conv_direct(g, q, x, w, bias, res, y, st, false, sib);
     if (e != cudaSuccess) return cuda_fail(e, "direct conv launch");
     return F8_OK;
 }
@@ -197,6 +222,8 @@ long long f8_tc_launch_count(void) { return g_tc_launches; }
 void f8_debug_force_direct(int on) { g_force_direct = on != 0; }
 
 void f8_debug_plan_options(unsigned off_mask) { g_plan_off = off_mask; }
+
+void f8_debug_set_micro_batch(int images) { g_micro_batch = images > 0 ? images : 0; }
 
 int f8_debug_last_plan(int *info, int n) {
     if (!info || n <= 0) return 0;
@@ -255,6 +282,25 @@ f8_status f8_conv2d_fixed(const f8_conv_desc *desc, const void *x, const int8_t 
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(residual) || !aligned16(bias))
         return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
     return run_dense(g, q, x, w, bias, residual, y, (cudaStream_t)cuda_stream);
+}
+
+f8_status f8_conv2d_siblings_fixed(const f8_conv_desc *desc, int y2_dtype, int fl_y2, const void *x, const int8_t *w,
+                                   const int32_t *bias, const void *residual, void *y, void *y2, void *, size_t,
+                                   void *cuda_stream) {
+    F8ConvGeom g;
+    F8Requant q;
+    f8_status s = check_conv(desc, false, residual != nullptr, &g, &q, true);
+    if (s != F8_OK) return s;
+    F8Sibling sib;
+    if (y2) {
+        s = make_sibling(desc, q, y2_dtype, fl_y2, y2, &sib);
+        if (s != F8_OK) return s;
+    }
+    if (g.n == 0) return F8_OK;
+    if (!x || !w || !y) return fail(F8_ERR_NULL, "x, w and y must not be NULL");
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(y2) || !aligned16(residual) || !aligned16(bias))
+        return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    return run_dense(g, q, x, w, bias, residual, y, (cudaStream_t)cuda_stream, y2 ? &sib : nullptr);
 }
 
 f8_status f8_dwconv_fixed(const f8_conv_desc *desc, const void *x, const int8_t *w, const int32_t *bias,
@@ -341,6 +387,8 @@ struct NetLayer {
     int8_t *w_packed = nullptr;
     int8_t *w_core = nullptr;   // the same window weights as [K / 16][c_out][16] (core-matrix order) for the stem kernel
     size_t out_bytes_per_image = 0;
+    F8Sibling sib;              // F8_LAYER_SIBLING: this layer's quantizer of its parent's sum (y2 filled per plan)
+    bool has_sibling = false;   // the next layer is an F8_LAYER_SIBLING of this one
 };
 
 struct Step {
@@ -351,6 +399,9 @@ struct Step {
     void *y = nullptr;
     bool use_tc = false;
     bool fused_pool = false;  // kind -2: the stem kernel also computes the max pool that follows (layer + 1)
+    bool has_sib = false;     // the launch also writes the output of the sibling layer behind it (layer + 1)
+    F8Sibling sib;
+    int img0 = 0;             // first image of the batch this step works on (micro-batched runs)
     PlanPtr plan;
     F8ConvGeom g;
 };
@@ -363,6 +414,8 @@ struct f8_net {
     bool overlap_layers = true;                  // programmatic dependent launch between layers
     bool sync_layers = false;                    // synchronize after every launch (fault attribution)
     unsigned plan_options = 0;                   // F8_PLAN_OFF_* mask the cached plan was made under
+    int plan_micro = 0;                          // forced micro-batch the cached plan was made under
+    int last_regions = 0, last_micro = 0;        // micro-batched runs of the cached plan and the smallest micro-batch
     std::vector<int> t_cp;                       // per tensor: channels as stored (intermediate 8-bit tensors are padded
                                                  // to a multiple of 16 so that every dense layer can use the TMA path)
     int max_batch = 0;
@@ -396,22 +449,139 @@ size_t tensor_bytes(const f8_net *net, int t, int batch) {
     return (size_t)batch * net->t_h[t] * net->t_w[t] * net->t_cp[t] * net->t_elem[t];
 }
 
+// A run of consecutive layers executed depth-first over micro-batches: layers first..last run on images
+// [0, mb), then on [mb, 2 mb), ...  Tensors that live entirely inside the run are allocated for mb images only and are
+// reused by every micro-batch, so a producer's output is still in the L2 cache when its consumer reads it (and is
+// overwritten there before it is ever written back); tensors that enter or leave the run keep their full size.
+struct Region { int first, last, mb; };
+
+size_t tensor_image_bytes(const f8_net *net, int t) {
+    return (size_t)net->t_h[t] * net->t_w[t] * net->t_cp[t] * net->t_elem[t];
+}
+
+// Bytes one image moves through layer i when every tensor comes from / goes to memory.
+size_t layer_image_bytes(const f8_net *net, int i) {
+    const NetLayer &L = net->layers[i];
+    if (L.d.kind == F8_LAYER_SIBLING) return tensor_image_bytes(net, i + 1);
+    size_t b = tensor_image_bytes(net, L.d.src) + tensor_image_bytes(net, i + 1);
+    if (L.q.has_res && L.d.res >= 0) b += tensor_image_bytes(net, L.d.res);
+    return b;
+}
+
+std::vector<Region> plan_regions(const f8_net *net, int batch) {
+    std::vector<Region> out;
+    if (g_plan_off & F8_PLAN_OFF_MICRO_BATCH) return out;
+    const int nl = (int)net->layers.size();
+    int dev = 0, l2 = 64 << 20, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+        cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    int i = 0;
+    while (i < nl) {
+        // a run of layers whose outputs have the same spatial size (one stage of a network)
+        const int oh = net->t_h[i + 1], ow = net->t_w[i + 1];
+        int j = i;
+        while (j + 1 < nl && net->t_h[j + 2] == oh && net->t_w[j + 2] == ow) ++j;
+        int first = i;
+        // a pooling layer that opens the run brings the convolution in front of it along (the two may be one kernel)
+        if (first > 0 && net->layers[first].d.kind == F8_LAYER_MAXPOOL && net->layers[first].d.src == first &&
+            net->layers[first - 1].d.kind == F8_LAYER_CONV && (out.empty() || out.back().last < first - 1))
+            --first;
+        if ((long long)oh * ow > 1 && j - first + 1 >= 3 && j < nl - 1) {
+            size_t worst = 0;
+            bool beyond_l2 = false;
+            for (int l = first; l <= j; ++l) {
+                const size_t b = layer_image_bytes(net, l);
+                worst = std::max(worst, b);
+                if (b * (size_t)batch > (size_t)l2) beyond_l2 = true;
+            }
+            int mb = 0;
+            if (g_micro_batch > 0) {
+                mb = g_micro_batch;
+            } else if (beyond_l2 && worst > 0) {
+                // the largest power of two whose heaviest layer moves at most half of the cache
+                mb = 1;
+                while ((size_t)(2 * mb) * worst <= (size_t)l2 / 2) mb *= 2;
+                // every dense layer must still fill the machine a few times over, or the tail of each launch costs
+                // more than the memory traffic saved
+                for (int l = first; l <= j && mb > 0; ++l) {
+                    const NetLayer &L = net->layers[l];
+                    if (L.d.kind != F8_LAYER_CONV) continue;
+                    const long long tiles = (((long long)mb * L.g.ho * L.g.wo + 127) / 128) * ((L.g.c_out + 255) / 256);
+                    if (tiles < 2ll * sms) mb = 0;
+                }
+            }
+            if (mb > 0 && mb < batch) out.push_back({first, j, mb});
+        }
+        i = j + 1;
+    }
+    return out;
+}
+
+// Which run a layer belongs to (-1: none), and which tensors live entirely inside one run.
+void classify_tensors(const f8_net *net, const std::vector<Region> &regions, std::vector<int> *layer_region,
+                      std::vector<int> *tensor_region /* run a tensor is internal to, or -1 */) {
+    const int nl = (int)net->layers.size();
+    layer_region->assign(nl, -1);
+    for (int r = 0; r < (int)regions.size(); ++r)
+        for (int l = regions[r].first; l <= regions[r].last; ++l) (*layer_region)[l] = r;
+    tensor_region->assign(nl + 1, -1);
+    for (int t = 1; t < nl; ++t) {
+        const int producer = net->layers[t - 1].d.kind == F8_LAYER_SIBLING ? t - 2 : t - 1;
+        const int r = (*layer_region)[producer];
+        if (r < 0 || (*layer_region)[t - 1] != r) continue;
+        bool inside = true;
+        for (int l = 0; l < nl && inside; ++l) {
+            const NetLayer &L = net->layers[l];
+            const bool reads = L.d.src == t || (L.q.has_res && L.d.res == t && L.d.kind != F8_LAYER_SIBLING);
+            if (reads && (*layer_region)[l] != r) inside = false;
+        }
+        if (inside) (*tensor_region)[t] = r;
+    }
+}
+
 // Assigns workspace offsets: tensors whose lifetimes do not overlap may share memory (first fit).
-size_t assign_offsets(const f8_net *net, int batch, std::vector<size_t> *off, size_t *pack_off) {
-    const int nt = (int)net->layers.size() + 1;
-    std::vector<int> last(nt, -1);
-    for (int i = 0; i < (int)net->layers.size(); ++i) {
+size_t assign_offsets(const f8_net *net, int batch, std::vector<size_t> *off, size_t *pack_off,
+                      const std::vector<Region> &regions) {
+    const int nl = (int)net->layers.size();
+    const int nt = nl + 1;
+    std::vector<int> layer_region, tensor_region;
+    classify_tensors(net, regions, &layer_region, &tensor_region);
+    std::vector<int> last(nt, -1), born(nt, 0);
+    for (int i = 0; i < nl; ++i) {
         last[net->layers[i].d.src] = i;
         if (net->layers[i].d.res >= 0) last[net->layers[i].d.res] = i;
+    }
+    for (int t = 1; t < nt; ++t) {
+        // written by layer t-1; a sibling's tensor is written by the launch of the layer before it
+        born[t] = net->layers[t - 1].d.kind == F8_LAYER_SIBLING ? t - 2 : t - 1;
+        last[t] = std::max(last[t], born[t]);
+    }
+    // A full-size tensor that a micro-batched run writes is filled slice by slice over the whole run, and one that the
+    // run reads is read again by every micro-batch: both are live from the run's first layer to its last.
+    for (int t = 1; t < nt; ++t) {
+        if (tensor_region[t] >= 0) continue;
+        const int rp = layer_region[born[t]];
+        if (rp >= 0) { born[t] = std::min(born[t], regions[rp].first); last[t] = std::max(last[t], regions[rp].last); }
+        for (int l = 0; l < nl; ++l) {
+            const NetLayer &L = net->layers[l];
+            const bool reads = L.d.src == t || (L.d.res == t && L.d.res >= 0);
+            if (reads && layer_region[l] >= 0) last[t] = std::max(last[t], regions[layer_region[l]].last);
+        }
     }
     struct Live { size_t off, size; int until; };
     std::vector<Live> live;
     off->assign(nt, 0);
     size_t top = 0;
-    for (int t = 1; t < nt - 1; ++t) {          // tensor 0 = caller's x, tensor nt-1 = caller's y
-        const int born = t - 1;                 // written by layer t-1
-        const size_t size = round256(tensor_bytes(net, t, batch));
-        live.erase(std::remove_if(live.begin(), live.end(), [&](const Live &l) { return l.until < born; }), live.end());
+    // in order of birth (a tensor a run writes in full may be born before tensors with smaller numbers)
+    std::vector<int> order;
+    for (int t = 1; t < nt - 1; ++t) order.push_back(t);      // tensor 0 = caller's x, tensor nt-1 = caller's y
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return born[a] < born[b]; });
+    for (int t : order) {
+        const int images = tensor_region[t] >= 0 ? std::min(batch, regions[tensor_region[t]].mb) : batch;
+        const size_t size = round256((size_t)images * tensor_image_bytes(net, t));
+        live.erase(std::remove_if(live.begin(), live.end(), [&](const Live &l) { return l.until < born[t]; }), live.end());
         std::sort(live.begin(), live.end(), [](const Live &a, const Live &b) { return a.off < b.off; });
         size_t pos = 0;
         for (const Live &l : live) {
@@ -419,7 +589,7 @@ size_t assign_offsets(const f8_net *net, int batch, std::vector<size_t> *off, si
             pos = std::max(pos, l.off + l.size);
         }
         (*off)[t] = pos;
-        live.push_back({pos, size, std::max(last[t], born)});
+        live.push_back({pos, size, last[t]});
         top = std::max(top, pos + size);
     }
     *pack_off = top;
@@ -456,12 +626,40 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
     net->t_c.assign(n_layers + 1, 0);
     net->t_elem.assign(n_layers + 1, 1);
     std::vector<int> t_dtype(n_layers + 1, -1), t_fl(n_layers + 1, 0);
+    std::vector<long long> t_bound(n_layers + 1, 0);       // largest magnitude an element of a 32-bit tensor can take
     auto cleanup = [&](f8_status s) { free_layers(net.get()); return s; };
     for (int i = 0; i < n_layers; ++i) {
         NetLayer &L = net->layers[i];
         L.d = layers[i];
         f8_conv_desc &d = L.d.conv;
         d.n = 1;
+        if (L.d.kind == F8_LAYER_SIBLING) {
+            // a second consumer of the 32-bit sum of the layer right before it, with its private format (Sec. 4.3)
+            if (i == 0 || L.d.src != i || net->layers[i - 1].d.kind != F8_LAYER_CONV)
+                return cleanup(fail(F8_ERR_SHAPE, "layer %d: a sibling layer must directly follow the dense convolution whose output tensor it names", i));
+            NetLayer &P = net->layers[i - 1];
+            const int yd = d.y_dtype, fy = d.fl_y;
+            const f8_status s = make_sibling(&P.d.conv, P.q, yd, fy, nullptr, &L.sib);
+            if (s != F8_OK) {
+                char msg[400];
+                snprintf(msg, sizeof(msg), "layer %d: %.300s", i, g_err);
+                return cleanup(fail(s, "%s", msg));
+            }
+            d = P.d.conv;
+            d.y_dtype = yd;
+            d.fl_y = fy;
+            L.d.res = -1;
+            L.g = P.g;
+            L.q = P.q;
+            P.has_sibling = true;
+            const bool wide = yd == F8_S32 || yd == F8_S32_RELU;
+            net->t_h[i + 1] = net->t_h[i]; net->t_w[i + 1] = net->t_w[i]; net->t_c[i + 1] = net->t_c[i];
+            net->t_elem[i + 1] = wide ? 4 : 1;
+            t_dtype[i + 1] = wide ? F8_S32 : yd;
+            t_fl[i + 1] = wide ? P.d.conv.fl_x + P.d.conv.fl_w + P.q.sh_acc : fy;
+            t_bound[i + 1] = t_bound[i];       // the same sum as the parent's output
+            continue;
+        }
         if (L.d.src < 0 || L.d.src > i) return cleanup(fail(F8_ERR_SHAPE, "layer %d: src %d is not an earlier tensor", i, L.d.src));
         if (L.d.res > i) return cleanup(fail(F8_ERR_SHAPE, "layer %d: res %d is not an earlier tensor", i, L.d.res));
         const int kind = L.d.kind;
@@ -472,6 +670,8 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
         f8_status s;
         switch (kind) {
             case F8_LAYER_CONV:
+                s = check_conv(&d, false, has_res, &L.g, &L.q, true);
+                break;
             case F8_LAYER_LINEAR:
                 s = check_conv(&d, false, has_res, &L.g, &L.q);
                 break;
@@ -517,9 +717,12 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
                 return cleanup(fail(F8_ERR_DTYPE, "layer %d: r_dtype / fl_r do not match the producer of tensor %d", i, r));
         }
         net->t_h[i + 1] = ho; net->t_w[i + 1] = wo; net->t_c[i + 1] = d.c_out;
-        net->t_elem[i + 1] = d.y_dtype == F8_S32 ? 4 : 1;
-        t_dtype[i + 1] = d.y_dtype;
-        t_fl[i + 1] = d.y_dtype == F8_S32 ? d.fl_x + d.fl_w : d.fl_y;
+        const bool wide_out = d.y_dtype == F8_S32 || d.y_dtype == F8_S32_RELU;
+        net->t_elem[i + 1] = wide_out ? 4 : 1;
+        t_dtype[i + 1] = wide_out ? F8_S32 : d.y_dtype;
+        t_fl[i + 1] = wide_out ? d.fl_x + d.fl_w + L.q.sh_acc : d.fl_y;
+        if (has_res && L.q.r_s32 && d.c_out % 16 != 0)
+            return cleanup(fail(F8_ERR_UNSUPPORTED, "layer %d: a 32-bit shortcut needs c_out to be a multiple of 16", i));
         L.out_bytes_per_image = (size_t)ho * wo * d.c_out * net->t_elem[i + 1];
 
         // parameters
@@ -531,16 +734,19 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
         const size_t per_out = (size_t)d.kh * d.kw * (kind == F8_LAYER_DWCONV ? 1 : d.c);
         // exact accumulator bound per output channel from the actual parameters
         const long long xmax = d.x_dtype == F8_U8 ? 255 : 128;
-        const long long rmax = has_res ? (d.r_dtype == F8_U8 ? 255 : 128) : 0;
+        const long long rmax = has_res ? (L.q.r_s32 ? t_bound[L.d.res] : (d.r_dtype == F8_U8 ? 255 : 128)) : 0;
+        long long layer_bound = 0;
         for (int co = 0; co < d.c_out; ++co) {
             long long sum = 0;
             for (size_t j = 0; j < per_out; ++j) sum += llabs((long long)hw[co * per_out + j]);
             long long bound = sum * xmax + (hb ? llabs((long long)hb[co]) : 0);
             bound = (bound << L.q.sh_acc) + (rmax << L.q.sh_res);
-            if (L.q.y_kind != F8_S32 && L.q.s >= 1) bound += 1ll << (L.q.s - 1);      // room for the rounding constant
+            layer_bound = std::max(layer_bound, bound);
+            if (L.q.y_kind != F8_S32 && L.q.y_kind != F8_S32_RELU && L.q.s >= 1) bound += 1ll << (L.q.s - 1);      // room for the rounding constant
             if (bound >= (1ll << 31) - 1)
                 return cleanup(fail(F8_ERR_ACC_BOUND, "layer %d channel %d: accumulator bound %lld exceeds int32", i, co, bound));
         }
+        t_bound[i + 1] = layer_bound;       // what a 32-bit output of this layer (its own or a sibling's) can reach
     }
     // Stored channel counts: intermediate 8-bit tensors whose channel count is not a multiple of 16 (24 in
     // MobileNetV2) are padded with channels that are identically zero -- zero weights and bias produce them,
@@ -548,6 +754,13 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
     net->t_cp = net->t_c;
     for (int t = 1; t < n_layers; ++t)
         if (net->t_elem[t] == 1 && net->t_c[t] % 16 != 0) net->t_cp[t] = (net->t_c[t] + 15) / 16 * 16;
+    // both outputs of a launch have the same number of stored channels
+    for (int i = 1; i < n_layers; ++i)
+        if (net->layers[i].d.kind == F8_LAYER_SIBLING) {
+            if (i + 1 == n_layers && net->t_cp[i] != net->t_c[i])
+                return cleanup(fail(F8_ERR_UNSUPPORTED, "layer %d: the network output cannot be the sibling of a layer with padded channels", i));
+            net->t_cp[i + 1] = net->t_cp[i];
+        }
     // second pass (everything validated): upload the parameters
     for (int i = 0; i < n_layers; ++i) {
         NetLayer &L = net->layers[i];
@@ -597,7 +810,7 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
         // the kh rows; taps that fall outside the filter get zero weights), which the tensor-core path takes
         // with few, long TMA rows.  Kernel row r sits in pair j, half e with r = 2j + e + pad - 2*top.
         if (kind == F8_LAYER_CONV && cp_in == d.c && cp_out == d.c_out && d.c <= 8 && d.stride == 2 &&
-            d.kw * 16 <= 256) {
+            d.kw * 16 <= 256 && !L.has_sibling && !L.q.r_s32 && d.y_dtype != F8_S32_RELU) {
             L.packed = true;
             L.pack_left = d.pad;
             L.pack_cpad = d.c <= 4 ? 4 : 8;
@@ -653,10 +866,15 @@ size_t f8_net_workspace_bytes(const f8_net *net, int batch) {
     if (!net || batch <= 0) return 0;
     std::vector<size_t> off;
     size_t pack_off;
-    return assign_offsets(net, batch, &off, &pack_off) + 256;
+    return assign_offsets(net, batch, &off, &pack_off, plan_regions(net, batch)) + 256;
 }
 
 int f8_net_last_launch_count(const f8_net *net) { return net ? net->last_launches : 0; }
+
+int f8_net_micro_batching(const f8_net *net, int *images) {
+    if (images) *images = net ? net->last_micro : 0;
+    return net ? net->last_regions : 0;
+}
 
 f8_status f8_net_set_profiling(f8_net *net, int on) {
     if (!net) return fail(F8_ERR_NULL, "net is NULL");
@@ -729,37 +947,60 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
             if (net->layers[i].w_core && layer_dump[i]) dump_fusable = true;
     const bool replan = net->plan_batch != batch || net->plan_x != x || net->plan_y != y || net->plan_ws != workspace ||
                         net->plan_force_direct != g_force_direct || net->plan_dump_first != dump_fusable ||
-                        net->plan_options != g_plan_off;
+                        net->plan_options != g_plan_off || net->plan_micro != g_micro_batch;
     net->overlap_layers = !(g_plan_off & F8_PLAN_OFF_LAYER_OVERLAP);
     net->sync_layers = (g_plan_off & F8_PLAN_SYNC_LAYERS) != 0;
     if (replan) {
         net->steps.clear();
         net->plan_batch = -1;
-        assign_offsets(net, batch, &net->t_off, &net->pack_off);
-        auto tensor_ptr = [&](int t) -> void * {
-            if (t == 0) return const_cast<void *>(x);
-            if (t == nl) return y;
-            return (uint8_t *)workspace + net->t_off[t];
-        };
+        const std::vector<Region> regions = plan_regions(net, batch);
+        assign_offsets(net, batch, &net->t_off, &net->pack_off, regions);
+        std::vector<int> layer_region, tensor_region;
+        classify_tensors(net, regions, &layer_region, &tensor_region);
+        net->last_regions = (int)regions.size();
+        net->last_micro = 0;
+        for (const Region &r : regions) net->last_micro = net->last_micro ? std::min(net->last_micro, r.mb) : r.mb;
+
+        // Plans layer i for images [img0, img0 + n) of the batch.  Inside a micro-batched run (in_run) tensors that live
+        // entirely in the run hold one micro-batch and always start at their base address; all other tensors are
+        // addressed at the slice of these images.
         int skip_layer = -1;          // a pooling layer the stem kernel has taken over
-        for (int i = 0; i < nl; ++i) {
+        auto plan_layer = [&](int i, int n, int img0, bool in_run) {
             NetLayer &L = net->layers[i];
-            if (i == skip_layer) continue;
+            if (i == skip_layer || L.d.kind == F8_LAYER_SIBLING) return;      // a sibling is written by its parent's launch
+            auto tensor_ptr = [&](int t) -> void * {
+                uint8_t *base = t == 0 ? (uint8_t *)const_cast<void *>(x)
+                                       : (t == nl ? (uint8_t *)y : (uint8_t *)workspace + net->t_off[t]);
+                if (in_run && tensor_region[t] < 0) {
+                    const size_t per_image = t == 0 ? (size_t)net->t_h[0] * net->t_w[0] * net->t_c[0]
+                                                    : (t == nl ? (size_t)net->t_h[nl] * net->t_w[nl] * net->t_c[nl] * net->t_elem[nl]
+                                                               : tensor_image_bytes(net, t));
+                    base += (size_t)img0 * per_image;
+                }
+                return base;
+            };
             Step stp;
             stp.kind = L.d.kind;
             stp.layer = i;
+            stp.img0 = img0;
             stp.x = tensor_ptr(L.d.src);
             stp.res = (L.q.has_res) ? tensor_ptr(L.d.res) : nullptr;
             stp.y = tensor_ptr(i + 1);
             stp.g = L.g;
-            stp.g.n = batch;
+            stp.g.n = n;
+            if (L.has_sibling) {
+                stp.has_sib = true;
+                stp.sib = net->layers[i + 1].sib;
+                stp.sib.y2 = tensor_ptr(i + 2);
+            }
             if ((L.d.kind == F8_LAYER_CONV || L.d.kind == F8_LAYER_LINEAR) && !g_force_direct) {
                 const char *why = "";
                 if (L.packed && L.w_core && !(g_plan_off & F8_PLAN_OFF_STEM_KERNEL) &&
                     f8_stem_tc_supported(stp.g, L.q, L.pack_kh, L.pack_kw8 / 32)) {
                     // the stem kernel; it also takes the 3x3 / 2 / pad 1 max pool behind the layer when nothing else
                     // reads the layer's output
-                    bool fuse = !dump_fusable && i + 1 < nl && !(g_plan_off & F8_PLAN_OFF_STEM_POOL_FUSION);
+                    bool fuse = !dump_fusable && i + 1 < nl && !(g_plan_off & F8_PLAN_OFF_STEM_POOL_FUSION) &&
+                                layer_region[i] == layer_region[i + 1];
                     if (fuse) {
                         const NetLayer &P = net->layers[i + 1];
                         fuse = P.d.kind == F8_LAYER_MAXPOOL && P.d.src == i + 1 && P.d.conv.kh == 3 && P.d.conv.kw == 3 &&
@@ -780,11 +1021,11 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                     pg.h = L.pack_hp;
                     void *pbuf = (uint8_t *)workspace + net->pack_off;
                     const uint64_t cb = 2 * (uint64_t)L.pack_cpad;
-                    const size_t pbytes = (size_t)batch * L.pack_hp * L.pack_wp * cb;
+                    const size_t pbytes = (size_t)n * L.pack_hp * L.pack_wp * cb;
                     if (f8_tc_supported(pg, pbytes)) {
                         F8TcTensorView v;
                         v.base = pbuf;
-                        v.dim_c = L.pack_kw8; v.dim_w = L.g.wo; v.dim_h = L.pack_hp; v.dim_n = batch;
+                        v.dim_c = L.pack_kw8; v.dim_w = L.g.wo; v.dim_h = L.pack_hp; v.dim_n = n;
                         v.stride_w = (uint64_t)L.g.stride_w * cb;
                         v.stride_h = (uint64_t)L.pack_wp * cb;
                         v.stride_n = (uint64_t)L.pack_wp * cb * L.pack_hp;
@@ -794,6 +1035,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                             Step pre;
                             pre.kind = -1;
                             pre.layer = i;
+                            pre.img0 = img0;
                             pre.x = stp.x;
                             pre.y = pbuf;
                             pre.g = stp.g;
@@ -803,10 +1045,10 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                             stp.plan = std::move(plan);
                         }
                     }
-                } else if (f8_tc_supported(stp.g, (size_t)batch * L.g.h * L.g.w * L.g.c)) {
+                } else if (f8_tc_supported(stp.g, (size_t)n * L.g.h * L.g.w * L.g.c)) {
                     PlanPtr plan = alloc_plan();
                     if (plan && f8_tc_plan_init(plan.get(), stp.g, L.q, dense_view(stp.x, stp.g), L.w, L.b, stp.res,
-                                                stp.y, f8_status_word(), &why) == cudaSuccess) {
+                                                stp.y, f8_status_word(), &why, stp.has_sib ? &stp.sib : nullptr) == cudaSuccess) {
                         stp.use_tc = true;
                         f8_tc_plan_set_tag(plan.get(), i + 1);
                         stp.plan = std::move(plan);
@@ -814,6 +1056,22 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                 }
             }
             net->steps.push_back(std::move(stp));
+        };
+        for (int i = 0; i < nl;) {
+            const int r = layer_region[i];
+            if (r < 0) {
+                plan_layer(i, batch, 0, false);
+                ++i;
+                continue;
+            }
+            // depth first: the whole run on one micro-batch, then on the next
+            for (int img0 = 0; img0 < batch; img0 += regions[r].mb) {
+                skip_layer = -1;
+                for (int l = regions[r].first; l <= regions[r].last; ++l)
+                    plan_layer(l, std::min(regions[r].mb, batch - img0), img0, true);
+            }
+            i = regions[r].last + 1;
+            skip_layer = -1;
         }
         net->plan_batch = batch;
         net->plan_x = x;
@@ -822,6 +1080,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         net->plan_force_direct = g_force_direct;
         net->plan_dump_first = dump_fusable;
         net->plan_options = g_plan_off;
+        net->plan_micro = g_micro_batch;
     }
 
     int launches = 0;
@@ -845,7 +1104,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                 ++g_tc_launches;
                 break;
             case -1:
-                e = f8_launch_pack_stem_pairs(batch, L.g.h, L.g.w, L.g.c, L.pack_cpad, L.pack_hp, L.pack_wp, L.pack_left, stp.x, stp.y, st,
+                e = f8_launch_pack_stem_pairs(stp.g.n, L.g.h, L.g.w, L.g.c, L.pack_cpad, L.pack_hp, L.pack_wp, L.pack_left, stp.x, stp.y, st,
                                               net->overlap_layers);
                 break;
             case F8_LAYER_CONV:
@@ -853,17 +1112,18 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                 // the net owns its weights (uploaded at creation), so a layer's prologue and weight loads may
                 // overlap the tail of the previous layer
                 if (stp.use_tc) { e = f8_tc_launch(stp.plan.get(), net->overlap_layers, st); ++g_tc_launches; }
-                else e = f8_launch_conv_direct(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st, net->overlap_layers);
+                else e = f8_launch_conv_direct(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st, net->overlap_layers,
+                                               stp.has_sib ? &stp.sib : nullptr);
                 break;
             case F8_LAYER_DWCONV:
                 e = f8_launch_dwconv(stp.g, L.q, stp.x, L.w, L.b, stp.res, stp.y, st, net->overlap_layers);
                 break;
             case F8_LAYER_MAXPOOL:
-                e = f8_launch_maxpool(batch, L.g.h, L.g.w, L.g.c, L.d.conv.kh, L.d.conv.stride, L.d.conv.pad, L.g.x_signed,
+                e = f8_launch_maxpool(stp.g.n, L.g.h, L.g.w, L.g.c, L.d.conv.kh, L.d.conv.stride, L.d.conv.pad, L.g.x_signed,
                                       stp.x, stp.y, st, net->overlap_layers);
                 break;
             case F8_LAYER_GAP:
-                e = f8_launch_gap(batch, L.g.h, L.g.w, L.g.c, L.g.x_signed, L.q.s, stp.x, stp.y, st, net->overlap_layers);
+                e = f8_launch_gap(stp.g.n, L.g.h, L.g.w, L.g.c, L.g.x_signed, L.q.s, stp.x, stp.y, st, net->overlap_layers);
                 break;
         }
         if (e != cudaSuccess) return fail(F8_ERR_CUDA, "launch of layer %d: %s", stp.layer, cudaGetErrorString(e));
@@ -876,16 +1136,23 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
             cudaEventRecord(net->events[launches], st);
             net->event_layer.push_back(stp.fused_pool ? stp.layer + 1 : stp.layer);
         }
-        const int out_layer = stp.fused_pool ? stp.layer + 1 : stp.layer;      // the layer whose output this step wrote
-        if (layer_dump && stp.kind != -1 && layer_dump[out_layer]) {
+        // copies of the outputs this step wrote: its layer's (the pooling layer's when fused), and a sibling's
+        auto dump_layer = [&](int out_layer, const void *src) -> cudaError_t {
+            if (!layer_dump || !layer_dump[out_layer]) return cudaSuccess;
             const int c_true = net->t_c[out_layer + 1], c_stored = net->t_cp[out_layer + 1];
+            const size_t elem = (size_t)net->t_elem[out_layer + 1];
+            const size_t pixels_per_image = (size_t)net->t_h[out_layer + 1] * net->t_w[out_layer + 1];
+            const size_t pixels = (size_t)stp.g.n * pixels_per_image;
+            uint8_t *dst = (uint8_t *)layer_dump[out_layer] + (size_t)stp.img0 * pixels_per_image * c_true * elem;
             if (c_true == c_stored)
-                e = cudaMemcpyAsync(layer_dump[out_layer], stp.y, (size_t)batch * net->layers[out_layer].out_bytes_per_image,
-                                    cudaMemcpyDeviceToDevice, st);
-            else   // drop the zero padding channels: one row per pixel
-                e = cudaMemcpy2DAsync(layer_dump[out_layer], (size_t)c_true, stp.y, (size_t)c_stored, (size_t)c_true,
-                                      (size_t)batch * net->t_h[out_layer + 1] * net->t_w[out_layer + 1],
-                                      cudaMemcpyDeviceToDevice, st);
+                return cudaMemcpyAsync(dst, src, pixels * c_true * elem, cudaMemcpyDeviceToDevice, st);
+            // drop the zero padding channels: one row per pixel
+            return cudaMemcpy2DAsync(dst, c_true * elem, src, c_stored * elem, c_true * elem, pixels,
+                                     cudaMemcpyDeviceToDevice, st);
+        };
+        if (stp.kind != -1) {
+            e = dump_layer(stp.fused_pool ? stp.layer + 1 : stp.layer, stp.y);
+            if (e == cudaSuccess && stp.has_sib) e = dump_layer(stp.layer + 1, stp.sib.y2);
             if (e != cudaSuccess) return cuda_fail(e, "layer dump copy");
         }
     }

@@ -39,7 +39,7 @@ __device__ __forceinline__ int dp4a_ss(uint32_t a, uint32_t b, int c) {   // s8 
 }
 
 __device__ __forceinline__ void store_out(void *y, size_t i, int v, int y_kind) {
-    if (y_kind == F8_S32) ((int32_t *)y)[i] = v;
+    if (y_kind == F8_S32 || y_kind == F8_S32_RELU) ((int32_t *)y)[i] = v;
     else ((uint8_t *)y)[i] = (uint8_t)(v & 0xff);
 }
 
@@ -51,7 +51,8 @@ template <bool VEC4>
 __global__ void __launch_bounds__(256) conv_direct_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
                                                           const int8_t *__restrict__ w,
                                                           const int32_t *__restrict__ bias,
-                                                          const void *__restrict__ res, void *__restrict__ y) {
+                                                          const void *__restrict__ res, void *__restrict__ y,
+                                                          F8Sibling sib) {
     grid_dependency_sync();
     const size_t total = (size_t)g.n * g.ho * g.wo * g.c_out;
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
@@ -88,8 +89,11 @@ __global__ void __launch_bounds__(256) conv_direct_kernel(F8ConvGeom g, F8Requan
                 }
             }
         }
-        const int rv = q.has_res ? f8_load8(res, idx, q.r_signed) : 0;
-        store_out(y, idx, f8_requant(acc, rv, q), q.y_kind);
+        const int rv = q.has_res ? (q.r_s32 ? ((const int32_t *)res)[idx] : f8_load8(res, idx, q.r_signed)) : 0;
+        // one 32-bit sum, one quantisation per consumer (Sec. 4.3)
+        const int v = f8_align_add(acc, rv, q);
+        store_out(y, idx, f8_quantize_child(v, q.y_kind, q.s, q.lo, q.hi), q.y_kind);
+        if (sib.y2) store_out(sib.y2, idx, f8_quantize_child(v, sib.y_kind, sib.s, sib.lo, sib.hi), sib.y_kind);
     }
 }
 
@@ -694,14 +698,16 @@ inline int grid_for(size_t total, int block) {
 }   // namespace
 
 cudaError_t f8_launch_conv_direct(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
-                                  const int32_t *bias, const void *res, void *y, cudaStream_t st, bool overlap_previous) {
+                                  const int32_t *bias, const void *res, void *y, cudaStream_t st, bool overlap_previous,
+                                  const F8Sibling *sib) {
     const size_t total = (size_t)g.n * g.ho * g.wo * g.c_out;
     if (total == 0) return cudaSuccess;
     const bool vec = (g.c % 4 == 0) && (((uintptr_t)x | (uintptr_t)w) % 4 == 0);
+    const F8Sibling sb = sib ? *sib : F8Sibling();
     if (vec)
-        launch_k(conv_direct_kernel<true>, grid_for(total, 256), 256, overlap_previous, st, g, q, (const uint8_t *)x, w, bias, res, y);
+        launch_k(conv_direct_kernel<true>, grid_for(total, 256), 256, overlap_previous, st, g, q, (const uint8_t *)x, w, bias, res, y, sb);
     else
-        launch_k(conv_direct_kernel<false>, grid_for(total, 256), 256, overlap_previous, st, g, q, (const uint8_t *)x, w, bias, res, y);
+        launch_k(conv_direct_kernel<false>, grid_for(total, 256), 256, overlap_previous, st, g, q, (const uint8_t *)x, w, bias, res, y, sb);
     return cudaGetLastError();
 }
 

@@ -9,20 +9,30 @@ __device__ __forceinline__ int f8_rshift_round(int v, int s) {
     return (v >> s) + ((v >> (s - 1)) & 1);
 }
 
-// acc already holds sum + bias.  r is the residual code (ignored unless q.has_res).
-__device__ __forceinline__ int f8_requant(int acc, int r, const F8Requant &q) {
-    int v = acc;
-    if (q.has_res) v = (acc << q.sh_acc) + (r << q.sh_res);
-    if (q.y_kind == F8_S32) return v;
+// One consumer's view of the aligned 32-bit sum v: the quantizer of Eq. 2 / its signed form with this consumer's
+// shift, or the 32-bit value itself (kind F8_S32), or that value behind a ReLU (F8_S32_RELU).
+__device__ __forceinline__ int f8_quantize_child(int v, int y_kind, int s, int lo, int hi) {
+    if (y_kind == F8_S32) return v;
+    if (y_kind == F8_S32_RELU) return max(v, 0);
     int t;
-    if (q.s > 0) {
-        t = f8_rshift_round(v, q.s);
+    if (s > 0) {
+        t = f8_rshift_round(v, s);
     } else {
         // left shift by at most 8; clamping first keeps the product inside int32 and
         // cannot change the clipped result because |lo|, |hi| <= 255 < 256
-        t = min(max(v, -256), 256) << (-q.s);
+        t = min(max(v, -256), 256) << (-s);
     }
-    return min(max(t, q.lo), q.hi);
+    return min(max(t, lo), hi);
+}
+
+// acc already holds sum + bias.  r is the residual operand (ignored unless q.has_res): the accumulator and the
+// shortcut are brought to the finer of their two formats by shifts and added (Sec. 4.3).
+__device__ __forceinline__ int f8_align_add(int acc, int r, const F8Requant &q) {
+    return q.has_res ? (acc << q.sh_acc) + (r << q.sh_res) : acc;
+}
+
+__device__ __forceinline__ int f8_requant(int acc, int r, const F8Requant &q) {
+    return f8_quantize_child(f8_align_add(acc, r, q), q.y_kind, q.s, q.lo, q.hi);
 }
 
 __device__ __forceinline__ int f8_load8(const void *p, size_t i, int is_signed) {

@@ -125,6 +125,8 @@ struct TcParams {
                                            // tiles, int32 bias' of all padded columns
     uint32_t ktab_off;        // table of k-iteration coordinates (8 bytes each)
     F8Requant q;
+    F8Sibling sib;            // second consumer of the same sums (generic epilogue only)
+    int vec_bytes2;           // widest aligned store of the second output's rows
     int mul_acc, mul_res;     // 2^q.sh_acc, 2^q.sh_res (kept opaque to the compiler, see the epilogue)
     int *status;
     // Windowed 3x3 (stride 1, pad 1, resident weights).  A tile is win_r whole output rows of one image; its M index runs
@@ -143,50 +145,80 @@ struct TcParams {
 
 // ----------------------------------------------------------------------------- epilogue helpers
 
-__device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int (&acc)[16], size_t row, int co0,
-                                               bool row_valid) {
-    // how many of the 16 channels exist
-    const int nvalid = min(16, p.c_out - co0);
-    int v[16];
-    uint32_t rw[4] = {0u, 0u, 0u, 0u};
-    const size_t o = row * (size_t)p.c_out + co0;
-    if (p.q.has_res && row_valid) {
-        if (p.vec_bytes == 16 && nvalid == 16) {
-            const uint4 t = *(const uint4 *)(p.res + o);
-            rw[0] = t.x; rw[1] = t.y; rw[2] = t.z; rw[3] = t.w;
-        } else {
-            for (int j = 0; j < nvalid; ++j) rw[j >> 2] |= (uint32_t)p.res[o + j] << (8 * (j & 3));
-        }
-    }
+// Writes 16 consecutive channels of one output row for one consumer of the aligned sums v[].
+__device__ __forceinline__ void store_chunk(uint8_t *ybase, int y_kind, int s, int lo, int hi, const int (&v)[16], size_t o,
+                                            int nvalid, int c_out, int vec_bytes) {
+    int t[16];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        const int b = (j < nvalid && p.bias) ? __ldg(p.bias + co0 + j) : 0;
-        v[j] = f8_requant(acc[j] + b, f8_byte(rw[j >> 2], j & 3, p.q.r_signed), p.q);
-    }
-    if (!row_valid) return;
-    if (p.q.y_kind == F8_S32) {
-        int32_t *y32 = (int32_t *)p.y + o;
-        if (nvalid == 16 && (p.c_out & 3) == 0) {
+    for (int j = 0; j < 16; ++j) t[j] = f8_quantize_child(v[j], y_kind, s, lo, hi);
+    if (y_kind == F8_S32 || y_kind == F8_S32_RELU) {
+        int32_t *y32 = (int32_t *)ybase + o;
+        if (nvalid == 16 && (c_out & 3) == 0) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) *(int4 *)(y32 + 4 * j) = make_int4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            for (int j = 0; j < 4; ++j) *(int4 *)(y32 + 4 * j) = make_int4(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3]);
         } else {
-            for (int j = 0; j < nvalid; ++j) y32[j] = v[j];
+            for (int j = 0; j < nvalid; ++j) y32[j] = t[j];
         }
         return;
     }
     uint32_t ow[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) ow[j] = f8_pack4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-    uint8_t *yo = p.y + o;
-    if (nvalid == 16 && p.vec_bytes == 16) {
+    for (int j = 0; j < 4; ++j) ow[j] = f8_pack4(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3]);
+    uint8_t *yo = ybase + o;
+    if (nvalid == 16 && vec_bytes == 16) {
         *(uint4 *)yo = make_uint4(ow[0], ow[1], ow[2], ow[3]);
-    } else if (p.vec_bytes >= 8 && (nvalid & 7) == 0) {
+    } else if (vec_bytes >= 8 && (nvalid & 7) == 0) {
         for (int j = 0; j < nvalid / 8; ++j) *(uint2 *)(yo + 8 * j) = make_uint2(ow[2 * j], ow[2 * j + 1]);
-    } else if (p.vec_bytes >= 4 && (nvalid & 3) == 0) {
+    } else if (vec_bytes >= 4 && (nvalid & 3) == 0) {
         for (int j = 0; j < nvalid / 4; ++j) *(uint32_t *)(yo + 4 * j) = ow[j];
     } else {
         for (int j = 0; j < nvalid; ++j) yo[j] = (uint8_t)(ow[j >> 2] >> (8 * (j & 3)));
     }
+}
+
+// Generic epilogue with direct stores: any output kind, any channel count, an 8-bit or 32-bit shortcut, and
+// optionally a second consumer of the same sums with its private fractional length (Sec. 4.3).
+__device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int (&acc)[16], size_t row, int co0,
+                                               bool row_valid) {
+    // how many of the 16 channels exist
+    const int nvalid = min(16, p.c_out - co0);
+    int v[16];
+    const size_t o = row * (size_t)p.c_out + co0;
+    int r[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) r[j] = 0;
+    if (p.q.has_res && row_valid) {
+        if (p.q.r_s32) {
+            const int32_t *r32 = (const int32_t *)p.res + o;
+            if (nvalid == 16 && (p.c_out & 3) == 0) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int4 t = *(const int4 *)(r32 + 4 * j);
+                    r[4 * j] = t.x; r[4 * j + 1] = t.y; r[4 * j + 2] = t.z; r[4 * j + 3] = t.w;
+                }
+            } else {
+                for (int j = 0; j < nvalid; ++j) r[j] = r32[j];
+            }
+        } else {
+            uint32_t rw[4] = {0u, 0u, 0u, 0u};
+            if ((p.c_out & 15) == 0 && nvalid == 16) {      // 8-bit rows of c_out bytes: 16-byte aligned chunks
+                const uint4 t = *(const uint4 *)(p.res + o);
+                rw[0] = t.x; rw[1] = t.y; rw[2] = t.z; rw[3] = t.w;
+            } else {
+                for (int j = 0; j < nvalid; ++j) rw[j >> 2] |= (uint32_t)p.res[o + j] << (8 * (j & 3));
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) r[j] = f8_byte(rw[j >> 2], j & 3, p.q.r_signed);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int b = (j < nvalid && p.bias) ? __ldg(p.bias + co0 + j) : 0;
+        v[j] = f8_align_add(acc[j] + b, r[j], p.q);
+    }
+    if (!row_valid) return;
+    store_chunk(p.y, p.q.y_kind, p.q.s, p.q.lo, p.q.hi, v, o, nvalid, p.c_out, p.vec_bytes);
+    if (p.sib.y2) store_chunk((uint8_t *)p.sib.y2, p.sib.y_kind, p.sib.s, p.sib.lo, p.sib.hi, v, o, nvalid, p.c_out, p.vec_bytes2);
 }
 
 // ----------------------------------------------------------------------------- the kernel
@@ -826,7 +858,7 @@ bool f8_tc_supported(const F8ConvGeom &g, size_t x_bytes) {
 
 cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant &q, const F8TcTensorView &xv,
                             const int8_t *w, const int32_t *bias, const void *res, void *y, int *status_word,
-                            const char **why) {
+                            const char **why, const F8Sibling *sib) {
     *why = "";
     if (!load_driver_entry_points()) {
         *why = "cuTensorMapEncode entry points not available";
@@ -850,7 +882,8 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     if (q.has_res && g.c_out > 128 && p.kb == 128 && g.c <= 256) p.kb = 64;
     p.c_chunks = (g.c + p.kb - 1) / p.kb;
     p.epi = EPI_GENERIC;
-    if (q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24 && g.c_out % 16 == 0)
+    const bool has_sib = sib && sib->y2;
+    if ((q.y_kind == F8_U8 || q.y_kind == F8_S8) && q.s >= 1 && q.s <= 24 && g.c_out % 16 == 0 && !has_sib && !q.r_s32)
         p.epi = q.y_kind == F8_U8 ? (q.has_res ? EPI_U8_RES : EPI_U8) : (q.has_res ? EPI_S8_RES : EPI_S8);
     const bool staged = p.epi != EPI_GENERIC;
     p.bn = staged ? choose_bn_staged(g.c_out, q.has_res != 0, p.kb) : choose_bn(g.c_out);
@@ -988,9 +1021,14 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.mul_acc = 1 << q.sh_acc;
     p.mul_res = 1 << q.sh_res;
     p.status = status_word;
-    const int ysz = q.y_kind == F8_S32 ? 4 : 1;
+    const int ysz = (q.y_kind == F8_S32 || q.y_kind == F8_S32_RELU) ? 4 : 1;
     const size_t row_bytes = (size_t)g.c_out * ysz;
     p.vec_bytes = (row_bytes % 16 == 0) ? 16 : (row_bytes % 8 == 0 ? 8 : (row_bytes % 4 == 0 ? 4 : 1));
+    if (has_sib) p.sib = *sib;
+    {
+        const size_t rb2 = (size_t)g.c_out * ((p.sib.y_kind == F8_S32 || p.sib.y_kind == F8_S32_RELU) ? 4 : 1);
+        p.vec_bytes2 = (rb2 % 16 == 0) ? 16 : (rb2 % 8 == 0 ? 8 : (rb2 % 4 == 0 ? 4 : 1));
+    }
 
     const bool dense_x = xv.stride_w == xv.dim_c && xv.stride_h == xv.dim_c * xv.dim_w && xv.stride_n == xv.dim_c * xv.dim_w * xv.dim_h;
     p.a_plain = (g.kh == 1 && g.kw == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 && g.pad_w == 0 && dense_x &&

@@ -16,9 +16,18 @@ struct F8Requant {
     int sh_res;     // F - fl_r
     int s;          // F - fl_y   in [-8, 31]
     int lo, hi;     // clip bounds of the output quantizer
-    int y_kind;     // F8_U8 / F8_S8 / F8_S32
+    int y_kind;     // F8_U8 / F8_S8 / F8_S32 / F8_S32_RELU
     int has_res;
     int r_signed;
+    int r_s32 = 0;  // the residual operand is an int32 tensor (a shortcut kept in 32 bits, Sec. 4.3)
+};
+
+// A second consumer of the same 32-bit sum, quantised with its private fractional length (Sec. 4.3).
+struct F8Sibling {
+    void *y2 = nullptr;     // nullptr: none
+    int y_kind = 0;         // F8_U8 / F8_S8 / F8_S32 / F8_S32_RELU
+    int s = 0;              // F - fl_y2
+    int lo = 0, hi = 0;
 };
 
 // Geometry of one convolution-shaped launch (dense or depthwise).
@@ -37,7 +46,7 @@ struct F8ConvGeom {
 // before it prior to touching memory, so this is always safe; it lets launch latency overlap their tail).
 cudaError_t f8_launch_conv_direct(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
                                   const int32_t *bias, const void *res, void *y, cudaStream_t st,
-                                  bool overlap_previous = false);
+                                  bool overlap_previous = false, const F8Sibling *sib = nullptr);
 cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void *x, const int8_t *w,
                              const int32_t *bias, const void *res, void *y, cudaStream_t st,
                              bool overlap_previous = false);
@@ -70,7 +79,7 @@ size_t f8_tc_plan_size();
 // Encodes tensor maps and tile schedule; returns cudaSuccess or an error (no launch).
 cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant &q, const F8TcTensorView &xv,
                             const int8_t *w /* [c_out][kh][kw][g.c] */, const int32_t *bias, const void *res,
-                            void *y, int *status_word, const char **why);
+                            void *y, int *status_word, const char **why, const F8Sibling *sib = nullptr);
 // Label reported (with the wait's site) when a bounded wait of this launch gives up; 0 = none.
 void f8_tc_plan_set_tag(F8TcPlan *plan, int tag);
 // overlap_previous: the grid may start before the preceding work of the stream has finished; only its weight

@@ -106,6 +106,38 @@ def bench_net(name: str, batch: int, iters: int, warmup: int):
                       "launches": net.last_launch_count}), flush=True)
 
 
+def shape_key(l: synth.Layer) -> str:
+    return f"{l.h}x{l.w}x{l.c}->{l.c_out} k{l.kh} s{l.stride} res{1 if l.res >= 0 else 0}"
+
+
+def run_distinct_shapes(name: str, batch: int):
+    """Every distinct dense-layer shape of a synthetic network once, as single-layer calls on fresh buffers, in the order
+    printed: the launch list of a profiler run of this command maps one to one onto the printed shapes (layers that do
+    not take the tensor-core kernel are listed with "tensor_cores": false and launch another kernel)."""
+    rng = np.random.default_rng(0)
+    seen = set()
+    for l in synth.make_net(name, 0):
+        if l.kind != synth.CONV or shape_key(l) in seen:
+            continue
+        seen.add(shape_key(l))
+        if l.x_dtype == synth.S8:
+            x = rng.integers(-128, 128, size=(batch, l.h, l.w, l.c), dtype=np.int64).astype(np.int8)
+        else:
+            x = rng.integers(0, 256, size=(batch, l.h, l.w, l.c), dtype=np.int64).astype(np.uint8)
+        res = None
+        if l.res >= 0:
+            res = torch.randint(0, 255, (batch, l.ho, l.wo, l.c_out), dtype=torch.uint8, device="cuda")
+            if l.r_dtype == synth.S8:
+                res = res.view(torch.int8)
+        before = api.f8_tc_launch_count()
+        api.run_layer(l, api.to_device(x), res)
+        torch.cuda.synchronize()
+        print(json.dumps({"shape": shape_key(l), "layer": l.name, "batch": batch,
+                          "tensor_cores": api.f8_tc_launch_count() - before == 1,
+                          "algorithmic_bytes": batch * l.bytes_per_image() + l.param_bytes()}), flush=True)
+    api.f8_device_status()
+
+
 def bench_fold(c_out: int, k: int, iters: int, warmup: int):
     """Device time of the weight compile step (f8_fold_quantize_fixed) on one [c_out, k] fp32 tensor.  Algorithmic
     bytes: 4 read + 1 written per weight (the fp32 tensor has to be read twice -- statistics, then quantisation --
@@ -157,6 +189,7 @@ def main():
     ap.add_argument("--fold", action="store_true", help="time the weight compile step on a [c-out, k * k * c] tensor")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--net", default="", help="time every layer of a synthetic network: resnet18, resnet50, mobilenetv2")
+    ap.add_argument("--distinct-shapes", default="", help="run every distinct dense-layer shape of this network once (for a profiler)")
     ap.add_argument("--h", type=int, default=56)
     ap.add_argument("--w", type=int, default=0)
     ap.add_argument("--c", type=int, default=64)
@@ -176,7 +209,9 @@ def main():
     if args.fold:
         bench_fold(args.c_out, args.k * args.k * args.c, args.iters, args.warmup)
         return
-    if args.net:
+    if args.distinct_shapes:
+        run_distinct_shapes(args.distinct_shapes, args.batch)
+    elif args.net:
         bench_net(args.net, args.batch, args.iters, args.warmup)
     elif args.sweep:
         for i in range(len(synth.SWEEP_SHAPES)):

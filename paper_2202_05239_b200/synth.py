@@ -37,8 +37,10 @@ from typing import List, Optional, Tuple
 import numpy as np
 
 U8, S8, S32 = 0, 1, 2
+S32_RELU = 3      # output kind of sibling handling only: the 32-bit sum behind a ReLU (stored like S32)
 CONV, DWCONV, MAXPOOL, GAP, LINEAR = 0, 1, 2, 3, 4
-KIND_NAMES = {CONV: "conv", DWCONV: "dwconv", MAXPOOL: "maxpool", GAP: "gap", LINEAR: "linear"}
+SIBLING = 5       # a second consumer's view of the previous layer's 32-bit sum, with its private format (Sec. 4.3)
+KIND_NAMES = {CONV: "conv", DWCONV: "dwconv", MAXPOOL: "maxpool", GAP: "gap", LINEAR: "linear", SIBLING: "sibling"}
 
 
 @dataclass
@@ -68,7 +70,7 @@ class Layer:
     wo: int = field(init=False, default=0)
 
     def __post_init__(self):
-        if self.kind in (CONV, DWCONV, MAXPOOL):
+        if self.kind in (CONV, DWCONV, MAXPOOL, SIBLING):
             self.ho = (self.h + 2 * self.pad - self.kh) // self.stride + 1
             self.wo = (self.w + 2 * self.pad - self.kw) // self.stride + 1
         else:
@@ -86,9 +88,12 @@ class Layer:
 
     def bytes_per_image(self) -> int:
         """Algorithmic activation bytes per image: input + output (+ residual)."""
-        ysz = 4 if self.y_dtype == S32 else 1
+        ysz = 4 if self.y_dtype in (S32, S32_RELU) else 1
         out = self.ho * self.wo * self.c_out * ysz
-        return self.h * self.w * self.c + out + (self.ho * self.wo * self.c_out if self.res >= 0 else 0)
+        if self.kind == SIBLING:
+            return out                      # a second output of the parent's launch: written, nothing read
+        rsz = 4 if self.r_dtype == S32 else 1
+        return self.h * self.w * self.c + out + (self.ho * self.wo * self.c_out * rsz if self.res >= 0 else 0)
 
     def param_bytes(self) -> int:
         b = 0
@@ -229,13 +234,16 @@ class _NetBuilder:
     def __init__(self, seed: int, stream: int, h: int, w: int, c: int):
         self.seed, self.stream = seed, stream
         self.layers: List[Layer] = []
+        self.drawn = 0            # layers that drew random numbers so far (sibling layers draw none)
         # image: N(0,1) real values in s8 FL 6
         self.stats: List[_Stat] = [_Stat(0.0, 1.0, S8, 6, h, w, c)]
 
     def _rng(self) -> np.random.Generator:
-        return _rng(self.seed, self.stream, len(self.layers))
+        # one stream per layer, numbered without the sibling layers: a net with sibling layers draws the same
+        # weights as the same net without them
+        return _rng(self.seed, self.stream, len(self.layers) - sum(1 for l in self.layers if l.kind == SIBLING))
 
-    def _finish(self, layer: Layer, pre_mean: float, pre_var: float, relu: bool) -> int:
+    def _finish(self, layer: Layer, pre_mean: float, pre_var: float, relu: bool, keep32: bool = False) -> int:
         sd = math.sqrt(pre_var)
         if relu:
             layer.y_dtype, layer.fl_y = U8, fl_unsigned(sd)
@@ -243,12 +251,28 @@ class _NetBuilder:
         else:
             layer.y_dtype, layer.fl_y = S8, fl_signed(sd)
             m1, v = pre_mean, pre_var
+        fl_out = layer.fl_y
+        if keep32:      # the sum itself, in the format of the aligned sum
+            layer.y_dtype = S32_RELU if relu else S32
+            fl_out = max(layer.fl_x + layer.fl_w, layer.fl_r) if layer.res >= 0 else layer.fl_x + layer.fl_w
         self.layers.append(layer)
-        self.stats.append(_Stat(m1, v, layer.y_dtype, layer.fl_y, layer.ho, layer.wo, layer.c_out))
+        self.stats.append(_Stat(m1, v, S32 if keep32 else layer.y_dtype, fl_out, layer.ho, layer.wo, layer.c_out))
+        return len(self.stats) - 1
+
+    def sibling(self, name: str, parent: int, y_dtype: int, fl_y: int = 0) -> int:
+        """Second consumer of the sum that produced tensor `parent` (which must be the newest tensor)."""
+        assert parent == len(self.stats) - 1 and self.layers[-1].kind == CONV
+        p, ps = self.layers[-1], self.stats[parent]
+        layer = Layer(SIBLING, name, parent, -1, ps.h, ps.w, ps.c, ps.c, 1, 1, 1, 0, p.x_dtype, y_dtype, U8,
+                      p.fl_x, p.fl_w, fl_y, 0)
+        self.layers.append(layer)
+        wide = y_dtype in (S32, S32_RELU)
+        fl_sum = max(p.fl_x + p.fl_w, p.fl_r) if p.res >= 0 else p.fl_x + p.fl_w
+        self.stats.append(_Stat(ps.mean, ps.var, S32 if wide else y_dtype, fl_sum if wide else fl_y, ps.h, ps.w, ps.c))
         return len(self.stats) - 1
 
     def conv(self, name: str, src: int, c_out: int, k: int, stride: int, relu: bool, res: int = -1,
-             depthwise: bool = False) -> int:
+             depthwise: bool = False, keep32: bool = False) -> int:
         s = self.stats[src]
         rng = self._rng()
         fan_in = k * k * (1 if depthwise else s.c)
@@ -266,7 +290,7 @@ class _NetBuilder:
             layer.r_dtype, layer.fl_r = r.dtype, r.fl
             pre_mean += r.mean
             pre_var += r.var
-        return self._finish(layer, pre_mean, pre_var, relu)
+        return self._finish(layer, pre_mean, pre_var, relu, keep32)
 
     def maxpool(self, name: str, src: int, k: int = 3, stride: int = 2, pad: int = 1) -> int:
         s = self.stats[src]
@@ -310,18 +334,35 @@ class _NetBuilder:
 # the paper under study names the networks but does not list their layers)
 # --------------------------------------------------------------------------
 
-def resnet18(seed: int = 0, image: int = 224) -> List[Layer]:
+def resnet18(seed: int = 0, image: int = 224, siblings: bool = False) -> List[Layer]:
+    """siblings=False: every activation is one 8-bit tensor that all of its consumers read (re-aligned by shifts
+    where their formats differ).  siblings=True: the handling the paper describes for layers with two children
+    (Sec. 4.3, Fig. 4) -- the sum of a block's last layer stays in 32 bits and is quantised once per child: the next
+    block's first convolution reads the master format, its down-sampling convolution (where there is one) a private
+    format one bit finer (a synthetic stand-in: trained formats are not available), and an identity shortcut takes
+    the 32-bit value itself (behind the ReLU, unrounded); a down-sampling convolution also hands its sum on in 32 bits.
+    Weights are the same in both variants."""
     b = _NetBuilder(seed, 18, image, image, 3)
     t = b.conv("stem", 0, 64, 7, 2, True)
     t = b.maxpool("pool", t)
-    for si, width in enumerate([64, 128, 256, 512]):
+    t_private, t_wide = None, None          # the newest block output in a private 8-bit format / in 32 bits
+    widths = [64, 128, 256, 512]
+    for si, width in enumerate(widths):
         for bi in range(2):
             stride = 2 if (bi == 0 and si > 0) else 1
-            short = t
+            short = t_wide if t_wide is not None else t
             if stride != 1 or b.stats[t].c != width:
-                short = b.conv(f"s{si}b{bi}.down", t, width, 1, stride, False)
+                short = b.conv(f"s{si}b{bi}.down", t_private if t_private is not None else t, width, 1, stride, False,
+                               keep32=siblings)
             u = b.conv(f"s{si}b{bi}.conv1", t, width, 3, stride, True)
             t = b.conv(f"s{si}b{bi}.conv2", u, width, 3, 1, True, res=short)
+            t_private, t_wide = None, None
+            last = si == len(widths) - 1 and bi == 1
+            if siblings and not last:
+                if bi == 1:      # the next block starts a stage: its down-sampling convolution is the second child
+                    t_private = b.sibling(f"s{si}b{bi}.conv2.private", t, U8, min(8, b.stats[t].fl + 1))
+                else:            # the next block adds this block's output back in: kept in 32 bits
+                    t_wide = b.sibling(f"s{si}b{bi}.conv2.wide", t, S32_RELU)
     t = b.gap("gap", t)
     b.linear("fc", t, 1000)
     return b.layers
@@ -383,6 +424,13 @@ def mobilenetv1(seed: int = 0, image: int = 224) -> List[Layer]:
 
 
 NETS = {"resnet18": resnet18, "resnet50": resnet50, "mobilenetv2": mobilenetv2, "mobilenetv1": mobilenetv1}
+
+
+def resnet18_siblings(seed: int = 0, image: int = 224) -> List[Layer]:
+    return resnet18(seed, image, siblings=True)
+
+
+NETS["resnet18_siblings"] = resnet18_siblings
 
 
 def make_net(name: str, seed: int = 0, image: int = 224) -> List[Layer]:

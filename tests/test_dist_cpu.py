@@ -62,3 +62,17 @@ def test_reference_arm_runs_on_rank_zero_only(tmp_path):
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
                           "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_gpus_flag_without_a_launcher_starts_that_many_ranks():
+    """`bench.py --gpus 2` with no launcher in the environment starts two local ranks itself (here only their
+    plumbing, on CPU with gloo) and rank 0 reports the world size it actually ran with."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dist-selftest"], env=env,
+                         capture_output=True, text=True, timeout=180)
+    assert out.returncode == 0, out.stderr
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    import json
+    rec = json.loads(lines[0])
+    assert rec["n_gpus"] == 2 and rec["requested"] == 2

@@ -13,7 +13,7 @@ def _layer_shape(l, batch):
     return (batch, l.c_out) if l.kind in (synth.LINEAR, synth.GAP) else (batch, l.ho, l.wo, l.c_out)
 
 
-def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0):
+def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0, micro_batch=0):
     """Every layer's output against the oracle.  The dump buffers, the network output and the workspace sit between
     poisoned guard bands that must come back untouched."""
     a = api()
@@ -22,6 +22,7 @@ def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0
     want = ref.net_forward(layers, x)
     a.f8_debug_force_direct(force_direct)
     a.f8_debug_plan_options(plan_off)
+    a.f8_debug_set_micro_batch(micro_batch)
     before = a.f8_tc_launch_count()
     try:
         net = a.Net(layers, batch)
@@ -35,17 +36,23 @@ def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0
     finally:
         a.f8_debug_force_direct(False)
         a.f8_debug_plan_options(0)
+        a.f8_debug_set_micro_batch(0)
+    if micro_batch:
+        runs, images = net.micro_batching()
+        assert runs >= 1 and images == micro_batch, "the forward pass was not micro-batched"
     for i, l in enumerate(layers):
         got = dump[i].cpu().numpy().reshape(want[i + 1].shape)
         assert_equal_arrays(got, want[i + 1], f"{name} layer {i} ({l.name}): ")
         assert guards[i].intact(), f"{name} layer {i} ({l.name}): bytes next to the dump buffer were overwritten"
     assert np.array_equal(out.t.cpu().numpy(), want[-1])
     assert out.intact() and ws.intact(), "bytes next to the output or the workspace were overwritten"
-    assert net.last_launch_count >= len(layers)
+    # one launch per layer, except that a sibling layer is written by its parent's launch and a first layer may take
+    # the pooling layer behind it along
+    assert net.last_launch_count >= sum(1 for l in layers if l.kind != synth.SIBLING) - 1
     tc = a.f8_tc_launch_count() - before
     if force_direct:
         assert tc == 0
-    elif image == 224:
+    elif image == 224 and not micro_batch:
         # every dense layer whose input is at least 128 KiB and has c % 16 == 0 (or is a packed stem)
         assert tc >= sum(1 for l in layers if l.kind == synth.CONV and l.c % 16 == 0 and batch * l.h * l.w * l.c >= 131072)
     net.close()
@@ -82,6 +89,15 @@ def test_net_parity_with_planning_choices_switched_off(ref, case):
     _compare_net(ref, "resnet50", 4, 224, plan_off=_off_masks()[case])
 
 
+@pytest.mark.parametrize("name,batch,micro,direct", [("resnet50", 8, 3, False), ("resnet18", 7, 2, False), ("mobilenetv2", 5, 2, False),
+                                                     ("mobilenetv1", 6, 4, False), ("resnet18_siblings", 5, 2, False),
+                                                     ("resnet50", 3, 1, True), ("resnet50", 64, 16, False)])
+def test_net_parity_micro_batched(ref, name, batch, micro, direct):
+    """Depth-first execution of runs of layers over micro-batches (tensors inside a run hold one micro-batch and are
+    reused; the last micro-batch may be ragged): every layer's output is unchanged."""
+    _compare_net(ref, name, batch, 224 if not direct else 64, force_direct=direct, micro_batch=micro)
+
+
 def test_mobilenet_parity_with_the_strip_kernel(ref):
     a = api()
     _compare_net(ref, "mobilenetv1", 3, 224, plan_off=a.PLAN_OFF_DW_WALK)
@@ -98,6 +114,7 @@ def _sampled_full_batch(ref, name, batch, samples):
     out = net.forward(a.to_device(x), dump=dump)
     torch.cuda.synchronize()
     a.f8_device_status()
+    print(f"{name} batch {batch}: micro-batched runs, smallest micro-batch = {net.micro_batching()}")
     for i in samples:
         want = ref.net_forward(layers, x[i:i + 1])
         for li, l in enumerate(layers):
