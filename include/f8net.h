@@ -181,10 +181,12 @@ size_t f8_net_workspace_bytes(const f8_net *net, int batch);
  * input; y: the last layer's output ([batch, out] int32 logits for a net ending in a linear
  * layer).  layer_dump: NULL, or an array of n_layers device pointers; a non-NULL entry i
  * receives a copy of layer i's output (for parity checks).
- * Schedule: layers run one after the other over the whole batch, except that a run of layers with equal output
- * size whose tensors do not fit the L2 cache at the full batch may be executed depth-first over micro-batches
- * (images are independent, so no result changes): tensors inside the run then hold one micro-batch and stay in
- * the cache between producer and consumer.  Status: if a kernel of an earlier pass on this object gave up a bounded
+ * Schedule: layers run one after the other over the whole batch on cuda_stream.  Two alternatives exist, both off
+ * by default because they measured slower on this GPU (every extra launch costs about 5 us of drained SMs):
+ * f8_debug_set_lanes(2) cuts the batch into two halves that run as two independent passes, one on cuda_stream and
+ * one on a stream the network owns, launched alternately (the call returns with cuda_stream waiting for both);
+ * f8_debug_set_micro_batch executes a run of layers with equal output size depth-first over micro-batches so that
+ * the tensors inside the run stay in the L2 cache.  Images are independent, so neither changes a result.  Status: if a kernel of an earlier pass on this object gave up a bounded
  * wait, the call returns F8_ERR_TIMEOUT before enqueuing anything (see f8_device_status). */
 f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *workspace,
                          size_t workspace_bytes, void *const *layer_dump, void *cuda_stream);
@@ -315,24 +317,29 @@ void f8_debug_force_direct(int on);
  *   F8_PLAN_OFF_STEM_KERNEL       first layers take the packed-row-pair GEMM instead of the first-layer kernel
  *   F8_PLAN_OFF_STEM_POOL_FUSION  the max pool behind a first layer runs as its own kernel
  *   F8_PLAN_OFF_LAYER_OVERLAP     f8_net_forward launches without programmatic dependent launch
- *   F8_PLAN_OFF_MICRO_BATCH       f8_net_forward runs every layer over the whole batch
+ *   F8_PLAN_OFF_LANES             f8_net_forward runs the whole batch as one sequence of launches on the caller's stream
  *   F8_PLAN_SYNC_LAYERS           f8_net_forward synchronises after every launch, so that a device fault is
  *                                 reported with the layer that raised it */
 enum {
     F8_PLAN_OFF_RESIDENT_WEIGHTS = 1, F8_PLAN_OFF_WINDOWED = 2, F8_PLAN_OFF_DUAL_ISSUE = 4, F8_PLAN_OFF_ALT_PRODUCERS = 8,
     F8_PLAN_OFF_PAIRS = 16, F8_PLAN_OFF_DW_WALK = 32, F8_PLAN_OFF_STEM_KERNEL = 64, F8_PLAN_OFF_STEM_POOL_FUSION = 128,
-    F8_PLAN_OFF_LAYER_OVERLAP = 256, F8_PLAN_OFF_MICRO_BATCH = 512, F8_PLAN_SYNC_LAYERS = 1024
+    F8_PLAN_OFF_LAYER_OVERLAP = 256, F8_PLAN_OFF_LANES = 512, F8_PLAN_SYNC_LAYERS = 1024
 };
 void f8_debug_plan_options(unsigned off_mask);
 
-/* Test hook for the micro-batch schedule of f8_net_forward.  By default a run of layers whose tensors exceed the L2
- * cache at the full batch is executed depth-first over micro-batches sized to the cache, provided every dense layer
- * of the run still has a few tiles per SM (see f8_net_forward).  images > 0 forces that micro-batch for every run of
- * three or more layers with equal output size (whatever the sizes); 0 restores the rule.  f8_net_micro_batching
- * reports what the last forward pass of a network did: the number of micro-batched runs (return value) and the
- * smallest micro-batch (*images). */
+/* The micro-batch schedule of f8_net_forward (off by default: on this GPU the extra launches cost more than the
+ * memory traffic they save).  images = -1: a run of layers whose tensors exceed the L2 cache at the full batch is
+ * executed depth-first over micro-batches sized to half the cache, provided every dense layer of the run still has
+ * two tiles per SM; images > 0 forces that micro-batch for every run of three or more layers with equal output
+ * size; 0 switches it off.  f8_net_micro_batching reports what the last forward pass of a network did: the number
+ * of micro-batched runs (return value) and the smallest micro-batch (*images). */
 void f8_debug_set_micro_batch(int images);
 int f8_net_micro_batching(const f8_net *net, int *images);
+
+/* Lanes of f8_net_forward: 0 = the library's rule (one lane: two measured slower on this GPU), 1 / 2 = that many.
+ * f8_net_lanes reports what the last forward pass used. */
+void f8_debug_set_lanes(int lanes);
+int f8_net_lanes(const f8_net *net);
 
 /* What the most recent tensor-core plan of this process decided (n <= 10 ints are written, the count is returned):
  * [0] flags below, [1] epilogue variant (0 generic, 1 u8, 2 u8 + residual, 3 s8, 4 s8 + residual), [2] N tile,

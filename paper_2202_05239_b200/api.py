@@ -239,7 +239,7 @@ _lib.f8_debug_wait_timeout_probe.argtypes = [ctypes.c_double, _vp]
 # f8_debug_plan_options bits (planning choices switched off) and f8_debug_last_plan flags
 PLAN_OFF_RESIDENT_WEIGHTS, PLAN_OFF_WINDOWED, PLAN_OFF_DUAL_ISSUE, PLAN_OFF_ALT_PRODUCERS = 1, 2, 4, 8
 PLAN_OFF_PAIRS, PLAN_OFF_DW_WALK, PLAN_OFF_STEM_KERNEL, PLAN_OFF_STEM_POOL_FUSION = 16, 32, 64, 128
-PLAN_OFF_LAYER_OVERLAP, PLAN_OFF_MICRO_BATCH, PLAN_SYNC_LAYERS = 256, 512, 1024
+PLAN_OFF_LAYER_OVERLAP, PLAN_OFF_LANES, PLAN_SYNC_LAYERS = 256, 512, 1024
 PLAN_RESIDENT_WEIGHTS, PLAN_WINDOWED, PLAN_DUAL_ISSUE, PLAN_ALT_PRODUCERS = 1, 2, 4, 8
 PLAN_PLAIN_MATRIX, PLAN_STAGED_EPILOGUE, PLAN_PAIRS = 16, 32, 64
 
@@ -254,8 +254,18 @@ _lib.f8_net_micro_batching.argtypes = [_vp, ctypes.POINTER(_ci)]
 
 
 def f8_debug_set_micro_batch(images: int):
-    """Forces the micro-batch of f8_net_forward's depth-first runs (0: the library's own rule)."""
+    """Micro-batch of f8_net_forward's depth-first runs: 0 off (default), -1 the L2-size rule, > 0 that many images."""
     _lib.f8_debug_set_micro_batch(images)
+
+
+_lib.f8_debug_set_lanes.argtypes = [_ci]
+_lib.f8_debug_set_lanes.restype = None
+_lib.f8_net_lanes.argtypes = [_vp]
+
+
+def f8_debug_set_lanes(lanes: int):
+    """Concurrent lanes of f8_net_forward: 0 the library's rule, 1 or 2 that many."""
+    _lib.f8_debug_set_lanes(lanes)
 
 
 def f8_debug_last_plan() -> dict:
@@ -395,6 +405,10 @@ class Net:
     @property
     def last_launch_count(self) -> int:
         return int(_lib.f8_net_last_launch_count(self._h))
+
+    @property
+    def lanes(self) -> int:
+        return int(_lib.f8_net_lanes(self._h))
 
     def micro_batching(self):
         """(number of runs of layers the last forward pass executed depth-first over micro-batches, smallest micro-batch)."""

@@ -21,7 +21,8 @@ long long g_tc_launches = 0;
 unsigned g_plan_off = 0;                      // F8_PLAN_OFF_* bits (test hook)
 unsigned long long g_wait_limit_cycles = 0;   // 0: the kernels' default
 int g_last_plan[10] = {0};
-int g_micro_batch = 0;                        // test hook: > 0 forces this micro-batch in every eligible run of layers
+int g_micro_batch = 0;                        // 0: no micro-batching; > 0: this micro-batch in every eligible run; -1: the L2 rule
+int g_lanes = 0;                              // 0: automatic; 1 / 2: that many concurrent lanes in f8_net_forward
 
 f8_status fail(f8_status s, const char *fmt, ...) {
     va_list ap;
@@ -223,7 +224,9 @@ void f8_debug_force_direct(int on) { g_force_direct = on != 0; }
 
 void f8_debug_plan_options(unsigned off_mask) { g_plan_off = off_mask; }
 
-void f8_debug_set_micro_batch(int images) { g_micro_batch = images > 0 ? images : 0; }
+void f8_debug_set_micro_batch(int images) { g_micro_batch = images > 0 ? images : (images < 0 ? -1 : 0); }
+
+void f8_debug_set_lanes(int lanes) { g_lanes = lanes == 1 || lanes == 2 ? lanes : 0; }
 
 int f8_debug_last_plan(int *info, int n) {
     if (!info || n <= 0) return 0;
@@ -401,7 +404,8 @@ struct Step {
     bool fused_pool = false;  // kind -2: the stem kernel also computes the max pool that follows (layer + 1)
     bool has_sib = false;     // the launch also writes the output of the sibling layer behind it (layer + 1)
     F8Sibling sib;
-    int img0 = 0;             // first image of the batch this step works on (micro-batched runs)
+    int img0 = 0;             // first image of the batch this step works on (lanes, micro-batched runs)
+    int lane = 0;             // 0: the caller's stream; 1: the network's second stream
     PlanPtr plan;
     F8ConvGeom g;
 };
@@ -414,7 +418,12 @@ struct f8_net {
     bool overlap_layers = true;                  // programmatic dependent launch between layers
     bool sync_layers = false;                    // synchronize after every launch (fault attribution)
     unsigned plan_options = 0;                   // F8_PLAN_OFF_* mask the cached plan was made under
-    int plan_micro = 0;                          // forced micro-batch the cached plan was made under
+    int plan_micro = 0, plan_lanes = 0;          // micro-batch / lane settings the cached plan was made under
+    bool plan_profiling = false;
+    int last_lanes = 1;
+    // second lane: its own stream, joined to the caller's stream by events
+    cudaStream_t lane_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     int last_regions = 0, last_micro = 0;        // micro-batched runs of the cached plan and the smallest micro-batch
     std::vector<int> t_cp;                       // per tensor: channels as stored (intermediate 8-bit tensors are padded
                                                  // to a multiple of 16 so that every dense layer can use the TMA path)
@@ -470,7 +479,7 @@ size_t layer_image_bytes(const f8_net *net, int i) {
 
 std::vector<Region> plan_regions(const f8_net *net, int batch) {
     std::vector<Region> out;
-    if (g_plan_off & F8_PLAN_OFF_MICRO_BATCH) return out;
+    if (g_micro_batch == 0) return out;
     const int nl = (int)net->layers.size();
     int dev = 0, l2 = 64 << 20, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) {
@@ -517,6 +526,23 @@ std::vector<Region> plan_regions(const f8_net *net, int batch) {
         i = j + 1;
     }
     return out;
+}
+
+// Lanes: the batch is cut into two halves that run as two independent forward passes on two streams, launched
+// alternately layer by layer.  Every launch starts and ends with a few microseconds in which most SMs idle (the
+// last tiles of a layer drain, the first tiles of the next one wait for memory); the idea is that with a second,
+// independent launch queue the SMs one lane leaves idle take blocks of the other lane.  Images are independent, so
+// no result changes.
+int lanes_for(const f8_net *net, int batch) {
+    if (g_plan_off & F8_PLAN_OFF_LANES) return 1;
+    if (g_lanes == 1 || batch < 2 || net->profiling) return 1;
+    // measured slower than one lane on every configuration tried (the waiting blocks of a lane's next launch hold the
+    // SMs its sibling could use): two lanes only on request
+    return g_lanes == 2 ? 2 : 1;
+}
+int lane_images(int batch, int lanes, int lane) {
+    const int first = (batch + lanes - 1) / lanes;
+    return lane == 0 ? first : batch - first;
 }
 
 // Which run a layer belongs to (-1: none), and which tensors live entirely inside one run.
@@ -858,6 +884,14 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
         return cleanup(fail(F8_ERR_CUDA, "could not create the status mirror"));
     }
     memset(net->host_status, 0, 64);
+    if (cudaStreamCreateWithFlags(&net->lane_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&net->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&net->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        (void)cudaGetLastError();
+        f8_net *raw = net.release();
+        f8_net_destroy(raw);
+        return fail(F8_ERR_CUDA, "could not create the second lane's stream");
+    }
     *out = net.release();
     return F8_OK;
 }
@@ -866,10 +900,22 @@ size_t f8_net_workspace_bytes(const f8_net *net, int batch) {
     if (!net || batch <= 0) return 0;
     std::vector<size_t> off;
     size_t pack_off;
-    return assign_offsets(net, batch, &off, &pack_off, plan_regions(net, batch)) + 256;
+    // enough for one lane and for two (a profiled pass runs as one lane whatever the rule says)
+    size_t most = 0;
+    for (int lanes = 1; lanes <= (batch >= 2 ? 2 : 1); ++lanes) {
+        size_t total = 256;
+        for (int lane = 0; lane < lanes; ++lane) {
+            const int n = lane_images(batch, lanes, lane);
+            total += round256(assign_offsets(net, n, &off, &pack_off, plan_regions(net, n)));
+        }
+        most = std::max(most, total);
+    }
+    return most;
 }
 
 int f8_net_last_launch_count(const f8_net *net) { return net ? net->last_launches : 0; }
+
+int f8_net_lanes(const f8_net *net) { return net ? net->last_lanes : 0; }
 
 int f8_net_micro_batching(const f8_net *net, int *images) {
     if (images) *images = net ? net->last_micro : 0;
@@ -907,6 +953,9 @@ void f8_net_destroy(f8_net *net) {
     if (!net) return;
     for (cudaEvent_t ev : net->events) cudaEventDestroy(ev);
     if (net->status_ev) cudaEventDestroy(net->status_ev);
+    if (net->ev_fork) cudaEventDestroy(net->ev_fork);
+    if (net->ev_join) cudaEventDestroy(net->ev_join);
+    if (net->lane_stream) cudaStreamDestroy(net->lane_stream);
     if (net->host_status) cudaFreeHost(net->host_status);
     free_layers(net);
     delete net;
@@ -947,42 +996,70 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
             if (net->layers[i].w_core && layer_dump[i]) dump_fusable = true;
     const bool replan = net->plan_batch != batch || net->plan_x != x || net->plan_y != y || net->plan_ws != workspace ||
                         net->plan_force_direct != g_force_direct || net->plan_dump_first != dump_fusable ||
-                        net->plan_options != g_plan_off || net->plan_micro != g_micro_batch;
+                        net->plan_options != g_plan_off || net->plan_micro != g_micro_batch || net->plan_lanes != g_lanes ||
+                        net->plan_profiling != net->profiling;
     net->overlap_layers = !(g_plan_off & F8_PLAN_OFF_LAYER_OVERLAP);
     net->sync_layers = (g_plan_off & F8_PLAN_SYNC_LAYERS) != 0;
     if (replan) {
         net->steps.clear();
         net->plan_batch = -1;
-        const std::vector<Region> regions = plan_regions(net, batch);
-        assign_offsets(net, batch, &net->t_off, &net->pack_off, regions);
-        std::vector<int> layer_region, tensor_region;
-        classify_tensors(net, regions, &layer_region, &tensor_region);
-        net->last_regions = (int)regions.size();
+        const int lanes = lanes_for(net, batch);
+        net->last_lanes = lanes;
+        net->last_regions = 0;
         net->last_micro = 0;
-        for (const Region &r : regions) net->last_micro = net->last_micro ? std::min(net->last_micro, r.mb) : r.mb;
+        // every lane is a forward pass of its own over its share of the images, with its own part of the workspace
+        struct Lane {
+            int img0 = 0, n = 0;
+            uint8_t *ws = nullptr;
+            std::vector<size_t> t_off;
+            size_t pack_off = 0;
+            std::vector<Region> regions;
+            std::vector<int> layer_region, tensor_region;
+            std::vector<Step> steps;
+            int skip_layer = -1;      // a pooling layer the stem kernel has taken over
+        };
+        std::vector<Lane> lane_list(lanes);
+        {
+            uint8_t *base = (uint8_t *)workspace;
+            int img = 0;
+            for (int k = 0; k < lanes; ++k) {
+                Lane &ln = lane_list[k];
+                ln.img0 = img;
+                ln.n = lane_images(batch, lanes, k);
+                img += ln.n;
+                ln.regions = plan_regions(net, ln.n);
+                ln.ws = base;
+                base += round256(assign_offsets(net, ln.n, &ln.t_off, &ln.pack_off, ln.regions));
+                classify_tensors(net, ln.regions, &ln.layer_region, &ln.tensor_region);
+                net->last_regions = std::max(net->last_regions, (int)ln.regions.size());
+                for (const Region &r : ln.regions) net->last_micro = net->last_micro ? std::min(net->last_micro, r.mb) : r.mb;
+            }
+        }
+        const size_t x_image_bytes = (size_t)net->t_h[0] * net->t_w[0] * net->t_c[0];
+        const size_t y_image_bytes = (size_t)net->t_h[nl] * net->t_w[nl] * net->t_c[nl] * net->t_elem[nl];
 
         // Plans layer i for images [img0, img0 + n) of the batch.  Inside a micro-batched run (in_run) tensors that live
         // entirely in the run hold one micro-batch and always start at their base address; all other tensors are
         // addressed at the slice of these images.
-        int skip_layer = -1;          // a pooling layer the stem kernel has taken over
-        auto plan_layer = [&](int i, int n, int img0, bool in_run) {
+        // img0: first image relative to the lane's share
+        auto plan_layer = [&](Lane &ln, int lane_index, int i, int n, int img0, bool in_run) {
             NetLayer &L = net->layers[i];
+            int &skip_layer = ln.skip_layer;
+            const std::vector<int> &layer_region = ln.layer_region, &tensor_region = ln.tensor_region;
             if (i == skip_layer || L.d.kind == F8_LAYER_SIBLING) return;      // a sibling is written by its parent's launch
             auto tensor_ptr = [&](int t) -> void * {
-                uint8_t *base = t == 0 ? (uint8_t *)const_cast<void *>(x)
-                                       : (t == nl ? (uint8_t *)y : (uint8_t *)workspace + net->t_off[t]);
-                if (in_run && tensor_region[t] < 0) {
-                    const size_t per_image = t == 0 ? (size_t)net->t_h[0] * net->t_w[0] * net->t_c[0]
-                                                    : (t == nl ? (size_t)net->t_h[nl] * net->t_w[nl] * net->t_c[nl] * net->t_elem[nl]
-                                                               : tensor_image_bytes(net, t));
-                    base += (size_t)img0 * per_image;
-                }
+                // the caller's tensors are addressed by the image's place in the whole batch
+                if (t == 0) return (uint8_t *)const_cast<void *>(x) + (size_t)(ln.img0 + img0) * x_image_bytes;
+                if (t == nl) return (uint8_t *)y + (size_t)(ln.img0 + img0) * y_image_bytes;
+                uint8_t *base = ln.ws + ln.t_off[t];
+                if (in_run && tensor_region[t] < 0) base += (size_t)img0 * tensor_image_bytes(net, t);
                 return base;
             };
             Step stp;
             stp.kind = L.d.kind;
             stp.layer = i;
-            stp.img0 = img0;
+            stp.lane = lane_index;
+            stp.img0 = ln.img0 + img0;
             stp.x = tensor_ptr(L.d.src);
             stp.res = (L.q.has_res) ? tensor_ptr(L.d.res) : nullptr;
             stp.y = tensor_ptr(i + 1);
@@ -1019,7 +1096,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                     pg.c = L.pack_kw8; pg.kw = 1; pg.stride_w = 1; pg.pad_w = 0;
                     pg.kh = L.pack_kh; pg.stride_h = 1; pg.pad_h = L.pack_top; pg.pad_h_end = L.pack_bottom;
                     pg.h = L.pack_hp;
-                    void *pbuf = (uint8_t *)workspace + net->pack_off;
+                    void *pbuf = ln.ws + ln.pack_off;
                     const uint64_t cb = 2 * (uint64_t)L.pack_cpad;
                     const size_t pbytes = (size_t)n * L.pack_hp * L.pack_wp * cb;
                     if (f8_tc_supported(pg, pbytes)) {
@@ -1035,11 +1112,12 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                             Step pre;
                             pre.kind = -1;
                             pre.layer = i;
-                            pre.img0 = img0;
+                            pre.img0 = ln.img0 + img0;
+                            pre.lane = lane_index;
                             pre.x = stp.x;
                             pre.y = pbuf;
                             pre.g = stp.g;
-                            net->steps.push_back(std::move(pre));
+                            ln.steps.push_back(std::move(pre));
                             stp.use_tc = true;
                             f8_tc_plan_set_tag(plan.get(), i + 1);
                             stp.plan = std::move(plan);
@@ -1055,23 +1133,34 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                     }
                 }
             }
-            net->steps.push_back(std::move(stp));
+            ln.steps.push_back(std::move(stp));
         };
-        for (int i = 0; i < nl;) {
-            const int r = layer_region[i];
-            if (r < 0) {
-                plan_layer(i, batch, 0, false);
-                ++i;
-                continue;
+        for (int k = 0; k < lanes; ++k) {
+            Lane &ln = lane_list[k];
+            for (int i = 0; i < nl;) {
+                const int r = ln.layer_region[i];
+                if (r < 0) {
+                    plan_layer(ln, k, i, ln.n, 0, false);
+                    ++i;
+                    continue;
+                }
+                // depth first: the whole run on one micro-batch, then on the next
+                for (int img0 = 0; img0 < ln.n; img0 += ln.regions[r].mb) {
+                    ln.skip_layer = -1;
+                    for (int l = ln.regions[r].first; l <= ln.regions[r].last; ++l)
+                        plan_layer(ln, k, l, std::min(ln.regions[r].mb, ln.n - img0), img0, true);
+                }
+                i = ln.regions[r].last + 1;
+                ln.skip_layer = -1;
             }
-            // depth first: the whole run on one micro-batch, then on the next
-            for (int img0 = 0; img0 < batch; img0 += regions[r].mb) {
-                skip_layer = -1;
-                for (int l = regions[r].first; l <= regions[r].last; ++l)
-                    plan_layer(l, std::min(regions[r].mb, batch - img0), img0, true);
-            }
-            i = regions[r].last + 1;
-            skip_layer = -1;
+        }
+        // launch order: the lanes take turns, one launch each
+        {
+            size_t longest = 0;
+            for (const Lane &ln : lane_list) longest = std::max(longest, ln.steps.size());
+            for (size_t j = 0; j < longest; ++j)
+                for (Lane &ln : lane_list)
+                    if (j < ln.steps.size()) net->steps.push_back(std::move(ln.steps[j]));
         }
         net->plan_batch = batch;
         net->plan_x = x;
@@ -1081,6 +1170,8 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         net->plan_dump_first = dump_fusable;
         net->plan_options = g_plan_off;
         net->plan_micro = g_micro_batch;
+        net->plan_lanes = g_lanes;
+        net->plan_profiling = net->profiling;
     }
 
     int launches = 0;
@@ -1094,9 +1185,18 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         net->event_layer.clear();
         cudaEventRecord(net->events[0], st);
     }
+    const cudaStream_t caller_stream = st;
+    const bool two_lanes = net->last_lanes == 2;
+    if (two_lanes) {
+        // the second lane starts when the caller's stream has reached this point ...
+        cudaError_t e = cudaEventRecord(net->ev_fork, caller_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(net->lane_stream, net->ev_fork, 0);
+        if (e != cudaSuccess) return cuda_fail(e, "second lane fork");
+    }
     for (Step &stp : net->steps) {
         NetLayer &L = net->layers[stp.layer];
         cudaError_t e = cudaSuccess;
+        st = stp.lane == 1 ? net->lane_stream : caller_stream;
         switch (stp.kind) {
             case -2:
                 e = f8_launch_stem_tc(stp.g, L.q, L.pack_kh, L.pack_top, L.pack_left, L.pack_kw8 / 32, stp.fused_pool ? 1 : 0, stp.x,
@@ -1155,6 +1255,13 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
             if (e == cudaSuccess && stp.has_sib) e = dump_layer(stp.layer + 1, stp.sib.y2);
             if (e != cudaSuccess) return cuda_fail(e, "layer dump copy");
         }
+    }
+    st = caller_stream;
+    if (two_lanes) {
+        // ... and the caller's stream continues when the second lane has finished
+        cudaError_t e = cudaEventRecord(net->ev_join, net->lane_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(caller_stream, net->ev_join, 0);
+        if (e != cudaSuccess) return cuda_fail(e, "second lane join");
     }
     net->last_launches = launches;
     if (int *word = f8_status_word()) {

@@ -128,6 +128,7 @@ struct TcParams {
     F8Sibling sib;            // second consumer of the same sums (generic epilogue only)
     int vec_bytes2;           // widest aligned store of the second output's rows
     int mul_acc, mul_res;     // 2^q.sh_acc, 2^q.sh_res (kept opaque to the compiler, see the epilogue)
+    int shr_mul;              // 2^(32 - q.s): the rounding shift as the high word of a product (staged epilogues, s >= 2)
     int *status;
     // Windowed 3x3 (stride 1, pad 1, resident weights).  A tile is win_r whole output rows of one image; its M index runs
     // over the rows of the zero-padded image (win_wp = W + 2 positions per row, the last two of each row are discarded).
@@ -619,6 +620,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const int ch_begin = min(group * per_group, chunks);
         const int nch = min(ch_begin + per_group, chunks) - ch_begin;
         const int mul_acc = p.mul_acc, mul_res = p.mul_res;     // 2^sh_acc, 2^sh_res
+        const int shr_mul = p.shr_mul;                          // 2^(32 - s)
         int local = 0;
         int ob = 0;                 // buffer of the output ring for the current tile and the parity of its use
         uint32_t ophase = 0;
@@ -663,14 +665,14 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         if (RES) rw = lds128(res_buf + so[i]);
                         tmem_ld_wait();
                         if (i + 1 < my_nch) tmem_ld16(t_addr + (i + 1) * 16, vb);
-                        sts128(out_buf + so[i], epilogue_fast16<RES, SGN>(va, bias_s + 64 * (i), rw, mul_acc, mul_res, rsel, p.q.s));
+                        sts128(out_buf + so[i], epilogue_fast16<RES, SGN>(va, bias_s + 64 * (i), rw, mul_acc, mul_res, rsel, shr_mul));
                     }
                     if (i + 1 < my_nch) {
                         uint4 rw = make_uint4(0, 0, 0, 0);
                         if (RES) rw = lds128(res_buf + so[i + 1]);
                         tmem_ld_wait();
                         if (i + 2 < my_nch) tmem_ld16(t_addr + (i + 2) * 16, va);
-                        sts128(out_buf + so[i + 1], epilogue_fast16<RES, SGN>(vb, bias_s + 64 * (i + 1), rw, mul_acc, mul_res, rsel, p.q.s));
+                        sts128(out_buf + so[i + 1], epilogue_fast16<RES, SGN>(vb, bias_s + 64 * (i + 1), rw, mul_acc, mul_res, rsel, shr_mul));
                     }
                 }
                 // accumulator and residual have been read, the output part is written: make the writes
@@ -883,7 +885,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.c_chunks = (g.c + p.kb - 1) / p.kb;
     p.epi = EPI_GENERIC;
     const bool has_sib = sib && sib->y2;
-    if ((q.y_kind == F8_U8 || q.y_kind == F8_S8) && q.s >= 1 && q.s <= 24 && g.c_out % 16 == 0 && !has_sib && !q.r_s32)
+    if ((q.y_kind == F8_U8 || q.y_kind == F8_S8) && q.s >= 2 && q.s <= 24 && g.c_out % 16 == 0 && !has_sib && !q.r_s32)
         p.epi = q.y_kind == F8_U8 ? (q.has_res ? EPI_U8_RES : EPI_U8) : (q.has_res ? EPI_S8_RES : EPI_S8);
     const bool staged = p.epi != EPI_GENERIC;
     p.bn = staged ? choose_bn_staged(g.c_out, q.has_res != 0, p.kb) : choose_bn(g.c_out);
@@ -1020,6 +1022,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.q = q;
     p.mul_acc = 1 << q.sh_acc;
     p.mul_res = 1 << q.sh_res;
+    p.shr_mul = (q.s >= 2 && q.s <= 30) ? (1 << (32 - q.s)) : 0;
     p.status = status_word;
     const int ysz = (q.y_kind == F8_S32 || q.y_kind == F8_S32_RELU) ? 4 : 1;
     const size_t row_bytes = (size_t)g.c_out * ysz;

@@ -254,7 +254,8 @@ __host__ __device__ inline uint64_t smem_desc_hi(int kb) {
 // Branch-free epilogue for the common case (8-bit output, 1 <= s <= 24, c_out % 16 == 0).
 //   v = acc * 2^sh_acc + bias'          bias' = (bias << sh_acc) + 2^(s-1), staged in shared memory
 //   v += r << sh_res                    (RES only)
-//   t = v >> s                          = floor((acc' + 2^(s-1)) / 2^s), round half up
+//   t = v >> s                          = floor((acc' + 2^(s-1)) / 2^s), round half up; computed as the high word of
+//                                       v * 2^(32-s) (2 <= s), which is the same floor and runs on the multiplier pipe
 //   y = clamp(t, lo, hi)                saturating pack; the signed quantizer additionally excludes -128
 // cvt.pack.sat packs two saturated values into the low half of d and moves the low half of c above
 // them: d = (c << 16) | (sat(a) << 8) | sat(b).
@@ -274,7 +275,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
 
 template <bool RES, bool SIGNED_OUT>
 __device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], uint32_t bias_addr, uint4 rw, int mul_acc,
-                                                 int mul_res, const uint32_t (&rsel)[4], int s) {
+                                                 int mul_res, const uint32_t (&rsel)[4], int shr_mul /* 2^(32-s), opaque */) {
     int t[16];
     const uint32_t rwords[4] = {rw.x, rw.y, rw.z, rw.w};
 #pragma unroll
@@ -290,7 +291,7 @@ __device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], uint32_t 
                 asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(rwords[g]), "r"(rsel[k]));
                 v += r * mul_res;
             }
-            v >>= s;
+            v = __mulhi(v, shr_mul);
             t[j] = SIGNED_OUT ? max(v, -127) : v;
         }
     }

@@ -13,7 +13,7 @@ def _layer_shape(l, batch):
     return (batch, l.c_out) if l.kind in (synth.LINEAR, synth.GAP) else (batch, l.ho, l.wo, l.c_out)
 
 
-def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0, micro_batch=0):
+def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0, micro_batch=0, lanes=0):
     """Every layer's output against the oracle.  The dump buffers, the network output and the workspace sit between
     poisoned guard bands that must come back untouched."""
     a = api()
@@ -23,6 +23,7 @@ def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0
     a.f8_debug_force_direct(force_direct)
     a.f8_debug_plan_options(plan_off)
     a.f8_debug_set_micro_batch(micro_batch)
+    a.f8_debug_set_lanes(lanes)
     before = a.f8_tc_launch_count()
     try:
         net = a.Net(layers, batch)
@@ -37,6 +38,9 @@ def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0
         a.f8_debug_force_direct(False)
         a.f8_debug_plan_options(0)
         a.f8_debug_set_micro_batch(0)
+        a.f8_debug_set_lanes(0)
+    if lanes:
+        assert net.lanes == lanes
     if micro_batch:
         runs, images = net.micro_batching()
         assert runs >= 1 and images == micro_batch, "the forward pass was not micro-batched"
@@ -52,7 +56,7 @@ def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0
     tc = a.f8_tc_launch_count() - before
     if force_direct:
         assert tc == 0
-    elif image == 224 and not micro_batch:
+    elif image == 224 and not micro_batch and lanes != 2:
         # every dense layer whose input is at least 128 KiB and has c % 16 == 0 (or is a packed stem)
         assert tc >= sum(1 for l in layers if l.kind == synth.CONV and l.c % 16 == 0 and batch * l.h * l.w * l.c >= 131072)
     net.close()
@@ -78,7 +82,7 @@ def test_net_parity_batch_64_every_layer(ref, name):
 
 def _off_masks():
     from paper_2202_05239_b200 import api as a
-    return [a.PLAN_OFF_STEM_KERNEL, a.PLAN_OFF_STEM_POOL_FUSION, a.PLAN_OFF_LAYER_OVERLAP, a.PLAN_OFF_MICRO_BATCH,
+    return [a.PLAN_OFF_STEM_KERNEL, a.PLAN_OFF_STEM_POOL_FUSION, a.PLAN_OFF_LAYER_OVERLAP, a.PLAN_OFF_LANES,
             a.PLAN_OFF_DUAL_ISSUE | a.PLAN_OFF_ALT_PRODUCERS, a.PLAN_OFF_RESIDENT_WEIGHTS, a.PLAN_OFF_PAIRS,
             a.PLAN_SYNC_LAYERS]
 
@@ -98,6 +102,14 @@ def test_net_parity_micro_batched(ref, name, batch, micro, direct):
     _compare_net(ref, name, batch, 224 if not direct else 64, force_direct=direct, micro_batch=micro)
 
 
+@pytest.mark.parametrize("name,batch,micro", [("resnet50", 5, 0), ("resnet18", 2, 0), ("mobilenetv2", 7, 0), ("mobilenetv1", 4, 0),
+                                              ("resnet18_siblings", 3, 0), ("resnet50", 9, 2)])
+def test_net_parity_two_lanes(ref, name, batch, micro):
+    """The batch cut into two halves (the first one larger when the batch is odd) that run as two passes on two
+    streams, launched alternately -- optionally with micro-batched runs inside each lane: every layer unchanged."""
+    _compare_net(ref, name, batch, 224, lanes=2, micro_batch=micro)
+
+
 def test_mobilenet_parity_with_the_strip_kernel(ref):
     a = api()
     _compare_net(ref, "mobilenetv1", 3, 224, plan_off=a.PLAN_OFF_DW_WALK)
@@ -114,7 +126,6 @@ def _sampled_full_batch(ref, name, batch, samples):
     out = net.forward(a.to_device(x), dump=dump)
     torch.cuda.synchronize()
     a.f8_device_status()
-    print(f"{name} batch {batch}: micro-batched runs, smallest micro-batch = {net.micro_batching()}")
     for i in samples:
         want = ref.net_forward(layers, x[i:i + 1])
         for li, l in enumerate(layers):
