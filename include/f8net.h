@@ -347,7 +347,7 @@ int f8_net_lanes(const f8_net *net);
  * [9] staged output buffers.  Lets a test assert which path a case took and how many tiles each CTA walked. */
 enum {
     F8_PLAN_RESIDENT_WEIGHTS = 1, F8_PLAN_WINDOWED = 2, F8_PLAN_DUAL_ISSUE = 4, F8_PLAN_ALT_PRODUCERS = 8,
-    F8_PLAN_PLAIN_MATRIX = 16, F8_PLAN_STAGED_EPILOGUE = 32, F8_PLAN_PAIRS = 64
+    F8_PLAN_PLAIN_MATRIX = 16, F8_PLAN_STAGED_EPILOGUE = 32, F8_PLAN_PAIRS = 64, F8_PLAN_ROW_TILES = 128
 };
 int f8_debug_last_plan(int *info, int n);
 

@@ -60,8 +60,10 @@ constexpr int MAX_STAGES = 16;
 constexpr int MAX_OUT_BUFS = 4;             // ring of staged output tiles; with a residual, the residual tile lands in the
                                             // buffer first and the epilogue converts it in place
 constexpr int TMEM_COLS = 512;
-constexpr size_t SMEM_LIMIT = 220 * 1024;     // shared memory budget of stages, staging and resident weights
-constexpr uint32_t CONTROL_BYTES = 1024;      // control block in front of them (plus up to 1023 bytes of alignment slack)
+// Shared memory budget of stages, staging and resident weights: the 227 KiB a block may have, minus the control block
+// in front of them and up to 1023 bytes of alignment slack (the kernel has no static shared memory).
+constexpr size_t SMEM_LIMIT = 225 * 1024;
+constexpr uint32_t CONTROL_BYTES = 1024;
 
 struct TcControl {
     uint64_t bars[2 * MAX_STAGES + 5];        // full[], empty[], tfull[2], tempty[2], bres
@@ -136,6 +138,11 @@ struct TcParams {
     // filter tap (r, s) is then the same shared-memory tile read from (r * win_wp + s) pixel rows further down, so the
     // activations cross the L2 -> SM path once instead of nine times.
     int win;
+    // Row-tiled geometry (rows = 1): a tile is win_r whole output rows of one image (win_wp positions per row, win_bands
+    // tiles per image), stored / fetched with 4-D tensor maps.  The windowed mode uses it with win_wp = W + 2; small
+    // tensors (for which no im2col map is made) use it with win_wp = W_out and one tiled load per filter tap, whose box
+    // starts at the tap's offset and whose out-of-image elements are zero filled (rowt = 1).
+    int rows, rowt;
     int win_r, win_wp, win_bands;
     FastDiv div_bands;
     uint32_t tx_win;          // bytes of one window load
@@ -373,12 +380,20 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
             const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
             const int m0 = m_t * TILE_M;
-            const int t1 = fast_div(m0, p.div_wo);
-            const int ow = m0 - t1 * p.wo;
-            const int img = fast_div(t1, p.div_ho);
-            const int oh = t1 - img * p.ho;
-            const int base_w = ow * p.stride_w - p.pad_w;
-            const int base_h = oh * p.stride_h - p.pad_h;
+            int img, base_w, base_h;
+            if (p.rowt) {
+                // whole output rows y0 .. y0 + win_r - 1 of one image; tap (r, s) starts at input (s - pad, y0 * stride + r - pad)
+                img = fast_div(m_t, p.div_bands);
+                base_w = -p.pad_w;
+                base_h = (m_t - img * p.win_bands) * p.win_r * p.stride_h - p.pad_h;
+            } else {
+                const int t1 = fast_div(m0, p.div_wo);
+                const int ow = m0 - t1 * p.wo;
+                img = fast_div(t1, p.div_ho);
+                const int oh = t1 - img * p.ho;
+                base_w = ow * p.stride_w - p.pad_w;
+                base_h = oh * p.stride_h - p.pad_h;
+            }
             const int n_base = n_t * p.bn;
             for (int kc = 0; kc < k_iters; kc += p.group, ++use_idx) {
                 if (p.alt && (use_idx & 1) != half) {
@@ -411,6 +426,8 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     const uint32_t dst = smem_base + stage * p.stage_bytes + j * p.sub_bytes;
                     if ((opnd == 0 || a_helper) && p.a_plain)
                         tma_load_2d(dst, &map_a, fb, (int)e.x, m0);
+                    else if ((opnd == 0 || a_helper) && p.rowt)
+                        tma_load_4d(dst, &map_a, fb, (int)e.x, base_w + (int)(e.y & 0xff), base_h + (int)((e.y >> 8) & 0xff), img);
                     else if (opnd == 0 || a_helper)
                         tma_load_im2col(dst, &map_a, fb, (int)e.x, base_w, base_h, img, (uint16_t)(e.y & 0xff),
                                         (uint16_t)((e.y >> 8) & 0xff));
@@ -553,7 +570,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
                 if (!mbar_wait(out_full + 8 * b, bphase, wc, tagbits | 108)) break;
                 const uint32_t src = smem_base + p.out_off + b * p.out_bytes;
-                if (p.win) {
+                if (p.rows) {
                     const int img = fast_div(m_t, p.div_bands);
                     const int y0 = (m_t - img * p.win_bands) * p.win_r;
                     // positions W and W + 1 of every row and rows below the image are clipped by the hardware
@@ -587,7 +604,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 if (!mbar_wait(out_free + 8 * rb, rphase ^ 1, wc, tagbits | 106)) { ok = false; break; }
                 const uint32_t fb = res_full + 8 * rb;
                 mbar_expect_tx(fb, p.tx_res);
-                if (p.win) {
+                if (p.rows) {
                     const int img = fast_div(m_t, p.div_bands);
                     const int y0 = (m_t - img * p.win_bands) * p.win_r;
                     for (int sl = 0; sl < p.n_slabs; ++sl)
@@ -694,8 +711,16 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const uint32_t acc_phase = (local >> 1) & 1;
                 const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
                 const int n0 = n_t * p.bn;
-                const size_t row = (size_t)m_t * TILE_M + tile_row;
-                const bool row_valid = row < (size_t)p.M;
+                size_t row = (size_t)m_t * TILE_M + tile_row;
+                bool row_valid = row < (size_t)p.M;
+                if (p.rows) {
+                    // row-tiled geometry: tile row -> (row of the band, position in the row) -> output pixel
+                    const int img = fast_div(m_t, p.div_bands);
+                    const int y0 = (m_t - img * p.win_bands) * p.win_r;
+                    const int ry = tile_row / p.win_wp, rx = tile_row - ry * p.win_wp;
+                    row_valid = ry < p.win_r && y0 + ry < p.ho && rx < p.wo;
+                    row = ((size_t)img * p.ho + (size_t)(y0 + ry)) * p.wo + rx;
+                }
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
                 if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar + 8 * acc, acc_phase, wc, tagbits | 104))) { ok = false; break; }
                 tc_fence_after();
@@ -846,13 +871,22 @@ struct F8TcPlan {
 size_t f8_tc_plan_size() { return sizeof(F8TcPlan); }
 void f8_tc_plan_set_tag(F8TcPlan *plan, int tag) { plan->p.tag = tag; }
 
+// Whole output rows fit a tile and the boxes of a tap stay inside the limits of a tiled tensor map.
+bool f8_tc_rowtile_ok(const F8ConvGeom &g) {
+    if (g.wo > TILE_M || g.pad_h_end >= 0) return false;
+    const int r = std::min(TILE_M / g.wo, g.ho);
+    return g.wo * g.stride_w <= 256 && r * g.stride_h <= 256 && g.stride_w <= 8 && g.stride_h <= 8;
+}
+
 bool f8_tc_supported(const F8ConvGeom &g, size_t x_bytes) {
     if (g.c % 16 != 0) return false;                 // TMA strides are multiples of 16 bytes
     // im2col tensor maps of tensors below 128 KiB are avoided.  A pointwise layer (1x1, stride 1, no padding) needs no
     // im2col: its activations are a plain [pixels, channels] matrix read through a tiled map, whatever their size;
-    // other small problems go to the CUDA-core kernel.
+    // other layers on small tensors take whole output rows per tile and one tiled load per filter tap; what fits
+    // neither goes to the CUDA-core kernel.
     const bool pointwise = g.kh == 1 && g.kw == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 && g.pad_w == 0;
-    if (x_bytes < 128 * 1024 && !(pointwise && x_bytes >= 4096)) return false;
+    if (x_bytes < 4096) return false;
+    if (x_bytes < 128 * 1024 && !pointwise && !f8_tc_rowtile_ok(g)) return false;
     if (g.kh > 255 || g.kw > 255) return false;
     if ((long long)g.n * g.ho * g.wo > 0x7fffff00ll) return false;
     return true;
@@ -948,8 +982,9 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // Windowed mode for 3x3 / stride 1 / pad 1 layers whose weights can stay resident: whole padded rows are loaded once
     // per tile and every filter tap reads them at a shifted row offset.  Worth it when whole rows fill most of a tile
     // and the im2col loads are what bounds the layer: measured, 128-channel layers gain 1.8x (the resident weights
-    // leave room for two im2col stages only), 64-channel layers lose a little (their tiles are bound by per-tile
-    // costs, and whole-row tiles are 12.5 % more tiles).
+    // leave room for two im2col stages only); 64-channel layers gain nothing (62 against 64 us: their tiles are bound
+    // by the rate at which the tensor core accepts N = 64 instructions, about one per 90 cycles whoever issues them,
+    // and whole-row tiles are 12.5 % more tiles).
     p.win = 0;
     if (staged && p.kb == 128 && g.kh == 3 && g.kw == 3 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 1 && g.pad_w == 1 &&
         g.pad_h_end < 0 && p.n_tiles == 1 && g.w + 2 <= TILE_M && g.w == g.wo && g.h == g.ho && g.c % p.kb == 0 &&
@@ -979,6 +1014,29 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
             p.m_tiles = g.n * bands;
             p.sub_bytes = win_stage;
         }
+    }
+    p.rows = p.win;
+    p.rowt = 0;
+    // Small tensors: no im2col map is made for tensors below 128 KiB.  Pointwise layers read them as a plain matrix; other
+    // layers take whole output rows per tile and fetch every filter tap with an ordinary tiled load.
+    const bool dense_x = xv.stride_w == xv.dim_c && xv.stride_h == xv.dim_c * xv.dim_w && xv.stride_n == xv.dim_c * xv.dim_w * xv.dim_h;
+    const bool pointwise = g.kh == 1 && g.kw == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 && g.pad_w == 0;
+    const bool small_x = xv.dim_c * xv.dim_w * xv.dim_h * xv.dim_n < 128 * 1024;
+    if (small_x && !pointwise && !p.win) {
+        if (!dense_x || !f8_tc_rowtile_ok(g)) {
+            *why = "small tensor whose rows do not fit a tile";
+            return cudaErrorInvalidValue;
+        }
+        const int r = std::min(TILE_M / g.wo, g.ho);
+        p.rows = p.rowt = 1;
+        p.win_r = r;
+        p.win_wp = g.wo;
+        p.win_bands = (g.ho + r - 1) / r;
+        p.div_bands = make_fast_div(p.win_bands);
+        p.m_tiles = g.n * p.win_bands;
+        p.tx_a = (uint32_t)p.kb * g.wo * r;            // bytes one tap's box delivers (zero fill included)
+        p.tx_sub = p.tx_a + (p.b_res ? 0u : p.tx_b);
+        p.tx_res = (uint32_t)p.bn * g.wo * r;
     }
     if (p.win) {
         p.group = 1;
@@ -1033,7 +1091,6 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         p.vec_bytes2 = (rb2 % 16 == 0) ? 16 : (rb2 % 8 == 0 ? 8 : (rb2 % 4 == 0 ? 4 : 1));
     }
 
-    const bool dense_x = xv.stride_w == xv.dim_c && xv.stride_h == xv.dim_c * xv.dim_w && xv.stride_n == xv.dim_c * xv.dim_w * xv.dim_h;
     p.a_plain = (g.kh == 1 && g.kw == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 && g.pad_w == 0 && dense_x &&
                  xv.dim_c * xv.dim_w * xv.dim_h * xv.dim_n < 128 * 1024) ? 1 : 0;
     if (p.a_plain) {
@@ -1047,6 +1104,20 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) {
             *why = "cuTensorMapEncodeTiled rejected the activation matrix";
+            return cudaErrorInvalidValue;
+        }
+    } else if (p.rowt) {
+        // A: plain tiles of win_r output rows: one box per filter tap, traversed with the convolution stride (a box of
+        // n * stride elements delivers n of them), out-of-image elements zero filled
+        cuuint64_t dims[4] = {xv.dim_c, xv.dim_w, xv.dim_h, xv.dim_n};
+        cuuint64_t strides[3] = {xv.stride_w, xv.stride_h, xv.stride_n};
+        cuuint32_t box[4] = {(cuuint32_t)p.kb, (cuuint32_t)(g.wo * g.stride_w), (cuuint32_t)(p.win_r * g.stride_h), 1};
+        cuuint32_t estr[4] = {1, (cuuint32_t)g.stride_w, (cuuint32_t)g.stride_h, 1};
+        CUresult r = g_encode_tiled(&plan->map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(xv.base), dims, strides,
+                                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(p.kb),
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            *why = "cuTensorMapEncodeTiled rejected the activation tensor";
             return cudaErrorInvalidValue;
         }
     } else if (p.win) {
@@ -1097,7 +1168,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // output / residual [M, c_out] bytes, one box = one column slab of a tile
     plan->map_y = plan->map_b;
     plan->map_r = plan->map_b;
-    if (staged && p.win) {
+    if (staged && p.rows) {
         // output / residual as (C_out, W, H, N); one box = one column slab of win_r rows of W + 2 positions
         cuuint64_t dims[4] = {(cuuint64_t)g.c_out, (cuuint64_t)g.wo, (cuuint64_t)g.ho, (cuuint64_t)g.n};
         cuuint64_t strides[3] = {(cuuint64_t)g.c_out, (cuuint64_t)g.c_out * g.wo, (cuuint64_t)g.c_out * g.wo * g.ho};
@@ -1150,7 +1221,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     {
         int *info = f8_last_plan_info();
         info[0] = (p.b_res ? F8_PLAN_RESIDENT_WEIGHTS : 0) | (p.win ? F8_PLAN_WINDOWED : 0) | (p.dual_issue ? F8_PLAN_DUAL_ISSUE : 0) |
-                  (p.alt ? F8_PLAN_ALT_PRODUCERS : 0) | (p.a_plain ? F8_PLAN_PLAIN_MATRIX : 0) | (staged ? F8_PLAN_STAGED_EPILOGUE : 0);
+                  (p.alt ? F8_PLAN_ALT_PRODUCERS : 0) | (p.a_plain ? F8_PLAN_PLAIN_MATRIX : 0) | (staged ? F8_PLAN_STAGED_EPILOGUE : 0) | (p.rowt ? F8_PLAN_ROW_TILES : 0);
         info[1] = p.epi; info[2] = p.bn; info[3] = p.kb; info[4] = p.stages; info[5] = p.group;
         info[6] = p.m_tiles; info[7] = p.n_tiles; info[8] = plan->grid; info[9] = staged ? p.out_bufs : 0;
     }

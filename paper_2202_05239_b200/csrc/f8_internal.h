@@ -75,6 +75,7 @@ struct F8TcTensorView {
 
 // True when this geometry can run on the tensor-core path.
 bool f8_tc_supported(const F8ConvGeom &g, size_t x_bytes);
+bool f8_tc_rowtile_ok(const F8ConvGeom &g);
 size_t f8_tc_plan_size();
 // Encodes tensor maps and tile schedule; returns cudaSuccess or an error (no launch).
 cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant &q, const F8TcTensorView &xv,

@@ -76,6 +76,37 @@ def test_small_pointwise_on_tensor_cores(ref, case):
     check_layer(ref, layer, x, res, expect_tc=True)
 
 
+# layers that are not pointwise on tensors below 128 KiB (single-image inference): whole output rows per tile, one tiled
+# load per filter tap (no im2col map)
+# (h, w, c, c_out, k, stride, pad, n, x_signed, y_dtype, res)
+SMALL_ROW_TILED = [
+    (28, 28, 128, 128, 3, 1, 1, 1, False, synth.U8, False),     # 98 KB: four rows per tile, seven bands
+    (14, 14, 256, 256, 3, 1, 1, 1, False, synth.U8, True),      # nine rows per tile, second band partial; residual
+    (7, 7, 512, 512, 3, 1, 1, 2, True, synth.S8, False),        # 49 of 128 tile rows used; two N tiles, streamed weights
+    (14, 14, 512, 512, 3, 2, 1, 1, False, synth.U8, False),     # stride 2: boxes traversed with the convolution stride
+    (28, 28, 96, 48, 1, 2, 0, 1, True, synth.U8, False),        # 1x1 stride 2 (a down-sampling shortcut), ragged K chunk
+    (15, 17, 32, 40, 3, 1, 1, 3, False, synth.S32, False),      # int32 output through the generic epilogue, odd sizes
+    (20, 20, 64, 32, 5, 1, 2, 2, False, synth.U8, True),        # 5x5
+    (9, 31, 16, 24, 3, 2, 0, 5, True, synth.S8, False),         # no padding, stride 2, c_out = 24
+    (6, 100, 128, 64, 3, 1, 1, 1, False, synth.U8, False),      # one row of 100 positions per tile
+    (6, 100, 64, 64, 3, 1, 1, 2, False, synth.U8, False),       # the same with 64-byte rows: row tiles
+]
+
+
+@pytest.mark.parametrize("case", range(len(SMALL_ROW_TILED)))
+def test_small_layers_row_tiled_on_tensor_cores(ref, case):
+    from paper_2202_05239_b200 import api as a
+    h, w, c, c_out, k, stride, pad, n, xs, y_dtype, with_res = SMALL_ROW_TILED[case]
+    rng = np.random.default_rng(800 + case)
+    layer = random_conv_layer(rng, h=h, w=w, c=c, c_out=c_out, k=k, stride=stride, pad=pad, x_signed=xs, y_dtype=y_dtype,
+                              with_res=with_res)
+    x = random_input(rng, n, layer)
+    assert 4096 <= x.size < 128 * 1024
+    res = random_residual(rng, n, layer) if with_res else None
+    # the first and the last case are also eligible for the windowed mode (which reads through a tiled map as well)
+    check_layer(ref, layer, x, res, expect_tc=True, expect_flags=a.PLAN_WINDOWED if case in (0, 8) else a.PLAN_ROW_TILES)
+
+
 def test_extreme_operands_on_tensor_cores(ref):
     """-128 weights against 255 / -128 activations: the signedness selection of the MMA must be right."""
     rng = np.random.default_rng(5)
