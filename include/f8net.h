@@ -313,7 +313,8 @@ void f8_debug_force_direct(int on);
  *   F8_PLAN_OFF_DUAL_ISSUE        one MMA-issuing thread per CTA
  *   F8_PLAN_OFF_ALT_PRODUCERS     one pair of TMA producer warps
  *   F8_PLAN_OFF_PAIRS             no two-CTA tiles (tcgen05 cta_group::2)
- *   F8_PLAN_OFF_DW_WALK           depthwise 3x3 stride-1 layers take the strip kernel
+ *   F8_PLAN_OFF_DW_DP4A           depthwise 3x3 layers do not use the packed-dot-product kernels
+ *   F8_PLAN_OFF_DW_WALK           depthwise 3x3 stride-1 layers do not use the row-walking kernel (with both off: the strip kernel)
  *   F8_PLAN_OFF_STEM_KERNEL       first layers take the packed-row-pair GEMM instead of the first-layer kernel
  *   F8_PLAN_OFF_STEM_POOL_FUSION  the max pool behind a first layer runs as its own kernel
  *   F8_PLAN_OFF_LAYER_OVERLAP     f8_net_forward launches without programmatic dependent launch
@@ -323,7 +324,7 @@ void f8_debug_force_direct(int on);
 enum {
     F8_PLAN_OFF_RESIDENT_WEIGHTS = 1, F8_PLAN_OFF_WINDOWED = 2, F8_PLAN_OFF_DUAL_ISSUE = 4, F8_PLAN_OFF_ALT_PRODUCERS = 8,
     F8_PLAN_OFF_PAIRS = 16, F8_PLAN_OFF_DW_WALK = 32, F8_PLAN_OFF_STEM_KERNEL = 64, F8_PLAN_OFF_STEM_POOL_FUSION = 128,
-    F8_PLAN_OFF_LAYER_OVERLAP = 256, F8_PLAN_OFF_LANES = 512, F8_PLAN_SYNC_LAYERS = 1024
+    F8_PLAN_OFF_LAYER_OVERLAP = 256, F8_PLAN_OFF_LANES = 512, F8_PLAN_SYNC_LAYERS = 1024, F8_PLAN_OFF_DW_DP4A = 2048
 };
 void f8_debug_plan_options(unsigned off_mask);
 

@@ -413,6 +413,327 @@ __global__ void __launch_bounds__(128) dwconv3x3_walk_kernel(F8ConvGeom g, F8Req
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Depthwise 3x3, pad 1, stride 1 with packed dot products.  Same walk as above (a thread owns 4 consecutive channels
+// and 2 output columns and walks down a band of rows with the three open output rows in registers), but the
+// multiply-accumulates run as dp4a: the four words of an input row that a thread needs (columns ow0 - 1 .. ow0 + 2,
+// four channels each) are transposed in registers into one word per channel holding that channel's four columns
+// (8 PRMT), and a filter row of a channel is kept as one packed word [w0 w1 w2 0], applied to that word for the left
+// output column and to the word shifted down by one column for the right one, so that one dp4a does the three products of
+// a filter row.  Per input row and thread: 4 copies, 8 permutes, 4 shifts and 24 dp4a for 72 multiply-accumulates, against
+// 72 multiply-adds and 16 unpacks before.
+// ---------------------------------------------------------------------------------------
+template <bool XS>
+__device__ __forceinline__ int dw_dot4(uint32_t x, uint32_t w, int acc) {
+    return XS ? dp4a_ss(x, w, acc) : dp4a_us(x, w, acc);
+}
+
+// input row (transposed: t[j] = the four columns of channel j) into the three open output rows; slot (K + 1 - r) mod 3
+// holds output row ih + 1 - r.  The top filter row opens an output row: its product starts the sum.
+template <int K, bool XS>
+__device__ __forceinline__ void dw_dp4a_accumulate(const uint32_t (&t)[4], const uint32_t (&wa)[3][4], const int (&open)[4],
+                                                   int (&acc)[3][2][4]) {
+    // the right output column reads columns 1..3: the same packed filter row against the word shifted down by one column
+    uint32_t tr[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) tr[j] = t[j] >> 8;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        const int slot = (K + 1 - r + 3) % 3;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            // open[j] = bias + rounding constant: the value an output row's sum starts from
+            acc[slot][0][j] = dw_dot4<XS>(t[j], wa[r][j], r == 0 ? open[j] : acc[slot][0][j]);
+            acc[slot][1][j] = dw_dot4<XS>(tr[j], wa[r][j], r == 0 ? open[j] : acc[slot][1][j]);
+        }
+    }
+}
+
+// Input rows reach the thread through a private ring in shared memory filled by asynchronous copies issued DW_AHEAD rows
+// ahead (no registers are tied up by loads in flight, so every thread keeps 4 * DW_AHEAD words on their way: with
+// loads into registers, one row ahead, the kernel was bound by memory latency at a quarter of the HBM bandwidth).
+constexpr int DW_AHEAD = 8;
+
+__device__ __forceinline__ void cp_async4_zfill(uint32_t dst, const void *src, bool valid) {
+    // 4-byte asynchronous copy global -> shared; with a source size of 0 nothing is read and zeros are written
+    const int bytes = valid ? 4 : 0;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <bool XS, bool SIGNED_OUT>
+__global__ void __launch_bounds__(128) dwconv3x3_dp4a_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
+                                                             const int8_t *__restrict__ w,
+                                                             const int32_t *__restrict__ bias, uint8_t *__restrict__ y,
+                                                             int strips, int bands, int band_rows, int total) {
+    grid_dependency_sync();
+    __shared__ uint32_t ring[DW_AHEAD][4][128];          // [row slot][column][thread]: a thread only touches its own words
+    const uint32_t ring_base = (uint32_t)__cvta_generic_to_shared(&ring[0][0][threadIdx.x]);
+    const int c4 = g.c >> 2;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int cg = idx % c4;
+        int tt = idx / c4;
+        const int strip = tt % strips;
+        tt /= strips;
+        const int band = tt % bands;
+        const int in = tt / bands;
+        const int c0 = cg * 4;
+        const int ow0 = strip * 2;
+        const int oh0 = band * band_rows, oh1 = min(g.ho, oh0 + band_rows);
+        // filter rows as packed words: bytes (w0, w1, w2, 0)
+        uint32_t wa[3][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int r = 0; r < 3; ++r) {
+                const uint32_t b0 = (uint8_t)w[(c0 + j) * 9 + 3 * r], b1 = (uint8_t)w[(c0 + j) * 9 + 3 * r + 1],
+                               b2 = (uint8_t)w[(c0 + j) * 9 + 3 * r + 2];
+                wa[r][j] = b0 | (b1 << 8) | (b2 << 16);
+            }
+        int4 b = bias ? *(const int4 *)(bias + c0) : make_int4(0, 0, 0, 0);
+        const int rnd = 1 << (q.s - 1);
+        const int bb[4] = {b.x + rnd, b.y + rnd, b.z + rnd, b.w + rnd};
+        int acc[3][2][4];
+#pragma unroll
+        for (int a = 0; a < 3; ++a)
+#pragma unroll
+            for (int o = 0; o < 2; ++o)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[a][o][j] = bb[j];
+        const int iw0 = ow0 - 1;
+        bool col_ok[4];
+        int col_off[4];                     // byte offset of the column inside a row (0 for columns outside the image)
+#pragma unroll
+        for (int xx = 0; xx < 4; ++xx) {
+            col_ok[xx] = iw0 + xx >= 0 && iw0 + xx < g.w;
+            col_off[xx] = col_ok[xx] ? (iw0 + xx) * g.c : 0;
+        }
+        const int row_stride = g.w * g.c;
+        const uint8_t *img = x + (size_t)in * g.h * row_stride + c0;
+
+        // request input row ih into ring slot `slot` (rows / columns outside the image: zeros)
+        auto request_row = [&](int ih, int slot) {
+            const bool row_ok = ih >= 0 && ih < g.h;
+            const uint8_t *rp = img + (size_t)(row_ok ? ih : 0) * row_stride;
+#pragma unroll
+            for (int xx = 0; xx < 4; ++xx)
+                cp_async4_zfill(ring_base + (uint32_t)((slot * 4 + xx) * 128 * 4), rp + col_off[xx], row_ok && col_ok[xx]);
+            cp_async_commit();
+        };
+        // the four words of the oldest requested row, transposed: words of four channels per column -> words of four
+        // columns per channel
+        auto take_row = [&](int slot, uint32_t (&t)[4]) {
+            cp_async_wait<DW_AHEAD - 1>();
+            uint32_t cw[4];
+#pragma unroll
+            for (int xx = 0; xx < 4; ++xx) cw[xx] = ring[slot][xx][threadIdx.x];
+            const uint32_t lo01 = __byte_perm(cw[0], cw[1], 0x5140), hi01 = __byte_perm(cw[0], cw[1], 0x7362);
+            const uint32_t lo23 = __byte_perm(cw[2], cw[3], 0x5140), hi23 = __byte_perm(cw[2], cw[3], 0x7362);
+            t[0] = __byte_perm(lo01, lo23, 0x5410);
+            t[1] = __byte_perm(lo01, lo23, 0x7632);
+            t[2] = __byte_perm(hi01, hi23, 0x5410);
+            t[3] = __byte_perm(hi01, hi23, 0x7632);
+        };
+        auto emit = [&](int oh, int (&a)[2][4]) {
+            if (oh >= oh0 && oh < oh1) {
+                uint8_t *out = y + ((size_t)(in * g.ho + oh) * g.wo + ow0) * g.c + c0;
+#pragma unroll
+                for (int o = 0; o < 2; ++o) {
+                    if (ow0 + o < g.wo) {
+                        int tv[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int vv = a[o][j] >> q.s;
+                            tv[j] = SIGNED_OUT ? max(vv, -127) : vv;
+                        }
+                        uint32_t hi2, word;
+                        if (SIGNED_OUT) {
+                            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+                            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+                        } else {
+                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+                        }
+                        *(uint32_t *)(out + o * g.c) = word;
+                    }
+                }
+            }
+        };
+
+        // input rows oh0 - 1 .. oh1; DW_AHEAD rows are on their way at any time (requests past the band are zero fills that
+        // nobody reads: they keep the group count regular); three rows per trip so that the accumulator slots are
+        // compile-time
+        const int first = oh0 - 1;
+#pragma unroll
+        for (int d = 0; d < DW_AHEAD; ++d) request_row(first + d, d);
+        int ih = first, slot = 0;
+        uint32_t t[4];
+        while (ih <= oh1) {
+            take_row(slot, t);
+            request_row(ih + DW_AHEAD <= oh1 ? ih + DW_AHEAD : -1, slot);
+            slot = (slot + 1) & (DW_AHEAD - 1);
+            dw_dp4a_accumulate<0, XS>(t, wa, bb, acc);
+            emit(ih - 1, acc[2]);
+            if (++ih > oh1) break;
+            take_row(slot, t);
+            request_row(ih + DW_AHEAD <= oh1 ? ih + DW_AHEAD : -1, slot);
+            slot = (slot + 1) & (DW_AHEAD - 1);
+            dw_dp4a_accumulate<1, XS>(t, wa, bb, acc);
+            emit(ih - 1, acc[0]);
+            if (++ih > oh1) break;
+            take_row(slot, t);
+            request_row(ih + DW_AHEAD <= oh1 ? ih + DW_AHEAD : -1, slot);
+            slot = (slot + 1) & (DW_AHEAD - 1);
+            dw_dp4a_accumulate<2, XS>(t, wa, bb, acc);
+            emit(ih - 1, acc[1]);
+            ++ih;
+        }
+        cp_async_wait<0>();          // nothing of this item is in flight when the ring is reused for the next one
+    }
+}
+
+// The same for stride 2.  A thread owns 4 channels and 2 output columns, i.e. the five input columns 2 ow0 - 1 .. 2 ow0 + 3:
+// columns 0..2 feed the left output, columns 2..4 the right one, so a filter row is one packed word (w0 w1 w2 0) for both
+// and the transposition yields two words per channel (12 PRMT).  Output row oh takes input rows 2 oh - 1, 2 oh and 2 oh + 1;
+// an odd input row closes one output row and opens the next, so a single set of accumulators walks down the band.
+template <bool XS, bool SIGNED_OUT>
+__global__ void __launch_bounds__(128) dwconv3x3s2_dp4a_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
+                                                               const int8_t *__restrict__ w,
+                                                               const int32_t *__restrict__ bias, uint8_t *__restrict__ y,
+                                                               int strips, int bands, int band_rows, int total) {
+    grid_dependency_sync();
+    __shared__ uint32_t ring[DW_AHEAD][5][128];
+    const uint32_t ring_base = (uint32_t)__cvta_generic_to_shared(&ring[0][0][threadIdx.x]);
+    const int c4 = g.c >> 2;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int cg = idx % c4;
+        int tt = idx / c4;
+        const int strip = tt % strips;
+        tt /= strips;
+        const int band = tt % bands;
+        const int in = tt / bands;
+        const int c0 = cg * 4;
+        const int ow0 = strip * 2;
+        const int oh0 = band * band_rows, oh1 = min(g.ho, oh0 + band_rows);
+        uint32_t wr[3][4];                  // filter row r of channel j: bytes (w0, w1, w2, 0)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int r = 0; r < 3; ++r) {
+                const uint32_t b0 = (uint8_t)w[(c0 + j) * 9 + 3 * r], b1 = (uint8_t)w[(c0 + j) * 9 + 3 * r + 1],
+                               b2 = (uint8_t)w[(c0 + j) * 9 + 3 * r + 2];
+                wr[r][j] = b0 | (b1 << 8) | (b2 << 16);
+            }
+        int4 b = bias ? *(const int4 *)(bias + c0) : make_int4(0, 0, 0, 0);
+        const int rnd = 1 << (q.s - 1);
+        const int bb[4] = {b.x + rnd, b.y + rnd, b.z + rnd, b.w + rnd};
+        const int iw0 = 2 * ow0 - 1;
+        bool col_ok[5];
+        int col_off[5];
+#pragma unroll
+        for (int xx = 0; xx < 5; ++xx) {
+            col_ok[xx] = iw0 + xx >= 0 && iw0 + xx < g.w;
+            col_off[xx] = col_ok[xx] ? (iw0 + xx) * g.c : 0;
+        }
+        const int row_stride = g.w * g.c;
+        const uint8_t *img = x + (size_t)in * g.h * row_stride + c0;
+        const int last_row = 2 * (oh1 - 1) + 1;            // last input row of the band
+
+        auto request_row = [&](int ih, int slot) {
+            const bool row_ok = ih >= 0 && ih < g.h && ih <= last_row;
+            const uint8_t *rp = img + (size_t)(row_ok ? ih : 0) * row_stride;
+#pragma unroll
+            for (int xx = 0; xx < 5; ++xx)
+                cp_async4_zfill(ring_base + (uint32_t)((slot * 5 + xx) * 128 * 4), rp + col_off[xx], row_ok && col_ok[xx]);
+            cp_async_commit();
+        };
+        // ta[j]: columns 0..3 of channel j (the left output reads bytes 0..2); tb[j]: columns 2, 3, 4 (the right output)
+        auto take_row = [&](int slot, uint32_t (&ta)[4], uint32_t (&tb)[4]) {
+            cp_async_wait<DW_AHEAD - 1>();
+            uint32_t cw[5];
+#pragma unroll
+            for (int xx = 0; xx < 5; ++xx) cw[xx] = ring[slot][xx][threadIdx.x];
+            const uint32_t lo01 = __byte_perm(cw[0], cw[1], 0x5140), hi01 = __byte_perm(cw[0], cw[1], 0x7362);
+            const uint32_t lo23 = __byte_perm(cw[2], cw[3], 0x5140), hi23 = __byte_perm(cw[2], cw[3], 0x7362);
+            ta[0] = __byte_perm(lo01, lo23, 0x5410);
+            ta[1] = __byte_perm(lo01, lo23, 0x7632);
+            ta[2] = __byte_perm(hi01, hi23, 0x5410);
+            ta[3] = __byte_perm(hi01, hi23, 0x7632);
+            tb[0] = __byte_perm(lo23, cw[4], 0x4410);
+            tb[1] = __byte_perm(lo23, cw[4], 0x5532);
+            tb[2] = __byte_perm(hi23, cw[4], 0x6610);
+            tb[3] = __byte_perm(hi23, cw[4], 0x7732);
+        };
+        auto emit = [&](int oh, const int (&a)[2][4]) {
+            uint8_t *out = y + ((size_t)(in * g.ho + oh) * g.wo + ow0) * g.c + c0;
+#pragma unroll
+            for (int o = 0; o < 2; ++o) {
+                if (ow0 + o < g.wo) {
+                    int tv[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int vv = a[o][j] >> q.s;
+                        tv[j] = SIGNED_OUT ? max(vv, -127) : vv;
+                    }
+                    uint32_t hi2, word;
+                    if (SIGNED_OUT) {
+                        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+                        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+                    } else {
+                        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+                        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+                    }
+                    *(uint32_t *)(out + o * g.c) = word;
+                }
+            }
+        };
+
+        const int first = 2 * oh0 - 1;
+#pragma unroll
+        for (int d = 0; d < DW_AHEAD; ++d) request_row(first + d, d);
+        int slot = 0, ih = first;
+        int acc[2][4];
+        uint32_t ta[4], tb[4];
+        // the row above the band opens the first output row
+        take_row(slot, ta, tb);
+        request_row(ih + DW_AHEAD, slot);
+        slot = (slot + 1) & (DW_AHEAD - 1);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            acc[0][j] = dw_dot4<XS>(ta[j], wr[0][j], bb[j]);
+            acc[1][j] = dw_dot4<XS>(tb[j], wr[0][j], bb[j]);
+        }
+        for (int oh = oh0; oh < oh1; ++oh) {
+            ih = 2 * oh;
+            take_row(slot, ta, tb);                         // the middle filter row
+            request_row(ih + DW_AHEAD, slot);
+            slot = (slot + 1) & (DW_AHEAD - 1);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc[0][j] = dw_dot4<XS>(ta[j], wr[1][j], acc[0][j]);
+                acc[1][j] = dw_dot4<XS>(tb[j], wr[1][j], acc[1][j]);
+            }
+            take_row(slot, ta, tb);                         // the bottom filter row of this output row, the top one of the next
+            request_row(ih + 1 + DW_AHEAD, slot);
+            slot = (slot + 1) & (DW_AHEAD - 1);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc[0][j] = dw_dot4<XS>(ta[j], wr[2][j], acc[0][j]);
+                acc[1][j] = dw_dot4<XS>(tb[j], wr[2][j], acc[1][j]);
+            }
+            emit(oh, acc);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc[0][j] = dw_dot4<XS>(ta[j], wr[0][j], bb[j]);
+                acc[1][j] = dw_dot4<XS>(tb[j], wr[0][j], bb[j]);
+            }
+        }
+        cp_async_wait<0>();
+    }
+}
+
 __global__ void __launch_bounds__(256) dwconv_scalar_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
                                                             const int8_t *__restrict__ w,
                                                             const int32_t *__restrict__ bias,
@@ -721,7 +1042,39 @@ cudaError_t f8_launch_dwconv(const F8ConvGeom &g, const F8Requant &q, const void
                           (size_t)g.n * g.h * g.w * g.c < (1u << 31) && total * (q.y_kind == F8_S32 ? 4 : 1) < (1u << 31);
     const bool walk_ok = strip_ok && g.stride_h == 1 && !q.has_res && q.y_kind != F8_S32 && q.s >= 1 && q.s <= 24 &&
                          q.sh_acc == 0 && !(f8_plan_options_off() & F8_PLAN_OFF_DW_WALK);
-    if (walk_ok) {
+    const bool dp4a_ok = strip_ok && !q.has_res && (q.y_kind == F8_U8 || q.y_kind == F8_S8) && q.s >= 1 &&
+                         q.s <= 24 && q.sh_acc == 0 && !(f8_plan_options_off() & F8_PLAN_OFF_DW_DP4A);
+    if (dp4a_ok && g.stride_h == 2) {
+        const int strips = (g.wo + 1) / 2;
+        int band_rows = g.ho;
+        while (band_rows > 4 && (long long)g.n * ((g.ho + band_rows - 1) / band_rows) * strips * (g.c / 4) < 148 * 128 * 8)
+            band_rows = (band_rows + 1) / 2;
+        const int bands = (g.ho + band_rows - 1) / band_rows;
+        const int threads = g.n * bands * strips * (g.c / 4);
+        const int grid = grid_for((size_t)threads, 128);
+        const uint8_t *xp = (const uint8_t *)x;
+#define F8_DW_DP4A2(XS_, SO_) \
+    launch_k(dwconv3x3s2_dp4a_kernel<XS_, SO_>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads)
+        const bool so = q.y_kind == F8_S8;
+        if (g.x_signed) { if (so) F8_DW_DP4A2(true, true); else F8_DW_DP4A2(true, false); }
+        else { if (so) F8_DW_DP4A2(false, true); else F8_DW_DP4A2(false, false); }
+#undef F8_DW_DP4A2
+    } else if (dp4a_ok) {
+        const int strips = (g.wo + 1) / 2;
+        int band_rows = g.ho;
+        while (band_rows > 8 && (long long)g.n * ((g.ho + band_rows - 1) / band_rows) * strips * (g.c / 4) < 148 * 128 * 8)
+            band_rows = (band_rows + 1) / 2;
+        const int bands = (g.ho + band_rows - 1) / band_rows;
+        const int threads = g.n * bands * strips * (g.c / 4);
+        const int grid = grid_for((size_t)threads, 128);
+        const uint8_t *xp = (const uint8_t *)x;
+#define F8_DW_DP4A(XS_, SO_) \
+    launch_k(dwconv3x3_dp4a_kernel<XS_, SO_>, grid, 128, overlap_previous, st, g, q, xp, w, bias, (uint8_t *)y, strips, bands, band_rows, threads)
+        const bool so = q.y_kind == F8_S8;
+        if (g.x_signed) { if (so) F8_DW_DP4A(true, true); else F8_DW_DP4A(true, false); }
+        else { if (so) F8_DW_DP4A(false, true); else F8_DW_DP4A(false, false); }
+#undef F8_DW_DP4A
+    } else if (walk_ok) {
         // two columns per thread measured slightly ahead of four (96 against 128 registers: 20 against 16 warps per SM)
         const int wcols = 2;
         const int strips = (g.wo + wcols - 1) / wcols;

@@ -45,6 +45,24 @@ def test_depthwise(ref, case):
     check_layer(ref, layer, x, res)
 
 
+@pytest.mark.parametrize("c,h,w,n,stride,x_signed,y_dtype", [
+    (32, 112, 112, 3, 1, False, synth.U8), (512, 14, 14, 5, 1, False, synth.U8), (1024, 7, 7, 4, 1, True, synth.S8),
+    (8, 5, 1, 2, 1, False, synth.U8), (4, 1, 9, 3, 1, True, synth.U8), (96, 37, 23, 2, 1, False, synth.S8),
+    (64, 112, 112, 2, 2, False, synth.U8), (256, 28, 28, 3, 2, True, synth.U8), (512, 14, 14, 4, 2, False, synth.S8),
+    (16, 7, 5, 2, 2, False, synth.U8), (12, 1, 2, 3, 2, True, synth.U8), (48, 33, 18, 2, 2, False, synth.U8)])
+def test_depthwise_packed_dot_products(ref, c, h, w, n, stride, x_signed, y_dtype):
+    """The dp4a depthwise kernels with every byte value on both sides (-128 weights against 255 / -128 activations),
+    widths of one and two, odd sizes, single rows."""
+    rng = np.random.default_rng(c * 1000 + h)
+    layer = random_conv_layer(rng, h=h, w=w, c=c, c_out=c, k=3, stride=stride, pad=1, x_signed=x_signed, y_dtype=y_dtype,
+                              with_res=False, kind=synth.DWCONV, fl_w=4, wide=True)
+    check_layer(ref, layer, random_input(rng, n, layer))
+    # the older kernels behind the planning switch give the same bits
+    from paper_2202_05239_b200 import api as a
+    if c <= 96:
+        check_layer(ref, layer, random_input(rng, n, layer), plan_off=a.PLAN_OFF_DW_DP4A)
+
+
 @pytest.mark.parametrize("c,signed,h,k,stride,pad", [(64, False, 112, 3, 2, 1), (16, True, 9, 3, 2, 1), (20, False, 11, 2, 2, 0),
                                                       (7, True, 10, 3, 1, 1), (128, False, 7, 3, 2, 1)])
 def test_maxpool(ref, c, signed, h, k, stride, pad):

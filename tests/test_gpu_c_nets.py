@@ -110,9 +110,13 @@ def test_net_parity_two_lanes(ref, name, batch, micro):
     _compare_net(ref, name, batch, 224, lanes=2, micro_batch=micro)
 
 
-def test_mobilenet_parity_with_the_strip_kernel(ref):
+@pytest.mark.parametrize("which", ["walk", "strip"])
+def test_mobilenet_parity_with_the_older_depthwise_kernels(ref, which):
+    """Stride-1 depthwise layers default to the packed-dot-product kernel; the row-walking kernel and the strip kernel
+    behind it stay selectable and must give the same bits."""
     a = api()
-    _compare_net(ref, "mobilenetv1", 3, 224, plan_off=a.PLAN_OFF_DW_WALK)
+    off = a.PLAN_OFF_DW_DP4A | (a.PLAN_OFF_DW_WALK if which == "strip" else 0)
+    _compare_net(ref, "mobilenetv1", 3, 224, plan_off=off)
 
 
 def _sampled_full_batch(ref, name, batch, samples):
