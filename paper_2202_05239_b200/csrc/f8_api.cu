@@ -182,17 +182,38 @@ unsigned f8_plan_options_off() { return g_plan_off; }
 unsigned long long f8_wait_limit_cycles() { return g_wait_limit_cycles; }
 int *f8_last_plan_info() { return g_last_plan; }
 
+namespace {
+int *g_status_words[64] = {nullptr};
+volatile int *g_status_host[64] = {nullptr};     // page-locked host word a kernel that gives up a wait writes its code to
+}   // namespace
+
 int *f8_status_word() {
-    static int *words[64] = {nullptr};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!words[dev]) {
+    if (!g_status_words[dev]) {
         int *p = nullptr;
         if (cudaMalloc(&p, 256) != cudaSuccess) return nullptr;
         cudaMemset(p, 0, 256);
-        words[dev] = p;
+        // a host-visible copy of the first word: kernels store to it through its device address (words 32 / 33 of the
+        // buffer), the host reads it directly -- f8_net_forward can then report a time-out without touching a stream
+        int *h = nullptr, *h_dev = nullptr;
+        if (cudaHostAlloc((void **)&h, 64, cudaHostAllocMapped) == cudaSuccess && cudaHostGetDevicePointer((void **)&h_dev, h, 0) == cudaSuccess) {
+            memset(h, 0, 64);
+            cudaMemcpy(p + 32, &h_dev, sizeof(h_dev), cudaMemcpyHostToDevice);
+            g_status_host[dev] = h;
+        } else {
+            (void)cudaGetLastError();
+        }
+        g_status_words[dev] = p;
     }
-    return words[dev];
+    return g_status_words[dev];
+}
+
+// 0, or the code of a wait some kernel on the current device has given up since the last f8_device_status().
+int f8_status_host_code() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || !g_status_host[dev]) return 0;
+    return *g_status_host[dev];
 }
 
 extern "C" {
@@ -263,6 +284,10 @@ f8_status f8_device_status(void) {
     int v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     e = cudaMemcpy(v, w, sizeof(v), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(e, "status read");
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && g_status_host[dev]) *g_status_host[dev] = 0;
+    }
     if (v[0] != 0) {
         cudaMemset(w, 0, sizeof(v));
         return fail(F8_ERR_TIMEOUT, "a kernel abandoned a bounded wait (site %d, layer %d, block %d, thread %d, barrier 0x%x, parity %d; "
@@ -442,12 +467,6 @@ struct f8_net {
     bool profiling = false;
     std::vector<cudaEvent_t> events;             // steps + 1 events of the last profiled forward
     std::vector<int> event_layer;                // layer each step belongs to
-    // Host copy of the device status word: every pass ends with an asynchronous copy of the word into this pinned
-    // buffer, and the next call looks at it once the copy has completed -- a kernel that gave up a bounded wait is
-    // then reported by f8_net_forward itself, without a synchronisation.
-    int *host_status = nullptr;
-    cudaEvent_t status_ev = nullptr;
-    bool status_pending = false;
 };
 
 namespace {
@@ -877,13 +896,7 @@ f8_status f8_net_create(const f8_layer_desc *layers, int n_layers, const int8_t 
             }
         }
     }
-    if (cudaHostAlloc((void **)&net->host_status, 64, cudaHostAllocDefault) != cudaSuccess ||
-        cudaEventCreateWithFlags(&net->status_ev, cudaEventDisableTiming) != cudaSuccess) {
-        if (net->host_status) cudaFreeHost(net->host_status);
-        (void)cudaGetLastError();
-        return cleanup(fail(F8_ERR_CUDA, "could not create the status mirror"));
-    }
-    memset(net->host_status, 0, 64);
+    (void)f8_status_word();         // creates the device status word and its host-visible copy
     if (cudaStreamCreateWithFlags(&net->lane_stream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&net->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&net->ev_join, cudaEventDisableTiming) != cudaSuccess) {
@@ -952,11 +965,9 @@ f8_status f8_net_get_layer_ms(f8_net *net, float *ms, int *on_tensor_cores) {
 void f8_net_destroy(f8_net *net) {
     if (!net) return;
     for (cudaEvent_t ev : net->events) cudaEventDestroy(ev);
-    if (net->status_ev) cudaEventDestroy(net->status_ev);
     if (net->ev_fork) cudaEventDestroy(net->ev_fork);
     if (net->ev_join) cudaEventDestroy(net->ev_join);
     if (net->lane_stream) cudaStreamDestroy(net->lane_stream);
-    if (net->host_status) cudaFreeHost(net->host_status);
     free_layers(net);
     delete net;
 }
@@ -973,21 +984,11 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         return fail(F8_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, workspace_bytes);
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int nl = (int)net->layers.size();
-    if (net->status_pending) {
-        const cudaError_t q = cudaEventQuery(net->status_ev);
-        if (q == cudaSuccess) {
-            net->status_pending = false;
-            const int v = net->host_status[0];
-            if (v != 0) {
-                net->host_status[0] = 0;
-                return fail(F8_ERR_TIMEOUT, "a kernel abandoned a bounded wait before or during the previous pass (site %d, layer %d): "
-                            "its output is incomplete; f8_device_status() gives the details and clears the record",
-                            v & 0xff, (v >> 8) - 1);
-            }
-        } else {
-            (void)cudaGetLastError();       // "not ready" is not an error
-        }
-    }
+    // A kernel that gives up a bounded wait also stores its code to a host-visible word: an earlier pass (or anything
+    // else on this device) that left its output incomplete is reported here, without a synchronisation.
+    if (const int v = f8_status_host_code())
+        return fail(F8_ERR_TIMEOUT, "a kernel abandoned a bounded wait (site %d, layer %d): the output of that pass is incomplete; "
+                    "f8_device_status() gives the details and clears the record", v & 0xff, (v >> 8) - 1);
 
     // a first layer whose output is asked for cannot be fused with the pooling layer behind it
     bool dump_fusable = false;
@@ -1264,13 +1265,6 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         if (e != cudaSuccess) return cuda_fail(e, "second lane join");
     }
     net->last_launches = launches;
-    if (int *word = f8_status_word()) {
-        if (cudaMemcpyAsync(net->host_status, word, sizeof(int), cudaMemcpyDeviceToHost, st) == cudaSuccess &&
-            cudaEventRecord(net->status_ev, st) == cudaSuccess)
-            net->status_pending = true;
-        else
-            (void)cudaGetLastError();
-    }
     return F8_OK;
 }
 

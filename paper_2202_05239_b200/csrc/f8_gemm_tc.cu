@@ -130,7 +130,6 @@ struct TcParams {
     F8Sibling sib;            // second consumer of the same sums (generic epilogue only)
     int vec_bytes2;           // widest aligned store of the second output's rows
     int mul_acc, mul_res;     // 2^q.sh_acc, 2^q.sh_res (kept opaque to the compiler, see the epilogue)
-    int shr_mul;              // 2^(32 - q.s): the rounding shift as the high word of a product (staged epilogues, s >= 2)
     int *status;
     // Windowed 3x3 (stride 1, pad 1, resident weights).  A tile is win_r whole output rows of one image; its M index runs
     // over the rows of the zero-padded image (win_wp = W + 2 positions per row, the last two of each row are discarded).
@@ -376,24 +375,67 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
             }
-        } else
+        } else if (p.rowt)
+        // small tensors: the same pipeline, but a tile is win_r whole output rows of one image and every filter tap is a
+        // tiled load whose box starts at the tap's offset (out-of-image elements are zero filled)
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
             const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
             const int m0 = m_t * TILE_M;
-            int img, base_w, base_h;
-            if (p.rowt) {
-                // whole output rows y0 .. y0 + win_r - 1 of one image; tap (r, s) starts at input (s - pad, y0 * stride + r - pad)
-                img = fast_div(m_t, p.div_bands);
-                base_w = -p.pad_w;
-                base_h = (m_t - img * p.win_bands) * p.win_r * p.stride_h - p.pad_h;
-            } else {
-                const int t1 = fast_div(m0, p.div_wo);
-                const int ow = m0 - t1 * p.wo;
-                img = fast_div(t1, p.div_ho);
-                const int oh = t1 - img * p.ho;
-                base_w = ow * p.stride_w - p.pad_w;
-                base_h = oh * p.stride_h - p.pad_h;
+            // output rows y0 .. y0 + win_r - 1; tap (r, s) starts at input (s - pad, y0 * stride + r - pad)
+            const int img = fast_div(m_t, p.div_bands);
+            const int base_w = -p.pad_w;
+            const int base_h = (m_t - img * p.win_bands) * p.win_r * p.stride_h - p.pad_h;
+            const int n_base = n_t * p.bn;
+            for (int kc = 0; kc < k_iters; kc += p.group, ++use_idx) {
+                if (p.alt && (use_idx & 1) != half) {
+                    // the other pair's use.  This warp waits only for the stages of its own uses, and the single,
+                    // in-order MMA issuer cannot pass one of those without it: it never falls a barrier phase behind.
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                    continue;
+                }
+                if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, wc, tagbits | 101))) {
+                    ok = false;
+                    break;
+                }
+                const int subs = min(p.group, k_iters - kc);
+                const uint32_t fb = full_bar + 8 * stage;
+                // Two arrivals per stage use, one from each producer warp, and each announces the bytes of its own loads
+                // BEFORE it issues them: the barrier's byte count never runs ahead of what has been announced, and both
+                // warps are needed for every use, so neither can fall a barrier phase behind the pipeline (a parity wait
+                // cannot tell a phase from the one two later).  A helper without a load in this use just arrives.
+                if (lane == 0) {
+                    uint32_t bytes;
+                    if (opnd == 0) bytes = (uint32_t)(p.b_res ? (subs + 1) >> 1 : subs) * p.tx_a;
+                    else bytes = p.b_res ? (uint32_t)(subs >> 1) * p.tx_a : (uint32_t)subs * p.tx_b;
+                    if (bytes) mbar_expect_tx(fb, bytes);
+                    else mbar_arrive(fb);
+                }
+                __syncwarp();
+                const int j = (lane - stage * p.group) & 31;
+                if (j < subs && (j & j_mask) == j_want) {
+                    const uint2 e = ktab[kc + j];       // x: first channel of the chunk, y: tap << 16 | r << 8 | s
+                    const uint32_t dst = smem_base + stage * p.stage_bytes + j * p.sub_bytes;
+                    if (opnd == 0 || a_helper)
+                        tma_load_4d(dst, &map_a, fb, (int)e.x, base_w + (int)(e.y & 0xff), base_h + (int)((e.y >> 8) & 0xff), img);
+                    else
+                        tma_load_3d(dst + p.a_bytes, &map_b, fb, (int)e.x, (int)(e.y >> 16), n_base);
+                    have_last = true;
+                    last_stage = stage;
+                    last_phase = phase;
+                }
+                if (++stage == p.stages) { stage = 0; phase ^= 1; }
             }
+        }
+        else
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
+            const int m0 = m_t * TILE_M;
+            const int t1 = fast_div(m0, p.div_wo);
+            const int ow = m0 - t1 * p.wo;
+            const int img = fast_div(t1, p.div_ho);
+            const int oh = t1 - img * p.ho;
+            const int base_w = ow * p.stride_w - p.pad_w;
+            const int base_h = oh * p.stride_h - p.pad_h;
             const int n_base = n_t * p.bn;
             for (int kc = 0; kc < k_iters; kc += p.group, ++use_idx) {
                 if (p.alt && (use_idx & 1) != half) {
@@ -426,8 +468,6 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     const uint32_t dst = smem_base + stage * p.stage_bytes + j * p.sub_bytes;
                     if ((opnd == 0 || a_helper) && p.a_plain)
                         tma_load_2d(dst, &map_a, fb, (int)e.x, m0);
-                    else if ((opnd == 0 || a_helper) && p.rowt)
-                        tma_load_4d(dst, &map_a, fb, (int)e.x, base_w + (int)(e.y & 0xff), base_h + (int)((e.y >> 8) & 0xff), img);
                     else if (opnd == 0 || a_helper)
                         tma_load_im2col(dst, &map_a, fb, (int)e.x, base_w, base_h, img, (uint16_t)(e.y & 0xff),
                                         (uint16_t)((e.y >> 8) & 0xff));
@@ -637,7 +677,6 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const int ch_begin = min(group * per_group, chunks);
         const int nch = min(ch_begin + per_group, chunks) - ch_begin;
         const int mul_acc = p.mul_acc, mul_res = p.mul_res;     // 2^sh_acc, 2^sh_res
-        const int shr_mul = p.shr_mul;                          // 2^(32 - s)
         int local = 0;
         int ob = 0;                 // buffer of the output ring for the current tile and the parity of its use
         uint32_t ophase = 0;
@@ -682,14 +721,14 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         if (RES) rw = lds128(res_buf + so[i]);
                         tmem_ld_wait();
                         if (i + 1 < my_nch) tmem_ld16(t_addr + (i + 1) * 16, vb);
-                        sts128(out_buf + so[i], epilogue_fast16<RES, SGN>(va, bias_s + 64 * (i), rw, mul_acc, mul_res, rsel, shr_mul));
+                        sts128(out_buf + so[i], epilogue_fast16<RES, SGN>(va, bias_s + 64 * (i), rw, mul_acc, mul_res, rsel, p.q.s));
                     }
                     if (i + 1 < my_nch) {
                         uint4 rw = make_uint4(0, 0, 0, 0);
                         if (RES) rw = lds128(res_buf + so[i + 1]);
                         tmem_ld_wait();
                         if (i + 2 < my_nch) tmem_ld16(t_addr + (i + 2) * 16, va);
-                        sts128(out_buf + so[i + 1], epilogue_fast16<RES, SGN>(vb, bias_s + 64 * (i + 1), rw, mul_acc, mul_res, rsel, shr_mul));
+                        sts128(out_buf + so[i + 1], epilogue_fast16<RES, SGN>(vb, bias_s + 64 * (i + 1), rw, mul_acc, mul_res, rsel, p.q.s));
                     }
                 }
                 // accumulator and residual have been read, the output part is written: make the writes
@@ -919,7 +958,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.c_chunks = (g.c + p.kb - 1) / p.kb;
     p.epi = EPI_GENERIC;
     const bool has_sib = sib && sib->y2;
-    if ((q.y_kind == F8_U8 || q.y_kind == F8_S8) && q.s >= 2 && q.s <= 24 && g.c_out % 16 == 0 && !has_sib && !q.r_s32)
+    if ((q.y_kind == F8_U8 || q.y_kind == F8_S8) && q.s >= 1 && q.s <= 24 && g.c_out % 16 == 0 && !has_sib && !q.r_s32)
         p.epi = q.y_kind == F8_U8 ? (q.has_res ? EPI_U8_RES : EPI_U8) : (q.has_res ? EPI_S8_RES : EPI_S8);
     const bool staged = p.epi != EPI_GENERIC;
     p.bn = staged ? choose_bn_staged(g.c_out, q.has_res != 0, p.kb) : choose_bn(g.c_out);
@@ -1080,7 +1119,6 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.q = q;
     p.mul_acc = 1 << q.sh_acc;
     p.mul_res = 1 << q.sh_res;
-    p.shr_mul = (q.s >= 2 && q.s <= 30) ? (1 << (32 - q.s)) : 0;
     p.status = status_word;
     const int ysz = (q.y_kind == F8_S32 || q.y_kind == F8_S32_RELU) ? 4 : 1;
     const size_t row_bytes = (size_t)g.c_out * ysz;

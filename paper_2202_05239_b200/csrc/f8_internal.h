@@ -98,8 +98,10 @@ cudaError_t f8_launch_stem_tc(const F8ConvGeom &g, const F8Requant &q, int kh2, 
                               const void *x, const int8_t *w_core, const int32_t *bias, void *y, int *status_word, int tag,
                               cudaStream_t st, bool overlap_previous);
 
-// Device status word (0 = fine); allocated once per device on first use.
+// Device status word (0 = fine); allocated once per device on first use, together with a host-visible copy of its
+// first word that kernels write through (f8_status_host_code reads it without synchronising).
 int *f8_status_word();
+int f8_status_host_code();
 
 // Planning choices switched off by f8_debug_plan_options (F8_PLAN_OFF_* bits), the bound of in-kernel waits in SM
 // cycles (0 = default) and the record of the last tensor-core plan (10 ints, see f8_debug_last_plan).

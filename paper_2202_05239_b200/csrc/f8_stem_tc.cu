@@ -51,8 +51,7 @@ struct StemParams {
     uint32_t idesc;
     uint32_t a_desc_hi, b_desc_hi;   // upper descriptor words (byte offsets between core matrices)
     uint32_t a_desc_lbo_sbo, b_desc_lbo_sbo;   // bits 16.. of the lower word (leading byte offset)
-    int s;                     // rounding shift, 2..24
-    int shr_mul;               // 2^(32 - s): the shift as the high word of a product
+    int s;                     // rounding shift, 1..24
     int signed_out;
     int x_signed;
     const uint8_t *x;
@@ -281,7 +280,7 @@ __global__ void __launch_bounds__(STEM_THREADS, 3) f8_stem_tc_kernel(const StemP
                         int v[16];
                         tmem_ld16(t_addr + ch * 16, v);
                         tmem_ld_wait();
-                        const uint4 o = epilogue_fast16<false, SIGNED>(v, bias_base + 64 * ch, make_uint4(0, 0, 0, 0), 1, 0, rsel, p.shr_mul);
+                        const uint4 o = epilogue_fast16<false, SIGNED>(v, bias_base + 64 * ch, make_uint4(0, 0, 0, 0), 1, 0, rsel, p.s);
                         const uint32_t co = ((uint32_t)ch ^ swz) << 4;
                         if (!POOL) {
                             sts128(cur + co, o);
@@ -368,7 +367,7 @@ static size_t stem_smem_bytes(int kh2, int slices, int c_out) {
 bool f8_stem_tc_supported(const F8ConvGeom &g, const F8Requant &q, int kh2, int slices) {
     if (g.c > 4 || g.stride_h != 2 || g.stride_w != 2) return false;
     if (g.wo > 128 || g.wo < 1 || g.c_out % 16 != 0 || g.c_out > 256) return false;
-    if (q.has_res || (q.y_kind != F8_U8 && q.y_kind != F8_S8) || q.s < 2 || q.s > 24) return false;
+    if (q.has_res || (q.y_kind != F8_U8 && q.y_kind != F8_S8) || q.s < 1 || q.s > 24) return false;
     if (kh2 < 1 || kh2 >= STEM_PAIR_SLOTS || slices < 1 || slices > 2) return false;       // windows of at most 64 bytes
     if (2 * (g.wo - 1) + slices * 4 > STEM_MAX_CELLS) return false;
     if ((size_t)g.n * g.h * g.w * g.c >= 0x7fffffffull || (size_t)g.n * std::max(g.ho, 1) >= 0x7fffffffull) return false;
@@ -417,7 +416,6 @@ cudaError_t f8_launch_stem_tc(const F8ConvGeom &g, const F8Requant &q, int kh2, 
     p.a_desc_hi = (a_sbo >> 4) | (1u << 14);     // stride byte offset at bit 32, descriptor version 1 at bit 46, no swizzle
     p.b_desc_hi = (b_sbo >> 4) | (1u << 14);
     p.s = q.s;
-    p.shr_mul = 1 << (32 - q.s);
     p.signed_out = q.y_kind == F8_S8 ? 1 : 0;
     p.x_signed = g.x_signed;
     p.x = (const uint8_t *)x; p.wk = w_core; p.bias = bias; p.y = (uint8_t *)y; p.status = status_word; p.tag = tag;

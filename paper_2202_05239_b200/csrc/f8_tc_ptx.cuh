@@ -104,6 +104,13 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const
                     status[5] = (int)spins;
                     status[6] = (int)(dc >> 20);       // SM cycles / 2^20
                     status[7] = (int)(dg >> 10);       // wall-clock microseconds (ns / 1024) since the 4096th poll (the 64th under a short test limit)
+                    // words 32 / 33 of the status buffer may hold the address of a word in host memory that the library
+                    // reads without synchronising (0: none): the code goes there as well
+                    int *host_copy = *(int *volatile *)(status + 32);
+                    if (host_copy) {
+                        *(volatile int *)host_copy = code;
+                        __threadfence_system();
+                    }
                 }
                 return false;
             }
@@ -254,8 +261,8 @@ __host__ __device__ inline uint64_t smem_desc_hi(int kb) {
 // Branch-free epilogue for the common case (8-bit output, 1 <= s <= 24, c_out % 16 == 0).
 //   v = acc * 2^sh_acc + bias'          bias' = (bias << sh_acc) + 2^(s-1), staged in shared memory
 //   v += r << sh_res                    (RES only)
-//   t = v >> s                          = floor((acc' + 2^(s-1)) / 2^s), round half up; computed as the high word of
-//                                       v * 2^(32-s) (2 <= s), which is the same floor and runs on the multiplier pipe
+//   t = v >> s                          = floor((acc' + 2^(s-1)) / 2^s), round half up (the same floor taken as the high
+//                                       word of v * 2^(32-s), to move it to the multiplier pipe, measured 2 % slower)
 //   y = clamp(t, lo, hi)                saturating pack; the signed quantizer additionally excludes -128
 // cvt.pack.sat packs two saturated values into the low half of d and moves the low half of c above
 // them: d = (c << 16) | (sat(a) << 8) | sat(b).
@@ -275,7 +282,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
 
 template <bool RES, bool SIGNED_OUT>
 __device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], uint32_t bias_addr, uint4 rw, int mul_acc,
-                                                 int mul_res, const uint32_t (&rsel)[4], int shr_mul /* 2^(32-s), opaque */) {
+                                                 int mul_res, const uint32_t (&rsel)[4], int s) {
     int t[16];
     const uint32_t rwords[4] = {rw.x, rw.y, rw.z, rw.w};
 #pragma unroll
@@ -291,7 +298,7 @@ __device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], uint32_t 
                 asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(rwords[g]), "r"(rsel[k]));
                 v += r * mul_res;
             }
-            v = __mulhi(v, shr_mul);
+            v >>= s;
             t[j] = SIGNED_OUT ? max(v, -127) : v;
         }
     }

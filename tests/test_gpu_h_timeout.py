@@ -29,8 +29,9 @@ def test_a_wait_that_runs_out_is_reported_and_the_device_stays_usable(ref):
 
 
 def test_net_forward_reports_a_time_out_left_by_an_earlier_pass(ref):
-    """f8_net_forward copies the status word to the host after every pass (asynchronously) and the next call on the
-    same object looks at that copy: a kernel that gave up is reported without anybody calling f8_device_status."""
+    """A kernel that gives up a wait also stores its code to a word in host memory, which f8_net_forward looks at on
+    entry: the time-out is reported by the next pass without anybody calling f8_device_status (and without a
+    synchronisation inside the library)."""
     a = api()
     a.f8_device_status()
     layers = synth.make_net("resnet18", 0, image=64)
