@@ -97,6 +97,8 @@ struct TcParams {
     int uses;                 // stage uses per tile: ceil(k_iters / group)
     int dual_issue;           // 1: two MMA-issuing threads (needs stages >= 2 * uses)
     int a_plain;              // 1: pointwise layer on a small tensor: activations read as a plain [M, C] matrix (tiled map)
+    int pair;                 // 1: CTA pairs (the PAIR instantiation): 256-row tiles, half of a weight tile per CTA
+    int pair_tiles;           // 256-row tiles x N tiles
     int alt;                  // 1: two pairs of producer warps, pair h takes the stage uses of parity h (streamed weights,
                               // one MMA issuer: fills may then complete out of order, the consumer is in order)
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
@@ -232,7 +234,9 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int (&ac
 
 enum { EPI_GENERIC = 0, EPI_U8 = 1, EPI_U8_RES = 2, EPI_S8 = 3, EPI_S8_RES = 4 };
 
-template <int EPI>
+// PAIR: two CTAs of a cluster share 256-row tiles (tcgen05 cta_group::2): each loads its own 128 rows of activations and
+// half of the weight tile, so a weight byte crosses the L2 -> SM path once per 256 rows; the even CTA issues the MMAs.
+template <int EPI, bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_r,
@@ -256,6 +260,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    // persistent workers: CTAs, or CTA pairs (rank 0 = the even CTA, which owns the stage barriers and issues the MMAs)
+    const uint32_t cta_rank = PAIR ? cluster_cta_rank() : 0u;
+    const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     const uint32_t full_bar = smem_u32(&bars[0]);
     const uint32_t empty_bar = smem_u32(&bars[MAX_STAGES]);
     const uint32_t tfull_bar = smem_u32(&bars[2 * MAX_STAGES]);
@@ -274,7 +282,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         mbar_init(bres_bar, 1);
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
-            mbar_init(tempty_bar + 8 * a, NUM_EPI_WARPS);
+            mbar_init(tempty_bar + 8 * a, PAIR ? 2 * NUM_EPI_WARPS : NUM_EPI_WARPS);     // the epilogue warps of both CTAs
         }
         for (int a = 0; a < MAX_OUT_BUFS; ++a) {
             mbar_init(out_full + 8 * a, NUM_EPI_WARPS);   // every epilogue warp has written its part of the tile
@@ -300,16 +308,20 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         for (int i = threadIdx.x; i < p.n_tiles * p.bn; i += NUM_THREADS)
             bias_all[i] = ((i < p.c_out && p.bias) ? (__ldg(p.bias + i) << p.q.sh_acc) : 0) + rnd;
     }
-    if (warp == MMA_WARP) tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+    if (warp == MMA_WARP) {
+        if (PAIR) tmem_alloc_pair(smem_u32(&tmem_base_slot), TMEM_COLS);
+        else tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+    }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();      // the partner's barriers exist before anything is sent to them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     // the next grid in the stream may be scheduled from here on: its CTAs take over an SM when this grid's
     // CTA there has exited, and run their prologue while the rest of this grid finishes
     grid_launch_dependents();
 
-    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int total_tiles = PAIR ? p.pair_tiles : p.m_tiles * p.n_tiles;      // per worker: 128-row tiles, or 256-row tiles of a pair
     const int k_iters = p.kh * p.kw * p.c_chunks;
     const WaitCtx wc = make_wait_ctx(&abort_flag, p.status, p.wait_limit);
     const int tagbits = p.tag << 8;     // status word of a timed-out wait: tag << 8 | site
@@ -355,7 +367,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         bool ok = true;
         if (p.win) {
             // one load per (tile, channel chunk): the padded rows of the band, requested by the lane that owns the stage
-            for (int tile = blockIdx.x; ok && opnd == 0 && tile < total_tiles; tile += gridDim.x) {
+            for (int tile = worker; ok && opnd == 0 && tile < total_tiles; tile += n_workers) {
                 const int m_t = fast_div(tile, p.div_n_tiles);
                 const int img = fast_div(m_t, p.div_bands);
                 const int y0 = (m_t - img * p.win_bands) * p.win_r;
@@ -378,8 +390,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         } else if (p.rowt)
         // small tensors: the same pipeline, but a tile is win_r whole output rows of one image and every filter tap is a
         // tiled load whose box starts at the tap's offset (out-of-image elements are zero filled)
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-            const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
+        for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+            const int m_q = fast_div(tile, p.div_n_tiles), n_t = tile - m_q * p.n_tiles;
+            const int m_t = PAIR ? 2 * m_q + (int)cta_rank : m_q;
             const int m0 = m_t * TILE_M;
             // output rows y0 .. y0 + win_r - 1; tap (r, s) starts at input (s - pad, y0 * stride + r - pad)
             const int img = fast_div(m_t, p.div_bands);
@@ -427,8 +440,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             }
         }
         else
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-            const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
+        for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+            const int m_q = fast_div(tile, p.div_n_tiles), n_t = tile - m_q * p.n_tiles;
+            const int m_t = PAIR ? 2 * m_q + (int)cta_rank : m_q;
             const int m0 = m_t * TILE_M;
             const int t1 = fast_div(m0, p.div_wo);
             const int ow = m0 - t1 * p.wo;
@@ -454,10 +468,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 // BEFORE it issues them: the barrier's byte count never runs ahead of what has been announced, and both
                 // warps are needed for every use, so neither can fall a barrier phase behind the pipeline (a parity wait
                 // cannot tell a phase from the one two later).  A helper without a load in this use just arrives.
-                if (lane == 0) {
+                // (A pair has one barrier per stage, in its even CTA: the even CTA's warps announce the bytes of both CTAs,
+                // the odd CTA's loads complete there without an arrival of their own.)
+                if (lane == 0 && (!PAIR || cta_rank == 0)) {
                     uint32_t bytes;
                     if (opnd == 0) bytes = (uint32_t)(p.b_res ? (subs + 1) >> 1 : subs) * p.tx_a;
                     else bytes = p.b_res ? (uint32_t)(subs >> 1) * p.tx_a : (uint32_t)subs * p.tx_b;
+                    if (PAIR) bytes *= 2;
                     if (bytes) mbar_expect_tx(fb, bytes);
                     else mbar_arrive(fb);
                 }
@@ -466,7 +483,17 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 if (j < subs && (j & j_mask) == j_want) {
                     const uint2 e = ktab[kc + j];       // x: first channel of the chunk, y: tap << 16 | r << 8 | s
                     const uint32_t dst = smem_base + stage * p.stage_bytes + j * p.sub_bytes;
-                    if ((opnd == 0 || a_helper) && p.a_plain)
+                    if (PAIR) {
+                        // this CTA's 128 rows of activations, its half of the weight tile; completion on the even CTA's barrier
+                        if (opnd == 0 && p.a_plain)
+                            tma_load_2d_pair(dst, &map_a, fb, (int)e.x, m0);
+                        else if (opnd == 0)
+                            tma_load_im2col_pair(dst, &map_a, fb, (int)e.x, base_w, base_h, img, (uint16_t)(e.y & 0xff),
+                                                 (uint16_t)((e.y >> 8) & 0xff));
+                        else
+                            tma_load_3d_pair(dst + p.a_bytes, &map_b, fb, (int)e.x, (int)(e.y >> 16),
+                                             n_base + (int)cta_rank * (p.bn >> 1));
+                    } else if ((opnd == 0 || a_helper) && p.a_plain)
                         tma_load_2d(dst, &map_a, fb, (int)e.x, m0);
                     else if (opnd == 0 || a_helper)
                         tma_load_im2col(dst, &map_a, fb, (int)e.x, base_w, base_h, img, (uint16_t)(e.y & 0xff),
@@ -500,7 +527,17 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // plan enables the second issuer only when stages >= 2 * uses per tile, which guarantees that (the
         // previous use of the stage then belongs to a tile this issuer, or the other one before it, is done with).
         const int q_issuer = warp == MMA_WARP ? 0 : 1;
-        if (lane == 0 && (q_issuer == 0 || p.dual_issue)) {
+        if (PAIR && cta_rank != 0) {
+            // The odd CTA of a pair issues nothing; the commits of the even CTA's issuer arrive on its barriers too.  Before
+            // the CTA may go, the arrivals that free its last stage uses must have landed (see below).
+            if (lane == 0 && q_issuer == 0) {
+                int local = 0;
+                for (int tile = worker; tile < total_tiles; tile += n_workers) ++local;
+                const int total_uses = local * p.uses;
+                for (int g = max(0, total_uses - p.stages); g < total_uses; ++g)
+                    mbar_wait(empty_bar + 8 * (g % p.stages), (uint32_t)(g / p.stages) & 1u, wc, tagbits | 113);
+            }
+        } else if (lane == 0 && (q_issuer == 0 || p.dual_issue)) {
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -517,7 +554,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const uint32_t b_step = p.b_res ? b16 : sub16;
             if (p.b_res && !mbar_wait(bres_bar, 0, wc, tagbits | 111)) ok = false;
             const int mmas = p.kb >> 5;      // 1, 2 or 4 instructions per stage
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+            for (int tile = worker; ok && tile < total_tiles; tile += n_workers, ++local) {
                 const int acc = local & 1;
                 if (p.dual_issue && acc != q_issuer) {
                     // the other issuer's tile: step over its stage uses
@@ -565,15 +602,24 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     const int subs = min(p.group, k_iters - kc);
                     const uint32_t first = kc != 0 ? 1u : 0u;      // the tile's first MMA overwrites the accumulator
                     const uint32_t b_lo = p.b_res ? b_tile_lo + (uint32_t)kc * b16 : stage_lo + a16;
+                    if (PAIR) {
+                        // 256-row instructions over both CTAs' tiles (128-byte K chunks only); the commit frees the stage in both
+                        uint32_t a_lo = stage_lo, bb_lo = b_lo;
+                        for (int j = 0; j < subs; ++j, a_lo += sub16, bb_lo += b_step)
+                            mma_i8_sub_pair4(d_tmem, a_lo, bb_lo, desc_hi32, p.idesc, j == 0 ? first : 1u);
+                        mma_commit_pair(empty_bar + 8 * stage);
+                    } else {
                     if (mmas == 4) mma_i8_stage<4>(d_tmem, stage_lo, b_lo, sub16, b_step, desc_hi32, p.idesc, subs, first);
                     else if (mmas == 2) mma_i8_stage<2>(d_tmem, stage_lo, b_lo, sub16, b_step, desc_hi32, p.idesc, subs, first);
                     else mma_i8_stage<1>(d_tmem, stage_lo, b_lo, sub16, b_step, desc_hi32, p.idesc, subs, first);
                     mma_commit(empty_bar + 8 * stage);    // frees the stage when these MMAs have read it
+                    }
                     stage_lo += stage16;
                     if (++stage == p.stages) { stage = 0; phase ^= 1; stage_lo = desc_lo0; }
                 }
                 if (!ok) break;
-                mma_commit(tfull_bar + 8 * acc);          // accumulator complete
+                if (PAIR) mma_commit_pair(tfull_bar + 8 * acc);      // both CTAs' halves of the accumulator are complete
+                else mma_commit(tfull_bar + 8 * acc);          // accumulator complete
                 committed_any = true;
                 last_acc = acc;
                 last_acc_phase = acc_phase;
@@ -606,8 +652,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             // stores: a tile leaves from its buffer of the ring once all epilogue warps have written it
             int b = 0;
             uint32_t bphase = 0;
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-                const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
+            for (int tile = worker; tile < total_tiles; tile += n_workers) {
+                const int m_q = fast_div(tile, p.div_n_tiles), n_t = tile - m_q * p.n_tiles;
+            const int m_t = PAIR ? 2 * m_q + (int)cta_rank : m_q;
                 if (!mbar_wait(out_full + 8 * b, bphase, wc, tagbits | 108)) break;
                 const uint32_t src = smem_base + p.out_off + b * p.out_bytes;
                 if (p.rows) {
@@ -639,8 +686,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             int rb = 0;
             uint32_t rphase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
-                const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
+            for (int tile = worker; tile < total_tiles; tile += n_workers, ++local) {
+                const int m_q = fast_div(tile, p.div_n_tiles), n_t = tile - m_q * p.n_tiles;
+            const int m_t = PAIR ? 2 * m_q + (int)cta_rank : m_q;
                 if (!mbar_wait(out_free + 8 * rb, rphase ^ 1, wc, tagbits | 106)) { ok = false; break; }
                 const uint32_t fb = res_full + 8 * rb;
                 mbar_expect_tx(fb, p.tx_res);
@@ -696,7 +744,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 off ^= ((off >> 7) & p.swz_mask) << 4;
                 so[i] = (uint32_t)(ch / p.slab_chunks) * (TILE_M * p.slab_w) + off;
             }
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+            for (int tile = worker; tile < total_tiles; tile += n_workers, ++local) {
                 const int acc = local & 1;                   // accumulator, output buffer and residual buffer in use
                 const uint32_t acc_phase = (local >> 1) & 1;
                 const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
@@ -737,7 +785,8 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(tempty_bar + 8 * acc);
+                    if (PAIR && cta_rank != 0) mbar_arrive_cluster(tempty_bar + 8 * acc, 0);     // the issuer's barrier
+                    else mbar_arrive(tempty_bar + 8 * acc);
                     mbar_arrive(out_full + 8 * ob);
                 }
                 if (++ob == p.out_bufs) { ob = 0; ophase ^= 1; }
@@ -745,10 +794,11 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         } else {
             grid_dependency_wait();     // direct stores (and residual reads) from these warps
             const int tile_row = quarter * 32 + lane;   // this thread's row of the tile
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+            for (int tile = worker; ok && tile < total_tiles; tile += n_workers, ++local) {
                 const int acc = local & 1;
                 const uint32_t acc_phase = (local >> 1) & 1;
-                const int m_t = fast_div(tile, p.div_n_tiles), n_t = tile - m_t * p.n_tiles;
+                const int m_q = fast_div(tile, p.div_n_tiles), n_t = tile - m_q * p.n_tiles;
+            const int m_t = PAIR ? 2 * m_q + (int)cta_rank : m_q;
                 const int n0 = n_t * p.bn;
                 size_t row = (size_t)m_t * TILE_M + tile_row;
                 bool row_valid = row < (size_t)p.M;
@@ -780,9 +830,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 
     tc_fence_before();
     __syncthreads();
+    // a pair leaves together: the issuer's instructions read the partner's shared memory and tensor memory, and arrivals
+    // go to the partner's barriers
+    if (PAIR) cluster_sync_all();
     if (warp == MMA_WARP) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS);
+        else tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -976,11 +1030,22 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.div_wo = make_fast_div(g.wo);
     p.div_ho = make_fast_div(g.ho);
     p.a_bytes = (uint32_t)(TILE_M * p.kb + 1023) / 1024 * 1024;
-    const uint32_t b_bytes = (uint32_t)(p.bn * p.kb + 1023) / 1024 * 1024;
+    // CTA pairs for the K-heavy layers with 256-wide tiles, whose main loop is bound by the bytes a CTA has to pull
+    // through the L2 -> SM path per tensor-core cycle (48 KiB per 128-byte K chunk alone, 32 KiB in a pair: the weight
+    // tile is split between the two CTAs)
+    {
+        const unsigned off0 = f8_plan_options_off();
+        const size_t xb = (size_t)xv.dim_c * xv.dim_w * xv.dim_h * xv.dim_n;
+        p.pair = (staged && p.kb == 128 && g.c % 128 == 0 && p.bn == 256 && g.c_out % 256 == 0 &&
+                  g.kh * g.kw * ((g.c + p.kb - 1) / p.kb) >= 8 && xb >= 128 * 1024 && p.m_tiles >= 2 && !(off0 & F8_PLAN_OFF_PAIRS)) ? 1 : 0;
+    }
+    const int bn_load = p.pair ? p.bn / 2 : p.bn;        // rows of a weight tile one CTA loads
+    const uint32_t b_bytes = (uint32_t)(bn_load * p.kb + 1023) / 1024 * 1024;
     p.b_bytes = b_bytes;
     p.sub_bytes = p.a_bytes + b_bytes;
     p.tx_a = (uint32_t)(TILE_M * p.kb);
-    p.tx_b = (uint32_t)(p.bn * p.kb);
+    p.tx_b = (uint32_t)(bn_load * p.kb);
+    p.pair_tiles = ((p.m_tiles + 1) / 2) * p.n_tiles;
     size_t staging = 0;
     if (staged) {
         p.slab_w = p.bn < 128 ? p.bn : 128;
@@ -1010,7 +1075,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // 3x3 layer of 128 channels waits on every im2col load: measured 62 us against 48 us with streamed weights)
     const size_t b_all = (size_t)p.n_tiles * k_iters * b_bytes;
     const unsigned off = f8_plan_options_off();
-    p.b_res = (p.n_tiles == 1 && b_all + 4 * (size_t)p.a_bytes <= avail && b_all + 32 * 1024 <= avail &&
+    p.b_res = (!p.pair && p.n_tiles == 1 && b_all + 4 * (size_t)p.a_bytes <= avail && b_all + 32 * 1024 <= avail &&
                !(off & F8_PLAN_OFF_RESIDENT_WEIGHTS)) ? 1 : 0;
     if (p.b_res) {
         avail -= b_all;
@@ -1025,7 +1090,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // by the rate at which the tensor core accepts N = 64 instructions, about one per 90 cycles whoever issues them,
     // and whole-row tiles are 12.5 % more tiles).
     p.win = 0;
-    if (staged && p.kb == 128 && g.kh == 3 && g.kw == 3 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 1 && g.pad_w == 1 &&
+    if (staged && !p.pair && p.kb == 128 && g.kh == 3 && g.kw == 3 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 1 && g.pad_w == 1 &&
         g.pad_h_end < 0 && p.n_tiles == 1 && g.w + 2 <= TILE_M && g.w == g.wo && g.h == g.ho && g.c % p.kb == 0 &&
         !(off & (F8_PLAN_OFF_WINDOWED | F8_PLAN_OFF_RESIDENT_WEIGHTS))) {
         const int wp = g.w + 2;
@@ -1089,6 +1154,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     int group = (k_iters + uses - 1) / uses;
     while (group > 1 && avail / ((size_t)group * p.sub_bytes) < 2) --group;
     group = (k_iters + (k_iters + group - 1) / group - 1) / ((k_iters + group - 1) / group);   // same uses, evenly split
+    if (p.pair) group = 1;      // 32-KiB stage uses, as many stages in flight as fit
     p.group = group;
     p.stage_bytes = (uint32_t)group * p.sub_bytes;
     int stages = (int)(avail / p.stage_bytes);
@@ -1111,7 +1177,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // instruction descriptor: D = s32 (2 at bit 4), A format at bit 7 (0 = u8, 1 = s8), B = s8 at bit 10,
     // both operands K-major, N/8 at bit 17, M/16 at bit 24
     p.idesc = (2u << 4) | ((g.x_signed ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) |
-              ((uint32_t)(TILE_M >> 4) << 24);
+              ((uint32_t)((p.pair ? 2 * TILE_M : TILE_M) >> 4) << 24);
     p.desc_hi = smem_desc_hi(p.kb);
     p.bias = bias;
     p.res = (const uint8_t *)res;
@@ -1193,7 +1259,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     {
         cuuint64_t dims[3] = {(cuuint64_t)g.c, (cuuint64_t)(g.kh * g.kw), (cuuint64_t)g.c_out};
         cuuint64_t strides[2] = {(cuuint64_t)g.c, (cuuint64_t)g.c * g.kh * g.kw};
-        cuuint32_t box[3] = {(cuuint32_t)p.kb, 1, (cuuint32_t)p.bn};
+        cuuint32_t box[3] = {(cuuint32_t)p.kb, 1, (cuuint32_t)bn_load};
         cuuint32_t estr[3] = {1, 1, 1};
         CUresult r = g_encode_tiled(&plan->map_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t *>(w), dims,
                                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(p.kb),
@@ -1251,6 +1317,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int total_tiles = p.m_tiles * p.n_tiles;
     plan->grid = total_tiles < sms ? total_tiles : sms;
+    if (p.pair) plan->grid = 2 * std::min(p.pair_tiles, sms / 2);        // clusters of two; trimmed to what fits at launch
     // at least half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
     plan->smem = (size_t)p.stages * p.stage_bytes + staging + (p.b_res ? b_all : 0) + 1024 + CONTROL_BYTES;
     if (plan->smem < 120 * 1024) plan->smem = 120 * 1024;
@@ -1259,7 +1326,8 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     {
         int *info = f8_last_plan_info();
         info[0] = (p.b_res ? F8_PLAN_RESIDENT_WEIGHTS : 0) | (p.win ? F8_PLAN_WINDOWED : 0) | (p.dual_issue ? F8_PLAN_DUAL_ISSUE : 0) |
-                  (p.alt ? F8_PLAN_ALT_PRODUCERS : 0) | (p.a_plain ? F8_PLAN_PLAIN_MATRIX : 0) | (staged ? F8_PLAN_STAGED_EPILOGUE : 0) | (p.rowt ? F8_PLAN_ROW_TILES : 0);
+                  (p.alt ? F8_PLAN_ALT_PRODUCERS : 0) | (p.a_plain ? F8_PLAN_PLAIN_MATRIX : 0) | (staged ? F8_PLAN_STAGED_EPILOGUE : 0) | (p.rowt ? F8_PLAN_ROW_TILES : 0) |
+                  (p.pair ? F8_PLAN_PAIRS : 0);
         info[1] = p.epi; info[2] = p.bn; info[3] = p.kb; info[4] = p.stages; info[5] = p.group;
         info[6] = p.m_tiles; info[7] = p.n_tiles; info[8] = plan->grid; info[9] = staged ? p.out_bufs : 0;
     }
@@ -1271,11 +1339,15 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     }
     if (!attr_set[dev]) {
         const int bytes = (int)(SMEM_LIMIT + CONTROL_BYTES);
-        cudaError_t e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_GENERIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        cudaError_t e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_GENERIC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e != cudaSuccess) {
             *why = "cudaFuncSetAttribute(MaxDynamicSharedMemorySize) failed";
             return e;
@@ -1286,30 +1358,59 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
 }
 
 namespace {
-template <int EPI>
+template <int EPI, bool PAIR>
 cudaError_t launch_variant(const F8TcPlan *plan, bool overlap_previous, cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)plan->grid);
     cfg.blockDim = dim3(NUM_THREADS);
     cfg.dynamicSmemBytes = plan->smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (PAIR) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = 2;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (overlap_previous) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = overlap_previous ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, f8_conv_gemm_tc_kernel<EPI>, plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p);
+    cfg.numAttrs = n;
+    if (PAIR) {
+        // persistent pairs: no more clusters than the device can hold at once
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, f8_conv_gemm_tc_kernel<EPI, PAIR>, &cfg) == cudaSuccess && clusters > 0 &&
+            2 * clusters < plan->grid)
+            cfg.gridDim = dim3((unsigned)(2 * clusters));
+        else
+            (void)cudaGetLastError();
+    }
+    return cudaLaunchKernelEx(&cfg, f8_conv_gemm_tc_kernel<EPI, PAIR>, plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p);
 }
 }   // namespace
 
 cudaError_t f8_tc_launch(const F8TcPlan *plan, bool overlap_previous, cudaStream_t st) {
     if (plan->p.M == 0) return cudaSuccess;
+    if (plan->p.pair) {
+        switch (plan->p.epi) {
+            case EPI_U8: return launch_variant<EPI_U8, true>(plan, overlap_previous, st);
+            case EPI_U8_RES: return launch_variant<EPI_U8_RES, true>(plan, overlap_previous, st);
+            case EPI_S8: return launch_variant<EPI_S8, true>(plan, overlap_previous, st);
+            case EPI_S8_RES: return launch_variant<EPI_S8_RES, true>(plan, overlap_previous, st);
+            default: return cudaErrorInvalidValue;
+        }
+    }
     switch (plan->p.epi) {
-        case EPI_U8: return launch_variant<EPI_U8>(plan, overlap_previous, st);
-        case EPI_U8_RES: return launch_variant<EPI_U8_RES>(plan, overlap_previous, st);
-        case EPI_S8: return launch_variant<EPI_S8>(plan, overlap_previous, st);
-        case EPI_S8_RES: return launch_variant<EPI_S8_RES>(plan, overlap_previous, st);
-        default: return launch_variant<EPI_GENERIC>(plan, overlap_previous, st);
+        case EPI_U8: return launch_variant<EPI_U8, false>(plan, overlap_previous, st);
+        case EPI_U8_RES: return launch_variant<EPI_U8_RES, false>(plan, overlap_previous, st);
+        case EPI_S8: return launch_variant<EPI_S8, false>(plan, overlap_previous, st);
+        case EPI_S8_RES: return launch_variant<EPI_S8_RES, false>(plan, overlap_previous, st);
+        default: return launch_variant<EPI_GENERIC, false>(plan, overlap_previous, st);
     }
 }
 

@@ -237,6 +237,81 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
                  : "memory");
 }
 
+// ----------------------------------------------------------------------------- CTA pairs (tcgen05 cta_group::2)
+// Two CTAs of a cluster work on one 256-row tile: each holds its own 128 rows of A and half of the B tile in its shared
+// memory (same offsets in both), the even CTA issues the instructions, each tensor core accumulates its 128 rows in its own
+// tensor memory.  Loads of the odd CTA complete on the even CTA's barrier; commits arrive on the barriers of both.
+
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+}
+// arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar, uint32_t rank) {
+    asm volatile(
+        "{\n\t.reg .b32 remote;\n\t"
+        "mapa.shared::cluster.u32 remote, %0, %1;\n\t"
+        "mbarrier.arrive.shared::cluster.b64 _, [remote];\n\t}" ::"r"(bar), "r"(rank)
+        : "memory");
+}
+// the barrier at the same offset in the even CTA of the pair (the CTA rank is bit 24 of a shared-window address)
+__device__ __forceinline__ uint32_t pair_leader_bar(uint32_t bar) { return bar & 0xFEFFFFFFu; }
+
+__device__ __forceinline__ void tma_load_im2col_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w, int h,
+                                                     int n, uint16_t off_w, uint16_t off_h) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};" ::"r"(dst),
+        "l"(map), "r"(pair_leader_bar(bar)), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+        "l"(map), "r"(pair_leader_bar(bar)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(map), "r"(pair_leader_bar(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// arrives on the barrier at this offset in both CTAs of the pair once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                 "h"(both)
+                 : "memory");
+}
+// The K = 32 slices of one 128-byte sub-chunk (four of them) as 256-row instructions of the pair, from one asm block.
+#define F8_MMA_I8_PAIR "tcgen05.mma.cta_group::2.kind::i8 [%0], a, b, %4, {%6, %6, %6, %6, %6, %6, %6, %6}, "
+#define F8_MMA_NEXT_PAIR(off) \
+    "add.u32 x, %1, " #off ";\n\tadd.u32 y, %2, " #off ";\n\tmov.b64 a, {x, %3};\n\tmov.b64 b, {y, %3};\n\t" F8_MMA_I8_PAIR "t;\n\t"
+__device__ __forceinline__ void mma_i8_sub_pair4(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                                 uint32_t accumulate) {
+    const uint32_t zero = 0;      // no output lane is disabled
+    asm volatile("{\n\t.reg .pred p, t;\n\t.reg .b64 a, b;\n\t.reg .b32 x, y;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "setp.eq.b32 t, 0, 0;\n\tmov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t" F8_MMA_I8_PAIR "p;\n\t"
+                 F8_MMA_NEXT_PAIR(2) F8_MMA_NEXT_PAIR(4) F8_MMA_NEXT_PAIR(6) "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi),
+                 "r"(idesc), "r"(accumulate), "r"(zero)
+                 : "memory");
+}
+
 // 16 consecutive accumulator columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
     asm volatile(

@@ -162,6 +162,32 @@ def _modes():
     ]
 
 
+# CTA pairs (tcgen05 cta_group::2): K-heavy layers with 256-wide tiles; 256-row tiles shared by two CTAs
+# (h, w, c, c_out, k, stride, n, x_signed, y_dtype, res)
+PAIR_CASES = [
+    (14, 14, 1024, 256, 1, 1, 64, False, synth.U8, False),      # eight K chunks, 98 M tiles: 49 pair tiles
+    (14, 14, 512, 256, 3, 1, 33, True, synth.U8, False),        # 3x3 through im2col, signed input; 51 M tiles: the last pair is half empty
+    (7, 7, 512, 512, 3, 1, 64, True, synth.S8, False),          # two N tiles, 36 K iterations, signed
+    (14, 14, 1024, 2048, 1, 2, 40, False, synth.S8, False),     # stride-2 shortcut convolution, eight N tiles
+    (7, 7, 2048, 512, 1, 1, 256, False, synth.U8, False),       # 98 M tiles x 2 N tiles on 74 pairs: several tiles per pair
+    (9, 9, 1024, 256, 1, 1, 3, False, synth.U8, False),         # 243 pixels: one pair, second CTA nearly empty
+]
+
+
+@pytest.mark.parametrize("case", range(len(PAIR_CASES)))
+def test_cta_pairs(ref, case):
+    from paper_2202_05239_b200 import api as a
+    h, w, c, c_out, k, stride, n, xs, y_dtype, with_res = PAIR_CASES[case]
+    rng = np.random.default_rng(1200 + case)
+    layer = random_conv_layer(rng, h=h, w=w, c=c, c_out=c_out, k=k, stride=stride, pad=k // 2, x_signed=xs, y_dtype=y_dtype,
+                              with_res=with_res)
+    x = random_input(rng, n, layer)
+    res = random_residual(rng, n, layer) if with_res else None
+    check_layer(ref, layer, x, res, expect_tc=True, expect_flags=a.PLAN_PAIRS)
+    if case in (0, 2):      # the same layer on single CTAs
+        check_layer(ref, layer, x, res, expect_tc=True, plan_off=a.PLAN_OFF_PAIRS, forbid_flags=a.PLAN_PAIRS)
+
+
 @pytest.mark.parametrize("case", range(13))
 def test_many_tiles_per_cta_in_every_plan_mode(ref, case):
     h, w, c, c_out, k, stride, n, xs, y_dtype, with_res, off, expect, forbid = _modes()[case]
