@@ -12,7 +12,12 @@
  * ReLU / PACT clip, Eq. 4) or its signed form from the appendix (clip
  * [-127, 127]).  Because all formats are powers of two, the quantizer is a
  * rounding arithmetic shift by  s = FL_x + FL_w - FL_y  followed by the clip;
- * no int32 or floating-point multiplication is used for rescaling.
+ * no int32 or floating-point multiplication by a learned scale is needed for
+ * rescaling.  (Where an accumulator or a shortcut has to be moved to a finer
+ * format, the tensor-core epilogue does that left shift as a multiply-add with
+ * the power of two 2^shift, which this GPU executes on a less loaded pipe; the
+ * result is the shift's, bit for bit.  Building with -DF8_EPILOGUE_SHIFTS_ONLY
+ * uses shift instructions instead.)
  *
  * For one output element, with FA = FL_x + FL_w:
  *
@@ -39,7 +44,14 @@
  *     f8_device_status() reads.
  *   - Preconditions the library cannot check on device data: every accumulator
  *     (including the aligned residual sum) fits in int32.  f8_net_create checks
- *     this bound from the host copies of the parameters.
+ *     this bound from the host copies of the parameters.  The single-layer entry
+ *     points only see the shapes: they reject layers whose worst case
+ *     K * 255 * 128 * 2^sh_acc reaches 2^30 and otherwise rely on the caller for
+ *         |sum + bias| * 2^sh_acc + 255 * 2^sh_res + 2^(s-1) < 2^31
+ *     (sh_acc / sh_res: the alignment shifts of accumulator and residual, s the
+ *     requantisation shift): the fast epilogue adds the rounding constant 2^(s-1)
+ *     to the bias once per layer and forms this sum in int32; a bias beyond that
+ *     bound wraps silently.
  */
 #ifndef F8NET_H
 #define F8NET_H

@@ -1,6 +1,6 @@
 // Sibling layers with private fractional lengths (Sec. 4.3 "Clipping-Level Sharing", appendix "Private Fractional
 // Lengths"): a value that feeds several layers is kept in 32 bits and quantised once per consumer, each with its own
-// format -- "the cost is only some bit shifting".  This kernel takes the int32 tensor a layer produced (format fa,
+// format; the formats differ by powers of two, so each consumer's view costs a shift.  This kernel takes the int32 tensor a layer produced (format fa,
 // e.g. the F8_S32 output of a convolution) and emits one or two 8-bit tensors:
 //
 //     y_k = clip(rshift_round(acc, fa - fl_k), lo_k, hi_k)        k = 1, 2;   rshift_round = round half up

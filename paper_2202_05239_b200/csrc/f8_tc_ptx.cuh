@@ -367,12 +367,22 @@ __device__ __forceinline__ uint4 epilogue_fast16(const int (&acc)[16], uint32_t 
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const int j = 4 * g + k;
+#ifdef F8_EPILOGUE_SHIFTS_ONLY
+            // the letter of the method: alignment by shift instructions (the factors are powers of two)
+            int v = (acc[j] << (31 - __clz(mul_acc))) + bb[k];
+            if (RES) {
+                int r;
+                asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(rwords[g]), "r"(rsel[k]));
+                v += r << (31 - __clz(mul_res));
+            }
+#else
             int v = acc[j] * mul_acc + bb[k];
             if (RES) {
                 int r;
                 asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(rwords[g]), "r"(rsel[k]));
                 v += r * mul_res;
             }
+#endif
             v >>= s;
             t[j] = SIGNED_OUT ? max(v, -127) : v;
         }
