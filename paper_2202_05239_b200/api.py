@@ -9,7 +9,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from typing import List, Optional, Sequence
+from typing import Optional, Sequence
 
 import numpy as np
 import torch
@@ -282,15 +282,6 @@ def f8_debug_set_wait_limit_ms(ms: float):
 
 def f8_debug_wait_timeout_probe(limit_ms: float, stream=None):
     _check(_lib.f8_debug_wait_timeout_probe(limit_ms, _stream(stream)))
-
-
-def exported_symbols() -> List[str]:
-    return ["f8_conv2d_fixed", "f8_dwconv_fixed", "f8_linear_fixed", "f8_maxpool_fixed", "f8_global_avgpool_fixed",
-            "f8_conv_workspace_bytes", "f8_net_create", "f8_net_workspace_bytes", "f8_net_forward",
-            "f8_net_last_launch_count", "f8_net_set_profiling", "f8_net_get_layer_ms", "f8_net_destroy", "f8_status_str", "f8_last_error", "f8_device_status",
-            "f8_mma_i8_probe", "f8_stem_conv2d_fixed_static", "f8_fold_quantize_fixed", "f8_fold_workspace_bytes", "f8_format_study_fixed", "f8_format_study_workspace_bytes", "f8_requantize_dual_fixed",
-            "f8_tc_launch_count", "f8_debug_force_direct", "f8_debug_plan_options", "f8_debug_last_plan",
-            "f8_debug_set_wait_limit_ms", "f8_debug_wait_timeout_probe"]
 
 
 def layer_output_shape(layer: "synth.Layer", n: int):

@@ -273,6 +273,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const uint32_t out_full = smem_u32(&epi_bars[0]), out_free = smem_u32(&epi_bars[MAX_OUT_BUFS]);
     const uint32_t res_full = smem_u32(&epi_bars[2 * MAX_OUT_BUFS]);
 
+    if (threadIdx.x == 32) {
+        // the first copy through a tensor map otherwise pays for fetching the map itself, at the head of every layer
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+        if (STAGED) prefetch_tensormap(&map_y);
+        if (RES) prefetch_tensormap(&map_r);
+    }
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) {
@@ -300,13 +307,6 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int r = tap / p.kw, sx = tap - r * p.kw;
             ktab[i] = make_uint2((uint32_t)(cc * p.kb), ((uint32_t)tap << 16) | ((uint32_t)r << 8) | (uint32_t)sx);
         }
-    }
-    if (STAGED) {
-        // bias' = (bias << sh_acc) + 2^(s-1) for every (padded) output column, once per CTA
-        int *bias_all = (int *)(smem + p.bias_off);
-        const int rnd = 1 << (p.q.s - 1);
-        for (int i = threadIdx.x; i < p.n_tiles * p.bn; i += NUM_THREADS)
-            bias_all[i] = ((i < p.c_out && p.bias) ? (__ldg(p.bias + i) << p.q.sh_acc) : 0) + rnd;
     }
     if (warp == MMA_WARP) {
         if (PAIR) tmem_alloc_pair(smem_u32(&tmem_base_slot), TMEM_COLS);
@@ -730,6 +730,17 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         uint32_t ophase = 0;
         bool ok = true;
         if (STAGED) {
+            {
+                // bias' = (bias << sh_acc) + 2^(s-1) for every (padded) output column, once per CTA.  Only these warps
+                // read the table, so they build it -- behind a barrier of their own -- while the producers and the MMA
+                // issuers are already at work: the prologue of a CTA starts when the previous layer's CTA has left the SM,
+                // and a round trip to global memory there would be paid by every layer.
+                int *bias_all = (int *)(smem + p.bias_off);
+                const int rnd = 1 << (p.q.s - 1);
+                for (int i = (int)threadIdx.x - FIRST_EPI_WARP * 32; i < p.n_tiles * p.bn; i += NUM_EPI_WARPS * 32)
+                    bias_all[i] = ((i < p.c_out && p.bias) ? (__ldg(p.bias + i) << p.q.sh_acc) : 0) + rnd;
+                asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
+            }
             const int tile_row = quarter * 32 + lane;
             // PRMT selectors that turn byte k of a residual word into an int (zero- or sign-extended)
             uint32_t rsel[4];
