@@ -1098,8 +1098,9 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     // per tile and every filter tap reads them at a shifted row offset.  Worth it when whole rows fill most of a tile
     // and the im2col loads are what bounds the layer: measured, 128-channel layers gain 1.8x (the resident weights
     // leave room for two im2col stages only); 64-channel layers gain nothing (62 against 64 us: their tiles are bound
-    // by the rate at which the tensor core accepts N = 64 instructions, about one per 90 cycles whoever issues them,
-    // and whole-row tiles are 12.5 % more tiles).
+    // by the MMA-issuing threads, which need about 150 cycles per N = 64 instruction while the epilogue warps of their
+    // scheduler partition are busy -- an MMA-only loop issues one every 52 cycles -- and whole-row tiles are 12.5 % more
+    // tiles).
     p.win = 0;
     if (staged && !p.pair && p.kb == 128 && g.kh == 3 && g.kw == 3 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 1 && g.pad_w == 1 &&
         g.pad_h_end < 0 && p.n_tiles == 1 && g.w + 2 <= TILE_M && g.w == g.wo && g.h == g.ho && g.c % p.kb == 0 &&
