@@ -235,8 +235,9 @@ def shape_key(l) -> str:
 
 def measured_traffic(layers, tc_flags, batch):
     """DRAM bytes per step of the tensor-core conv kernel: per-launch counters of every distinct layer shape, captured
-    one launch at a time at a reduced batch (profiles/dram_traffic_conv_gemm_tc_shapes.md), scaled by the batch and
-    summed over the layers.  None when the kernel source has changed since, or a shape is missing."""
+    one single-layer launch at a time (profiles/dram_traffic_conv_gemm_tc_shapes.md; scaled by batch / capture batch
+    when the two differ) and summed over the layers.  None when the kernel source has changed since, or a shape is
+    missing."""
     try:
         text = open(os.path.join(ROOT, "profiles", "dram_traffic_conv_gemm_tc_shapes.md")).read()
         sha = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text).group(1)
@@ -550,9 +551,10 @@ def run_ours(args):
         "bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
         "peak_source": f"{peak_kind} HBM copy bandwidth",
         "traffic": measured_traffic(layers, tc_flags, BATCH),
-        "traffic_note": "DRAM bytes of this kernel's launches in one step: single-launch ncu counters per distinct layer shape at a "
-                        "reduced batch, scaled by the batch (profiles/dram_traffic_conv_gemm_tc_shapes.md); tensors that stay in "
-                        "L2 between two layers of a real step are not captured this way",
+        "traffic_note": "DRAM bytes of this kernel's launches in one step: ncu counters of one cold single-layer launch per distinct layer "
+                        "shape at the bench batch (profiles/dram_traffic_conv_gemm_tc_shapes.md), summed over the layers; tensors that "
+                        "stay in L2 between two layers of a real step, and lines still dirty in L2 when a launch ends, are not "
+                        "captured this way",
         "launches_per_step": n_tc, "kernel_ms_per_step": tc_ms, "kernel_ms_per_step_events": tc_ms / scale if scale > 0 else None,
         "event_sum_ms": event_sum, "event_to_step_scale": scale,
         "algorithmic_bytes_per_step": tc_bytes,

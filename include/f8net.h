@@ -40,8 +40,12 @@
  *   - Errors are reported by the return code; nothing is launched when validation
  *     fails.  f8_last_error() gives a message for the calling thread's last
  *     failure.  Kernels never trap: a wait that does not complete within its
- *     bound makes the kernel return early and sets a device status word that
- *     f8_device_status() reads.
+ *     bound makes the kernel return early (its output is then incomplete) and
+ *     records itself in a device status word and in a host-visible copy of it.
+ *     Every entry point that enqueues work looks at that copy first (a host
+ *     load, no synchronisation) and returns F8_ERR_TIMEOUT without enqueuing
+ *     anything while a record is pending; f8_device_status() synchronises,
+ *     reports the details and clears it.
  *   - Preconditions the library cannot check on device data: every accumulator
  *     (including the aligned residual sum) fits in int32.  f8_net_create checks
  *     this bound from the host copies of the parameters.  The single-layer entry

@@ -216,6 +216,15 @@ int f8_status_host_code() {
     return *g_status_host[dev];
 }
 
+// A kernel that gives up a bounded wait also stores its code to a host-visible word.  Every entry point that enqueues work
+// looks at it first (a plain host load, no synchronisation), so an incomplete earlier result is reported by the next call.
+static f8_status pending_timeout() {
+    if (const int v = f8_status_host_code())
+        return fail(F8_ERR_TIMEOUT, "a kernel abandoned a bounded wait (site %d, layer %d): the output of that launch is incomplete; "
+                    "f8_device_status() gives the details and clears the record", v & 0xff, (v >> 8) - 1);
+    return F8_OK;
+}
+
 extern "C" {
 
 const char *f8_status_str(f8_status s) {
@@ -309,6 +318,7 @@ f8_status f8_conv2d_fixed(const f8_conv_desc *desc, const void *x, const int8_t 
     if (!x || !w || !y) return fail(F8_ERR_NULL, "x, w and y must not be NULL");
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(residual) || !aligned16(bias))
         return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    if (pending_timeout() != F8_OK) return F8_ERR_TIMEOUT;
     return run_dense(g, q, x, w, bias, residual, y, (cudaStream_t)cuda_stream);
 }
 
@@ -328,6 +338,7 @@ f8_status f8_conv2d_siblings_fixed(const f8_conv_desc *desc, int y2_dtype, int f
     if (!x || !w || !y) return fail(F8_ERR_NULL, "x, w and y must not be NULL");
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(y2) || !aligned16(residual) || !aligned16(bias))
         return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    if (pending_timeout() != F8_OK) return F8_ERR_TIMEOUT;
     return run_dense(g, q, x, w, bias, residual, y, (cudaStream_t)cuda_stream, y2 ? &sib : nullptr);
 }
 
@@ -341,6 +352,7 @@ f8_status f8_dwconv_fixed(const f8_conv_desc *desc, const void *x, const int8_t 
     if (!x || !w || !y) return fail(F8_ERR_NULL, "x, w and y must not be NULL");
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(residual) || !aligned16(bias))
         return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    if (pending_timeout() != F8_OK) return F8_ERR_TIMEOUT;
     cudaError_t e = f8_launch_dwconv(g, q, x, w, bias, residual, y, (cudaStream_t)cuda_stream);
     if (e != cudaSuccess) return cuda_fail(e, "depthwise launch");
     return F8_OK;
@@ -364,6 +376,7 @@ f8_status f8_maxpool_fixed(int n, int h, int w, int c, int k, int stride, int pa
     if (n == 0) return F8_OK;
     if (!x || !y) return fail(F8_ERR_NULL, "x and y must not be NULL");
     if (!aligned16(x) || !aligned16(y)) return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    if (pending_timeout() != F8_OK) return F8_ERR_TIMEOUT;
     cudaError_t e = f8_launch_maxpool(n, h, w, c, k, stride, pad, x_dtype == F8_S8, x, y, (cudaStream_t)cuda_stream);
     if (e != cudaSuccess) return cuda_fail(e, "max-pool launch");
     return F8_OK;
@@ -380,6 +393,7 @@ f8_status f8_global_avgpool_fixed(int n, int h, int w, int c, int x_dtype, int f
     if (n == 0) return F8_OK;
     if (!x || !y) return fail(F8_ERR_NULL, "x and y must not be NULL");
     if (!aligned16(x) || !aligned16(y)) return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    if (pending_timeout() != F8_OK) return F8_ERR_TIMEOUT;
     cudaError_t e = f8_launch_gap(n, h, w, c, x_dtype == F8_S8, s, x, y, (cudaStream_t)cuda_stream);
     if (e != cudaSuccess) return cuda_fail(e, "global-average-pool launch");
     return F8_OK;
@@ -986,9 +1000,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
     const int nl = (int)net->layers.size();
     // A kernel that gives up a bounded wait also stores its code to a host-visible word: an earlier pass (or anything
     // else on this device) that left its output incomplete is reported here, without a synchronisation.
-    if (const int v = f8_status_host_code())
-        return fail(F8_ERR_TIMEOUT, "a kernel abandoned a bounded wait (site %d, layer %d): the output of that pass is incomplete; "
-                    "f8_device_status() gives the details and clears the record", v & 0xff, (v >> 8) - 1);
+    if (pending_timeout() != F8_OK) return F8_ERR_TIMEOUT;
 
     // a first layer whose output is asked for cannot be fused with the pooling layer behind it
     bool dump_fusable = false;

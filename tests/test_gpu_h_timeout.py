@@ -17,14 +17,20 @@ def test_a_wait_that_runs_out_is_reported_and_the_device_stays_usable(ref):
     a.f8_device_status()                                  # clean to begin with
     a.f8_debug_wait_timeout_probe(1.0)
     torch.cuda.synchronize()                              # the kernel returned by itself
+    rng = np.random.default_rng(1)
+    layer = random_conv_layer(rng, h=28, w=28, c=128, c_out=128, k=1, stride=1, pad=0, x_signed=False, y_dtype=synth.U8,
+                              with_res=False)
+    # while the record is pending, a call that would enqueue work reports it instead (no synchronisation involved)
+    x = a.to_device(random_input(rng, 2, layer))
+    y = torch.empty((2, layer.ho, layer.wo, layer.c_out), dtype=torch.uint8, device="cuda")
+    with pytest.raises(a.F8Error) as e:
+        a.f8_conv2d_fixed(a.conv_desc(layer, 2), x, a.to_device(layer.weight), a.to_device(layer.bias), None, y)
+    assert e.value.status == 11
     with pytest.raises(a.F8Error) as e:
         a.f8_device_status()
     assert e.value.status == 11                           # F8_ERR_TIMEOUT
     assert "site 199" in str(e.value)
     a.f8_device_status()                                  # reading the word cleared it
-    rng = np.random.default_rng(1)
-    layer = random_conv_layer(rng, h=28, w=28, c=128, c_out=128, k=1, stride=1, pad=0, x_signed=False, y_dtype=synth.U8,
-                              with_res=False)
     check_layer(ref, layer, random_input(rng, 2, layer), expect_tc=True)
 
 
