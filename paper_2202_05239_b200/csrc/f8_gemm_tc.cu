@@ -101,6 +101,8 @@ struct TcParams {
     int pair_tiles;           // 256-row tiles x N tiles
     int alt;                  // 1: two pairs of producer warps, pair h takes the stage uses of parity h (streamed weights,
                               // one MMA issuer: fills may then complete out of order, the consumer is in order)
+    int epi_groups;           // 1, 2 or 4: the tile's columns are split over this many groups of four epilogue warps (one warp per
+                              // tensor-memory lane quarter); the warps of the other groups stay out of the tile loop
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
     uint32_t stage_bytes;     // group * sub_bytes
     uint32_t a_bytes;         // bytes of the A part (rounded to 1024)
@@ -289,10 +291,10 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         mbar_init(bres_bar, 1);
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
-            mbar_init(tempty_bar + 8 * a, PAIR ? 2 * NUM_EPI_WARPS : NUM_EPI_WARPS);     // the epilogue warps of both CTAs
+            mbar_init(tempty_bar + 8 * a, (PAIR ? 8 : 4) * p.epi_groups);     // the active epilogue warps (of both CTAs)
         }
         for (int a = 0; a < MAX_OUT_BUFS; ++a) {
-            mbar_init(out_full + 8 * a, NUM_EPI_WARPS);   // every epilogue warp has written its part of the tile
+            mbar_init(out_full + 8 * a, 4 * p.epi_groups);   // every active epilogue warp has written its part of the tile
             mbar_init(out_free + 8 * a, 1);               // the store has finished reading the tile
             mbar_init(res_full + 8 * a, 1);               // the residual tile has landed in the buffer (transaction count)
         }
@@ -721,7 +723,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const int ew = warp - FIRST_EPI_WARP;
         const int group = ew >> 2;                  // which quarter of the tile's columns this warp converts
         const int chunks = p.bn / 16;
-        const int per_group = (chunks + 3) / 4;     // <= 4 chunks of 16 columns per warp
+        const int per_group = (chunks + p.epi_groups - 1) / p.epi_groups;     // <= 4 chunks of 16 columns per warp
         const int ch_begin = min(group * per_group, chunks);
         const int nch = min(ch_begin + per_group, chunks) - ch_begin;
         const int mul_acc = p.mul_acc, mul_res = p.mul_res;     // 2^sh_acc, 2^sh_res
@@ -742,6 +744,9 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
             }
             const int tile_row = quarter * 32 + lane;
+            // Narrow tiles are converted by fewer warps: the MMA-issuing threads share their scheduler partitions with the
+            // epilogue warps, and every warp that is ready to issue slows them down.
+            const int my_tiles_end = group < p.epi_groups ? total_tiles : 0;
             // PRMT selectors that turn byte k of a residual word into an int (zero- or sign-extended)
             uint32_t rsel[4];
 #pragma unroll
@@ -755,7 +760,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 off ^= ((off >> 7) & p.swz_mask) << 4;
                 so[i] = (uint32_t)(ch / p.slab_chunks) * (TILE_M * p.slab_w) + off;
             }
-            for (int tile = worker; tile < total_tiles; tile += n_workers, ++local) {
+            for (int tile = worker; tile < my_tiles_end; tile += n_workers, ++local) {
                 const int acc = local & 1;                   // accumulator, output buffer and residual buffer in use
                 const uint32_t acc_phase = (local >> 1) & 1;
                 const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
@@ -1006,6 +1011,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     }
     memset(plan, 0, sizeof(*plan));
     TcParams &p = plan->p;
+    p.epi_groups = 4;
     p.M = g.n * g.ho * g.wo;
     p.ho = g.ho;
     p.wo = g.wo;
@@ -1069,6 +1075,9 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         // before.  With a residual a buffer goes through load -> convert in place -> store, and a residual tile takes
         // about as long to arrive from HBM as a tile takes to compute: three buffers (four when they are small).
         p.out_bufs = !q.has_res ? 2 : (p.out_bytes <= 16 * 1024 ? 4 : 3);
+        // 64-wide tiles: eight epilogue warps (two chunks each) instead of sixteen -- measured, 3x3 64 -> 64 at 56 x 56 61 -> 57 us
+        // (one warp per quarter: the same); 128-wide tiles show no difference and keep all sixteen
+        p.epi_groups = p.bn <= 64 ? 2 : 4;
         staging = (size_t)p.out_bytes * p.out_bufs + bias_bytes;
     }
     const size_t ktab_bytes = ((size_t)g.kh * g.kw * p.c_chunks * 8 + 1023) / 1024 * 1024;
