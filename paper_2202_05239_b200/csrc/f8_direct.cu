@@ -454,15 +454,39 @@ __device__ __forceinline__ void dw_dp4a_accumulate(const uint32_t (&t)[4], const
 // loads into registers, one row ahead, the kernel was bound by memory latency at a quarter of the HBM bandwidth).
 constexpr int DW_AHEAD = 8;
 
-__device__ __forceinline__ void cp_async4_zfill(uint32_t dst, const void *src, bool valid) {
-    // 4-byte asynchronous copy global -> shared; with a source size of 0 nothing is read and zeros are written
-    const int bytes = valid ? 4 : 0;
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+// four saturated bytes (channels 0..3 of one output pixel) from four sums that still carry the rounding constant
+template <bool SIGNED_OUT>
+__device__ __forceinline__ uint32_t dw_pack4(const int (&a)[4], int s) {
+    int tv[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int vv = a[j] >> s;
+        tv[j] = SIGNED_OUT ? max(vv, -127) : vv;
+    }
+    uint32_t hi2, word;
+    if (SIGNED_OUT) {
+        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+    } else {
+        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
+        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
+    }
+    return word;
+}
+
+// Addresses are 32-bit offsets that advance by a row per step (tensors on this path are below 2 GiB): with the offsets
+// recomputed from the row index for every copy and every store, address arithmetic was more than a third of the
+// instructions of a kernel that is bound by instruction issue.
 template <bool XS, bool SIGNED_OUT>
 __global__ void __launch_bounds__(128) dwconv3x3_dp4a_kernel(F8ConvGeom g, F8Requant q, const uint8_t *__restrict__ x,
                                                              const int8_t *__restrict__ w,
@@ -470,8 +494,10 @@ __global__ void __launch_bounds__(128) dwconv3x3_dp4a_kernel(F8ConvGeom g, F8Req
                                                              int strips, int bands, int band_rows, int total) {
     grid_dependency_sync();
     __shared__ uint32_t ring[DW_AHEAD][4][128];          // [row slot][column][thread]: a thread only touches its own words
+    constexpr uint32_t SLOT_BYTES = 4 * 128 * 4, RING_BYTES = DW_AHEAD * SLOT_BYTES;
     const uint32_t ring_base = (uint32_t)__cvta_generic_to_shared(&ring[0][0][threadIdx.x]);
     const int c4 = g.c >> 2;
+    const uint32_t row_stride = (uint32_t)(g.w * g.c), out_stride = (uint32_t)(g.wo * g.c);
     for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
         const int cg = idx % c4;
         int tt = idx / c4;
@@ -503,32 +529,46 @@ __global__ void __launch_bounds__(128) dwconv3x3_dp4a_kernel(F8ConvGeom g, F8Req
 #pragma unroll
                 for (int j = 0; j < 4; ++j) acc[a][o][j] = bb[j];
         const int iw0 = ow0 - 1;
-        bool col_ok[4];
-        int col_off[4];                     // byte offset of the column inside a row (0 for columns outside the image)
+        uint32_t col_off[4];                // byte offset of the column inside a row (0 for columns outside the image)
+        int col_bytes[4];                   // 4, or 0 for a column outside the image (the copy then writes zeros)
 #pragma unroll
         for (int xx = 0; xx < 4; ++xx) {
-            col_ok[xx] = iw0 + xx >= 0 && iw0 + xx < g.w;
-            col_off[xx] = col_ok[xx] ? (iw0 + xx) * g.c : 0;
+            const bool ok = (unsigned)(iw0 + xx) < (unsigned)g.w;
+            col_off[xx] = ok ? (uint32_t)(iw0 + xx) * (uint32_t)g.c : 0u;
+            col_bytes[xx] = ok ? 4 : 0;
         }
-        const int row_stride = g.w * g.c;
-        const uint8_t *img = x + (size_t)in * g.h * row_stride + c0;
+        const uint32_t img_off = (uint32_t)in * (uint32_t)g.h * row_stride + (uint32_t)c0;
+        const bool right_ok = ow0 + 1 < g.wo;
 
-        // request input row ih into ring slot `slot` (rows / columns outside the image: zeros)
-        auto request_row = [&](int ih, int slot) {
-            const bool row_ok = ih >= 0 && ih < g.h;
-            const uint8_t *rp = img + (size_t)(row_ok ? ih : 0) * row_stride;
+        // input rows oh0 - 1 .. oh1 are requested in order, DW_AHEAD rows ahead of their use (rows outside the image and
+        // requests past the band are zero fills that keep the group count regular)
+        int req_ih = oh0 - 1;
+        uint32_t req_off = img_off + (uint32_t)req_ih * row_stride;       // (wraps for row -1: used only for rows inside)
+        uint32_t req_slot = 0;                                            // byte offset of the ring slot
+        auto request_next = [&]() {
+            const bool row_ok = (unsigned)req_ih < (unsigned)g.h && req_ih <= oh1;
+            const uint32_t off = row_ok ? req_off : img_off;
 #pragma unroll
-            for (int xx = 0; xx < 4; ++xx)
-                cp_async4_zfill(ring_base + (uint32_t)((slot * 4 + xx) * 128 * 4), rp + col_off[xx], row_ok && col_ok[xx]);
+            for (int xx = 0; xx < 4; ++xx) {
+                const int bytes = row_ok ? col_bytes[xx] : 0;
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(ring_base + req_slot + (uint32_t)xx * 512u),
+                             "l"(x + (off + col_off[xx])), "r"(bytes)
+                             : "memory");
+            }
             cp_async_commit();
+            ++req_ih;
+            req_off += row_stride;
+            req_slot = (req_slot + SLOT_BYTES) & (RING_BYTES - 1);
         };
         // the four words of the oldest requested row, transposed: words of four channels per column -> words of four
         // columns per channel
-        auto take_row = [&](int slot, uint32_t (&t)[4]) {
+        uint32_t take_slot = 0;
+        auto take_row = [&](uint32_t (&t)[4]) {
             cp_async_wait<DW_AHEAD - 1>();
             uint32_t cw[4];
 #pragma unroll
-            for (int xx = 0; xx < 4; ++xx) cw[xx] = ring[slot][xx][threadIdx.x];
+            for (int xx = 0; xx < 4; ++xx) cw[xx] = lds32(ring_base + take_slot + (uint32_t)xx * 512u);
+            take_slot = (take_slot + SLOT_BYTES) & (RING_BYTES - 1);
             const uint32_t lo01 = __byte_perm(cw[0], cw[1], 0x5140), hi01 = __byte_perm(cw[0], cw[1], 0x7362);
             const uint32_t lo23 = __byte_perm(cw[2], cw[3], 0x5140), hi23 = __byte_perm(cw[2], cw[3], 0x7362);
             t[0] = __byte_perm(lo01, lo23, 0x5410);
@@ -536,58 +576,39 @@ __global__ void __launch_bounds__(128) dwconv3x3_dp4a_kernel(F8ConvGeom g, F8Req
             t[2] = __byte_perm(hi01, hi23, 0x5410);
             t[3] = __byte_perm(hi01, hi23, 0x7632);
         };
-        auto emit = [&](int oh, int (&a)[2][4]) {
-            if (oh >= oh0 && oh < oh1) {
-                uint8_t *out = y + ((size_t)(in * g.ho + oh) * g.wo + ow0) * g.c + c0;
-#pragma unroll
-                for (int o = 0; o < 2; ++o) {
-                    if (ow0 + o < g.wo) {
-                        int tv[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int vv = a[o][j] >> q.s;
-                            tv[j] = SIGNED_OUT ? max(vv, -127) : vv;
-                        }
-                        uint32_t hi2, word;
-                        if (SIGNED_OUT) {
-                            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
-                            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
-                        } else {
-                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
-                            asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
-                        }
-                        *(uint32_t *)(out + o * g.c) = word;
-                    }
-                }
+        // output rows leave in order, starting two rows above the band (those two belong to the band above)
+        int emit_left = -2;                                               // rows until the first one of this band
+        uint32_t out_off = ((uint32_t)(in * g.ho + oh0) * (uint32_t)g.wo + (uint32_t)ow0) * (uint32_t)g.c + (uint32_t)c0;
+        auto emit = [&](int (&a)[2][4]) {
+            if (emit_left >= 0) {
+                *(uint32_t *)(y + out_off) = dw_pack4<SIGNED_OUT>(a[0], q.s);
+                if (right_ok) *(uint32_t *)(y + out_off + (uint32_t)g.c) = dw_pack4<SIGNED_OUT>(a[1], q.s);
+                out_off += out_stride;
             }
+            ++emit_left;
         };
 
-        // input rows oh0 - 1 .. oh1; DW_AHEAD rows are on their way at any time (requests past the band are zero fills that
-        // nobody reads: they keep the group count regular); three rows per trip so that the accumulator slots are
-        // compile-time
-        const int first = oh0 - 1;
+        static_assert((RING_BYTES & (RING_BYTES - 1)) == 0, "ring size must be a power of two");
 #pragma unroll
-        for (int d = 0; d < DW_AHEAD; ++d) request_row(first + d, d);
-        int ih = first, slot = 0;
+        for (int d = 0; d < DW_AHEAD; ++d) request_next();
+        int ih = oh0 - 1;
         uint32_t t[4];
+        // three rows per trip so that the accumulator slots are compile-time; output row ih - 1 closes with input row ih
         while (ih <= oh1) {
-            take_row(slot, t);
-            request_row(ih + DW_AHEAD <= oh1 ? ih + DW_AHEAD : -1, slot);
-            slot = (slot + 1) & (DW_AHEAD - 1);
+            take_row(t);
+            request_next();
             dw_dp4a_accumulate<0, XS>(t, wa, bb, acc);
-            emit(ih - 1, acc[2]);
+            emit(acc[2]);
             if (++ih > oh1) break;
-            take_row(slot, t);
-            request_row(ih + DW_AHEAD <= oh1 ? ih + DW_AHEAD : -1, slot);
-            slot = (slot + 1) & (DW_AHEAD - 1);
+            take_row(t);
+            request_next();
             dw_dp4a_accumulate<1, XS>(t, wa, bb, acc);
-            emit(ih - 1, acc[0]);
+            emit(acc[0]);
             if (++ih > oh1) break;
-            take_row(slot, t);
-            request_row(ih + DW_AHEAD <= oh1 ? ih + DW_AHEAD : -1, slot);
-            slot = (slot + 1) & (DW_AHEAD - 1);
+            take_row(t);
+            request_next();
             dw_dp4a_accumulate<2, XS>(t, wa, bb, acc);
-            emit(ih - 1, acc[1]);
+            emit(acc[1]);
             ++ih;
         }
         cp_async_wait<0>();          // nothing of this item is in flight when the ring is reused for the next one
@@ -605,8 +626,10 @@ __global__ void __launch_bounds__(128) dwconv3x3s2_dp4a_kernel(F8ConvGeom g, F8R
                                                                int strips, int bands, int band_rows, int total) {
     grid_dependency_sync();
     __shared__ uint32_t ring[DW_AHEAD][5][128];
+    constexpr uint32_t SLOT_BYTES = 5 * 128 * 4;
     const uint32_t ring_base = (uint32_t)__cvta_generic_to_shared(&ring[0][0][threadIdx.x]);
     const int c4 = g.c >> 2;
+    const uint32_t row_stride = (uint32_t)(g.w * g.c), out_stride = (uint32_t)(g.wo * g.c);
     for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
         const int cg = idx % c4;
         int tt = idx / c4;
@@ -630,31 +653,48 @@ __global__ void __launch_bounds__(128) dwconv3x3s2_dp4a_kernel(F8ConvGeom g, F8R
         const int rnd = 1 << (q.s - 1);
         const int bb[4] = {b.x + rnd, b.y + rnd, b.z + rnd, b.w + rnd};
         const int iw0 = 2 * ow0 - 1;
-        bool col_ok[5];
-        int col_off[5];
+        uint32_t col_off[5];
+        int col_bytes[5];
 #pragma unroll
         for (int xx = 0; xx < 5; ++xx) {
-            col_ok[xx] = iw0 + xx >= 0 && iw0 + xx < g.w;
-            col_off[xx] = col_ok[xx] ? (iw0 + xx) * g.c : 0;
+            const bool ok = (unsigned)(iw0 + xx) < (unsigned)g.w;
+            col_off[xx] = ok ? (uint32_t)(iw0 + xx) * (uint32_t)g.c : 0u;
+            col_bytes[xx] = ok ? 4 : 0;
         }
-        const int row_stride = g.w * g.c;
-        const uint8_t *img = x + (size_t)in * g.h * row_stride + c0;
+        const uint32_t img_off = (uint32_t)in * (uint32_t)g.h * row_stride + (uint32_t)c0;
         const int last_row = 2 * (oh1 - 1) + 1;            // last input row of the band
+        const bool right_ok = ow0 + 1 < g.wo;
 
-        auto request_row = [&](int ih, int slot) {
-            const bool row_ok = ih >= 0 && ih < g.h && ih <= last_row;
-            const uint8_t *rp = img + (size_t)(row_ok ? ih : 0) * row_stride;
+        // input rows 2 oh0 - 1 .. last_row, requested in order DW_AHEAD rows ahead of their use (32-bit offsets that advance
+        // by a row per request; rows outside the image or past the band are zero fills)
+        int req_ih = 2 * oh0 - 1;
+        uint32_t req_off = img_off + (uint32_t)req_ih * row_stride;
+        int req_slot = 0;
+        auto request_next = [&]() {
+            const bool row_ok = (unsigned)req_ih < (unsigned)g.h && req_ih <= last_row;
+            const uint32_t off = row_ok ? req_off : img_off;
+            const uint32_t dst = ring_base + (uint32_t)req_slot * SLOT_BYTES;
 #pragma unroll
-            for (int xx = 0; xx < 5; ++xx)
-                cp_async4_zfill(ring_base + (uint32_t)((slot * 5 + xx) * 128 * 4), rp + col_off[xx], row_ok && col_ok[xx]);
+            for (int xx = 0; xx < 5; ++xx) {
+                const int bytes = row_ok ? col_bytes[xx] : 0;
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst + (uint32_t)xx * 512u),
+                             "l"(x + (off + col_off[xx])), "r"(bytes)
+                             : "memory");
+            }
             cp_async_commit();
+            ++req_ih;
+            req_off += row_stride;
+            req_slot = (req_slot + 1) & (DW_AHEAD - 1);
         };
         // ta[j]: columns 0..3 of channel j (the left output reads bytes 0..2); tb[j]: columns 2, 3, 4 (the right output)
-        auto take_row = [&](int slot, uint32_t (&ta)[4], uint32_t (&tb)[4]) {
+        int take_slot = 0;
+        auto take_row = [&](uint32_t (&ta)[4], uint32_t (&tb)[4]) {
             cp_async_wait<DW_AHEAD - 1>();
+            const uint32_t src = ring_base + (uint32_t)take_slot * SLOT_BYTES;
+            take_slot = (take_slot + 1) & (DW_AHEAD - 1);
             uint32_t cw[5];
 #pragma unroll
-            for (int xx = 0; xx < 5; ++xx) cw[xx] = ring[slot][xx][threadIdx.x];
+            for (int xx = 0; xx < 5; ++xx) cw[xx] = lds32(src + (uint32_t)xx * 512u);
             const uint32_t lo01 = __byte_perm(cw[0], cw[1], 0x5140), hi01 = __byte_perm(cw[0], cw[1], 0x7362);
             const uint32_t lo23 = __byte_perm(cw[2], cw[3], 0x5140), hi23 = __byte_perm(cw[2], cw[3], 0x7362);
             ta[0] = __byte_perm(lo01, lo23, 0x5410);
@@ -666,64 +706,41 @@ __global__ void __launch_bounds__(128) dwconv3x3s2_dp4a_kernel(F8ConvGeom g, F8R
             tb[2] = __byte_perm(hi23, cw[4], 0x6610);
             tb[3] = __byte_perm(hi23, cw[4], 0x7732);
         };
-        auto emit = [&](int oh, const int (&a)[2][4]) {
-            uint8_t *out = y + ((size_t)(in * g.ho + oh) * g.wo + ow0) * g.c + c0;
-#pragma unroll
-            for (int o = 0; o < 2; ++o) {
-                if (ow0 + o < g.wo) {
-                    int tv[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int vv = a[o][j] >> q.s;
-                        tv[j] = SIGNED_OUT ? max(vv, -127) : vv;
-                    }
-                    uint32_t hi2, word;
-                    if (SIGNED_OUT) {
-                        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
-                        asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
-                    } else {
-                        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, 0;" : "=r"(hi2) : "r"(tv[3]), "r"(tv[2]));
-                        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(tv[1]), "r"(tv[0]), "r"(hi2));
-                    }
-                    *(uint32_t *)(out + o * g.c) = word;
-                }
-            }
+        uint32_t out_off = ((uint32_t)(in * g.ho + oh0) * (uint32_t)g.wo + (uint32_t)ow0) * (uint32_t)g.c + (uint32_t)c0;
+        auto emit = [&](const int (&a)[2][4]) {
+            *(uint32_t *)(y + out_off) = dw_pack4<SIGNED_OUT>(a[0], q.s);
+            if (right_ok) *(uint32_t *)(y + out_off + (uint32_t)g.c) = dw_pack4<SIGNED_OUT>(a[1], q.s);
+            out_off += out_stride;
         };
 
-        const int first = 2 * oh0 - 1;
 #pragma unroll
-        for (int d = 0; d < DW_AHEAD; ++d) request_row(first + d, d);
-        int slot = 0, ih = first;
+        for (int d = 0; d < DW_AHEAD; ++d) request_next();
         int acc[2][4];
         uint32_t ta[4], tb[4];
         // the row above the band opens the first output row
-        take_row(slot, ta, tb);
-        request_row(ih + DW_AHEAD, slot);
-        slot = (slot + 1) & (DW_AHEAD - 1);
+        take_row(ta, tb);
+        request_next();
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             acc[0][j] = dw_dot4<XS>(ta[j], wr[0][j], bb[j]);
             acc[1][j] = dw_dot4<XS>(tb[j], wr[0][j], bb[j]);
         }
         for (int oh = oh0; oh < oh1; ++oh) {
-            ih = 2 * oh;
-            take_row(slot, ta, tb);                         // the middle filter row
-            request_row(ih + DW_AHEAD, slot);
-            slot = (slot + 1) & (DW_AHEAD - 1);
+            take_row(ta, tb);                               // the middle filter row
+            request_next();
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 acc[0][j] = dw_dot4<XS>(ta[j], wr[1][j], acc[0][j]);
                 acc[1][j] = dw_dot4<XS>(tb[j], wr[1][j], acc[1][j]);
             }
-            take_row(slot, ta, tb);                         // the bottom filter row of this output row, the top one of the next
-            request_row(ih + 1 + DW_AHEAD, slot);
-            slot = (slot + 1) & (DW_AHEAD - 1);
+            take_row(ta, tb);                               // the bottom filter row of this output row, the top one of the next
+            request_next();
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 acc[0][j] = dw_dot4<XS>(ta[j], wr[2][j], acc[0][j]);
                 acc[1][j] = dw_dot4<XS>(tb[j], wr[2][j], acc[1][j]);
             }
-            emit(oh, acc);
+            emit(acc);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 acc[0][j] = dw_dot4<XS>(ta[j], wr[0][j], bb[j]);
