@@ -1025,14 +1025,17 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     p.kb = choose_kb(g.c);
     // residual layers are bound by the epilogue, not by the main loop: prefer 64-byte K chunks so that a
     // 256-wide tile (half the tiles, half the A re-reads) still leaves room for the pipeline stages
-    if (q.has_res && g.c_out > 128 && p.kb == 128 && g.c <= 256) p.kb = 64;
+    // (not the K-heavy ones -- a 3x3 layer with a shortcut, as in basic residual blocks: those keep 128-byte chunks and
+    // 256-wide tiles, which makes them CTA pairs; the three 32-KiB buffers of the output ring leave three 32-KiB stages)
+    const bool k_heavy_res = q.has_res && g.c % 128 == 0 && g.c_out % 256 == 0 && g.kh * g.kw * (g.c / 128) >= 8;
+    if (q.has_res && g.c_out > 128 && p.kb == 128 && g.c <= 256 && !k_heavy_res) p.kb = 64;
     p.c_chunks = (g.c + p.kb - 1) / p.kb;
     p.epi = EPI_GENERIC;
     const bool has_sib = sib && sib->y2;
     if ((q.y_kind == F8_U8 || q.y_kind == F8_S8) && q.s >= 1 && q.s <= 24 && g.c_out % 16 == 0 && !has_sib && !q.r_s32)
         p.epi = q.y_kind == F8_U8 ? (q.has_res ? EPI_U8_RES : EPI_U8) : (q.has_res ? EPI_S8_RES : EPI_S8);
     const bool staged = p.epi != EPI_GENERIC;
-    p.bn = staged ? choose_bn_staged(g.c_out, q.has_res != 0, p.kb) : choose_bn(g.c_out);
+    p.bn = staged ? (k_heavy_res ? 256 : choose_bn_staged(g.c_out, q.has_res != 0, p.kb)) : choose_bn(g.c_out);
     p.m_tiles = (p.M + TILE_M - 1) / TILE_M;
     if (!staged) {
         // few output pixels (a fully connected layer): narrower N tiles until every SM has one, the weights are

@@ -171,6 +171,9 @@ PAIR_CASES = [
     (14, 14, 1024, 2048, 1, 2, 40, False, synth.S8, False),     # stride-2 shortcut convolution, eight N tiles
     (7, 7, 2048, 512, 1, 1, 256, False, synth.U8, False),       # 98 M tiles x 2 N tiles on 74 pairs: several tiles per pair
     (9, 9, 1024, 256, 1, 1, 3, False, synth.U8, False),         # 243 pixels: one pair, second CTA nearly empty
+    (14, 14, 256, 256, 3, 1, 96, False, synth.U8, True),        # K-heavy layer with a shortcut (basic residual block): 74 pair tiles
+    (7, 7, 512, 512, 3, 1, 64, False, synth.S8, True),          # the same with two N tiles and a signed output
+    (13, 13, 256, 256, 3, 1, 5, True, synth.U8, True),          # ragged: 845 pixels, the last pair tile half empty, signed input
 ]
 
 
