@@ -76,12 +76,19 @@ def test_maxpool(ref, c, signed, h, k, stride, pad):
 
 
 @pytest.mark.parametrize("c,signed,h,w,fl_x,fl_y", [(2048, False, 7, 7, 5, 6), (1280, False, 7, 7, 6, 7), (24, True, 5, 3, 4, 4),
-                                                     (512, False, 1, 1, 5, 5), (100, True, 8, 8, 7, 2)])
+                                                     (512, False, 1, 1, 5, 5), (100, True, 8, 8, 7, 2),
+                                                     # 257 positions: the largest sum the 16-bit lanes of the packed kernel hold;
+                                                     # 258: one more (the byte-wise kernel); 6 channels: not a multiple of four
+                                                     (8, False, 257, 1, 4, 4), (8, True, 257, 1, 4, 4), (8, False, 129, 2, 4, 4),
+                                                     (6, True, 4, 4, 5, 5)])
 def test_global_average_pool(ref, c, signed, h, w, fl_x, fl_y):
     rng = np.random.default_rng(c + h)
     dt = synth.S8 if signed else synth.U8
     layer = synth.Layer(synth.GAP, "gap", 0, -1, h, w, c, c, 1, 1, 1, 0, dt, dt, synth.U8, fl_x, 0, fl_y, 0)
-    check_layer(ref, layer, random_input(rng, 5, layer))
+    x = random_input(rng, 5, layer)
+    x[0, :, :, 0] = -128 if signed else 255          # a channel of extreme values: the largest / smallest possible sum
+    x[1, :, :, 1] = 127 if signed else 0
+    check_layer(ref, layer, x)
 
 
 @pytest.mark.parametrize("n,k,out,y_dtype", [(4, 512, 1000, synth.S32), (1, 2048, 1000, synth.S32), (3, 33, 10, synth.S8),
