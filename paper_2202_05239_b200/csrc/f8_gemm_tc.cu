@@ -767,17 +767,31 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int c_first = n_t * p.bn + ch_begin * 16;
                 const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
-                bool got = mbar_wait(tfull_bar + 8 * acc, acc_phase, wc, tagbits | 104);
-                // the buffer holds the residual tile (which implies that its previous store has left), or is free
-                if (RES) got = mbar_wait(res_full + 8 * ob, ophase, wc, tagbits | 107) && got;
-                else got = mbar_wait(out_free + 8 * ob, ophase ^ 1, wc, tagbits | 109) && got;
+                // The buffer first (it holds the residual tile, which implies that its previous store has left, or it is
+                // free): that wait is over long before the accumulator is complete, so it costs the chain accumulator ->
+                // epilogue -> accumulator nothing.
+                bool got;
+                if (RES) got = mbar_wait(res_full + 8 * ob, ophase, wc, tagbits | 107);
+                else got = mbar_wait(out_free + 8 * ob, ophase ^ 1, wc, tagbits | 109);
+                got = mbar_wait(tfull_bar + 8 * acc, acc_phase, wc, tagbits | 104) && got;
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t out_buf = smem_base + p.out_off + ob * p.out_bytes;
                 const uint32_t res_buf = out_buf;       // in place: a thread reads and then overwrites its own 16 bytes
                 const uint32_t bias_s = smem_base + p.bias_off + 4 * c_first;
+                // The accumulator goes back to the MMA issuer as soon as this warp's last load from it has completed -- before
+                // the last chunk is converted and written.
+                auto release_acc = [&]() {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (PAIR && cta_rank != 0) mbar_arrive_cluster(tempty_bar + 8 * acc, 0);     // the issuer's barrier
+                        else mbar_arrive(tempty_bar + 8 * acc);
+                    }
+                };
                 int va[16], vb[16];
                 if (my_nch > 0) tmem_ld16(t_addr, va);
+                else release_acc();
 #pragma unroll
                 for (int i = 0; i < 4; i += 2) {
                     if (i < my_nch) {
@@ -785,6 +799,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         if (RES) rw = lds128(res_buf + so[i]);
                         tmem_ld_wait();
                         if (i + 1 < my_nch) tmem_ld16(t_addr + (i + 1) * 16, vb);
+                        else release_acc();
                         sts128(out_buf + so[i], epilogue_fast16<RES, SGN>(va, bias_s + 64 * (i), rw, mul_acc, mul_res, rsel, p.q.s));
                     }
                     if (i + 1 < my_nch) {
@@ -792,19 +807,15 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         if (RES) rw = lds128(res_buf + so[i + 1]);
                         tmem_ld_wait();
                         if (i + 2 < my_nch) tmem_ld16(t_addr + (i + 2) * 16, va);
+                        else release_acc();
                         sts128(out_buf + so[i + 1], epilogue_fast16<RES, SGN>(vb, bias_s + 64 * (i + 1), rw, mul_acc, mul_res, rsel, p.q.s));
                     }
                 }
-                // accumulator and residual have been read, the output part is written: make the writes
-                // visible to the TMA and tell the MMA warp, the mover and the fetcher
-                tc_fence_before();
+                // the output part is written: make the writes visible to the TMA and tell the mover (and, through it, the
+                // fetcher)
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
-                if (lane == 0) {
-                    if (PAIR && cta_rank != 0) mbar_arrive_cluster(tempty_bar + 8 * acc, 0);     // the issuer's barrier
-                    else mbar_arrive(tempty_bar + 8 * acc);
-                    mbar_arrive(out_full + 8 * ob);
-                }
+                if (lane == 0) mbar_arrive(out_full + 8 * ob);
                 if (++ob == p.out_bufs) { ob = 0; ophase ^= 1; }
             }
         } else {
