@@ -330,6 +330,7 @@ void f8_debug_force_direct(int on);
  *   F8_PLAN_OFF_ALT_PRODUCERS     one pair of TMA producer warps
  *   F8_PLAN_OFF_PAIRS             no two-CTA tiles (tcgen05 cta_group::2)
  *   F8_PLAN_OFF_DW_DP4A           depthwise 3x3 layers do not use the packed-dot-product kernels
+ *   F8_PLAN_OFF_TILE_GROUPS       pointwise layers with a single K chunk do not hand several M tiles over at once
  *   F8_PLAN_OFF_DW_WALK           depthwise 3x3 stride-1 layers do not use the row-walking kernel (with both off: the strip kernel)
  *   F8_PLAN_OFF_STEM_KERNEL       first layers take the packed-row-pair GEMM instead of the first-layer kernel
  *   F8_PLAN_OFF_STEM_POOL_FUSION  the max pool behind a first layer runs as its own kernel
@@ -340,7 +341,8 @@ void f8_debug_force_direct(int on);
 enum {
     F8_PLAN_OFF_RESIDENT_WEIGHTS = 1, F8_PLAN_OFF_WINDOWED = 2, F8_PLAN_OFF_DUAL_ISSUE = 4, F8_PLAN_OFF_ALT_PRODUCERS = 8,
     F8_PLAN_OFF_PAIRS = 16, F8_PLAN_OFF_DW_WALK = 32, F8_PLAN_OFF_STEM_KERNEL = 64, F8_PLAN_OFF_STEM_POOL_FUSION = 128,
-    F8_PLAN_OFF_LAYER_OVERLAP = 256, F8_PLAN_OFF_LANES = 512, F8_PLAN_SYNC_LAYERS = 1024, F8_PLAN_OFF_DW_DP4A = 2048
+    F8_PLAN_OFF_LAYER_OVERLAP = 256, F8_PLAN_OFF_LANES = 512, F8_PLAN_SYNC_LAYERS = 1024, F8_PLAN_OFF_DW_DP4A = 2048,
+    F8_PLAN_OFF_TILE_GROUPS = 4096
 };
 void f8_debug_plan_options(unsigned off_mask);
 
@@ -364,7 +366,8 @@ int f8_net_lanes(const f8_net *net);
  * [9] staged output buffers.  Lets a test assert which path a case took and how many tiles each CTA walked. */
 enum {
     F8_PLAN_RESIDENT_WEIGHTS = 1, F8_PLAN_WINDOWED = 2, F8_PLAN_DUAL_ISSUE = 4, F8_PLAN_ALT_PRODUCERS = 8,
-    F8_PLAN_PLAIN_MATRIX = 16, F8_PLAN_STAGED_EPILOGUE = 32, F8_PLAN_PAIRS = 64, F8_PLAN_ROW_TILES = 128
+    F8_PLAN_PLAIN_MATRIX = 16, F8_PLAN_STAGED_EPILOGUE = 32, F8_PLAN_PAIRS = 64, F8_PLAN_ROW_TILES = 128,
+    F8_PLAN_TILE_GROUPS = 256
 };
 int f8_debug_last_plan(int *info, int n);
 

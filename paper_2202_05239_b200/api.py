@@ -240,8 +240,10 @@ _lib.f8_debug_wait_timeout_probe.argtypes = [ctypes.c_double, _vp]
 PLAN_OFF_RESIDENT_WEIGHTS, PLAN_OFF_WINDOWED, PLAN_OFF_DUAL_ISSUE, PLAN_OFF_ALT_PRODUCERS = 1, 2, 4, 8
 PLAN_OFF_PAIRS, PLAN_OFF_DW_WALK, PLAN_OFF_STEM_KERNEL, PLAN_OFF_STEM_POOL_FUSION = 16, 32, 64, 128
 PLAN_OFF_LAYER_OVERLAP, PLAN_OFF_LANES, PLAN_SYNC_LAYERS, PLAN_OFF_DW_DP4A = 256, 512, 1024, 2048
+PLAN_OFF_TILE_GROUPS = 4096
 PLAN_RESIDENT_WEIGHTS, PLAN_WINDOWED, PLAN_DUAL_ISSUE, PLAN_ALT_PRODUCERS = 1, 2, 4, 8
 PLAN_PLAIN_MATRIX, PLAN_STAGED_EPILOGUE, PLAN_PAIRS, PLAN_ROW_TILES = 16, 32, 64, 128
+PLAN_TILE_GROUPS = 256
 
 
 def f8_debug_plan_options(off_mask: int):

@@ -101,6 +101,11 @@ struct TcParams {
     int pair_tiles;           // 256-row tiles x N tiles
     int alt;                  // 1: two pairs of producer warps, pair h takes the stage uses of parity h (streamed weights,
                               // one MMA issuer: fills may then complete out of order, the consumer is in order)
+    int sup;                  // 0, or the number of M tiles (2..4) that share one stage use and one accumulator hand-over: layers
+                              // with a single k-iteration and narrow tiles, where the per-tile hand-overs between the roles cost
+                              // more than the tile's work.  M tile j of such a group takes columns j * bn of the accumulator and
+                              // column slab j of the staged output
+    int sup_tiles;            // groups of `sup` M tiles
     int epi_groups;           // 1, 2 or 4: the tile's columns are split over this many groups of four epilogue warps (one warp per
                               // tensor-memory lane quarter); the warps of the other groups stay out of the tile loop
     uint32_t sub_bytes;       // A + B bytes of one k-iteration (each rounded to 1024)
@@ -236,13 +241,16 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int (&ac
 
 enum { EPI_GENERIC = 0, EPI_U8 = 1, EPI_U8_RES = 2, EPI_S8 = 3, EPI_S8_RES = 4 };
 
+// MODE 0: one 128-row tile per hand-over.  MODE 2: groups of M tiles (TcParams::sup).  MODE 1 (PAIR below):
 // PAIR: two CTAs of a cluster share 256-row tiles (tcgen05 cta_group::2): each loads its own 128 rows of activations and
 // half of the weight tile, so a weight byte crosses the L2 -> SM path once per 256 rows; the even CTA issues the MMAs.
-template <int EPI, bool PAIR>
+template <int EPI, int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_r,
                        const TcParams p) {
+    constexpr bool PAIR = MODE == 1;                                // CTA pairs
+    constexpr bool SUP = MODE == 2;                                 // groups of M tiles per hand-over (TcParams::sup)
     constexpr bool STAGED = EPI != EPI_GENERIC;                     // output (and residual) through shared memory + TMA
     constexpr bool RES = EPI == EPI_U8_RES || EPI == EPI_S8_RES;
     constexpr bool SGN = EPI == EPI_S8 || EPI == EPI_S8_RES;
@@ -323,7 +331,8 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     // CTA there has exited, and run their prologue while the rest of this grid finishes
     grid_launch_dependents();
 
-    const int total_tiles = PAIR ? p.pair_tiles : p.m_tiles * p.n_tiles;      // per worker: 128-row tiles, or 256-row tiles of a pair
+    // per worker: 128-row tiles, 256-row tiles of a pair, or groups of p.sup M tiles
+    const int total_tiles = PAIR ? p.pair_tiles : (SUP ? p.sup_tiles : p.m_tiles * p.n_tiles);
     const int k_iters = p.kh * p.kw * p.c_chunks;
     const WaitCtx wc = make_wait_ctx(&abort_flag, p.status, p.wait_limit);
     const int tagbits = p.tag << 8;     // status word of a timed-out wait: tag << 8 | site
@@ -388,6 +397,42 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     }
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
+            }
+        } else if (SUP) {
+            // one stage use per group of M tiles: sub-chunk j is the activation tile of M tile first + j (a single k-iteration
+            // per tile; the weights are resident, so the two producer warps share the sub-chunks as usual)
+            for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+                if (!__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * stage, phase ^ 1, wc, tagbits | 101))) {
+                    ok = false;
+                    break;
+                }
+                const int first_m = tile * p.sup;
+                const int subs = min(p.sup, p.m_tiles - first_m);
+                const uint32_t fb = full_bar + 8 * stage;
+                if (lane == 0) {
+                    const uint32_t bytes = (uint32_t)(opnd == 0 ? (subs + 1) >> 1 : subs >> 1) * p.tx_a;
+                    if (bytes) mbar_expect_tx(fb, bytes);
+                    else mbar_arrive(fb);
+                }
+                __syncwarp();
+                const int j = (lane - stage * p.sup) & 31;
+                if (j < subs && (j & 1) == opnd) {
+                    const int m0 = (first_m + j) * TILE_M;
+                    const uint32_t dst = smem_base + stage * p.stage_bytes + j * p.a_bytes;
+                    if (p.a_plain) {
+                        tma_load_2d(dst, &map_a, fb, 0, m0);
+                    } else {
+                        const int t1 = fast_div(m0, p.div_wo);
+                        const int ow = m0 - t1 * p.wo;
+                        const int img = fast_div(t1, p.div_ho);
+                        const int oh = t1 - img * p.ho;
+                        tma_load_im2col(dst, &map_a, fb, 0, ow * p.stride_w - p.pad_w, oh * p.stride_h - p.pad_h, img, 0, 0);
+                    }
+                    have_last = true;
+                    last_stage = stage;
+                    last_phase = phase;
+                }
+                if (++stage == p.stages) { stage = 0; phase ^= 1; }
             }
         } else if (p.rowt)
         // small tensors: the same pipeline, but a tile is win_r whole output rows of one image and every filter tap is a
@@ -574,7 +619,23 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
                     b_tile_lo = bres_lo + (uint32_t)(n_t * k_iters) * b16;
                 }
-                if (p.win) {
+                if (SUP) {
+                    // one stage use: the activation tiles of up to p.sup M tiles, each accumulated (a single k-iteration) into
+                    // its own column range of this accumulator
+                    if (!mbar_wait(full_bar + 8 * stage, phase, wc, tagbits | 103)) { ok = false; break; }
+                    tc_fence_after();
+                    const int subs = min(p.sup, p.m_tiles - tile * p.sup);
+                    uint32_t a_lo = stage_lo;
+                    for (int j = 0; j < subs; ++j, a_lo += a16) {
+                        const uint32_t d_sub = d_tmem + (uint32_t)(j * p.bn);
+                        if (mmas == 4) mma_i8_sub<4>(d_sub, a_lo, b_tile_lo, desc_hi32, p.idesc, 0u);
+                        else if (mmas == 2) mma_i8_sub<2>(d_sub, a_lo, b_tile_lo, desc_hi32, p.idesc, 0u);
+                        else mma_i8_sub<1>(d_sub, a_lo, b_tile_lo, desc_hi32, p.idesc, 0u);
+                    }
+                    mma_commit(empty_bar + 8 * stage);
+                    stage_lo += stage16;
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; stage_lo = desc_lo0; }
+                } else if (p.win) {
                     // one stage use per channel chunk; the nine taps read the same tile at shifted row offsets
                     const uint32_t kb16 = (uint32_t)p.kb >> 4;
                     for (int cc = 0; cc < p.c_chunks; ++cc) {
@@ -631,7 +692,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 // are done).  Such an arrival must not land after this CTA has gone: the next kernel's CTA takes over
                 // the SM at once and keeps its own barriers at the same shared-memory addresses.  So every issuer waits
                 // for the last arrival on each stage that came from one of its own tiles.
-                const int uses_tile = p.win ? p.c_chunks : p.uses;
+                const int uses_tile = p.win ? p.c_chunks : p.uses;      // (p.sup: one use per group of M tiles, p.uses == 1)
                 const int total_uses = local * uses_tile;
                 for (int g = max(0, total_uses - p.stages); g < total_uses; ++g) {
                     const int t_of_g = g / uses_tile;
@@ -659,7 +720,12 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int m_t = PAIR ? 2 * m_q + (int)cta_rank : m_q;
                 if (!mbar_wait(out_full + 8 * b, bphase, wc, tagbits | 108)) break;
                 const uint32_t src = smem_base + p.out_off + b * p.out_bytes;
-                if (p.rows) {
+                if (SUP) {
+                    // column slab sl of the staged tile is M tile tile * sup + sl
+                    const int subs = min(p.sup, p.m_tiles - tile * p.sup);
+                    for (int sl = 0; sl < subs; ++sl)
+                        tma_store_2d(&map_y, src + sl * (TILE_M * p.slab_w), 0, (tile * p.sup + sl) * TILE_M);
+                } else if (p.rows) {
                     const int img = fast_div(m_t, p.div_bands);
                     const int y0 = (m_t - img * p.win_bands) * p.win_r;
                     // positions W and W + 1 of every row and rows below the image are clipped by the hardware
@@ -722,7 +788,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 belong to this warp
         const int ew = warp - FIRST_EPI_WARP;
         const int group = ew >> 2;                  // which quarter of the tile's columns this warp converts
-        const int chunks = p.bn / 16;
+        const int chunks = (SUP ? p.sup * p.bn : p.bn) / 16;
         const int per_group = (chunks + p.epi_groups - 1) / p.epi_groups;     // <= 4 chunks of 16 columns per warp
         const int ch_begin = min(group * per_group, chunks);
         const int nch = min(ch_begin + per_group, chunks) - ch_begin;
@@ -744,6 +810,7 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
             }
             const int tile_row = quarter * 32 + lane;
+            const int sup_sub = SUP ? (ch_begin * 16) / p.bn : 0, sup_col0 = ch_begin * 16 - sup_sub * p.bn;
             // Narrow tiles are converted by fewer warps: the MMA-issuing threads share their scheduler partitions with the
             // epilogue warps, and every warp that is ready to issue slows them down.
             const int my_tiles_end = group < p.epi_groups ? total_tiles : 0;
@@ -764,8 +831,13 @@ f8_conv_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 const int acc = local & 1;                   // accumulator, output buffer and residual buffer in use
                 const uint32_t acc_phase = (local >> 1) & 1;
                 const int n_t = tile - fast_div(tile, p.div_n_tiles) * p.n_tiles;
-                const int c_first = n_t * p.bn + ch_begin * 16;
-                const int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
+                int c_first = n_t * p.bn + ch_begin * 16;
+                int my_nch = min(nch, max(0, (p.c_out - c_first) / 16));      // chunks that exist in c_out
+                if (SUP) {
+                    // this warp's chunks lie in M tile sup_sub of the group (a chunk range never straddles two of them)
+                    c_first = sup_col0;
+                    my_nch = sup_sub < min(p.sup, p.m_tiles - tile * p.sup) ? min(nch, max(0, (p.c_out - c_first) / 16)) : 0;
+                }
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + ch_begin * 16;
                 // The buffer first (it holds the residual tile, which implies that its previous store has left, or it is
                 // free): that wait is over long before the accumulator is complete, so it costs the chain accumulator ->
@@ -1092,6 +1164,26 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         // 64-wide tiles: eight epilogue warps (two chunks each) instead of sixteen -- measured, 3x3 64 -> 64 at 56 x 56 61 -> 57 us
         // (one warp per quarter: the same); 128-wide tiles show no difference and keep all sixteen
         p.epi_groups = p.bn <= 64 ? 2 : 4;
+        // Groups of M tiles (see TcParams::sup): pointwise layers with one k-iteration, one N tile of at most 128 columns and
+        // no residual; enough tiles that every CTA still gets several groups
+        p.sup = 0;
+        {
+            const bool one_k = g.kh == 1 && g.kw == 1 && g.c <= p.kb;
+            const int gsz = p.bn <= 64 ? 4 : 2;
+            if (one_k && !q.has_res && p.bn <= 128 && g.c_out <= p.bn && g.c_out % 16 == 0 && !p.pair && g.stride_h == 1 &&
+                g.stride_w == 1 && g.pad_h == 0 && g.pad_w == 0 && p.m_tiles >= 148 * 4 * gsz &&
+                !(f8_plan_options_off() & (F8_PLAN_OFF_TILE_GROUPS | F8_PLAN_OFF_RESIDENT_WEIGHTS))) {
+                p.sup = gsz;
+                p.sup_tiles = (p.m_tiles + gsz - 1) / gsz;
+                p.slab_w = p.bn;
+                p.slab_chunks = p.slab_w / 16;
+                p.n_slabs = gsz;
+                p.swz_mask = p.slab_w == 128 ? 7u : (p.slab_w == 64 ? 3u : (p.slab_w == 32 ? 1u : 0u));
+                p.out_bytes = (uint32_t)(TILE_M * p.bn * gsz + 1023) / 1024 * 1024;
+                p.out_bufs = 2;
+                p.epi_groups = 4;
+            }
+        }
         staging = (size_t)p.out_bytes * p.out_bufs + bias_bytes;
     }
     const size_t ktab_bytes = ((size_t)g.kh * g.kw * p.c_chunks * 8 + 1023) / 1024 * 1024;
@@ -1114,6 +1206,10 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     if (p.b_res) {
         avail -= b_all;
         p.sub_bytes = p.a_bytes;
+    }
+    if (p.sup && !p.b_res) {
+        *why = "tile groups need resident weights";
+        return cudaErrorInvalidValue;
     }
     p.tx_sub = p.tx_a + (p.b_res ? 0u : p.tx_b);
     p.tx_res = p.out_bytes;
@@ -1190,6 +1286,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     while (group > 1 && avail / ((size_t)group * p.sub_bytes) < 2) --group;
     group = (k_iters + (k_iters + group - 1) / group - 1) / ((k_iters + group - 1) / group);   // same uses, evenly split
     if (p.pair) group = 1;      // 32-KiB stage uses, as many stages in flight as fit
+    if (p.sup) group = p.sup;   // a stage use holds the activation tiles of a group of M tiles (sub_bytes == a_bytes)
     p.group = group;
     p.stage_bytes = (uint32_t)group * p.sub_bytes;
     int stages = (int)(avail / p.stage_bytes);
@@ -1200,10 +1297,10 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         return cudaErrorInvalidValue;
     }
     p.stages = stages;
-    p.uses = (k_iters + group - 1) / group;
+    p.uses = p.sup ? 1 : (k_iters + group - 1) / group;
     }
     const int stages = p.stages;
-    p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !(off & F8_PLAN_OFF_DUAL_ISSUE)) ? 1 : 0;
+    p.dual_issue = (p.bn <= 128 && stages >= 2 * p.uses && !p.sup && !(off & F8_PLAN_OFF_DUAL_ISSUE)) ? 1 : 0;
     p.alt = (!p.b_res && !p.dual_issue && !p.win && p.stages >= 2 && !(off & F8_PLAN_OFF_ALT_PRODUCERS)) ? 1 : 0;
     p.out_off = (uint32_t)(p.stages * p.stage_bytes);
     p.bias_off = p.out_off + (uint32_t)p.out_bufs * p.out_bytes;
@@ -1350,7 +1447,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int total_tiles = p.sup ? p.sup_tiles : p.m_tiles * p.n_tiles;
     plan->grid = total_tiles < sms ? total_tiles : sms;
     if (p.pair) plan->grid = 2 * std::min(p.pair_tiles, sms / 2);        // clusters of two; trimmed to what fits at launch
     // at least half of an SM's shared memory so that two CTAs (each owning all of TMEM) never share an SM
@@ -1362,7 +1459,7 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
         int *info = f8_last_plan_info();
         info[0] = (p.b_res ? F8_PLAN_RESIDENT_WEIGHTS : 0) | (p.win ? F8_PLAN_WINDOWED : 0) | (p.dual_issue ? F8_PLAN_DUAL_ISSUE : 0) |
                   (p.alt ? F8_PLAN_ALT_PRODUCERS : 0) | (p.a_plain ? F8_PLAN_PLAIN_MATRIX : 0) | (staged ? F8_PLAN_STAGED_EPILOGUE : 0) | (p.rowt ? F8_PLAN_ROW_TILES : 0) |
-                  (p.pair ? F8_PLAN_PAIRS : 0);
+                  (p.pair ? F8_PLAN_PAIRS : 0) | (p.sup ? F8_PLAN_TILE_GROUPS : 0);
         info[1] = p.epi; info[2] = p.bn; info[3] = p.kb; info[4] = p.stages; info[5] = p.group;
         info[6] = p.m_tiles; info[7] = p.n_tiles; info[8] = plan->grid; info[9] = staged ? p.out_bufs : 0;
     }
@@ -1374,15 +1471,17 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
     }
     if (!attr_set[dev]) {
         const int bytes = (int)(SMEM_LIMIT + CONTROL_BYTES);
-        cudaError_t e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_GENERIC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        cudaError_t e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_GENERIC, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8_RES, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8_RES, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_U8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f8_conv_gemm_tc_kernel<EPI_S8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         if (e != cudaSuccess) {
             *why = "cudaFuncSetAttribute(MaxDynamicSharedMemorySize) failed";
             return e;
@@ -1393,8 +1492,9 @@ cudaError_t f8_tc_plan_init(F8TcPlan *plan, const F8ConvGeom &g, const F8Requant
 }
 
 namespace {
-template <int EPI, bool PAIR>
+template <int EPI, int MODE>
 cudaError_t launch_variant(const F8TcPlan *plan, bool overlap_previous, cudaStream_t st) {
+    constexpr bool PAIR = MODE == 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)plan->grid);
     cfg.blockDim = dim3(NUM_THREADS);
@@ -1419,13 +1519,13 @@ cudaError_t launch_variant(const F8TcPlan *plan, bool overlap_previous, cudaStre
     if (PAIR) {
         // persistent pairs: no more clusters than the device can hold at once
         int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, f8_conv_gemm_tc_kernel<EPI, PAIR>, &cfg) == cudaSuccess && clusters > 0 &&
+        if (cudaOccupancyMaxActiveClusters(&clusters, f8_conv_gemm_tc_kernel<EPI, MODE>, &cfg) == cudaSuccess && clusters > 0 &&
             2 * clusters < plan->grid)
             cfg.gridDim = dim3((unsigned)(2 * clusters));
         else
             (void)cudaGetLastError();
     }
-    return cudaLaunchKernelEx(&cfg, f8_conv_gemm_tc_kernel<EPI, PAIR>, plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p);
+    return cudaLaunchKernelEx(&cfg, f8_conv_gemm_tc_kernel<EPI, MODE>, plan->map_a, plan->map_b, plan->map_y, plan->map_r, plan->p);
 }
 }   // namespace
 
@@ -1433,19 +1533,26 @@ cudaError_t f8_tc_launch(const F8TcPlan *plan, bool overlap_previous, cudaStream
     if (plan->p.M == 0) return cudaSuccess;
     if (plan->p.pair) {
         switch (plan->p.epi) {
-            case EPI_U8: return launch_variant<EPI_U8, true>(plan, overlap_previous, st);
-            case EPI_U8_RES: return launch_variant<EPI_U8_RES, true>(plan, overlap_previous, st);
-            case EPI_S8: return launch_variant<EPI_S8, true>(plan, overlap_previous, st);
-            case EPI_S8_RES: return launch_variant<EPI_S8_RES, true>(plan, overlap_previous, st);
+            case EPI_U8: return launch_variant<EPI_U8, 1>(plan, overlap_previous, st);
+            case EPI_U8_RES: return launch_variant<EPI_U8_RES, 1>(plan, overlap_previous, st);
+            case EPI_S8: return launch_variant<EPI_S8, 1>(plan, overlap_previous, st);
+            case EPI_S8_RES: return launch_variant<EPI_S8_RES, 1>(plan, overlap_previous, st);
+            default: return cudaErrorInvalidValue;
+        }
+    }
+    if (plan->p.sup) {
+        switch (plan->p.epi) {
+            case EPI_U8: return launch_variant<EPI_U8, 2>(plan, overlap_previous, st);
+            case EPI_S8: return launch_variant<EPI_S8, 2>(plan, overlap_previous, st);
             default: return cudaErrorInvalidValue;
         }
     }
     switch (plan->p.epi) {
-        case EPI_U8: return launch_variant<EPI_U8, false>(plan, overlap_previous, st);
-        case EPI_U8_RES: return launch_variant<EPI_U8_RES, false>(plan, overlap_previous, st);
-        case EPI_S8: return launch_variant<EPI_S8, false>(plan, overlap_previous, st);
-        case EPI_S8_RES: return launch_variant<EPI_S8_RES, false>(plan, overlap_previous, st);
-        default: return launch_variant<EPI_GENERIC, false>(plan, overlap_previous, st);
+        case EPI_U8: return launch_variant<EPI_U8, 0>(plan, overlap_previous, st);
+        case EPI_U8_RES: return launch_variant<EPI_U8_RES, 0>(plan, overlap_previous, st);
+        case EPI_S8: return launch_variant<EPI_S8, 0>(plan, overlap_previous, st);
+        case EPI_S8_RES: return launch_variant<EPI_S8_RES, 0>(plan, overlap_previous, st);
+        default: return launch_variant<EPI_GENERIC, 0>(plan, overlap_previous, st);
     }
 }
 

@@ -191,6 +191,30 @@ def test_cta_pairs(ref, case):
         check_layer(ref, layer, x, res, expect_tc=True, plan_off=a.PLAN_OFF_PAIRS, forbid_flags=a.PLAN_PAIRS)
 
 
+# Pointwise layers with a single K chunk and narrow tiles: several M tiles share one stage use and one accumulator hand-over
+# (h, w, c, c_out, n, x_signed, y_dtype)
+GROUP_CASES = [
+    (56, 56, 64, 64, 100, False, synth.U8),       # groups of four 64-wide tiles; 2450 M tiles
+    (56, 56, 64, 64, 97, True, synth.S8),         # 2377 M tiles: the last group holds one tile, and that one is ragged
+    (112, 112, 32, 64, 25, False, synth.U8),      # 32-byte K chunk
+    (56, 56, 64, 128, 50, False, synth.U8),       # groups of two 128-wide tiles
+    (56, 56, 128, 96, 50, True, synth.U8),        # 96 of 128 columns exist: the last two chunks of every tile are skipped
+    (56, 56, 16, 32, 100, False, synth.S8),       # 16 channels in a 32-byte chunk, 32-wide tiles: half of the accumulator unused
+]
+
+
+@pytest.mark.parametrize("case", range(len(GROUP_CASES)))
+def test_groups_of_m_tiles(ref, case):
+    from paper_2202_05239_b200 import api as a
+    h, w, c, c_out, n, xs, y_dtype = GROUP_CASES[case]
+    rng = np.random.default_rng(1500 + case)
+    layer = random_conv_layer(rng, h=h, w=w, c=c, c_out=c_out, k=1, stride=1, pad=0, x_signed=xs, y_dtype=y_dtype, with_res=False)
+    x = random_input(rng, n, layer)
+    check_layer(ref, layer, x, None, expect_tc=True, expect_flags=a.PLAN_TILE_GROUPS | a.PLAN_RESIDENT_WEIGHTS)
+    if case in (1, 4):      # the same layer with one tile per hand-over
+        check_layer(ref, layer, x, None, expect_tc=True, plan_off=a.PLAN_OFF_TILE_GROUPS, forbid_flags=a.PLAN_TILE_GROUPS)
+
+
 @pytest.mark.parametrize("case", range(13))
 def test_many_tiles_per_cta_in_every_plan_mode(ref, case):
     h, w, c, c_out, k, stride, n, xs, y_dtype, with_res, off, expect, forbid = _modes()[case]
