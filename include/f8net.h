@@ -129,6 +129,24 @@ f8_status f8_conv2d_siblings_fixed(const f8_conv_desc *desc, int y2_dtype, int f
                                    const int8_t *w_ohwi, const int32_t *bias, const void *residual, void *y, void *y2,
                                    void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Two consecutive layers in one launch: a dense convolution `conv` (Eq. 6, quantizer of Eq. 2) and the pointwise (1x1,
+ * stride 1, no padding) convolution `pw` that reads its output, with the optional shortcut add of Sec. 4.3 behind the
+ * second layer -- the last two layers of a ResNet bottleneck block (Sec. 5 workloads).  Eq. 6 holds per layer, so both
+ * outputs are exactly what f8_conv2d_fixed(conv) followed by f8_conv2d_fixed(pw) give; the difference is that the
+ * first layer's output tile goes from the epilogue straight into the second GEMM through shared memory and is not
+ * written to device memory unless y_mid is given.
+ *   conv  c = 64, c_out = 64, any kh * kw <= 16, stride, pad; y_dtype F8_U8; input at least 128 KiB; no shortcut
+ *   pw    n / h / w / c = conv's output, c_out = 256, x_dtype / fl_x = conv's y_dtype / fl_y, y_dtype F8_U8 or F8_S8;
+ *         r_dtype / fl_r describe `residual` ([n, ho, wo, 256] 8-bit, NULL: none)
+ *   both requantisation shifts must lie in 1..24
+ *   w_conv [64, kh, kw, 64], w_pw [256, 64] int8; bias_conv [64], bias_pw [256] int32 or NULL; all pointers DEVICE,
+ *   16-byte aligned; y_mid NULL or [n, ho, wo, 64] (receives the first layer's output); y [n, ho, wo, 256].
+ * Errors: as f8_conv2d_fixed for each descriptor; F8_ERR_SHAPE / F8_ERR_DTYPE when pw does not continue conv;
+ * F8_ERR_UNSUPPORTED for shapes outside the list above (call the two layers separately). */
+f8_status f8_conv_pointwise_fixed(const f8_conv_desc *conv, const f8_conv_desc *pw, const void *x, const int8_t *w_conv,
+                                  const int32_t *bias_conv, const int8_t *w_pw, const int32_t *bias_pw, const void *residual,
+                                  void *y_mid, void *y, void *cuda_stream);
+
 /* Depthwise convolution (one kh x kw filter per channel; MobileNet layers of Sec. 5),
  * c_out must equal c.  w_chw [c, kh, kw] int8.  Everything else as f8_conv2d_fixed. */
 f8_status f8_dwconv_fixed(const f8_conv_desc *desc, const void *x, const int8_t *w_chw, const int32_t *bias,

@@ -127,6 +127,15 @@ def f8_conv2d_siblings_fixed(desc: ConvDesc, y2_dtype, fl_y2, x, w, bias, residu
                                          workspace.numel() if workspace is not None else 0, _stream(stream)))
 
 
+_lib.f8_conv_pointwise_fixed.argtypes = [ctypes.POINTER(ConvDesc), ctypes.POINTER(ConvDesc)] + [_vp] * 9
+
+
+def f8_conv_pointwise_fixed(conv: ConvDesc, pw: ConvDesc, x, w_conv, bias_conv, w_pw, bias_pw, residual, y_mid, y, stream=None):
+    """A 64 -> 64 convolution and the 64 -> 256 pointwise layer behind it in one launch (y_mid: optional copy of the first output)."""
+    _check(_lib.f8_conv_pointwise_fixed(ctypes.byref(conv), ctypes.byref(pw), _ptr(x), _ptr(w_conv), _ptr(bias_conv), _ptr(w_pw),
+                                        _ptr(bias_pw), _ptr(residual), _ptr(y_mid), _ptr(y), _stream(stream)))
+
+
 def f8_dwconv_fixed(desc: ConvDesc, x, w, bias, residual, y, workspace=None, stream=None):
     _check(_lib.f8_dwconv_fixed(ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y),
                                 _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))

@@ -342,6 +342,41 @@ f8_status f8_conv2d_siblings_fixed(const f8_conv_desc *desc, int y2_dtype, int f
     return run_dense(g, q, x, w, bias, residual, y, (cudaStream_t)cuda_stream, y2 ? &sib : nullptr);
 }
 
+f8_status f8_conv_pointwise_fixed(const f8_conv_desc *conv, const f8_conv_desc *pw, const void *x, const int8_t *w_conv,
+                                  const int32_t *bias_conv, const int8_t *w_pw, const int32_t *bias_pw, const void *residual,
+                                  void *y_mid, void *y, void *cuda_stream) {
+    F8ConvGeom g1, g2;
+    F8Requant q1, q2;
+    f8_status s = check_conv(conv, false, false, &g1, &q1);
+    if (s != F8_OK) return s;
+    s = check_conv(pw, false, residual != nullptr, &g2, &q2);
+    if (s != F8_OK) return s;
+    if (pw->n != conv->n || pw->h != g1.ho || pw->w != g1.wo || pw->c != conv->c_out || pw->kh != 1 || pw->kw != 1 || pw->stride != 1 ||
+        pw->pad != 0)
+        return fail(F8_ERR_SHAPE, "the second layer must be a 1x1 convolution over the first layer's output");
+    if (pw->x_dtype != conv->y_dtype || pw->fl_x != conv->fl_y)
+        return fail(F8_ERR_DTYPE, "the second layer's input format must be the first layer's output format");
+    if (g1.n == 0) return F8_OK;
+    if (!x || !w_conv || !w_pw || !y) return fail(F8_ERR_NULL, "x, both weight tensors and y must not be NULL");
+    if (!aligned16(x) || !aligned16(w_conv) || !aligned16(w_pw) || !aligned16(y) || !aligned16(y_mid) || !aligned16(residual) ||
+        !aligned16(bias_conv) || !aligned16(bias_pw))
+        return fail(F8_ERR_ALIGN, "device pointers must be 16-byte aligned");
+    if (!f8_fused_supported(g1, q1, g2.c_out, q2))
+        return fail(F8_ERR_UNSUPPORTED, "the two-layer kernel takes 64 -> 64 -> 256 channels, an unsigned 8-bit tensor between the layers, "
+                                        "shifts in 1..24 and an input of at least 128 KiB");
+    if (pending_timeout() != F8_OK) return F8_ERR_TIMEOUT;
+    const size_t size = (f8_fused_plan_size() + 63) / 64 * 64;
+    F8FusedPlan *plan = (F8FusedPlan *)aligned_alloc(64, size);
+    if (!plan) return fail(F8_ERR_CUDA, "out of host memory");
+    const char *why = "";
+    cudaError_t e = f8_fused_plan_init(plan, g1, q1, q2, x, w_conv, bias_conv, w_pw, bias_pw, residual, y_mid, y, f8_status_word(), &why);
+    if (e == cudaSuccess) e = f8_fused_launch(plan, false, (cudaStream_t)cuda_stream);
+    free(plan);
+    if (e != cudaSuccess) return cuda_fail(e, *why ? why : "two-layer kernel launch");
+    ++g_tc_launches;
+    return F8_OK;
+}
+
 f8_status f8_dwconv_fixed(const f8_conv_desc *desc, const void *x, const int8_t *w, const int32_t *bias,
                           const void *residual, void *y, void *, size_t, void *cuda_stream) {
     F8ConvGeom g;

@@ -90,6 +90,18 @@ cudaError_t f8_tc_probe(int iters, double *ops, int *status_word, cudaStream_t s
 // One thread waits `limit_cycles` on a barrier nothing arrives at, records the time-out (site 199) and returns.
 cudaError_t f8_tc_wait_probe(unsigned long long limit_cycles, int *status_word, cudaStream_t st);
 
+// ---- two layers in one launch (f8_fused_tc.cu): a dense convolution 64 -> 64 channels (unsigned 8-bit output, no shortcut)
+// followed by the pointwise convolution 64 -> 256 behind it (8-bit output, optional 8-bit shortcut).  The first layer's
+// output stays in shared memory; y_mid (may be NULL) receives a copy of it.
+struct F8FusedPlan;
+bool f8_fused_supported(const F8ConvGeom &g1, const F8Requant &q1, int c_out2, const F8Requant &q2);
+size_t f8_fused_plan_size();
+cudaError_t f8_fused_plan_init(F8FusedPlan *plan, const F8ConvGeom &g1, const F8Requant &q1, const F8Requant &q2, const void *x,
+                               const int8_t *w1, const int32_t *bias1, const int8_t *w2, const int32_t *bias2, const void *res,
+                               void *y_mid, void *y, int *status_word, const char **why);
+void f8_fused_plan_set_tag(F8FusedPlan *plan, int tag);
+cudaError_t f8_fused_launch(const F8FusedPlan *plan, bool overlap_previous, cudaStream_t st);
+
 // ---- first-layer kernel (f8_stem_tc.cu): stride-2 convolution over an image with <= 4 channels, optionally fused
 // with the 3x3 / 2 / pad 1 max pool behind it.  kh2 row pairs per window starting `top` pairs above the output row,
 // `left` zero cells in front of a row, `slices` 32-byte K slices per row pair; w_core is [K / 16][c_out][16].
