@@ -68,6 +68,7 @@ struct FtParams {
     int m_tiles;
     FtDiv div_wo, div_ho;
     int stages, out_bufs;
+    int stages_a;               // stages of the ring of the even taps (the odd taps' ring takes the rest)
     uint32_t w1_off, w2_off, t_off, out_off, bias_off;      // byte offsets behind the control block
     uint32_t idesc1, idesc2;
     uint64_t desc_hi;
@@ -146,9 +147,12 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 
     if (warp == FT_A_WARP || warp == FT_A2_WARP) {
         // ------------------------------------------------------------------ TMA producers
-        // Tap j of local tile l is stage use u = l * taps + j: stage u mod stages, use u div stages.  Lane j of the
-        // first warp requests the even taps, lane j of the second warp the odd ones (loads issued by different threads
-        // overlap; a single thread's loads are served one after the other).
+        // Two producer warps, two rings.  Warp h requests the taps of parity h (lane q: tap 2 q + h) into a ring of its
+        // own: S_h stages, T_h taps per tile, tap q of local tile l is use u = l * T_h + q of that ring (stage u mod S_h,
+        // use u div S_h).  A parity wait can only tell a phase from its neighbour, so the thread that refills a stage
+        // must know that the stage's previous refill has happened.  Inside one warp it does: that refill's wait comes
+        // earlier in the warp's program order (an earlier tile, or an earlier round below).  One ring shared by both
+        // warps would not give that: the stages would rotate between lanes of two warps that do not wait for each other.
         const int half = warp == FT_A2_WARP ? 1 : 0;
         if (half == 1) {
             // the weights of both layers, once per CTA: nothing the previous grid writes
@@ -159,38 +163,42 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
             else if (lane == n_loads - 1) tma_load_3d(smem_base + p.w2_off, &map_w2, wres_bar, 0, 0, 0);
         }
         grid_dependency_wait();
-        const bool mine = lane < p.taps && (lane & 1) == half;
-        const int r = lane / p.kw, sx = lane - r * p.kw;
-        int slot = lane % p.stages, use = lane / p.stages;
+        const int taps_h = half ? p.taps / 2 : (p.taps + 1) / 2;
+        const int S = half ? p.stages - p.stages_a : p.stages_a;
+        const int base = half ? p.stages_a : 0;
+        const int tap = 2 * lane + half;
+        const bool mine = lane < taps_h;
+        const int r = tap / p.kw, sx = tap - r * p.kw;
+        int slot = S > 0 ? lane % S : 0, use = S > 0 ? lane / S : 0;
         bool ok = true, have_last = false;
         int last_slot = 0;
         uint32_t last_par = 0;
-        for (int l = 0; l < n_local; ++l) {
+        for (int l = 0; taps_h > 0 && l < n_local; ++l) {
             const int m0 = (worker + l * n_workers) * FT_TILE_M;
             const int t1 = ft_div(m0, p.div_wo);
             const int ow = m0 - t1 * p.wo;
             const int img = ft_div(t1, p.div_ho);
             const int oh = t1 - img * p.ho;
-            // With fewer stages than taps the taps go in rounds of `stages`: the lanes of one round wait for different
-            // stages, and a stage a later round needs is freed by loads that were requested in an earlier one.
-            for (int j0 = 0; ok && j0 < p.taps; j0 += p.stages) {
-                const bool act = mine && lane >= j0 && lane < j0 + p.stages;
+            // With fewer stages than taps the taps go in rounds of S: the lanes of one round wait for different stages,
+            // and a stage a later round needs is freed by loads that were requested in an earlier one.
+            for (int q0 = 0; ok && q0 < taps_h; q0 += S) {
+                const bool act = mine && lane >= q0 && lane < q0 + S;
                 bool got = true;
-                if (act) got = mbar_wait(empty_bar + 8 * slot, (uint32_t)(use & 1) ^ 1u, wc, tagbits | 201);
+                if (act) got = mbar_wait(empty_bar + 8 * (base + slot), (uint32_t)(use & 1) ^ 1u, wc, tagbits | 201);
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 if (act) {
-                    const uint32_t fb = full_bar + 8 * slot;
+                    const uint32_t fb = full_bar + 8 * (base + slot);
                     mbar_expect_tx(fb, FT_A_BYTES);
-                    tma_load_im2col(smem_base + (uint32_t)slot * FT_A_BYTES, &map_a, fb, 0, ow * p.stride - p.pad,
+                    tma_load_im2col(smem_base + (uint32_t)(base + slot) * FT_A_BYTES, &map_a, fb, 0, ow * p.stride - p.pad,
                                     oh * p.stride - p.pad, img, (uint16_t)sx, (uint16_t)r);
                     have_last = true;
-                    last_slot = slot;
+                    last_slot = base + slot;
                     last_par = (uint32_t)(use & 1);
                 }
             }
             if (!ok) break;
-            slot += p.taps;
-            while (slot >= p.stages) { slot -= p.stages; ++use; }
+            slot += taps_h;
+            while (slot >= S) { slot -= S; ++use; }
         }
         if (!ok && have_last) {
             const unsigned long long t0 = clock64();
@@ -209,7 +217,8 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
             bool committed_any = false;
             int last_acc = 0;
             uint32_t last_acc_phase = 0;
-            int slot = 0, use = 0;
+            int slot_a = 0, use_a = 0, slot_b = 0, use_b = 0;       // position in the ring of the even / odd taps
+            const int size_a = p.stages_a, size_b = p.stages - p.stages_a;
             // GEMM 2 of local tile i: the staged tile times the pointwise weights
             auto gemm2 = [&](int i) -> bool {
                 if (!mbar_wait(tmid_full, (uint32_t)(i & 1), wc, tagbits | 205)) return false;
@@ -226,12 +235,14 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * FT_C;
                 for (int j = 0; j < p.taps; ++j) {
-                    if (!mbar_wait(full_bar + 8 * slot, (uint32_t)(use & 1), wc, tagbits | 203)) { ok = false; break; }
+                    const int h = j & 1, slot = h ? size_a + slot_b : slot_a;
+                    if (!mbar_wait(full_bar + 8 * slot, (uint32_t)((h ? use_b : use_a) & 1), wc, tagbits | 203)) { ok = false; break; }
                     tc_fence_after();
                     mma_i8_sub<2>(d_tmem, desc_lo0 + (uint32_t)slot * (FT_A_BYTES >> 4), w1_lo + (uint32_t)j * (FT_W1_BYTES >> 4), desc_hi32,
                                   p.idesc1, j != 0 ? 1u : 0u);
                     mma_commit(empty_bar + 8 * slot);
-                    if (++slot == p.stages) { slot = 0; ++use; }
+                    if (h) { if (++slot_b == size_b) { slot_b = 0; ++use_b; } }
+                    else if (++slot_a == size_a) { slot_a = 0; ++use_a; }
                 }
                 if (!ok) break;
                 mma_commit(tfull1 + 8 * acc);
@@ -244,9 +255,12 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
             if (ok) {
                 // arrivals nobody else waits for must land before the CTA goes: the releases of the last stage uses and of
                 // the staged tile
-                const int total = n_local * p.taps;
-                for (int g = max(0, total - p.stages); g < total; ++g)
-                    mbar_wait(empty_bar + 8 * (g % p.stages), (uint32_t)(g / p.stages) & 1u, wc, tagbits | 212);
+                for (int h = 0; h < 2; ++h) {
+                    const int total = n_local * (h ? p.taps / 2 : (p.taps + 1) / 2);
+                    const int size = h ? size_b : size_a, first = h ? size_a : 0;
+                    for (int g = max(0, total - size); g < total; ++g)
+                        mbar_wait(empty_bar + 8 * (first + g % size), (uint32_t)(g / size) & 1u, wc, tagbits | 212);
+                }
                 mbar_wait(tmid_free, (uint32_t)((n_local - 1) & 1), wc, tagbits | 213);
             } else if (committed_any) {
                 // let the tensor pipe finish what was issued before tensor memory is released
@@ -406,6 +420,14 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         if (ok && n_local > 0) epi2(n_local - 1);
     }
 
+    if (*(volatile int *)&ctl.abort_flag) {
+        // A wait gave up: the roles have left their loops with copies and tensor-core work possibly still on their way to
+        // this CTA's shared memory, barriers and tensor memory.  Give them time to land before the CTA goes (the
+        // failure is already on record; this only keeps it from turning into a fault).
+        const unsigned long long t0 = clock64();
+        while ((unsigned long long)(clock64() - t0) < 400000ull) {
+        }
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == FT_MMA_WARP) {
@@ -504,6 +526,11 @@ cudaError_t f8_fused_plan_init(F8FusedPlan *plan, const F8ConvGeom &g1, const F8
         return cudaErrorInvalidValue;
     }
     p.stages = stages;
+    {
+        // the ring of the even taps gets its share of the stages (all of them when there is a single tap)
+        const int taps_a = (p.taps + 1) / 2;
+        p.stages_a = p.taps == 1 ? stages : std::min(stages - 1, std::max(1, (stages * taps_a + p.taps - 1) / p.taps));
+    }
     p.w1_off = (uint32_t)stages * FT_A_BYTES;
     p.w2_off = p.w1_off + (uint32_t)p.taps * FT_W1_BYTES;
     p.t_off = p.w2_off + FT_W2_BYTES;

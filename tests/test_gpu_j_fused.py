@@ -19,6 +19,7 @@ FUSED_CASES = [
     (31, 31, 3, 2, 0, 10, True, synth.S8, True, False),      # stride 2 without padding
     (20, 20, 4, 1, 1, 12, False, synth.U8, False, True),     # sixteen taps: more taps than stages (two rounds per tile)
     (56, 56, 3, 1, 1, 64, False, synth.U8, True, True),      # 1568 tiles: ten or eleven per CTA
+    (56, 56, 3, 1, 1, 256, False, synth.U8, True, False),    # the bench shape: 6272 tiles, tensors beyond the L2 cache
 ]
 
 
@@ -80,3 +81,30 @@ def test_conv_pointwise_fused_rejects_what_it_cannot_run():
     d1 = a.conv_desc(first, 0)
     d2 = a.conv_desc(second, 0)
     a.f8_conv_pointwise_fixed(d1, d2, x, w1, b1, w2, b2, None, None, y)      # an empty batch is not an error
+
+
+def test_conv_pointwise_fused_many_launches(ref):
+    """Forty launches back to back (no synchronisation in between) over rotating buffers, every output compared with the
+    oracle's: the two producer warps, the issuer and the epilogue run at whatever skew the memory system gives them."""
+    a = api()
+    rng = np.random.default_rng(1700)
+    first, second = _pair(rng, 56, 56, 3, 1, 1, False, synth.U8, True)
+    n, sets = 48, 4
+    w1, b1, w2, b2 = (a.to_device(t) for t in (first.weight, first.bias, second.weight, second.bias))
+    xs, rs, wants, ys = [], [], [], []
+    for _ in range(sets):
+        x = random_input(rng, n, first)
+        res = random_residual(rng, n, second)
+        wants.append(ref.run_layer(second, ref.run_layer(first, x, None), res))
+        xs.append(a.to_device(x))
+        rs.append(a.to_device(res))
+    d1, d2 = a.conv_desc(first, n), a.conv_desc(second, n)
+    for rep in range(10):
+        ys = [Guarded((n, 56, 56, 256), torch.uint8) for _ in range(sets)]
+        for i in range(sets):
+            a.f8_conv_pointwise_fixed(d1, d2, xs[i], w1, b1, w2, b2, rs[i], None, ys[i].t)
+        torch.cuda.synchronize()
+        a.f8_device_status()
+        for i in range(sets):
+            assert ys[i].intact()
+            assert_equal_arrays(ys[i].t.cpu().numpy(), wants[i], f"round {rep}, set {i}: ")
