@@ -33,7 +33,8 @@ constexpr int FT_MAX_OUT_BUFS = 4;
 constexpr int FT_EPI_WARPS = 16;
 constexpr int FT_A_WARP = 0, FT_MMA_WARP = 1, FT_MOVER_WARP = 2, FT_FETCH_WARP = 3, FT_FIRST_EPI = 4;
 constexpr int FT_A2_WARP = FT_FIRST_EPI + FT_EPI_WARPS;
-constexpr int FT_THREADS = 32 * (FT_A2_WARP + 1);
+constexpr int FT_MMA2_WARP = FT_A2_WARP + 2;        // (the warp in between would share the first issuer's scheduler)
+constexpr int FT_THREADS = 32 * (FT_MMA2_WARP + 1);
 constexpr uint32_t FT_A_BYTES = FT_TILE_M * FT_C;          // one tap of a tile
 constexpr uint32_t FT_W1_BYTES = FT_C * FT_C;              // one tap of the first layer's weights
 constexpr uint32_t FT_W2_BYTES = FT_N2 * FT_C;
@@ -68,7 +69,7 @@ struct FtParams {
     int m_tiles;
     FtDiv div_wo, div_ho;
     int stages, out_bufs;
-    int stages_a;               // stages of the ring of the even taps (the odd taps' ring takes the rest)
+    int group, groups;          // taps per stage, stages uses per tile
     uint32_t w1_off, w2_off, t_off, out_off, bias_off;      // byte offsets behind the control block
     uint32_t idesc1, idesc2;
     uint64_t desc_hi;
@@ -114,7 +115,7 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     if (threadIdx.x == 0) {
         ctl.abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(full_bar + 8 * s, 1);        // the lane that requests the tap announces its bytes
+            mbar_init(full_bar + 8 * s, p.group);  // every lane that requests a tap of the group announces its bytes
             mbar_init(empty_bar + 8 * s, 1);       // commit of the MMAs that read the stage
         }
         mbar_init(wres_bar, 1);
@@ -147,12 +148,12 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 
     if (warp == FT_A_WARP || warp == FT_A2_WARP) {
         // ------------------------------------------------------------------ TMA producers
-        // Two producer warps, two rings.  Warp h requests the taps of parity h (lane q: tap 2 q + h) into a ring of its
-        // own: S_h stages, T_h taps per tile, tap q of local tile l is use u = l * T_h + q of that ring (stage u mod S_h,
-        // use u div S_h).  A parity wait can only tell a phase from its neighbour, so the thread that refills a stage
-        // must know that the stage's previous refill has happened.  Inside one warp it does: that refill's wait comes
-        // earlier in the warp's program order (an earlier tile, or an earlier round below).  One ring shared by both
-        // warps would not give that: the stages would rotate between lanes of two warps that do not wait for each other.
+        // A stage holds a group of G consecutive taps of one tile (one barrier pair per group: every wait, fence and commit
+        // costs the lone MMA-issuing thread a few hundred cycles, as much as several MMAs).  Group k of local tile l is
+        // use u = l * groups + k of the ring: stage u mod S, use u div S.  Warp h requests the uses of parity h, every
+        // tap in a lane of its own (loads issued by different threads overlap).  S is even, so a stage is always
+        // refilled by the same warp: the wait for its previous refill comes earlier in that warp's program order, and
+        // a parity wait (which can only tell a phase from its neighbour) cannot take an older release for the last one.
         const int half = warp == FT_A2_WARP ? 1 : 0;
         if (half == 1) {
             // the weights of both layers, once per CTA: nothing the previous grid writes
@@ -163,42 +164,45 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
             else if (lane == n_loads - 1) tma_load_3d(smem_base + p.w2_off, &map_w2, wres_bar, 0, 0, 0);
         }
         grid_dependency_wait();
-        const int taps_h = half ? p.taps / 2 : (p.taps + 1) / 2;
-        const int S = half ? p.stages - p.stages_a : p.stages_a;
-        const int base = half ? p.stages_a : 0;
-        const int tap = 2 * lane + half;
-        const bool mine = lane < taps_h;
-        const int r = tap / p.kw, sx = tap - r * p.kw;
-        int slot = S > 0 ? lane % S : 0, use = S > 0 ? lane / S : 0;
+        const int G = p.group, NG = p.groups, S = p.stages, per_round = S >> 1;
+        const int gi = lane / G, ti = lane - gi * G;       // this lane's group among the warp's groups of a tile, tap in the group
         bool ok = true, have_last = false;
         int last_slot = 0;
         uint32_t last_par = 0;
-        for (int l = 0; taps_h > 0 && l < n_local; ++l) {
+        for (int l = 0; l < n_local; ++l) {
             const int m0 = (worker + l * n_workers) * FT_TILE_M;
             const int t1 = ft_div(m0, p.div_wo);
             const int ow = m0 - t1 * p.wo;
             const int img = ft_div(t1, p.div_ho);
             const int oh = t1 - img * p.ho;
-            // With fewer stages than taps the taps go in rounds of S: the lanes of one round wait for different stages,
-            // and a stage a later round needs is freed by loads that were requested in an earlier one.
-            for (int q0 = 0; ok && q0 < taps_h; q0 += S) {
-                const bool act = mine && lane >= q0 && lane < q0 + S;
+            const int u0 = l * NG;
+            const int k0 = (half - u0) & 1;                          // this warp's first group of the tile
+            const int n_mine = k0 < NG ? (NG - k0 + 1) >> 1 : 0;     // groups k0, k0 + 2, ...
+            const int k = k0 + 2 * gi, u = u0 + k, tap = k * G + ti;
+            const int slot = u % S, use = u / S;
+            const int r = tap / p.kw, sx = tap - r * p.kw;
+            // at most S / 2 of the warp's groups at a time: they lie in different stages, and a stage a later round needs
+            // is freed by loads that were requested in an earlier one
+            for (int r0 = 0; ok && r0 < n_mine; r0 += per_round) {
+                const bool act = gi < n_mine && gi >= r0 && gi < r0 + per_round;
                 bool got = true;
-                if (act) got = mbar_wait(empty_bar + 8 * (base + slot), (uint32_t)(use & 1) ^ 1u, wc, tagbits | 201);
+                if (act) got = mbar_wait(empty_bar + 8 * slot, (uint32_t)(use & 1) ^ 1u, wc, tagbits | 201);
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 if (act) {
-                    const uint32_t fb = full_bar + 8 * (base + slot);
-                    mbar_expect_tx(fb, FT_A_BYTES);
-                    tma_load_im2col(smem_base + (uint32_t)(base + slot) * FT_A_BYTES, &map_a, fb, 0, ow * p.stride - p.pad,
-                                    oh * p.stride - p.pad, img, (uint16_t)sx, (uint16_t)r);
-                    have_last = true;
-                    last_slot = base + slot;
-                    last_par = (uint32_t)(use & 1);
+                    const uint32_t fb = full_bar + 8 * slot;
+                    if (tap < p.taps) {
+                        mbar_expect_tx(fb, FT_A_BYTES);
+                        tma_load_im2col(smem_base + (uint32_t)(slot * G + ti) * FT_A_BYTES, &map_a, fb, 0, ow * p.stride - p.pad,
+                                        oh * p.stride - p.pad, img, (uint16_t)sx, (uint16_t)r);
+                        have_last = true;
+                        last_slot = slot;
+                        last_par = (uint32_t)(use & 1);
+                    } else {
+                        mbar_arrive(fb);        // a tap the last group does not have
+                    }
                 }
             }
             if (!ok) break;
-            slot += taps_h;
-            while (slot >= S) { slot -= S; ++use; }
         }
         if (!ok && have_last) {
             const unsigned long long t0 = clock64();
@@ -212,62 +216,67 @@ f8_conv_pw_fused_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         if (lane == 0 && n_local > 0) {
             const uint32_t desc_lo0 = (uint32_t)p.desc_hi | ((smem_base & 0x3ffffu) >> 4);
             const uint32_t desc_hi32 = (uint32_t)(p.desc_hi >> 32);
-            const uint32_t w1_lo = desc_lo0 + (p.w1_off >> 4), w2_lo = desc_lo0 + (p.w2_off >> 4), t_lo = desc_lo0 + (p.t_off >> 4);
+            const uint32_t w1_lo = desc_lo0 + (p.w1_off >> 4);
             bool ok = mbar_wait(wres_bar, 0, wc, tagbits | 211);
             bool committed_any = false;
             int last_acc = 0;
             uint32_t last_acc_phase = 0;
-            int slot_a = 0, use_a = 0, slot_b = 0, use_b = 0;       // position in the ring of the even / odd taps
-            const int size_a = p.stages_a, size_b = p.stages - p.stages_a;
-            // GEMM 2 of local tile i: the staged tile times the pointwise weights
-            auto gemm2 = [&](int i) -> bool {
-                if (!mbar_wait(tmid_full, (uint32_t)(i & 1), wc, tagbits | 205)) return false;
-                if (!mbar_wait(tempty2, (uint32_t)(i & 1) ^ 1u, wc, tagbits | 206)) return false;
-                tc_fence_after();
-                mma_i8_sub<2>(tmem_base + FT_ACC2_COL, t_lo, w2_lo, desc_hi32, p.idesc2, 0u);
-                mma_commit(tmid_free);
-                mma_commit(tfull2);
-                return true;
-            };
+            int slot = 0, use = 0;
+            const int G = p.group, NG = p.groups;
             for (int l = 0; ok && l < n_local; ++l) {
                 const int acc = l & 1;
                 if (!mbar_wait(tempty1 + 8 * acc, (uint32_t)((l >> 1) & 1) ^ 1u, wc, tagbits | 202)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * FT_C;
-                for (int j = 0; j < p.taps; ++j) {
-                    const int h = j & 1, slot = h ? size_a + slot_b : slot_a;
-                    if (!mbar_wait(full_bar + 8 * slot, (uint32_t)((h ? use_b : use_a) & 1), wc, tagbits | 203)) { ok = false; break; }
+                int tap = 0;
+                for (int k = 0; k < NG; ++k) {
+                    if (!mbar_wait(full_bar + 8 * slot, (uint32_t)(use & 1), wc, tagbits | 203)) { ok = false; break; }
                     tc_fence_after();
-                    mma_i8_sub<2>(d_tmem, desc_lo0 + (uint32_t)slot * (FT_A_BYTES >> 4), w1_lo + (uint32_t)j * (FT_W1_BYTES >> 4), desc_hi32,
-                                  p.idesc1, j != 0 ? 1u : 0u);
+                    uint32_t a_lo = desc_lo0 + (uint32_t)(slot * G) * (FT_A_BYTES >> 4);
+                    for (int t = 0; t < G && tap < p.taps; ++t, ++tap, a_lo += FT_A_BYTES >> 4)
+                        mma_i8_sub<2>(d_tmem, a_lo, w1_lo + (uint32_t)tap * (FT_W1_BYTES >> 4), desc_hi32, p.idesc1, tap != 0 ? 1u : 0u);
                     mma_commit(empty_bar + 8 * slot);
-                    if (h) { if (++slot_b == size_b) { slot_b = 0; ++use_b; } }
-                    else if (++slot_a == size_a) { slot_a = 0; ++use_a; }
+                    if (++slot == p.stages) { slot = 0; ++use; }
                 }
                 if (!ok) break;
                 mma_commit(tfull1 + 8 * acc);
                 committed_any = true;
                 last_acc = acc;
                 last_acc_phase = (uint32_t)((l >> 1) & 1);
-                if (l >= 1 && !gemm2(l - 1)) { ok = false; break; }
             }
-            if (ok) ok = gemm2(n_local - 1);
             if (ok) {
-                // arrivals nobody else waits for must land before the CTA goes: the releases of the last stage uses and of
-                // the staged tile
-                for (int h = 0; h < 2; ++h) {
-                    const int total = n_local * (h ? p.taps / 2 : (p.taps + 1) / 2);
-                    const int size = h ? size_b : size_a, first = h ? size_a : 0;
-                    for (int g = max(0, total - size); g < total; ++g)
-                        mbar_wait(empty_bar + 8 * (first + g % size), (uint32_t)(g / size) & 1u, wc, tagbits | 212);
-                }
-                mbar_wait(tmid_free, (uint32_t)((n_local - 1) & 1), wc, tagbits | 213);
+                // the releases of the last stage uses, which nobody else waits for, must land before the CTA goes
+                const int total = n_local * NG;
+                for (int g = max(0, total - p.stages); g < total; ++g)
+                    mbar_wait(empty_bar + 8 * (g % p.stages), (uint32_t)(g / p.stages) & 1u, wc, tagbits | 212);
             } else if (committed_any) {
                 // let the tensor pipe finish what was issued before tensor memory is released
                 const unsigned long long t0 = clock64();
                 while (!mbar_try_wait(tfull1 + 8 * last_acc, last_acc_phase) && (unsigned long long)(clock64() - t0) < DRAIN_LIMIT_CYCLES) {
                 }
             }
+        }
+    } else if (warp == FT_MMA2_WARP) {
+        // ------------------------------------------------------------------ second issuer: the pointwise GEMM
+        // GEMM 2 of local tile i: the staged tile times the pointwise weights, as soon as the first layer's epilogue has
+        // written the tile and the second layer's epilogue has read the previous result out of the accumulator.  A thread
+        // of its own, so that these waits do not sit between the first issuer's instructions.
+        if (lane == 0 && n_local > 0) {
+            const uint32_t desc_lo0 = (uint32_t)p.desc_hi | ((smem_base & 0x3ffffu) >> 4);
+            const uint32_t desc_hi32 = (uint32_t)(p.desc_hi >> 32);
+            const uint32_t w2_lo = desc_lo0 + (p.w2_off >> 4), t_lo = desc_lo0 + (p.t_off >> 4);
+            bool ok = mbar_wait(wres_bar, 0, wc, tagbits | 214);
+            int i = 0;
+            for (; ok && i < n_local; ++i) {
+                if (!mbar_wait(tmid_full, (uint32_t)(i & 1), wc, tagbits | 205)) { ok = false; break; }
+                if (!mbar_wait(tempty2, (uint32_t)(i & 1) ^ 1u, wc, tagbits | 206)) { ok = false; break; }
+                tc_fence_after();
+                mma_i8_sub<2>(tmem_base + FT_ACC2_COL, t_lo, w2_lo, desc_hi32, p.idesc2, 0u);
+                mma_commit(tmid_free);
+                mma_commit(tfull2);
+            }
+            // the last release of the staged tile has no other waiter
+            if (ok) mbar_wait(tmid_free, (uint32_t)((n_local - 1) & 1), wc, tagbits | 213);
         }
     } else if (warp == FT_MOVER_WARP) {
         // ------------------------------------------------------------------ output mover
@@ -517,21 +526,22 @@ cudaError_t f8_fused_plan_init(F8FusedPlan *plan, const F8ConvGeom &g1, const F8
     p.div_ho = ft_make_div(g1.ho);
     // shared memory: stages | first layer's weights | pointwise weights | staged tile | output ring | bias tables.
     // With a shortcut a buffer of the ring goes through load -> convert in place -> store: three of them.
-    p.out_bufs = q2.has_res ? 3 : 2;
+    // Two buffers in the output ring (with a shortcut a buffer goes through load -> convert in place -> store; a third
+    // buffer measured no faster than two, and costs four stages).
+    p.out_bufs = 2;
+    p.group = p.taps >= 3 ? 3 : p.taps;
+    p.groups = (p.taps + p.group - 1) / p.group;
+    const size_t stage_bytes = (size_t)p.group * FT_A_BYTES;
     const size_t fixed = (size_t)p.taps * FT_W1_BYTES + FT_W2_BYTES + FT_T_BYTES + (size_t)p.out_bufs * FT_OUT_BYTES + 2048;
-    int stages = (int)((FT_SMEM_LIMIT - fixed) / FT_A_BYTES);
+    int stages = (int)((FT_SMEM_LIMIT - fixed) / stage_bytes);
     if (stages > FT_MAX_STAGES) stages = FT_MAX_STAGES;
+    stages &= ~1;           // even: a stage is always refilled by the same producer warp
     if (stages < 2) {
         *why = "stages do not fit";
         return cudaErrorInvalidValue;
     }
     p.stages = stages;
-    {
-        // the ring of the even taps gets its share of the stages (all of them when there is a single tap)
-        const int taps_a = (p.taps + 1) / 2;
-        p.stages_a = p.taps == 1 ? stages : std::min(stages - 1, std::max(1, (stages * taps_a + p.taps - 1) / p.taps));
-    }
-    p.w1_off = (uint32_t)stages * FT_A_BYTES;
+    p.w1_off = (uint32_t)(stages * stage_bytes);
     p.w2_off = p.w1_off + (uint32_t)p.taps * FT_W1_BYTES;
     p.t_off = p.w2_off + FT_W2_BYTES;
     p.out_off = p.t_off + FT_T_BYTES;
