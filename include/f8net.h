@@ -228,6 +228,11 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
 /* Number of kernels the last f8_net_forward on this object enqueued. */
 int f8_net_last_launch_count(const f8_net *net);
 
+/* Number of those kernels that ran two layers at once (a 64 -> 64 convolution and the 64 -> 256 pointwise layer that
+ * alone reads its output: see f8_conv_pointwise_fixed).  f8_net_forward does that wherever the shapes allow; the
+ * first layer's output then exists in device memory only in a pass that asks for layer dumps. */
+int f8_net_fused_pairs(const f8_net *net);
+
 /* Per-layer timing.  With profiling on, f8_net_forward records a CUDA event after every kernel it
  * enqueues; f8_net_get_layer_ms waits for the last profiled pass and writes the device time of
  * each layer (ms[n_layers]; a stem's packing pre-pass is added to its layer) and, if
@@ -353,6 +358,7 @@ void f8_debug_force_direct(int on);
  *   F8_PLAN_OFF_STEM_KERNEL       first layers take the packed-row-pair GEMM instead of the first-layer kernel
  *   F8_PLAN_OFF_STEM_POOL_FUSION  the max pool behind a first layer runs as its own kernel
  *   F8_PLAN_OFF_LAYER_OVERLAP     f8_net_forward launches without programmatic dependent launch
+ *   F8_PLAN_OFF_LAYER_FUSION      f8_net_forward runs a 64 -> 64 convolution and the 64 -> 256 pointwise layer behind it as two launches
  *   F8_PLAN_OFF_LANES             f8_net_forward runs the whole batch as one sequence of launches on the caller's stream
  *   F8_PLAN_SYNC_LAYERS           f8_net_forward synchronises after every launch, so that a device fault is
  *                                 reported with the layer that raised it */
@@ -360,7 +366,7 @@ enum {
     F8_PLAN_OFF_RESIDENT_WEIGHTS = 1, F8_PLAN_OFF_WINDOWED = 2, F8_PLAN_OFF_DUAL_ISSUE = 4, F8_PLAN_OFF_ALT_PRODUCERS = 8,
     F8_PLAN_OFF_PAIRS = 16, F8_PLAN_OFF_DW_WALK = 32, F8_PLAN_OFF_STEM_KERNEL = 64, F8_PLAN_OFF_STEM_POOL_FUSION = 128,
     F8_PLAN_OFF_LAYER_OVERLAP = 256, F8_PLAN_OFF_LANES = 512, F8_PLAN_SYNC_LAYERS = 1024, F8_PLAN_OFF_DW_DP4A = 2048,
-    F8_PLAN_OFF_TILE_GROUPS = 4096
+    F8_PLAN_OFF_TILE_GROUPS = 4096, F8_PLAN_OFF_LAYER_FUSION = 8192
 };
 void f8_debug_plan_options(unsigned off_mask);
 

@@ -250,6 +250,7 @@ PLAN_OFF_RESIDENT_WEIGHTS, PLAN_OFF_WINDOWED, PLAN_OFF_DUAL_ISSUE, PLAN_OFF_ALT_
 PLAN_OFF_PAIRS, PLAN_OFF_DW_WALK, PLAN_OFF_STEM_KERNEL, PLAN_OFF_STEM_POOL_FUSION = 16, 32, 64, 128
 PLAN_OFF_LAYER_OVERLAP, PLAN_OFF_LANES, PLAN_SYNC_LAYERS, PLAN_OFF_DW_DP4A = 256, 512, 1024, 2048
 PLAN_OFF_TILE_GROUPS = 4096
+PLAN_OFF_LAYER_FUSION = 8192
 PLAN_RESIDENT_WEIGHTS, PLAN_WINDOWED, PLAN_DUAL_ISSUE, PLAN_ALT_PRODUCERS = 1, 2, 4, 8
 PLAN_PLAIN_MATRIX, PLAN_STAGED_EPILOGUE, PLAN_PAIRS, PLAN_ROW_TILES = 16, 32, 64, 128
 PLAN_TILE_GROUPS = 256
@@ -272,6 +273,7 @@ def f8_debug_set_micro_batch(images: int):
 _lib.f8_debug_set_lanes.argtypes = [_ci]
 _lib.f8_debug_set_lanes.restype = None
 _lib.f8_net_lanes.argtypes = [_vp]
+_lib.f8_net_fused_pairs.argtypes = [_vp]
 
 
 def f8_debug_set_lanes(lanes: int):
@@ -411,6 +413,11 @@ class Net:
     @property
     def lanes(self) -> int:
         return int(_lib.f8_net_lanes(self._h))
+
+    @property
+    def fused_pairs(self) -> int:
+        """Launches of the last forward pass that ran two layers at once."""
+        return int(_lib.f8_net_fused_pairs(self._h))
 
     def micro_batching(self):
         """(number of runs of layers the last forward pass executed depth-first over micro-batches, smallest micro-batch)."""

@@ -130,6 +130,16 @@ PlanPtr alloc_plan() {
     return PlanPtr((F8TcPlan *)p);
 }
 
+struct FusedPlanDeleter { void operator()(F8FusedPlan *p) const { free(p); } };
+using FusedPlanPtr = std::unique_ptr<F8FusedPlan, FusedPlanDeleter>;
+
+FusedPlanPtr alloc_fused_plan() {
+    const size_t size = (f8_fused_plan_size() + 63) / 64 * 64;
+    void *p = aligned_alloc(64, size);
+    if (p) memset(p, 0, size);
+    return FusedPlanPtr((F8FusedPlan *)p);
+}
+
 // The second consumer of a layer's sum: its quantizer relative to the format F of the aligned sum.
 f8_status make_sibling(const f8_conv_desc *d, const F8Requant &q, int y2_dtype, int fl_y2, void *y2, F8Sibling *sib) {
     if (y2_dtype != F8_U8 && y2_dtype != F8_S8 && y2_dtype != F8_S32 && y2_dtype != F8_S32_RELU)
@@ -481,6 +491,10 @@ struct Step {
     int img0 = 0;             // first image of the batch this step works on (lanes, micro-batched runs)
     int lane = 0;             // 0: the caller's stream; 1: the network's second stream
     PlanPtr plan;
+    // kind -3: this layer and the pointwise layer behind it (layer + 1) in one launch; y is that layer's output,
+    // y_mid NULL or where a copy of this layer's own output goes
+    FusedPlanPtr fplan;
+    void *y_mid = nullptr;
     F8ConvGeom g;
 };
 
@@ -508,6 +522,7 @@ struct f8_net {
     void *plan_y = nullptr, *plan_ws = nullptr;
     bool plan_force_direct = false;
     bool plan_dump_first = false;                // the cached plan keeps the output of a fusable first layer
+    bool plan_dumping = false;                   // the cached plan was made for a pass that copies layer outputs
     std::vector<Step> steps;
     std::vector<size_t> t_off;                   // workspace offset per tensor
     size_t pack_off = 0;
@@ -636,6 +651,26 @@ void classify_tensors(const f8_net *net, const std::vector<Region> &regions, std
 }
 
 // Assigns workspace offsets: tensors whose lifetimes do not overlap may share memory (first fit).
+// Layer i and the pointwise layer behind it may run as one launch (the two-layer kernel): layer i + 1 is a 1x1 convolution
+// that alone reads layer i's output, and the channel counts are the kernel's.  (Whether they do is decided per plan: the
+// batch must make the input large enough, and both layers must lie in the same run of the schedule.)
+bool pair_candidate(const f8_net *net, int i) {
+    const int nl = (int)net->layers.size();
+    if (i + 1 >= nl) return false;
+    const NetLayer &L = net->layers[i], &P = net->layers[i + 1];
+    if (L.d.kind != F8_LAYER_CONV || L.packed || L.has_sibling || L.q.has_res) return false;
+    if (P.d.kind != F8_LAYER_CONV || P.has_sibling || P.packed || P.d.src != i + 1 || P.g.kh != 1 || P.g.kw != 1 || P.g.stride_h != 1 ||
+        P.g.stride_w != 1 || P.g.pad_h != 0 || P.g.pad_w != 0)
+        return false;
+    if (P.q.has_res && P.d.res == i + 1) return false;
+    if (net->t_cp[i + 1] != L.g.c_out) return false;
+    for (int l2 = i + 2; l2 < nl; ++l2)
+        if (net->layers[l2].d.src == i + 1 || (net->layers[l2].q.has_res && net->layers[l2].d.res == i + 1)) return false;
+    F8ConvGeom g = L.g;
+    g.n = net->max_batch;   // the size rule is checked again with the real batch when a plan is made
+    return f8_fused_supported(g, L.q, P.g.c_out, P.q);
+}
+
 size_t assign_offsets(const f8_net *net, int batch, std::vector<size_t> *off, size_t *pack_off,
                       const std::vector<Region> &regions) {
     const int nl = (int)net->layers.size();
@@ -652,6 +687,10 @@ size_t assign_offsets(const f8_net *net, int batch, std::vector<size_t> *off, si
         born[t] = net->layers[t - 1].d.kind == F8_LAYER_SIBLING ? t - 2 : t - 1;
         last[t] = std::max(last[t], born[t]);
     }
+    // the two-layer kernel writes the second layer's output while it still reads the first layer's input: that output is
+    // born with the first layer's launch, so that it shares memory with nothing the launch reads
+    for (int i = 0; i + 1 < nl; ++i)
+        if (pair_candidate(net, i)) born[i + 2] = std::min(born[i + 2], i);
     // A full-size tensor that a micro-batched run writes is filled slice by slice over the whole run, and one that the
     // run reads is read again by every micro-batch: both are live from the run's first layer to its last.
     for (int t = 1; t < nt; ++t) {
@@ -979,6 +1018,13 @@ int f8_net_last_launch_count(const f8_net *net) { return net ? net->last_launche
 
 int f8_net_lanes(const f8_net *net) { return net ? net->last_lanes : 0; }
 
+int f8_net_fused_pairs(const f8_net *net) {
+    int n = 0;
+    if (net)
+        for (const Step &stp : net->steps) n += stp.kind == -3 ? 1 : 0;
+    return n;
+}
+
 int f8_net_micro_batching(const f8_net *net, int *images) {
     if (images) *images = net ? net->last_micro : 0;
     return net ? net->last_regions : 0;
@@ -1008,6 +1054,7 @@ f8_status f8_net_get_layer_ms(f8_net *net, float *ms, int *on_tensor_cores) {
     if (on_tensor_cores)
         for (const Step &stp : net->steps)
             if (stp.kind >= 0 && stp.use_tc) on_tensor_cores[stp.layer] = 1;
+            else if (stp.kind == -3) on_tensor_cores[stp.layer] = on_tensor_cores[stp.layer + 1] = 1;
     return F8_OK;
 }
 
@@ -1044,6 +1091,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
             if (net->layers[i].w_core && layer_dump[i]) dump_fusable = true;
     const bool replan = net->plan_batch != batch || net->plan_x != x || net->plan_y != y || net->plan_ws != workspace ||
                         net->plan_force_direct != g_force_direct || net->plan_dump_first != dump_fusable ||
+                        net->plan_dumping != (layer_dump != nullptr) ||
                         net->plan_options != g_plan_off || net->plan_micro != g_micro_batch || net->plan_lanes != g_lanes ||
                         net->plan_profiling != net->profiling;
     net->overlap_layers = !(g_plan_off & F8_PLAN_OFF_LAYER_OVERLAP);
@@ -1171,6 +1219,33 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                             stp.plan = std::move(plan);
                         }
                     }
+                } else if ([&]() -> bool {
+                               // This layer and the pointwise layer behind it in one launch (the tail of a bottleneck block):
+                               // the next layer is a 1x1 convolution that alone reads this layer's output, both lie in the
+                               // same run of the schedule, and the shapes are the two-layer kernel's.
+                               if (g_plan_off & F8_PLAN_OFF_LAYER_FUSION) return false;
+                               if (!pair_candidate(net, i) || layer_region[i] != layer_region[i + 1]) return false;
+                               const NetLayer &P = net->layers[i + 1];
+                               if (!f8_fused_supported(stp.g, L.q, P.g.c_out, P.q)) return false;
+                               FusedPlanPtr fp = alloc_fused_plan();
+                               if (!fp) return false;
+                               const void *res2 = P.q.has_res ? tensor_ptr(P.d.res) : nullptr;
+                               void *mid = layer_dump ? tensor_ptr(i + 1) : nullptr;      // only a pass that copies outputs keeps it
+                               if (f8_fused_plan_init(fp.get(), stp.g, L.q, P.q, stp.x, L.w, L.b, P.w, P.b, res2, mid, tensor_ptr(i + 2),
+                                                      f8_status_word(), &why) != cudaSuccess) {
+                                   (void)cudaGetLastError();
+                                   return false;
+                               }
+                               f8_fused_plan_set_tag(fp.get(), i + 2);
+                               stp.kind = -3;
+                               stp.use_tc = true;
+                               stp.y = tensor_ptr(i + 2);
+                               stp.y_mid = mid;
+                               stp.fplan = std::move(fp);
+                               skip_layer = i + 1;
+                               return true;
+                           }()) {
+                    // planned above
                 } else if (f8_tc_supported(stp.g, (size_t)n * L.g.h * L.g.w * L.g.c)) {
                     PlanPtr plan = alloc_plan();
                     if (plan && f8_tc_plan_init(plan.get(), stp.g, L.q, dense_view(stp.x, stp.g), L.w, L.b, stp.res,
@@ -1216,6 +1291,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         net->plan_ws = workspace;
         net->plan_force_direct = g_force_direct;
         net->plan_dump_first = dump_fusable;
+        net->plan_dumping = layer_dump != nullptr;
         net->plan_options = g_plan_off;
         net->plan_micro = g_micro_batch;
         net->plan_lanes = g_lanes;
@@ -1251,6 +1327,10 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                                       L.w_core, L.b, stp.y, f8_status_word(), stp.layer + 1, st, net->overlap_layers);
                 ++g_tc_launches;
                 break;
+            case -3:
+                e = f8_fused_launch(stp.fplan.get(), net->overlap_layers, st);
+                ++g_tc_launches;
+                break;
             case -1:
                 e = f8_launch_pack_stem_pairs(stp.g.n, L.g.h, L.g.w, L.g.c, L.pack_cpad, L.pack_hp, L.pack_wp, L.pack_left, stp.x, stp.y, st,
                                               net->overlap_layers);
@@ -1282,7 +1362,7 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
         ++launches;
         if (prof) {
             cudaEventRecord(net->events[launches], st);
-            net->event_layer.push_back(stp.fused_pool ? stp.layer + 1 : stp.layer);
+            net->event_layer.push_back(stp.fused_pool || stp.kind == -3 ? stp.layer + 1 : stp.layer);
         }
         // copies of the outputs this step wrote: its layer's (the pooling layer's when fused), and a sibling's
         auto dump_layer = [&](int out_layer, const void *src) -> cudaError_t {
@@ -1299,7 +1379,8 @@ f8_status f8_net_forward(f8_net *net, int batch, const void *x, void *y, void *w
                                      cudaMemcpyDeviceToDevice, st);
         };
         if (stp.kind != -1) {
-            e = dump_layer(stp.fused_pool ? stp.layer + 1 : stp.layer, stp.y);
+            e = dump_layer(stp.fused_pool || stp.kind == -3 ? stp.layer + 1 : stp.layer, stp.y);
+            if (e == cudaSuccess && stp.kind == -3 && stp.y_mid) e = dump_layer(stp.layer, stp.y_mid);
             if (e == cudaSuccess && stp.has_sib) e = dump_layer(stp.layer + 1, stp.sib.y2);
             if (e != cudaSuccess) return cuda_fail(e, "layer dump copy");
         }

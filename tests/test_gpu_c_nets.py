@@ -52,13 +52,19 @@ def _compare_net(ref, name, batch, image, force_direct=False, seed=0, plan_off=0
     assert out.intact() and ws.intact(), "bytes next to the output or the workspace were overwritten"
     # one launch per layer, except that a sibling layer is written by its parent's launch and a first layer may take
     # the pooling layer behind it along
-    assert net.last_launch_count >= sum(1 for l in layers if l.kind != synth.SIBLING) - 1
+    # ... and a 64 -> 64 convolution runs in one launch with the 64 -> 256 pointwise layer behind it
+    fused = net.fused_pairs
+    if plan_off & a.PLAN_OFF_LAYER_FUSION or force_direct:
+        assert fused == 0
+    elif name == "resnet50" and image == 224 and not micro_batch:
+        assert fused == 3 * (2 if lanes == 2 else 1), "the three bottleneck tails of the first stage should each be one launch"
+    assert net.last_launch_count >= sum(1 for l in layers if l.kind != synth.SIBLING) - 1 - fused
     tc = a.f8_tc_launch_count() - before
     if force_direct:
         assert tc == 0
     elif image == 224 and not micro_batch and lanes != 2:
         # every dense layer whose input is at least 128 KiB and has c % 16 == 0 (or is a packed stem)
-        assert tc >= sum(1 for l in layers if l.kind == synth.CONV and l.c % 16 == 0 and batch * l.h * l.w * l.c >= 131072)
+        assert tc >= sum(1 for l in layers if l.kind == synth.CONV and l.c % 16 == 0 and batch * l.h * l.w * l.c >= 131072) - fused
     net.close()
 
 
@@ -84,10 +90,10 @@ def _off_masks():
     from paper_2202_05239_b200 import api as a
     return [a.PLAN_OFF_STEM_KERNEL, a.PLAN_OFF_STEM_POOL_FUSION, a.PLAN_OFF_LAYER_OVERLAP, a.PLAN_OFF_LANES,
             a.PLAN_OFF_DUAL_ISSUE | a.PLAN_OFF_ALT_PRODUCERS, a.PLAN_OFF_RESIDENT_WEIGHTS, a.PLAN_OFF_PAIRS,
-            a.PLAN_SYNC_LAYERS]
+            a.PLAN_SYNC_LAYERS, a.PLAN_OFF_LAYER_FUSION]
 
 
-@pytest.mark.parametrize("case", range(8))
+@pytest.mark.parametrize("case", range(9))
 def test_net_parity_with_planning_choices_switched_off(ref, case):
     """The alternative code paths behind f8_debug_plan_options give the same bits."""
     _compare_net(ref, "resnet50", 4, 224, plan_off=_off_masks()[case])
