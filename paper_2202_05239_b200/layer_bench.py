@@ -183,11 +183,55 @@ def bench_requant(n: int, iters: int, warmup: int):
     print(json.dumps({"op": "requantize_dual", "n": n, "ms": ms, "algorithmic_gbs": 6.0 * n / (ms * 1e-3) / 1e9}), flush=True)
 
 
+def bench_fused(h: int, batch: int, with_res: bool, iters: int, warmup: int):
+    """Device time of the two-layer kernel (f8_conv_pointwise_fixed): 3x3 64 -> 64 and 1x1 64 -> 256 (+ shortcut) at h x h,
+    over rotating buffer sets larger than twice the L2 cache.  Algorithmic bytes: the first layer's input, the shortcut,
+    the second layer's output, both layers' parameters (the tensor between the layers does not travel)."""
+    rng = np.random.default_rng(3)
+    w1, fl1 = synth.draw_weight(rng, (64, 3, 3, 64), math.sqrt(2.0 / 576))
+    w2, fl2 = synth.draw_weight(rng, (256, 1, 1, 64), math.sqrt(2.0 / 64))
+    first = synth.Layer(synth.CONV, "conv3x3", 0, -1, h, h, 64, 64, 3, 3, 1, 1, synth.U8, synth.U8, synth.U8, 5, fl1, 5, 5, w1,
+                        synth.draw_bias(rng, 64, 5 + fl1))
+    second = synth.Layer(synth.CONV, "conv1x1", 1, 0 if with_res else -1, h, h, 64, 256, 1, 1, 1, 0, synth.U8, synth.U8, synth.U8, 5, fl2,
+                         5, 5, w2, synth.draw_bias(rng, 256, 5 + fl2))
+    x_bytes, y_bytes = batch * h * h * 64, batch * h * h * 256
+    per_set = x_bytes + y_bytes * (2 if with_res else 1)
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    sets = min(16, max(2, math.ceil(2.2 * l2 / per_set)))
+    xs = [torch.randint(0, 255, (batch, h, h, 64), dtype=torch.uint8, device="cuda") for _ in range(sets)]
+    rs = [torch.randint(0, 255, (batch, h, h, 256), dtype=torch.uint8, device="cuda") if with_res else None for _ in range(sets)]
+    ys = [torch.empty((batch, h, h, 256), dtype=torch.uint8, device="cuda") for _ in range(sets)]
+    p1 = (api.to_device(first.weight), api.to_device(first.bias))
+    p2 = (api.to_device(second.weight), api.to_device(second.bias))
+    d1, d2 = api.conv_desc(first, batch), api.conv_desc(second, batch)
+
+    def run(i):
+        api.f8_conv_pointwise_fixed(d1, d2, xs[i % sets], p1[0], p1[1], p2[0], p2[1], rs[i % sets], None, ys[i % sets])
+
+    for i in range(warmup):
+        run(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        run(i)
+    e1.record()
+    torch.cuda.synchronize()
+    api.f8_device_status()
+    ms = e0.elapsed_time(e1) / iters
+    byts = per_set + first.param_bytes() + second.param_bytes()
+    macs = batch * (first.macs_per_image + second.macs_per_image)
+    print(json.dumps({"op": "conv3x3_64_64 + conv1x1_64_256" + (" + shortcut" if with_res else ""), "h": h, "batch": batch, "ms": ms,
+                      "gbs": byts / (ms * 1e-3) / 1e9, "tops": 2 * macs / (ms * 1e-3) / 1e12, "bytes": byts, "buffer_sets": sets}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--requant", type=int, default=0, help="time the dual requantisation on this many int32 values")
     ap.add_argument("--fold", action="store_true", help="time the weight compile step on a [c-out, k * k * c] tensor")
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--fused", action="store_true", help="time the two-layer kernel: 3x3 64 -> 64 + 1x1 64 -> 256 at --h, --batch, --res")
     ap.add_argument("--net", default="", help="time every layer of a synthetic network: resnet18, resnet50, mobilenetv2")
     ap.add_argument("--distinct-shapes", default="", help="run every distinct dense-layer shape of this network once (for a profiler)")
     ap.add_argument("--h", type=int, default=56)
@@ -208,6 +252,9 @@ def main():
         return
     if args.fold:
         bench_fold(args.c_out, args.k * args.k * args.c, args.iters, args.warmup)
+        return
+    if args.fused:
+        bench_fused(args.h, args.batch, args.res, args.iters, args.warmup)
         return
     if args.distinct_shapes:
         run_distinct_shapes(args.distinct_shapes, args.batch)
