@@ -590,6 +590,10 @@ def run_ours(args):
                              "gbs": pair_bytes / (pair_ms * 1e-3) / 1e9 if pair_ms > 0 else None,
                              "frac_of_hbm_peak": pair_bytes / (pair_ms * 1e-3) / 1e9 / peak_gbs if pair_ms > 0 else None,
                              "tops": pair_ops / (pair_ms * 1e-3) / 1e12 if pair_ms > 0 else None},
+        "both_tensor_core_kernels": {"ms_per_step": tc_ms + pair_ms, "algorithmic_bytes_per_step": tc_bytes + pair_bytes,
+                                     "gbs": (tc_bytes + pair_bytes) / ((tc_ms + pair_ms) * 1e-3) / 1e9 if tc_ms + pair_ms > 0 else None,
+                                     "frac_of_hbm_peak": (tc_bytes + pair_bytes) / ((tc_ms + pair_ms) * 1e-3) / 1e9 / peak_gbs
+                                     if tc_ms + pair_ms > 0 else None},
         "other_kernels": {"ms_per_step": other_ms, "gbs": other_bytes / (other_ms * 1e-3) / 1e9 if other_ms > 0 else None},
         "whole_step": {"tops": total_ops / (ms_per_step * 1e-3) / 1e12,
                        "gbs": (tc_bytes + pair_bytes + other_bytes) / (ms_per_step * 1e-3) / 1e9,
